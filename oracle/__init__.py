@@ -1,0 +1,116 @@
+"""Test infrastructure: loader for the fp64 CPU oracle of paged GQA decode attention.
+
+The oracle is the plain definition of softmax attention (two passes, fp64, no
+tiling, no splits) read through a block table; see ``decode_attn_oracle.c`` for
+the statement it follows.  Only the tests, the smoke check and the benchmark's
+CPU-baseline leg may import this package.  It imports nothing from the CUDA
+package and the CUDA package imports nothing from here.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "decode_attn_oracle.c")
+_LIB = os.path.join(_HERE, "libdecode_attn_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP) into a shared library beside its source."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+           "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build())
+            i64, i32, p = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p
+            lib.decode_attn_oracle.restype = ctypes.c_int
+            lib.decode_attn_oracle.argtypes = [
+                p, i64, i64, i64,            # q, B, Hq, D
+                p, p, i64, i64, i64,         # k_pages, v_pages, num_pages, Hkv, P
+                i64, i64, i64,               # strides (elements): page, head, token
+                p, i64, p,                   # block_table, max_pages, seq_lens
+                i32, ctypes.c_double,        # window, scale
+                p, p, i32,                   # out, lse, num_threads
+            ]
+            lib.decode_attn_oracle_max_threads.restype = ctypes.c_int
+            _lib = lib
+    return _lib
+
+
+def _bf16_bits(x) -> np.ndarray:
+    """View a bf16 tensor (torch CPU bfloat16, or numpy uint16 bit patterns) as uint16 bits."""
+    if isinstance(x, np.ndarray):
+        if x.dtype != np.uint16:
+            raise TypeError("numpy inputs must hold bf16 bit patterns as uint16")
+        return x
+    import torch  # only to reinterpret a CPU bf16 tensor's storage
+
+    if x.dtype != torch.bfloat16 or x.device.type != "cpu":
+        raise TypeError("expected a CPU torch.bfloat16 tensor")
+    return x.view(torch.int16).numpy().view(np.uint16)
+
+
+def max_threads() -> int:
+    return int(_load().decode_attn_oracle_max_threads())
+
+
+def decode_attn_oracle(q, k_pages, v_pages, block_table, seq_lens, window: int, scale: float,
+                       num_threads: int = 0):
+    """fp64 decode attention over a paged KV cache.
+
+    q            bf16 [B, Hq, D]
+    k_pages      bf16 [num_pages, Hkv, P, D] in any strides with a contiguous last dim
+    v_pages      same shape and strides as k_pages
+    block_table  int32 [B, max_pages]
+    seq_lens     int32 [B]
+    window       <= 0 for full attention, else the number of most recent tokens attended
+    scale        the float that multiplies q.k (taken at fp32 precision, as the C-ABI takes it)
+
+    Returns (out float64 [B, Hq, D], lse float64 [B, Hq]).
+    """
+    lib = _load()
+    qb = np.ascontiguousarray(_bf16_bits(q))
+    kb, vb = _bf16_bits(k_pages), _bf16_bits(v_pages)
+    if kb.shape != vb.shape or kb.strides != vb.strides:
+        raise ValueError("k_pages and v_pages must share shape and strides")
+    if kb.ndim != 4 or qb.ndim != 3:
+        raise ValueError("q must be [B,Hq,D] and k_pages [num_pages,Hkv,P,D]")
+    B, Hq, D = qb.shape
+    num_pages, Hkv, P, Dk = kb.shape
+    if Dk != D or kb.strides[3] != 2:
+        raise ValueError("head_dim mismatch or non-contiguous last dim")
+    bt = np.ascontiguousarray(np.asarray(block_table, dtype=np.int32))
+    sl = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32))
+    if bt.ndim != 2 or bt.shape[0] != B or sl.shape != (B,):
+        raise ValueError("block_table must be [B,max_pages] and seq_lens [B]")
+    out = np.empty((B, Hq, D), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    st = [s // 2 for s in kb.strides]
+    rc = lib.decode_attn_oracle(
+        qb.ctypes.data, B, Hq, D,
+        kb.ctypes.data, vb.ctypes.data, num_pages, Hkv, P,
+        st[0], st[1], st[2],
+        bt.ctypes.data, bt.shape[1], sl.ctypes.data,
+        int(window), float(np.float32(scale)),
+        out.ctypes.data, lse.ctypes.data, int(num_threads))
+    if rc != 0:
+        raise RuntimeError(f"decode_attn_oracle failed with code {rc}")
+    return out, lse

@@ -1,0 +1,176 @@
+/*
+ * decode_attn_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, fp64 CPU statement of grouped-query single-token ("decode")
+ * softmax attention over a paged bf16 KV cache.  It exists so that the CUDA
+ * library can be compared with something that is obviously the definition.
+ * Only the test-suite, the smoke check and the benchmark's CPU-baseline leg
+ * may load it; the product never does, and it shares no source, header, table
+ * or helper with the CUDA path.
+ *
+ * What it follows.  The paper's agent loop spends its run time in calls to a
+ * central LLM inference service (Sec. 3.2, "Large-scale runs"; Sec. 4 fixes a
+ * 131,072-token context, temperature 1.0 and up to 15 calls x 3 sessions per
+ * operator).  The paper gives no internals for that service; its only pointer
+ * to attention is the FlashAttention line of work cited under "Kernel
+ * Research" (Sec. 5).  Those works reach *exactly* softmax attention by
+ * re-associating it (tiling, online softmax, split-K with a log-sum-exp
+ * merge), so the oracle is the textbook definition written out, two passes,
+ * no tiling, no online rescaling, no splits:
+ *
+ *   for each sequence b with length L = seq_lens[b] (the current token's K/V
+ *   are already in the cache, so the query sits at position L-1):
+ *     lo = (window > 0 && window < L) ? L - window : 0
+ *     for each query head h, using KV head g = h / (Hq/Hkv):
+ *       s_t   = scale * sum_d q[b,h,d] * K[page(t), g, t % P, d]   t in [lo,L)
+ *       m     = max_t s_t
+ *       Z     = sum_t exp(s_t - m)
+ *       out   = sum_t (exp(s_t - m) / Z) * V[page(t), g, t % P, :]
+ *       lse   = m + log(Z)                       (natural log, scaled scores)
+ *     with page(t) = block_table[b][t / P].
+ *   L <= 0 gives out = 0 and lse = -inf.
+ *
+ * bf16 -> double conversion is exact (the 16 bits are the top half of an
+ * IEEE-754 binary32).  Sums run in a fixed order (d ascending, t ascending)
+ * so that results are reproducible bit for bit, whatever the thread count.
+ *
+ * Pins (tests/test_oracle_pins.py): one-token context, identical keys,
+ * scale 0, one dominant score, huge score offsets, page permutation, GQA head
+ * mapping, window identities, split/merge algebra, dense numpy brute force.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_bits_to_double(uint16_t bits)
+{
+    uint32_t u = ((uint32_t)bits) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Return codes. */
+enum { ORACLE_OK = 0, ORACLE_BAD_ARG = 1, ORACLE_BAD_PAGE = 2, ORACLE_NO_MEM = 3 };
+
+/*
+ * All pointers are HOST pointers; nothing is retained.
+ *   q            bf16 bits, [B, Hq, D] contiguous
+ *   k_pages,
+ *   v_pages      bf16 bits; element (page, g, r, d) lives at
+ *                page*stride_page + g*stride_head + r*stride_tok + d  (elements)
+ *   block_table  int32 [B, max_pages] contiguous; only entries with index
+ *                < ceil(L/P) are read
+ *   seq_lens     int32 [B]
+ *   window       <= 0: full attention; else the last `window` tokens
+ *   scale        multiplies q.k before the softmax
+ *   out          double [B, Hq, D] contiguous
+ *   lse          double [B, Hq]    contiguous (may be NULL)
+ *   num_threads  <= 0: let OpenMP decide
+ */
+int decode_attn_oracle(const uint16_t *q, int64_t B, int64_t Hq, int64_t D,
+                       const uint16_t *k_pages, const uint16_t *v_pages,
+                       int64_t num_pages, int64_t Hkv, int64_t P,
+                       int64_t stride_page, int64_t stride_head, int64_t stride_tok,
+                       const int32_t *block_table, int64_t max_pages,
+                       const int32_t *seq_lens, int32_t window, double scale,
+                       double *out, double *lse, int32_t num_threads)
+{
+    if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !out)
+        return ORACLE_BAD_ARG;
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || D <= 0 || P <= 0 || Hq % Hkv != 0 || num_pages < 0)
+        return ORACLE_BAD_ARG;
+
+    const int64_t G = Hq / Hkv; /* query heads per KV head; consecutive heads share one */
+    int status = ORACLE_OK;
+
+#ifdef _OPENMP
+    if (num_threads > 0)
+        omp_set_num_threads(num_threads);
+#else
+    (void)num_threads;
+#endif
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t bh = 0; bh < B * Hq; ++bh) {
+        const int64_t b = bh / Hq, h = bh % Hq, g = h / G;
+        double *o = out + bh * D;
+        const int64_t L = seq_lens[b];
+
+        for (int64_t d = 0; d < D; ++d)
+            o[d] = 0.0;
+        if (L <= 0) {
+            if (lse)
+                lse[bh] = -INFINITY;
+            continue;
+        }
+        if ((L + P - 1) / P > max_pages) {
+#pragma omp atomic write
+            status = ORACLE_BAD_ARG;
+            continue;
+        }
+        const int64_t lo = (window > 0 && (int64_t)window < L) ? L - window : 0;
+        const int64_t n = L - lo;
+        double *s = (double *)malloc((size_t)n * sizeof(double));
+        if (!s) {
+#pragma omp atomic write
+            status = ORACLE_NO_MEM;
+            continue;
+        }
+        const uint16_t *qv = q + bh * D;
+        int bad = 0;
+
+        /* pass 1: scores and their maximum */
+        double m = -INFINITY;
+        for (int64_t t = lo; t < L; ++t) {
+            const int64_t page = block_table[b * max_pages + t / P];
+            if (page < 0 || page >= num_pages) {
+                bad = 1;
+                break;
+            }
+            const uint16_t *kv = k_pages + page * stride_page + g * stride_head + (t % P) * stride_tok;
+            double acc = 0.0;
+            for (int64_t d = 0; d < D; ++d)
+                acc += bf16_bits_to_double(qv[d]) * bf16_bits_to_double(kv[d]);
+            s[t - lo] = scale * acc;
+            if (s[t - lo] > m)
+                m = s[t - lo];
+        }
+        if (bad) {
+#pragma omp atomic write
+            status = ORACLE_BAD_PAGE;
+            free(s);
+            continue;
+        }
+
+        /* pass 2: normaliser, then the weighted sum of V rows */
+        double Z = 0.0;
+        for (int64_t t = lo; t < L; ++t)
+            Z += exp(s[t - lo] - m);
+        for (int64_t t = lo; t < L; ++t) {
+            const int64_t page = block_table[b * max_pages + t / P];
+            const uint16_t *vv = v_pages + page * stride_page + g * stride_head + (t % P) * stride_tok;
+            const double w = exp(s[t - lo] - m) / Z;
+            for (int64_t d = 0; d < D; ++d)
+                o[d] += w * bf16_bits_to_double(vv[d]);
+        }
+        if (lse)
+            lse[bh] = m + log(Z);
+        free(s);
+    }
+    return status;
+}
+
+/* How many threads a call with num_threads <= 0 would use. */
+int decode_attn_oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

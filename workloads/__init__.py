@@ -1,0 +1,270 @@
+"""Seeded synthetic inputs for paged GQA decode attention.
+
+This module only *makes inputs* (lengths, block tables, random bf16 pools, NaN
+poison in the places that must never be read) and copies parts of them between
+devices.  It holds none of the attention arithmetic and is the one module that
+both the CUDA tests/benchmark and the CPU oracle's callers may import.
+
+The shapes stand in for long agent trajectories served by an LLM inference
+service (the paper, Sec. 3.2 and Sec. 4: hundreds of concurrent sessions that
+share one long initial prompt, contexts that grow by multi-thousand-token
+feedback prompts up to 131,072 tokens).  No dataset or benchmark item is
+involved: every value is drawn from a seeded generator.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+HQ, HKV, D = 48, 8, 128
+
+
+@dataclass
+class Case:
+    """One decode-attention problem.  Tensors live on ``device``."""
+    name: str
+    q: torch.Tensor            # bf16 [B, Hq, D]
+    k_pages: torch.Tensor      # bf16 [num_pages, Hkv, P, D] (logical shape; strides may differ)
+    v_pages: torch.Tensor      # bf16, same shape/strides as k_pages
+    block_table: torch.Tensor  # int32 [B, max_pages], unused entries = -1
+    seq_lens: torch.Tensor     # int32 [B]
+    window: int
+    scale: float
+    lens: np.ndarray = field(repr=False, default=None)  # host copy of seq_lens (int64)
+
+    @property
+    def B(self) -> int:
+        return self.q.shape[0]
+
+    @property
+    def P(self) -> int:
+        return self.k_pages.shape[2]
+
+    def attended_tokens(self) -> np.ndarray:
+        """Tokens each sequence attends (exact count, not rounded to pages)."""
+        L = self.lens.astype(np.int64)
+        w = self.window
+        n = np.where((w > 0) & (w < L), w, L)
+        return np.maximum(n, 0)
+
+    def algorithmic_bytes(self, out_itemsize: int = 4) -> int:
+        """Bytes the operation must move: attended K+V rows, block-table entries
+        touched, seq_len, q, out and lse.  Split-K partials are overhead and are
+        not counted."""
+        Hq, Dh = self.q.shape[1], self.q.shape[2]
+        Hkv = self.k_pages.shape[1]
+        n = self.attended_tokens()
+        L = np.maximum(self.lens.astype(np.int64), 0)
+        lo = L - n
+        P = self.P
+        pages_touched = np.where(n > 0, (L - 1) // P - lo // P + 1, 0)
+        per_seq = (n * (2 * Hkv * Dh * 2) + pages_touched * 4 + 4
+                   + Hq * Dh * 2 + Hq * Dh * out_itemsize + Hq * 4)
+        return int(per_seq.sum())
+
+
+def _randn_bf16(shape, gen: torch.Generator, device) -> torch.Tensor:
+    return torch.randn(shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+
+
+def build_case(name: str, lens: Sequence[int], P: int, seed: int, device="cpu", *,
+               Hq: int = HQ, Hkv: int = HKV, Dh: int = D, window: int = 0,
+               scale: Optional[float] = None, shuffle: bool = True,
+               pool_pages: Optional[int] = None, shared_prefix_tokens: int = 0,
+               layout: str = "head_major", poison: bool = True,
+               pad_table_to: Optional[int] = None, fill_chunk_pages: int = 16384) -> Case:
+    """Build one problem.
+
+    lens                  context length of each sequence (current token included)
+    shuffle               physical page ids are a random permutation of the pool
+                          (False: sequence pages laid out contiguously in order)
+    pool_pages            size of the physical pool (default: exactly the pages
+                          referenced); extra pages are NaN-filled
+    shared_prefix_tokens  the first this-many tokens of every sequence use the
+                          SAME physical pages (must be a multiple of P)
+    layout                "head_major": memory order [page, kv_head, token, d];
+                          "token_major": memory order [page, token, kv_head, d]
+                          (same logical shape, different strides)
+    poison                NaN in page tails past each sequence's end, in unused
+                          pool pages; block-table padding is -1 either way
+    """
+    rng = np.random.default_rng(seed)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    lens = np.asarray(lens, dtype=np.int64)
+    B = len(lens)
+    if shared_prefix_tokens % P:
+        raise ValueError("shared prefix must be whole pages")
+    pre_pages = shared_prefix_tokens // P
+    npg = np.maximum((lens + P - 1) // P, 0)
+    if pre_pages and (lens < shared_prefix_tokens).any():
+        raise ValueError("every sequence must contain the shared prefix")
+    own = npg - pre_pages if pre_pages else npg
+    referenced = int(own.sum()) + pre_pages
+    pool = referenced if pool_pages is None else int(pool_pages)
+    if pool < referenced:
+        raise ValueError("pool smaller than the pages referenced")
+    pool = max(pool, 1)
+    ids = rng.permutation(pool)[:referenced] if shuffle else np.arange(referenced)
+    max_pages = int(max(int(npg.max()) if B else 1, 1))
+    if pad_table_to is not None:
+        max_pages = max(max_pages, int(pad_table_to))
+    bt = np.full((B, max_pages), -1, dtype=np.int32)
+    cursor = pre_pages
+    for b in range(B):
+        if pre_pages:
+            bt[b, :pre_pages] = ids[:pre_pages]
+        k = int(own[b])
+        bt[b, pre_pages:pre_pages + k] = ids[cursor:cursor + k]
+        cursor += k
+
+    if layout == "head_major":
+        phys = (pool, Hkv, P, Dh)
+        to_logical = lambda t: t
+    elif layout == "token_major":
+        phys = (pool, P, Hkv, Dh)
+        to_logical = lambda t: t.permute(0, 2, 1, 3)
+    else:
+        raise ValueError(layout)
+
+    nan = float("nan")
+    pools = []
+    for _ in range(2):
+        if poison and pool > referenced:
+            t = torch.full(phys, nan, dtype=torch.bfloat16, device=device)
+        else:
+            t = torch.empty(phys, dtype=torch.bfloat16, device=device)
+        ids_t = torch.from_numpy(np.ascontiguousarray(ids)).to(device)
+        for s in range(0, referenced, fill_chunk_pages):
+            sel = ids_t[s:s + fill_chunk_pages]
+            t[sel] = _randn_bf16((len(sel),) + phys[1:], gen, device)
+        pools.append(t)
+    k_pages, v_pages = (to_logical(t) for t in pools)
+
+    if poison:
+        # rows past a sequence's end inside its last page must never be read
+        for b in range(B):
+            L = int(lens[b])
+            if L > 0 and L % P and not (pre_pages and L <= shared_prefix_tokens):
+                page = int(bt[b, (L - 1) // P])
+                k_pages[page, :, L % P:, :] = nan
+                v_pages[page, :, L % P:, :] = nan
+
+    q = _randn_bf16((B, Hq, Dh), gen, device)
+    return Case(
+        name=name, q=q, k_pages=k_pages, v_pages=v_pages,
+        block_table=torch.from_numpy(bt).to(device),
+        seq_lens=torch.from_numpy(lens.astype(np.int32)).to(device),
+        window=int(window), scale=float(scale if scale is not None else 1.0 / math.sqrt(Dh)),
+        lens=lens.copy())
+
+
+# ----------------------------------------------------------------------------
+# The five workload recipes.
+# ----------------------------------------------------------------------------
+
+def lengths_c2(seed: int = 1, B: int = 64) -> np.ndarray:
+    return np.random.default_rng(seed).integers(1024, 16385, size=B)
+
+
+def lengths_c3(seed: int = 2, B: int = 256) -> np.ndarray:
+    u = np.random.default_rng(seed).uniform(math.log(512.0), math.log(32768.0), size=B)
+    return np.clip(np.floor(np.exp(u)).astype(np.int64), 512, 32768)
+
+
+def lengths_c5(seed: int = 4, B: int = 128, prefix: int = 16384, max_suffix: int = 8192) -> np.ndarray:
+    return prefix + np.random.default_rng(seed).integers(0, max_suffix + 1, size=B)
+
+
+def c1(device="cpu") -> Case:
+    """1 sequence x 512 tokens, page 16, contiguous block table, seed 0, and three
+    key rows multiplied by 20 (all KV heads) to stress softmax stability."""
+    case = build_case("c1", [512], 16, 0, device, shuffle=False)
+    hot = np.random.default_rng(0).choice(512, size=3, replace=False)
+    for t in hot:
+        page = int(case.block_table[0, t // 16])
+        row = case.k_pages[page, :, t % 16, :].float() * 20.0
+        case.k_pages[page, :, t % 16, :] = row.to(torch.bfloat16)
+    return case
+
+
+def c2(device="cpu", B: int = 64) -> Case:
+    """64 sequences, lengths uniform in [1024, 16384], page 16, block tables dealt
+    from one random permutation of an exact-size pool, seed 1."""
+    return build_case("c2", lengths_c2(1, B), 16, 1, device)
+
+
+def c3(device="cpu", B: int = 256, pool_bytes: float = 20e9) -> Case:
+    """256 sequences, lengths log-uniform in [512, 32768], page 16, referenced pages
+    scattered through a ~20 GB pool (K + V) whose other pages are NaN, seed 2."""
+    lens = lengths_c3(2, B)
+    page_bytes = 2 * HKV * 16 * D * 2
+    referenced = int(((lens + 15) // 16).sum())
+    pool = max(int(pool_bytes // page_bytes), referenced)
+    return build_case("c3", lens, 16, 2, device, pool_pages=pool)
+
+
+def c4(device="cpu", B: int = 8, L: int = 131072) -> Case:
+    """8 sequences x 131,072 tokens, page 64, shuffled pool, seed 3."""
+    return build_case("c4", [L] * B, 64, 3, device)
+
+
+def c5(device="cpu", window: int = 0, B: int = 128) -> Case:
+    """128 sequences sharing a 16,384-token prefix (same physical pages in every
+    block table) plus unique suffixes uniform in [0, 8192], page 16, seed 4;
+    window = 0 (full) or 8192."""
+    return build_case("c5b" if window else "c5a", lengths_c5(4, B), 16, 4, device,
+                      shared_prefix_tokens=16384, window=window)
+
+
+RECIPES = {"c1": c1, "c2": c2, "c3": c3, "c4": c4,
+           "c5a": lambda device="cpu": c5(device, 0),
+           "c5b": lambda device="cpu": c5(device, 8192)}
+
+
+# ----------------------------------------------------------------------------
+# Moving parts of a case to the host (for the CPU oracle's callers).
+# ----------------------------------------------------------------------------
+
+def host_subcase(case: Case, seq_ids: Sequence[int]) -> Case:
+    """A CPU copy of the chosen sequences only: their pages are gathered into a
+    compact head-major pool and the block table is renumbered to match.  Pure
+    copying; values are untouched."""
+    seq_ids = list(seq_ids)
+    P = case.P
+    lens = case.lens[seq_ids]
+    npg = np.maximum((lens + P - 1) // P, 0)
+    bt_host = case.block_table[seq_ids].cpu().numpy()
+    used = np.unique(np.concatenate([bt_host[i, :npg[i]] for i in range(len(seq_ids))]
+                                    + [np.zeros(0, np.int32)]))
+    remap = {int(p): i for i, p in enumerate(used)}
+    new_bt = np.full_like(bt_host, -1)
+    for i in range(len(seq_ids)):
+        new_bt[i, :npg[i]] = [remap[int(p)] for p in bt_host[i, :npg[i]]]
+    sel = torch.from_numpy(used.astype(np.int64)).to(case.k_pages.device)
+    if len(used) == 0:
+        sel = torch.zeros(1, dtype=torch.int64, device=case.k_pages.device)
+    k = case.k_pages.index_select(0, sel).contiguous().cpu()
+    v = case.v_pages.index_select(0, sel).contiguous().cpu()
+    return Case(name=case.name + "/sub", q=case.q[seq_ids].cpu(), k_pages=k, v_pages=v,
+                block_table=torch.from_numpy(new_bt), seq_lens=torch.from_numpy(lens.astype(np.int32)),
+                window=case.window, scale=case.scale, lens=lens.copy())
+
+
+def to_device(case: Case, device) -> Case:
+    """Copy a case to another device, keeping the pools' strides."""
+    def mv(t):
+        if t.is_contiguous():
+            return t.to(device)
+        # keep memory order: move the underlying dense buffer, then re-view
+        order = sorted(range(t.dim()), key=lambda i: -t.stride(i))
+        dense = t.permute(order).contiguous().to(device)
+        inv = [order.index(i) for i in range(t.dim())]
+        return dense.permute(inv)
+    return Case(name=case.name, q=case.q.to(device), k_pages=mv(case.k_pages), v_pages=mv(case.v_pages),
+                block_table=case.block_table.to(device), seq_lens=case.seq_lens.to(device),
+                window=case.window, scale=case.scale, lens=case.lens.copy())
