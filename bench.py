@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the paged GQA decode-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5a|c5b] [--impl ours|reference]
+
+A step is one decode_attn call (plan + partition + merge kernels) over one synthetic batch whose
+KV cache is resident in HBM.  Rank 0 prints ONE JSON line.  The metric is KV-cache GB/s: the
+algorithmic bytes of the call (attended K+V rows, block-table entries touched, seq_lens, q, out,
+lse) divided by the CUDA-event time.  With N > 1 (torchrun, one rank per GPU) every rank runs an
+independent replica of the workload -- the path has no exchange step -- and the value is the sum
+of the replicas' bytes over the slowest rank's time.
+
+--impl reference times the fp64 CPU oracle, as it stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "decode-attn KV-cache GB/s (fraction of 8 TB/s HBM); sequences/s per layer"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+WORKLOAD_TEXT = {
+    "c1": "c1: 1 seq x 512 tok, page 16, contiguous, seed 0, 3 keys x20",
+    "c2": "c2: 64 seqs, len U[1024,16384], 48q/8kv heads, d128, page 16, permuted pool, seed 1",
+    "c3": "c3: 256 seqs, len log-uniform [512,32768], page 16, pages scattered in a ~20 GB pool, seed 2",
+    "c4": "c4: 8 seqs x 131072 tok, page 64, seed 3",
+    "c5a": "c5a: 128 seqs, 16384-token shared prefix + U[0,8192] suffix, page 16, full attention, seed 4",
+    "c5b": "c5b: same as c5a with a sliding window of 8192",
+}
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def reduce_over_ranks(value: float, op: str, device) -> float:
+    """max / sum of a scalar over all ranks (identity when not distributed)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX if op == "max" else dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def aggregate_replicas(bytes_per_step: float, seqs_per_step: float, ms_per_step: float, device):
+    """Whole-job numbers for independent replicas: units add up, time is the slowest rank's."""
+    ms = reduce_over_ranks(ms_per_step, "max", device)
+    total_bytes = reduce_over_ranks(bytes_per_step, "sum", device)
+    total_seqs = reduce_over_ranks(seqs_per_step, "sum", device)
+    return total_bytes / (ms * 1e-3) / 1e9, total_seqs / (ms * 1e-3), ms
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi samples of SM clock and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            text = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in text.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(case, every: int):
+    """Time the CPU oracle, as it stands, on every `every`-th sequence of the workload."""
+    import oracle
+    ids = list(range(0, case.B, every))
+    sub = workloads.host_subcase(case, ids)
+    threads = oracle.max_threads()
+    t0 = time.perf_counter()
+    oracle.decode_attn_oracle(sub.q, sub.k_pages, sub.v_pages, sub.block_table, sub.seq_lens,
+                              sub.window, sub.scale, 0)
+    dt = time.perf_counter() - t0
+    nbytes = sub.algorithmic_bytes(4)
+    return {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "sample": f"every {every}th sequence of {case.name} ({len(ids)} of {case.B} sequences, "
+                      f"{int(sub.attended_tokens().sum())} attended tokens, {dt:.2f} s wall)",
+            "seconds": dt, "seq_per_s": len(ids) / dt}
+
+
+# ----------------------------------------------------------------------------- reference arm
+
+def run_reference(args):
+    rank, world, local = dist_env()
+    if rank != 0:
+        return 0
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    case = workloads.RECIPES[args.workload](dev)
+    every = max(args.ref_every, 1)
+    for _ in range(args.warmup if args.warmup < 2 else 1):
+        oracle_sample(case, every * 4)
+    res = [oracle_sample(case, every) for _ in range(max(1, min(args.steps, 3)))]
+    best = max(res, key=lambda r: r["value"])
+    ms = statistics.mean(r["seconds"] for r in res) * 1e3
+    line = {
+        "impl": "reference", "metric": METRIC, "value": best["value"], "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": len(res), "warmup": 1, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.workload], "sample": best["sample"]},
+        "seq_per_s": best["seq_per_s"], "frac_of_8TBs": best["value"] / NOMINAL_HBM_GBS,
+        "cpu_baseline": {k: best[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": best["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import paper_2512_10977_b200 as da   # raises if the CUDA library is missing
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    case = workloads.RECIPES[args.workload](device)
+    out = torch.empty(case.q.shape, dtype=torch.float32, device=device)
+    lse = torch.empty(case.q.shape[:2], dtype=torch.float32, device=device)
+    nbytes = case.algorithmic_bytes(4)
+    stream = torch.cuda.current_stream()
+    lib = da.lib()
+
+    def step():
+        da.decode_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
+                       case.window, case.scale, out=out, lse=lse, stream=stream)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    assert da.read_device_status() == (0, 0, 0, 0)
+
+    # ---- device-resident timing: K steps, events on the launching stream
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    K = args.steps
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    stops = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    kev0 = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    kev1 = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    for e in kev0 + kev1:     # materialise the handles
+        e.record(stream)
+    barrier()
+    launches0 = da.launch_count()
+    t_all0 = torch.cuda.Event(enable_timing=True)
+    t_all1 = torch.cuda.Event(enable_timing=True)
+    t_all0.record(stream)
+    for i in range(K):
+        starts[i].record(stream)
+        step()
+        stops[i].record(stream)
+    t_all1.record(stream)
+    barrier()
+    launches = da.launch_count() - launches0
+    ms_total = t_all0.elapsed_time(t_all1)
+    per_step = [a.elapsed_time(b) for a, b in zip(starts, stops)]
+    ms_per_step = ms_total / K
+
+    # ---- the partition kernel alone (the dominant kernel), bracketed inside the library
+    kernel_ms = None
+    if hasattr(lib, "decode_attn_set_profile_events"):
+        import ctypes
+        lib.decode_attn_set_profile_events.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+        durs = []
+        for i in range(K):
+            lib.decode_attn_set_profile_events(kev0[i].cuda_event, kev1[i].cuda_event)
+            step()
+        lib.decode_attn_set_profile_events(None, None)
+        torch.cuda.synchronize()
+        durs = [a.elapsed_time(b) for a, b in zip(kev0, kev1)]
+        kernel_ms = statistics.mean(durs)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end: per-step inputs from pinned host memory, result read back to the host
+    q_h, bt_h, sl_h = (t.cpu().pin_memory() for t in (case.q, case.block_table, case.seq_lens))
+    out_h = torch.empty(case.q.shape, dtype=torch.float32).pin_memory()
+    lse_h = torch.empty(case.q.shape[:2], dtype=torch.float32).pin_memory()
+    h2d = q_h.numel() * 2 + bt_h.numel() * 4 + sl_h.numel() * 4
+    d2h = out_h.numel() * 4 + lse_h.numel() * 4
+
+    def e2e_step():
+        da.decode_attn_host_io(q_h, case.k_pages, case.v_pages, bt_h, sl_h, case.window, case.scale,
+                               out_h, lse_h, stream=stream)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(K):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / K
+    assert torch.equal(out_h, out.cpu()), "host-io result differs from the device-resident call"
+
+    gbs, seqs, ms = aggregate_replicas(nbytes, case.B, ms_per_step, device)
+    e2e_gbs, _, e2e_ms_max = aggregate_replicas(nbytes, case.B, e2e_ms, device)
+
+    if rank != 0:
+        return 0
+    peak, peak_src = measured_peak()
+    kms = kernel_ms if kernel_ms is not None else ms_per_step
+    achieved = nbytes / (kms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.workload], "sequences": case.B,
+                   "attended_tokens": int(case.attended_tokens().sum()), "algorithmic_bytes": nbytes,
+                   "l2": "inputs exceed L2 (no flush)" if nbytes > 4 * 126e6 else "inputs fit L2; not flushed",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "grid_blocks": da.get_option("grid_blocks")},
+        "frac_of_8TBs": gbs / world / NOMINAL_HBM_GBS, "seq_per_s": seqs,
+        "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
+        "roofline": {"bound": "hbm", "kernel": "partition_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                     "kernel_ms": kms, "traffic": None},
+        "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms_max,
+                "note": "q, block_table, seq_lens from pinned host memory and out, lse back to it every step; "
+                        "the KV cache is resident state"},
+        "gpu_launches": launches, "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = {k: v for k, v in oracle_sample(case, args.ref_every).items()
+                                if k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOAD_TEXT))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-every", type=int, default=2, help="oracle sample: every n-th sequence")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    return run_reference(args) if args.impl == "reference" else run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,184 @@
+/*
+ * decode_attn.h -- C ABI of the B200 (sm_100a) paged GQA decode-attention library.
+ *
+ * The operation.  For every sequence b of a batch and every query head h, one
+ * query vector (the token being decoded) attends over that sequence's cached
+ * keys and values, which live in fixed-size pages addressed through a block
+ * table:
+ *
+ *     L  = seq_lens[b]            (the current token's K/V are already cached)
+ *     lo = (window > 0 && window < L) ? L - window : 0
+ *     g  = h / (Hq / Hkv)         (consecutive query heads share one KV head)
+ *     s_t = scale * <q[b,h,:], K[block_table[b][t/P], g, t%P, :]>     lo <= t < L
+ *     out[b,h,:] = sum_t softmax(s)_t * V[block_table[b][t/P], g, t%P, :]
+ *     lse[b,h]   = ln sum_t exp(s_t)
+ *     L <= 0:  out = 0, lse = -inf.
+ *
+ * Where it comes from.  The paper's agent loop is bound by calls to a central
+ * LLM inference service (Sec. 3.2, last paragraph of "Large-scale runs"; Sec. 4
+ * sets a 131,072-token context, up to 15 calls x 3 sessions per operator,
+ * hundreds of sessions at once).  Per generated token and layer that service
+ * runs exactly this step.  The paper gives no internals for it; its pointer to
+ * the computation is the FlashAttention line of work cited in Sec. 5 ("Kernel
+ * Research"), which evaluates softmax attention exactly by tiling, online
+ * softmax and split-K with a log-sum-exp merge.  Those three are the stages
+ * behind decode_attn(): a plan kernel (split schedule), a partition kernel
+ * (page gather by TMA, QK^T, online fp32 softmax, PV on tensor cores) and a
+ * merge kernel (log-sum-exp combine).
+ *
+ * Conventions.  Every function returns a da_status (0 = ok) and never throws,
+ * aborts or synchronises unless it says so.  Pointers inside da_tensor are
+ * DEVICE pointers unless a function says HOST.  The library owns no memory:
+ * scratch comes from the caller through decode_attn_set_workspace().  Work is
+ * enqueued on the given CUDA stream and the call returns at once.  Arguments a
+ * host can check (NULL, dtype, shape, stride, alignment, workspace size) are
+ * rejected before anything is launched.  Errors that depend on device data (a
+ * page id outside the pool, a sequence longer than its block-table row) are
+ * found on the device: the offending access is skipped or clamped (never a
+ * trap, never an unbounded wait), a status word is set, and
+ * decode_attn_read_device_status() returns it.
+ */
+#ifndef DECODE_ATTN_H_
+#define DECODE_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DA_OK = 0,
+    DA_ERR_NULL = 1,         /* a required pointer is NULL                              */
+    DA_ERR_SHAPE = 2,        /* ranks or extents disagree                               */
+    DA_ERR_DTYPE = 3,        /* wrong element type                                      */
+    DA_ERR_STRIDE_ALIGN = 4, /* last dim not contiguous, or a stride/base not 16-B aligned */
+    DA_ERR_UNSUPPORTED = 5,  /* head_dim != 128, page size not in {16,32,64,128}, group > 16 */
+    DA_ERR_WORKSPACE = 6,    /* no workspace registered for this device, or too small   */
+    DA_ERR_CUDA = 7          /* a CUDA call failed; see decode_attn_last_cuda_error()   */
+} da_status;
+
+typedef enum { DA_BF16 = 1, DA_F32 = 2, DA_I32 = 3 } da_dtype;
+
+/* Device-side status codes (first word of the status record). */
+typedef enum {
+    DA_DEV_OK = 0,
+    DA_DEV_BAD_PAGE = 1,   /* block-table entry outside [0, num_pages); that load was skipped */
+    DA_DEV_BAD_SEQLEN = 2, /* seq_len < 0 or > max_pages * P; the sequence was treated as empty */
+    DA_DEV_TIMEOUT = 3     /* a bounded wait inside a kernel ran out; results are invalid  */
+} da_dev_status;
+
+/* A strided view.  `stride` is in ELEMENTS.  Nothing is owned. */
+typedef struct da_tensor {
+    void *data;
+    int32_t dtype; /* da_dtype */
+    int32_t ndim;
+    int64_t shape[4];
+    int64_t stride[4];
+} da_tensor;
+
+/*
+ * decode_attn -- the whole hot path (plan, partition, merge) on `stream`.
+ *
+ *   q            bf16 [B, Hq, D]          D = 128, last dim contiguous, rows 4-B aligned
+ *   k_pages      bf16 [num_pages, Hkv, P, D]   any strides with a contiguous last dim; base and
+ *                                         every stride a multiple of 16 bytes (so both
+ *                                         [page][head][token][d] and [page][token][head][d]
+ *                                         memory orders are accepted); P in {16, 32, 64, 128}
+ *   v_pages      same shape and rules as k_pages (a separate pool; strides may differ)
+ *   block_table  i32 [B, max_pages], last dim contiguous; entry i of row b is the physical page
+ *                holding tokens [i*P, (i+1)*P) of sequence b; entries at index >= ceil(L/P) are
+ *                never read
+ *   seq_lens     i32 [B]; includes the token being decoded
+ *   window       <= 0: attend everything; else attend the last `window` tokens, the current one
+ *                included (window >= L is the same as 0)
+ *   scale        multiplies q.k before the softmax
+ *   out          f32 or bf16 [B, Hq, D], last dim contiguous
+ *   lse          f32 [B, Hq] (natural log of the sum of exp of the scaled scores); may be NULL
+ *   stream       cudaStream_t (NULL = the legacy default stream)
+ *
+ * Rows of K/V past a sequence's end inside its last page, pages that no block table references
+ * and block-table padding may hold anything (NaN included); they do not reach the result.
+ * Hq % Hkv == 0 and Hq / Hkv <= 16 are required.  The registered workspace is read and written:
+ * two calls that share it must not overlap on the GPU (use one stream, or order them).
+ */
+int decode_attn(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                const da_tensor *block_table, const da_tensor *seq_lens, int32_t window, float scale,
+                da_tensor *out, da_tensor *lse, void *stream);
+
+/*
+ * decode_attn_host_io -- the same call for a caller whose per-step tensors are in HOST memory.
+ * q, block_table, seq_lens, out and lse are HOST views (pinned memory makes the copies
+ * asynchronous; they must stay valid until the stream reaches the end of the call); k_pages and
+ * v_pages stay DEVICE views (the cache is resident state).  The inputs are staged into the
+ * registered workspace with cudaMemcpyAsync, decode_attn() runs on the staged copies, and out/lse
+ * are copied back, all on `stream`, without synchronising.  Host views must be contiguous.
+ */
+int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tensor *v_pages,
+                        const da_tensor *block_table_host, const da_tensor *seq_lens_host,
+                        int32_t window, float scale, da_tensor *out_host, da_tensor *lse_host,
+                        void *stream);
+
+/*
+ * Scratch.  decode_attn_workspace_bytes() says how much device memory a call with these extents
+ * needs on the current device with the current launch options (split partials, the plan, a status
+ * record, and staging room for decode_attn_host_io).  decode_attn_set_workspace() registers a
+ * caller-owned, 256-B aligned device buffer for the current device (one per device, process-wide)
+ * and clears its status record with a cudaMemsetAsync on the legacy default stream followed by a
+ * synchronize.  Passing NULL unregisters.
+ */
+size_t decode_attn_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t P,
+                                   int64_t max_pages);
+int decode_attn_set_workspace(void *dev_ptr, size_t bytes);
+
+/*
+ * decode_attn_read_device_status -- synchronises `stream`, copies the 4-word status record
+ * {da_dev_status code, sequence index, block-table index, page id or length} of the current
+ * device's workspace to HOST memory and clears it on the device.  All zero = clean.
+ */
+int decode_attn_read_device_status(void *stream, int32_t *host_status4);
+
+/*
+ * decode_attn_plan -- runs only the plan kernel (the split schedule of the partition kernel) and
+ * copies it to HOST arrays, synchronising `stream`.  A debugging and test aid: it shows which
+ * token ranges each thread block will cover.
+ *   seq_lens        DEVICE i32 [B] view
+ *   host_seq_info   HOST int32 [B][4]: {lo, L, first_tile, num_tiles}; a tile is tile_tokens
+ *                   consecutive tokens starting at a multiple of tile_tokens
+ *   host_block_work HOST int32 [*num_blocks][4]: {b, kv_head, first tile of that pair relative to
+ *                   its first_tile, number of tiles}; a block walks forward from there through
+ *                   (b, kv_head) pairs in row-major order
+ *   num_blocks      HOST in: capacity of host_block_work in rows; out: the grid size
+ *   tile_tokens     HOST out
+ */
+int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int32_t P,
+                     int64_t max_pages, int32_t *host_seq_info, int32_t *host_block_work,
+                     int32_t *num_blocks, int32_t *tile_tokens, void *stream);
+
+/*
+ * Launch options, for tests and tuning.  Names: "grid_blocks" (thread blocks of the partition
+ * kernel; 0 = two per SM; every value gives the same result up to fp32 rounding and changes how
+ * sequences are split).  Returns DA_ERR_UNSUPPORTED for an unknown name or a value out of range.
+ */
+int decode_attn_set_option(const char *name, int64_t value);
+int64_t decode_attn_get_option(const char *name);
+
+/*
+ * decode_attn_set_profile_events -- timing aid.  While both handles are non-NULL, every
+ * decode_attn() call records `before` (a cudaEvent_t) on its stream just before the partition
+ * kernel's launch and `after` just after it, so that a benchmark can time that kernel alone.
+ * Pass NULL, NULL to stop.  The events stay owned by the caller.
+ */
+int decode_attn_set_profile_events(void *before, void *after);
+
+const char *decode_attn_strerror(int status);
+int decode_attn_last_cuda_error(void); /* cudaError_t of the last failing CUDA call, else 0 */
+int decode_attn_version(void);
+/* Kernel launches issued by this library since load (a counter for benchmarks). */
+int64_t decode_attn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DECODE_ATTN_H_ */

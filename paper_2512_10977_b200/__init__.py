@@ -1,0 +1,12 @@
+"""B200 (sm_100a) paged GQA decode attention: a C-ABI CUDA library and its thin Python binding.
+
+``decode_attn`` and friends marshal torch tensors (device memory and streams only) into the
+``extern "C"`` calls of ``include/decode_attn.h``; every step of the computation runs in the
+library's own kernels.  There is no CPU or PyTorch fallback: if the library is missing or no
+CUDA device is present, the calls raise.
+"""
+from .binding import (DecodeAttnError, decode_attn, decode_attn_host_io, ensure_workspace, get_option,
+                      launch_count, lib, plan, read_device_status, set_option, version, workspace_bytes)
+
+__all__ = ["DecodeAttnError", "decode_attn", "decode_attn_host_io", "ensure_workspace", "get_option",
+           "launch_count", "lib", "plan", "read_device_status", "set_option", "version", "workspace_bytes"]

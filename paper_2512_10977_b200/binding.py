@@ -1,0 +1,210 @@
+"""ctypes binding of include/decode_attn.h.  Argument marshalling only.
+
+torch is used for device buffers and streams; nothing here computes.  The shared library is
+loaded from this directory (built in-tree by ``build.py``); if it is missing, or a call is made
+without a CUDA device, an exception is raised -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libdecode_attn.so")
+_lock = threading.Lock()
+_lib = None
+_workspaces = {}   # device index -> torch uint8 tensor kept alive while registered
+
+DA_BF16, DA_F32, DA_I32 = 1, 2, 3
+_DTYPES = {torch.bfloat16: DA_BF16, torch.float32: DA_F32, torch.int32: DA_I32}
+
+
+class DecodeAttnError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"decode_attn status {status}: {what}")
+        self.status = status
+
+
+class DaTensor(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("ndim", ctypes.c_int32),
+                ("shape", ctypes.c_int64 * 4), ("stride", ctypes.c_int64 * 4)]
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library (raises if it has not been built)."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(_LIB_PATH):
+                raise FileNotFoundError(
+                    f"{_LIB_PATH} is missing: build it with `python -m paper_2512_10977_b200.build`")
+            L = ctypes.CDLL(_LIB_PATH)
+            T = ctypes.POINTER(DaTensor)
+            vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+            L.decode_attn.restype = ctypes.c_int
+            L.decode_attn.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_host_io.restype = ctypes.c_int
+            L.decode_attn_host_io.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_workspace_bytes.restype = ctypes.c_size_t
+            L.decode_attn_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i64]
+            L.decode_attn_set_workspace.restype = ctypes.c_int
+            L.decode_attn_set_workspace.argtypes = [vp, ctypes.c_size_t]
+            L.decode_attn_read_device_status.restype = ctypes.c_int
+            L.decode_attn_read_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+            L.decode_attn_plan.restype = ctypes.c_int
+            L.decode_attn_plan.argtypes = [T, i32, i32, i32, i64, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                           ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
+            L.decode_attn_set_option.restype = ctypes.c_int
+            L.decode_attn_set_option.argtypes = [ctypes.c_char_p, i64]
+            L.decode_attn_get_option.restype = i64
+            L.decode_attn_get_option.argtypes = [ctypes.c_char_p]
+            L.decode_attn_strerror.restype = ctypes.c_char_p
+            L.decode_attn_strerror.argtypes = [ctypes.c_int]
+            L.decode_attn_last_cuda_error.restype = ctypes.c_int
+            L.decode_attn_version.restype = ctypes.c_int
+            L.decode_attn_launch_count.restype = i64
+            _lib = L
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        L = lib()
+        msg = L.decode_attn_strerror(rc).decode()
+        if rc == 7:
+            msg += f" [cudaError {L.decode_attn_last_cuda_error()}]"
+        raise DecodeAttnError(rc, msg)
+
+
+def _view(t: Optional[torch.Tensor]) -> Optional[DaTensor]:
+    if t is None:
+        return None
+    if t.dtype not in _DTYPES:
+        raise TypeError(f"unsupported dtype {t.dtype}")
+    if t.dim() > 4:
+        raise ValueError("at most 4 dimensions")
+    d = DaTensor()
+    d.data = t.data_ptr()
+    d.dtype = _DTYPES[t.dtype]
+    d.ndim = t.dim()
+    for i in range(t.dim()):
+        d.shape[i] = t.shape[i]
+        d.stride[i] = t.stride(i)
+    return d
+
+
+def _ref(d: Optional[DaTensor]):
+    return ctypes.byref(d) if d is not None else None
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    if not torch.cuda.is_available():
+        raise RuntimeError("decode_attn needs a CUDA device; there is no CPU path")
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def version() -> int:
+    return lib().decode_attn_version()
+
+
+def launch_count() -> int:
+    return int(lib().decode_attn_launch_count())
+
+
+def set_option(name: str, value: int) -> None:
+    _check(lib().decode_attn_set_option(name.encode(), int(value)))
+
+
+def get_option(name: str) -> int:
+    return int(lib().decode_attn_get_option(name.encode()))
+
+
+def workspace_bytes(B: int, Hq: int, Hkv: int, D: int, P: int, max_pages: int) -> int:
+    return int(lib().decode_attn_workspace_bytes(B, Hq, Hkv, D, P, max_pages))
+
+
+def ensure_workspace(B: int, Hq: int, Hkv: int, D: int, P: int, max_pages: int,
+                     device: Optional[torch.device] = None) -> torch.Tensor:
+    """Make sure the current device has a registered workspace large enough for these extents.
+    The buffer is a torch allocation owned here; the library only borrows the pointer."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    with torch.cuda.device(dev):
+        need = workspace_bytes(B, Hq, Hkv, D, P, max_pages)
+        cur = _workspaces.get(dev.index)
+        if cur is None or cur.numel() < need:
+            torch.cuda.synchronize()
+            buf = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+            _check(lib().decode_attn_set_workspace(buf.data_ptr(), buf.numel()))
+            _workspaces[dev.index] = buf
+        return _workspaces[dev.index]
+
+
+def _auto_workspace(q, k_pages, block_table):
+    ensure_workspace(q.shape[0], q.shape[1], k_pages.shape[1], q.shape[2], k_pages.shape[2],
+                     block_table.shape[1], k_pages.device)
+
+
+def decode_attn(q, k_pages, v_pages, block_table, seq_lens, window: int, scale: float,
+                out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                stream: Optional[torch.cuda.Stream] = None, out_dtype=torch.float32, want_lse: bool = True):
+    """GQA decode attention over a paged bf16 KV cache (see include/decode_attn.h for the contract).
+
+    Allocates ``out`` / ``lse`` with torch when not given, registers a workspace on first use and
+    enqueues the library call on ``stream`` (default: torch's current stream).  Returns (out, lse).
+    """
+    if out is None:
+        out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+    with torch.cuda.device(k_pages.device):
+        _auto_workspace(q, k_pages, block_table)
+        tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
+        _check(lib().decode_attn(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
+                                 int(window), float(scale), _ref(tv[5]), _ref(tv[6]), _stream_ptr(stream)))
+    return out, lse
+
+
+def decode_attn_host_io(q_host, k_pages, v_pages, block_table_host, seq_lens_host, window: int, scale: float,
+                        out_host, lse_host=None, stream: Optional[torch.cuda.Stream] = None):
+    """Same call with q / block_table / seq_lens / out / lse in (pinned) HOST memory; the KV pools
+    stay on the device.  Copies and kernels are enqueued on ``stream``; nothing synchronises."""
+    with torch.cuda.device(k_pages.device):
+        _auto_workspace(q_host, k_pages, block_table_host)
+        tv = [_view(t) for t in (q_host, k_pages, v_pages, block_table_host, seq_lens_host, out_host, lse_host)]
+        _check(lib().decode_attn_host_io(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
+                                         int(window), float(scale), _ref(tv[5]), _ref(tv[6]),
+                                         _stream_ptr(stream)))
+    return out_host, lse_host
+
+
+def read_device_status(stream: Optional[torch.cuda.Stream] = None):
+    """Synchronise and return the device status record as a 4-tuple; (0, 0, 0, 0) is clean."""
+    buf = (ctypes.c_int32 * 4)()
+    _check(lib().decode_attn_read_device_status(_stream_ptr(stream), buf))
+    return tuple(int(x) for x in buf)
+
+
+def plan(seq_lens: torch.Tensor, window: int, Hkv: int, P: int, max_pages: int,
+         stream: Optional[torch.cuda.Stream] = None):
+    """Run only the plan kernel; returns (seq_info [B,4], block_work [nblocks,4], tile_tokens) as
+    host int32 tensors: per sequence {lo, L, first_tile, num_tiles}; per thread block
+    {b, kv_head, first tile relative to the pair's first_tile, tiles}."""
+    B = seq_lens.shape[0]
+    with torch.cuda.device(seq_lens.device):
+        ensure_workspace(B, 1, Hkv, 128, P, max_pages, seq_lens.device)
+        cap = 4096
+        seq_info = torch.zeros((max(B, 1), 4), dtype=torch.int32)
+        block_work = torch.zeros((cap, 4), dtype=torch.int32)
+        nb = ctypes.c_int32(cap)
+        tt = ctypes.c_int32(0)
+        sv = _view(seq_lens)
+        _check(lib().decode_attn_plan(_ref(sv), int(window), int(Hkv), int(P), int(max_pages),
+                                      ctypes.cast(seq_info.data_ptr(), ctypes.POINTER(ctypes.c_int32)),
+                                      ctypes.cast(block_work.data_ptr(), ctypes.POINTER(ctypes.c_int32)),
+                                      ctypes.byref(nb), ctypes.byref(tt), _stream_ptr(stream)))
+    return seq_info[:B], block_work[:nb.value], tt.value

@@ -1,0 +1,563 @@
+// Host side of the C ABI declared in include/decode_attn.h: argument checks, the workspace
+// layout, TMA descriptor creation and the three launches.  Nothing here allocates device memory.
+#include "../../include/decode_attn.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "da_kernels.cuh"
+
+namespace {
+
+using namespace da;
+
+constexpr int kVersion = 100;
+constexpr int kMaxDevices = 64;
+constexpr int kMaxGridBlocks = 4096;
+constexpr int kMaxGroup = 16;
+
+std::mutex g_mu;
+std::atomic<int> g_last_cuda_error{0};
+std::atomic<int64_t> g_launches{0};
+int64_t g_opt_grid_blocks = 0;   // 0 = two blocks per SM
+cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+
+struct DeviceState {
+    void *ws = nullptr;
+    size_t ws_bytes = 0;
+    int sm_count = 0;
+    bool attrs_set = false;
+};
+DeviceState g_dev[kMaxDevices];
+
+struct TmapKey {
+    const void *ptr;
+    int64_t shape[4];
+    int64_t stride[4];
+    int box_rows;
+};
+struct TmapEntry {
+    TmapKey key;
+    CUtensorMap map;
+    bool used = false;
+};
+constexpr int kTmapCache = 16;
+TmapEntry g_tmaps[kTmapCache];
+int g_tmap_next = 0;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int cuda_fail(cudaError_t e)
+{
+    g_last_cuda_error.store((int)e);
+    return DA_ERR_CUDA;
+}
+#define DA_CUDA(call)                      \
+    do {                                   \
+        cudaError_t e_ = (call);           \
+        if (e_ != cudaSuccess)             \
+            return cuda_fail(e_);          \
+    } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int current_device(int *dev, DeviceState **st)
+{
+    DA_CUDA(cudaGetDevice(dev));
+    if (*dev < 0 || *dev >= kMaxDevices)
+        return DA_ERR_UNSUPPORTED;
+    *st = &g_dev[*dev];
+    if ((*st)->sm_count == 0) {
+        int n = 0;
+        DA_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, *dev));
+        (*st)->sm_count = n;
+    }
+    return DA_OK;
+}
+
+int grid_blocks_for(const DeviceState *st)
+{
+    int64_t n = g_opt_grid_blocks > 0 ? g_opt_grid_blocks : 2 * (int64_t)st->sm_count;
+    if (n < 1) n = 1;
+    if (n > kMaxGridBlocks) n = kMaxGridBlocks;
+    return (int)n;
+}
+
+struct WsLayout {
+    size_t status, seq_info, prefix, block_work, part_lse, part_o;
+    size_t stg_q, stg_bt, stg_sl, stg_out, stg_lse, total;
+};
+
+WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int nblocks)
+{
+    WsLayout w;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    w.status = take(16);
+    w.seq_info = take((size_t)B * 16);
+    w.prefix = take((size_t)(B + 1) * 4);
+    w.block_work = take((size_t)nblocks * 16);
+    w.part_lse = take((size_t)2 * nblocks * kMaxGroup * 4);
+    w.part_o = take((size_t)2 * nblocks * kMaxGroup * HEAD_DIM * 4);
+    w.stg_q = take((size_t)B * Hq * D * 2);
+    w.stg_bt = take((size_t)B * max_pages * 4);
+    w.stg_sl = take((size_t)B * 4);
+    w.stg_out = take((size_t)B * Hq * D * 4);
+    w.stg_lse = take((size_t)B * Hq * 4);
+    w.total = off;
+    return w;
+}
+
+int get_encoder()
+{
+    if (g_encode)
+        return DA_OK;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    DA_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (qres != cudaDriverEntryPointSuccess || !fn)
+        return cuda_fail(cudaErrorNotSupported);
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return DA_OK;
+}
+
+// A 4-D view {d, token, kv head, page} of a K or V pool with box {64, box_rows, 1, 1} and the
+// 128-byte swizzle: one box is box_rows rows of 128 bytes, the unit tile_addr() indexes.
+int get_tmap(const da_tensor *t, int box_rows, CUtensorMap *out)
+{
+    TmapKey key;
+    std::memset(&key, 0, sizeof key);
+    key.ptr = t->data;
+    for (int i = 0; i < 4; ++i) {
+        key.shape[i] = t->shape[i];
+        key.stride[i] = t->stride[i];
+    }
+    key.box_rows = box_rows;
+    for (int i = 0; i < kTmapCache; ++i)
+        if (g_tmaps[i].used && std::memcmp(&g_tmaps[i].key, &key, sizeof key) == 0) {
+            *out = g_tmaps[i].map;
+            return DA_OK;
+        }
+    int rc = get_encoder();
+    if (rc != DA_OK)
+        return rc;
+    cuuint64_t gdim[4] = {(cuuint64_t)t->shape[3], (cuuint64_t)t->shape[2], (cuuint64_t)t->shape[1],
+                          (cuuint64_t)t->shape[0]};
+    cuuint64_t gstr[3] = {(cuuint64_t)t->stride[2] * 2, (cuuint64_t)t->stride[1] * 2, (cuuint64_t)t->stride[0] * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUtensorMap m;
+    CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, t->data, gdim, gstr, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_last_cuda_error.store((int)cudaErrorInvalidValue);
+        return DA_ERR_CUDA;
+    }
+    TmapEntry &e = g_tmaps[g_tmap_next];
+    g_tmap_next = (g_tmap_next + 1) % kTmapCache;
+    e.key = key;
+    e.map = m;
+    e.used = true;
+    *out = m;
+    return DA_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Dims {
+    int64_t B, Hq, Hkv, G, P, num_pages, max_pages;
+};
+
+int check_pool(const da_tensor *t)
+{
+    if (!t->data) return DA_ERR_NULL;
+    if (t->dtype != DA_BF16) return DA_ERR_DTYPE;
+    if (t->ndim != 4) return DA_ERR_SHAPE;
+    if (t->shape[3] != HEAD_DIM) return DA_ERR_UNSUPPORTED;
+    if (t->stride[3] != 1 || !aligned16(t->data)) return DA_ERR_STRIDE_ALIGN;
+    for (int i = 0; i < 3; ++i)
+        if (t->stride[i] <= 0 || (t->stride[i] * 2) % 16 != 0 || t->stride[i] * 2 >= (1ll << 40))
+            return DA_ERR_STRIDE_ALIGN;
+    return DA_OK;
+}
+
+int validate(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl,
+             const da_tensor *out, const da_tensor *lse, Dims *d)
+{
+    if (!q || !k || !v || !bt || !sl || !out) return DA_ERR_NULL;
+    if (!q->data || !bt->data || !sl->data || !out->data) return DA_ERR_NULL;
+    if (lse && !lse->data) return DA_ERR_NULL;
+    if (q->dtype != DA_BF16 || bt->dtype != DA_I32 || sl->dtype != DA_I32) return DA_ERR_DTYPE;
+    if (out->dtype != DA_F32 && out->dtype != DA_BF16) return DA_ERR_DTYPE;
+    if (lse && lse->dtype != DA_F32) return DA_ERR_DTYPE;
+    if (q->ndim != 3 || bt->ndim != 2 || sl->ndim != 1 || out->ndim != 3) return DA_ERR_SHAPE;
+    if (lse && lse->ndim != 2) return DA_ERR_SHAPE;
+    int rc = check_pool(k);
+    if (rc != DA_OK) return rc;
+    rc = check_pool(v);
+    if (rc != DA_OK) return rc;
+    for (int i = 0; i < 4; ++i)
+        if (k->shape[i] != v->shape[i]) return DA_ERR_SHAPE;
+    d->B = q->shape[0];
+    d->Hq = q->shape[1];
+    d->num_pages = k->shape[0];
+    d->Hkv = k->shape[1];
+    d->P = k->shape[2];
+    d->max_pages = bt->shape[1];
+    if (d->B < 0 || d->Hq <= 0 || d->Hkv <= 0 || d->num_pages <= 0 || d->max_pages <= 0) return DA_ERR_SHAPE;
+    if (d->B > (1 << 24) || d->num_pages > 0x7fffffffll || d->max_pages > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+    if (q->shape[2] != HEAD_DIM) return DA_ERR_UNSUPPORTED;
+    if (d->Hq % d->Hkv != 0) return DA_ERR_SHAPE;
+    d->G = d->Hq / d->Hkv;
+    if (d->G > kMaxGroup) return DA_ERR_UNSUPPORTED;
+    if (d->P != 16 && d->P != 32 && d->P != 64 && d->P != 128) return DA_ERR_UNSUPPORTED;
+    if (bt->shape[0] != d->B || sl->shape[0] != d->B) return DA_ERR_SHAPE;
+    if (out->shape[0] != d->B || out->shape[1] != d->Hq || out->shape[2] != HEAD_DIM) return DA_ERR_SHAPE;
+    if (lse && (lse->shape[0] != d->B || lse->shape[1] != d->Hq)) return DA_ERR_SHAPE;
+    if (q->stride[2] != 1 || out->stride[2] != 1 || bt->stride[1] != 1) return DA_ERR_STRIDE_ALIGN;
+    if ((q->stride[0] | q->stride[1]) & 1) return DA_ERR_STRIDE_ALIGN;   // rows read as 32-bit pairs
+    if (reinterpret_cast<uintptr_t>(q->data) & 3u) return DA_ERR_STRIDE_ALIGN;
+    return DA_OK;
+}
+
+template <int NT8>
+int set_kernel_attrs()
+{
+    DA_CUDA(cudaFuncSetAttribute(partition_kernel<NT8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PartCfg<NT8>::SMEM_BYTES));
+    return DA_OK;
+}
+
+int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws, const WsLayout &lay, int nblocks,
+                cudaStream_t stream)
+{
+    PlanParams pp;
+    pp.seq_lens = static_cast<const int32_t *>(sl->data);
+    pp.sl_stride = sl->stride[0];
+    pp.seq_info = reinterpret_cast<int4 *>(ws + lay.seq_info);
+    pp.prefix = reinterpret_cast<int32_t *>(ws + lay.prefix);
+    pp.block_work = reinterpret_cast<int4 *>(ws + lay.block_work);
+    pp.status = reinterpret_cast<int32_t *>(ws + lay.status);
+    pp.B = (int32_t)d.B;
+    pp.Hkv = (int32_t)d.Hkv;
+    pp.P = (int32_t)d.P;
+    pp.window = window;
+    pp.nblocks = nblocks;
+    pp.max_pages = d.max_pages;
+    plan_kernel<<<1, PLAN_THREADS, 0, stream>>>(pp);
+    g_launches.fetch_add(1);
+    DA_CUDA(cudaGetLastError());
+    return DA_OK;
+}
+
+int run(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl,
+        int32_t window, float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream)
+{
+    Dims d;
+    int rc = validate(q, k, v, bt, sl, out, lse, &d);
+    if (rc != DA_OK) return rc;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    rc = current_device(&dev, &st);
+    if (rc != DA_OK) return rc;
+    const int nblocks = grid_blocks_for(st);
+    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks);
+    if (!st->ws || st->ws_bytes < lay.stg_q) return DA_ERR_WORKSPACE;   // staging is only for host_io
+    if (d.B == 0) return DA_OK;
+    uint8_t *ws = static_cast<uint8_t *>(st->ws);
+
+    if (!st->attrs_set) {
+        rc = set_kernel_attrs<1>();
+        if (rc != DA_OK) return rc;
+        rc = set_kernel_attrs<2>();
+        if (rc != DA_OK) return rc;
+        st->attrs_set = true;
+    }
+    const int box_rows = d.P < TILE_T ? (int)d.P : TILE_T;
+    CUtensorMap tm_k, tm_v;
+    rc = get_tmap(k, box_rows, &tm_k);
+    if (rc != DA_OK) return rc;
+    rc = get_tmap(v, box_rows, &tm_v);
+    if (rc != DA_OK) return rc;
+
+    rc = launch_plan(sl, window, d, ws, lay, nblocks, stream);
+    if (rc != DA_OK) return rc;
+
+    PartParams pa;
+    pa.q = static_cast<const __nv_bfloat16 *>(q->data);
+    pa.q_sb = q->stride[0];
+    pa.q_sh = q->stride[1];
+    pa.block_table = static_cast<const int32_t *>(bt->data);
+    pa.bt_sb = bt->stride[0];
+    pa.out = out->data;
+    pa.o_sb = out->stride[0];
+    pa.o_sh = out->stride[1];
+    pa.lse = lse ? static_cast<float *>(lse->data) : nullptr;
+    pa.l_sb = lse ? lse->stride[0] : 0;
+    pa.l_sh = lse ? lse->stride[1] : 0;
+    pa.seq_info = reinterpret_cast<const int4 *>(ws + lay.seq_info);
+    pa.block_work = reinterpret_cast<const int4 *>(ws + lay.block_work);
+    pa.part_o = reinterpret_cast<float *>(ws + lay.part_o);
+    pa.part_lse = reinterpret_cast<float *>(ws + lay.part_lse);
+    pa.status = reinterpret_cast<int32_t *>(ws + lay.status);
+    pa.B = (int32_t)d.B;
+    pa.Hkv = (int32_t)d.Hkv;
+    pa.G = (int32_t)d.G;
+    pa.P = (int32_t)d.P;
+    pa.box_rows = box_rows;
+    pa.num_pages = (int32_t)d.num_pages;
+    pa.out_bf16 = out->dtype == DA_BF16;
+    pa.scale_log2 = scale * LOG2E;
+    const int nt8 = d.G <= 8 ? 1 : 2;
+    const bool timed = g_ev_before && g_ev_after;
+    if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
+    if (nt8 == 1)
+        partition_kernel<1><<<nblocks, NTHREADS, PartCfg<1>::SMEM_BYTES, stream>>>(tm_k, tm_v, pa);
+    else
+        partition_kernel<2><<<nblocks, NTHREADS, PartCfg<2>::SMEM_BYTES, stream>>>(tm_k, tm_v, pa);
+    g_launches.fetch_add(1);
+    DA_CUDA(cudaGetLastError());
+    if (timed) DA_CUDA(cudaEventRecord(g_ev_after, stream));
+
+    MergeParams mp;
+    mp.seq_info = pa.seq_info;
+    mp.prefix = reinterpret_cast<const int32_t *>(ws + lay.prefix);
+    mp.part_o = pa.part_o;
+    mp.part_lse = pa.part_lse;
+    mp.out = out->data;
+    mp.o_sb = pa.o_sb;
+    mp.o_sh = pa.o_sh;
+    mp.lse = pa.lse;
+    mp.l_sb = pa.l_sb;
+    mp.l_sh = pa.l_sh;
+    mp.B = pa.B;
+    mp.Hkv = pa.Hkv;
+    mp.G = pa.G;
+    mp.heads_pad = nt8 * 8;
+    mp.nblocks = nblocks;
+    mp.out_bf16 = pa.out_bf16;
+    merge_kernel<<<(unsigned)(d.B * d.Hkv), HEAD_DIM, 0, stream>>>(mp);
+    g_launches.fetch_add(1);
+    DA_CUDA(cudaGetLastError());
+    return DA_OK;
+}
+
+bool contiguous(const da_tensor *t)
+{
+    int64_t expect = 1;
+    for (int i = t->ndim - 1; i >= 0; --i) {
+        if (t->shape[i] != 1 && t->stride[i] != expect) return false;
+        expect *= t->shape[i];
+    }
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int decode_attn(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
+                const da_tensor *seq_lens, int32_t window, float scale, da_tensor *out, da_tensor *lse, void *stream)
+{
+    return run(q, k_pages, v_pages, block_table, seq_lens, window, scale, out, lse, static_cast<cudaStream_t>(stream));
+}
+
+int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tensor *v_pages,
+                        const da_tensor *block_table_host, const da_tensor *seq_lens_host, int32_t window, float scale,
+                        da_tensor *out_host, da_tensor *lse_host, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Dims d;
+    int rc = validate(q_host, k_pages, v_pages, block_table_host, seq_lens_host, out_host, lse_host, &d);
+    if (rc != DA_OK) return rc;
+    if (!contiguous(q_host) || !contiguous(block_table_host) || !contiguous(seq_lens_host) || !contiguous(out_host) ||
+        (lse_host && !contiguous(lse_host)))
+        return DA_ERR_STRIDE_ALIGN;
+    uint8_t *ws;
+    WsLayout lay;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        int dev;
+        DeviceState *st;
+        rc = current_device(&dev, &st);
+        if (rc != DA_OK) return rc;
+        lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, grid_blocks_for(st));
+        if (!st->ws || st->ws_bytes < lay.total) return DA_ERR_WORKSPACE;
+        ws = static_cast<uint8_t *>(st->ws);
+    }
+    if (d.B == 0) return DA_OK;
+    const size_t out_item = out_host->dtype == DA_BF16 ? 2 : 4;
+    DA_CUDA(cudaMemcpyAsync(ws + lay.stg_q, q_host->data, (size_t)d.B * d.Hq * HEAD_DIM * 2, cudaMemcpyHostToDevice, stream));
+    DA_CUDA(cudaMemcpyAsync(ws + lay.stg_bt, block_table_host->data, (size_t)d.B * d.max_pages * 4, cudaMemcpyHostToDevice, stream));
+    DA_CUDA(cudaMemcpyAsync(ws + lay.stg_sl, seq_lens_host->data, (size_t)d.B * 4, cudaMemcpyHostToDevice, stream));
+    da_tensor qd = *q_host, btd = *block_table_host, sld = *seq_lens_host, od = *out_host, ld;
+    qd.data = ws + lay.stg_q;
+    btd.data = ws + lay.stg_bt;
+    sld.data = ws + lay.stg_sl;
+    od.data = ws + lay.stg_out;
+    if (lse_host) {
+        ld = *lse_host;
+        ld.data = ws + lay.stg_lse;
+    }
+    rc = run(&qd, k_pages, v_pages, &btd, &sld, window, scale, &od, lse_host ? &ld : nullptr, stream);
+    if (rc != DA_OK) return rc;
+    DA_CUDA(cudaMemcpyAsync(out_host->data, ws + lay.stg_out, (size_t)d.B * d.Hq * HEAD_DIM * out_item, cudaMemcpyDeviceToHost, stream));
+    if (lse_host)
+        DA_CUDA(cudaMemcpyAsync(lse_host->data, ws + lay.stg_lse, (size_t)d.B * d.Hq * 4, cudaMemcpyDeviceToHost, stream));
+    return DA_OK;
+}
+
+size_t decode_attn_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D, int32_t P, int64_t max_pages)
+{
+    (void)Hkv;
+    (void)P;
+    if (B < 0 || Hq <= 0 || D <= 0 || max_pages < 0) return 0;
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    int nblocks = g_opt_grid_blocks > 0 ? (int)g_opt_grid_blocks : kMaxGridBlocks;
+    if (g_opt_grid_blocks <= 0 && current_device(&dev, &st) == DA_OK)
+        nblocks = grid_blocks_for(st);
+    return ws_layout(B, Hq, D, max_pages, nblocks).total;
+}
+
+int decode_attn_set_workspace(void *dev_ptr, size_t bytes)
+{
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    int rc = current_device(&dev, &st);
+    if (rc != DA_OK) return rc;
+    if (!dev_ptr) {
+        st->ws = nullptr;
+        st->ws_bytes = 0;
+        return DA_OK;
+    }
+    if (reinterpret_cast<uintptr_t>(dev_ptr) & 255u) return DA_ERR_STRIDE_ALIGN;
+    if (bytes < 256) return DA_ERR_WORKSPACE;
+    DA_CUDA(cudaMemsetAsync(dev_ptr, 0, 256, 0));
+    DA_CUDA(cudaStreamSynchronize(0));
+    st->ws = dev_ptr;
+    st->ws_bytes = bytes;
+    return DA_OK;
+}
+
+int decode_attn_read_device_status(void *stream_, int32_t *host_status4)
+{
+    if (!host_status4) return DA_ERR_NULL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    void *ws;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        int dev;
+        DeviceState *st;
+        int rc = current_device(&dev, &st);
+        if (rc != DA_OK) return rc;
+        if (!st->ws) return DA_ERR_WORKSPACE;
+        ws = st->ws;
+    }
+    DA_CUDA(cudaMemcpyAsync(host_status4, ws, 16, cudaMemcpyDeviceToHost, stream));
+    DA_CUDA(cudaMemsetAsync(ws, 0, 16, stream));
+    DA_CUDA(cudaStreamSynchronize(stream));
+    return DA_OK;
+}
+
+int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int32_t P, int64_t max_pages,
+                     int32_t *host_seq_info, int32_t *host_block_work, int32_t *num_blocks, int32_t *tile_tokens,
+                     void *stream_)
+{
+    if (!seq_lens || !seq_lens->data || !host_seq_info || !host_block_work || !num_blocks || !tile_tokens)
+        return DA_ERR_NULL;
+    if (seq_lens->dtype != DA_I32) return DA_ERR_DTYPE;
+    if (seq_lens->ndim != 1 || Hkv <= 0 || max_pages <= 0) return DA_ERR_SHAPE;
+    if (P != 16 && P != 32 && P != 64 && P != 128) return DA_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    int rc = current_device(&dev, &st);
+    if (rc != DA_OK) return rc;
+    const int nblocks = grid_blocks_for(st);
+    Dims d;
+    d.B = seq_lens->shape[0];
+    d.Hkv = Hkv;
+    d.P = P;
+    d.max_pages = max_pages;
+    const WsLayout lay = ws_layout(d.B, 1, HEAD_DIM, max_pages, nblocks);
+    if (!st->ws || st->ws_bytes < lay.part_lse) return DA_ERR_WORKSPACE;
+    if (*num_blocks < nblocks) return DA_ERR_SHAPE;
+    *num_blocks = nblocks;
+    *tile_tokens = TILE_T;
+    if (d.B == 0) return DA_OK;
+    uint8_t *ws = static_cast<uint8_t *>(st->ws);
+    rc = launch_plan(seq_lens, window, d, ws, lay, nblocks, stream);
+    if (rc != DA_OK) return rc;
+    DA_CUDA(cudaMemcpyAsync(host_seq_info, ws + lay.seq_info, (size_t)d.B * 16, cudaMemcpyDeviceToHost, stream));
+    DA_CUDA(cudaMemcpyAsync(host_block_work, ws + lay.block_work, (size_t)nblocks * 16, cudaMemcpyDeviceToHost, stream));
+    DA_CUDA(cudaStreamSynchronize(stream));
+    return DA_OK;
+}
+
+int decode_attn_set_option(const char *name, int64_t value)
+{
+    if (!name) return DA_ERR_NULL;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (std::strcmp(name, "grid_blocks") == 0) {
+        if (value < 0 || value > kMaxGridBlocks) return DA_ERR_UNSUPPORTED;
+        g_opt_grid_blocks = value;
+        return DA_OK;
+    }
+    return DA_ERR_UNSUPPORTED;
+}
+
+int64_t decode_attn_get_option(const char *name)
+{
+    if (!name) return -1;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (std::strcmp(name, "grid_blocks") == 0) return g_opt_grid_blocks;
+    return -1;
+}
+
+int decode_attn_set_profile_events(void *before, void *after)
+{
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_ev_before = static_cast<cudaEvent_t>(before);
+    g_ev_after = static_cast<cudaEvent_t>(after);
+    return DA_OK;
+}
+
+const char *decode_attn_strerror(int status)
+{
+    switch (status) {
+    case DA_OK: return "ok";
+    case DA_ERR_NULL: return "a required pointer is NULL";
+    case DA_ERR_SHAPE: return "tensor ranks or extents disagree";
+    case DA_ERR_DTYPE: return "wrong element type";
+    case DA_ERR_STRIDE_ALIGN: return "non-contiguous last dimension, or a base/stride that is not suitably aligned";
+    case DA_ERR_UNSUPPORTED: return "unsupported head_dim, page size, group size or option";
+    case DA_ERR_WORKSPACE: return "no workspace registered for this device, or it is too small";
+    case DA_ERR_CUDA: return "a CUDA call failed (see decode_attn_last_cuda_error)";
+    default: return "unknown status";
+    }
+}
+
+int decode_attn_last_cuda_error(void) { return g_last_cuda_error.load(); }
+int decode_attn_version(void) { return kVersion; }
+int64_t decode_attn_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"
