@@ -315,7 +315,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOAD_TEXT))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--ref-every", type=int, default=2, help="oracle sample: every n-th sequence")
+    ap.add_argument("--ref-every", type=int, default=1, help="oracle sample: every n-th sequence")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     return run_reference(args) if args.impl == "reference" else run_ours(args)
