@@ -263,24 +263,13 @@ int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws,
     return DA_OK;
 }
 
-int run(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl,
-        int32_t window, float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream)
+// The three launches of the hot path, with every scratch array taken from `ws` as laid out by `lay`.
+// Called with g_mu held.
+int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay, int nblocks, const da_tensor *q,
+                const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl, int32_t window,
+                float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream)
 {
-    Dims d;
-    int rc = validate(q, k, v, bt, sl, out, lse, &d);
-    if (rc != DA_OK) return rc;
-
-    std::lock_guard<std::mutex> lock(g_mu);
-    int dev;
-    DeviceState *st;
-    rc = current_device(&dev, &st);
-    if (rc != DA_OK) return rc;
-    const int nblocks = grid_blocks_for(st);
-    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks);
-    if (!st->ws || st->ws_bytes < lay.stg_q) return DA_ERR_WORKSPACE;   // staging is only for host_io
-    if (d.B == 0) return DA_OK;
-    uint8_t *ws = static_cast<uint8_t *>(st->ws);
-
+    int rc;
     if (!st->attrs_set) {
         rc = set_kernel_attrs<1>();
         if (rc != DA_OK) return rc;
@@ -355,6 +344,26 @@ int run(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_ten
     g_launches.fetch_add(1);
     DA_CUDA(cudaGetLastError());
     return DA_OK;
+}
+
+int run(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl,
+        int32_t window, float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream)
+{
+    Dims d;
+    int rc = validate(q, k, v, bt, sl, out, lse, &d);
+    if (rc != DA_OK) return rc;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    rc = current_device(&dev, &st);
+    if (rc != DA_OK) return rc;
+    const int nblocks = grid_blocks_for(st);
+    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks);
+    if (!st->ws || st->ws_bytes < lay.stg_q) return DA_ERR_WORKSPACE;   // staging is only for host_io
+    if (d.B == 0) return DA_OK;
+    return launch_path(st, d, static_cast<uint8_t *>(st->ws), lay, nblocks, q, k, v, bt, sl, window, scale, out, lse,
+                       stream);
 }
 
 bool contiguous(const da_tensor *t)
