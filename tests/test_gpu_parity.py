@@ -40,7 +40,8 @@ def gpu_of(da, case, out_dtype=torch.float32):
 def assert_close(got, ref, what, atol=ATOL, rtol=RTOL):
     got, ref = np.asarray(got), np.asarray(ref)
     both_ninf = np.isneginf(got) & np.isneginf(ref)
-    err = np.where(both_ninf, 0.0, np.abs(got - ref))
+    with np.errstate(invalid="ignore"):
+        err = np.where(both_ninf, 0.0, np.abs(got - ref))
     lim = atol + rtol * np.abs(np.where(both_ninf, 0.0, ref))
     bad = ~(err <= lim)
     if bad.any():
