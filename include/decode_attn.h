@@ -121,6 +121,37 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
                         void *stream);
 
 /*
+ * decode_attn_static_scratch -- decode_attn() for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a packaging variant of the same kernels.)
+ *
+ * Who needs it: an inference server that hands every free byte of HBM to its KV-cache pool at
+ * start-up has nothing left for a later cudaMalloc, and a caller in the middle of a decode step
+ * cannot afford cudaMalloc's device-wide synchronisation; neither may have an allocator whose
+ * buffer it could register with decode_attn_set_workspace().  This entry point needs no registered
+ * workspace and calls no cudaMalloc, cudaFree or any allocating routine: the plan arrays, the
+ * split partials and the status record live in one fixed 6 MiB array that is part of the library
+ * image (every GPU that loads the library holds those 6 MiB until the process exits).
+ *
+ * Arguments and results are those of decode_attn(), plus
+ *   dev_status4  DEVICE int32[4], may be NULL: receives the device status record of THIS call
+ *                ({da_dev_status code, sequence, block-table index, value}; all zero = clean),
+ *                copied on `stream` after the kernels.
+ * Limits: B <= 4096 sequences and at most 320 thread blocks in the partition kernel (the default
+ * of two per SM on a B200 is 296); beyond either, or if the layout would exceed the 6 MiB, the
+ * call returns DA_ERR_WORKSPACE and launches nothing.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call outside any stream capture.  All calls on a device
+ * share the one array, which still holds the previous call's contents when the next one starts
+ * (the call clears the only part that must start at zero, its status record): two calls that
+ * overlap on the GPU race on it, so keep them on one stream or order them yourself.
+ */
+int decode_attn_static_scratch(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                               const da_tensor *block_table, const da_tensor *seq_lens, int32_t window,
+                               float scale, da_tensor *out, da_tensor *lse, int32_t *dev_status4,
+                               void *stream);
+
+/*
  * Scratch.  decode_attn_workspace_bytes() says how much device memory a call with these extents
  * needs on the current device with the current launch options (split partials, the plan, a status
  * record, and staging room for decode_attn_host_io).  decode_attn_set_workspace() registers a

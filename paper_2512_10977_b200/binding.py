@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
             L.decode_attn.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_host_io.restype = ctypes.c_int
             L.decode_attn_host_io.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_static_scratch.restype = ctypes.c_int
+            L.decode_attn_static_scratch.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp, vp]
             L.decode_attn_workspace_bytes.restype = ctypes.c_size_t
             L.decode_attn_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i64]
             L.decode_attn_set_workspace.restype = ctypes.c_int
@@ -180,6 +182,25 @@ def decode_attn_host_io(q_host, k_pages, v_pages, block_table_host, seq_lens_hos
                                          int(window), float(scale), _ref(tv[5]), _ref(tv[6]),
                                          _stream_ptr(stream)))
     return out_host, lse_host
+
+
+def decode_attn_static_scratch(q, k_pages, v_pages, block_table, seq_lens, window: int, scale: float,
+                               out: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                               dev_status: Optional[torch.Tensor] = None,
+                               stream: Optional[torch.cuda.Stream] = None):
+    """decode_attn for callers that cannot allocate: scratch is the library's fixed 6 MiB device array.
+
+    Unlike ``decode_attn`` this wrapper allocates nothing either: ``out`` (and ``lse`` and the
+    optional int32[4] device tensor ``dev_status``) must be passed in, and no workspace is
+    registered.  Raises DecodeAttnError(6) beyond 4096 sequences or 320 partition blocks.
+    """
+    with torch.cuda.device(k_pages.device):
+        tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
+        _check(lib().decode_attn_static_scratch(
+            _ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]), int(window), float(scale),
+            _ref(tv[5]), _ref(tv[6]), dev_status.data_ptr() if dev_status is not None else None,
+            _stream_ptr(stream)))
+    return out, lse
 
 
 def read_device_status(stream: Optional[torch.cuda.Stream] = None):

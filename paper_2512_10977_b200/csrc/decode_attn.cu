@@ -50,6 +50,15 @@ constexpr int kTmapCache = 16;
 TmapEntry g_tmaps[kTmapCache];
 int g_tmap_next = 0;
 
+// Scratch for decode_attn_static_scratch(): part of the library image, so every GPU that loads the
+// library holds these bytes until the process exits.  In host code this name is only a stand-in
+// for the device object; its device address comes from cudaGetSymbolAddress (static_scratch_ptr).
+constexpr size_t kStaticScratchBytes = 6u << 20;   // 6 MiB
+constexpr int64_t kStaticMaxSeqs = 4096;
+constexpr int kStaticMaxBlocks = 320;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+uint8_t *g_static_scratch_addr[kMaxDevices] = {};
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -428,6 +437,45 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
     DA_CUDA(cudaMemcpyAsync(out_host->data, ws + lay.stg_out, (size_t)d.B * d.Hq * HEAD_DIM * out_item, cudaMemcpyDeviceToHost, stream));
     if (lse_host)
         DA_CUDA(cudaMemcpyAsync(lse_host->data, ws + lay.stg_lse, (size_t)d.B * d.Hq * 4, cudaMemcpyDeviceToHost, stream));
+    return DA_OK;
+}
+
+int decode_attn_static_scratch(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                               const da_tensor *block_table, const da_tensor *seq_lens, int32_t window, float scale,
+                               da_tensor *out, da_tensor *lse, int32_t *dev_status4, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Dims d;
+    int rc = validate(q, k_pages, v_pages, block_table, seq_lens, out, lse, &d);
+    if (rc != DA_OK) return rc;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    rc = current_device(&dev, &st);
+    if (rc != DA_OK) return rc;
+    const int nblocks = grid_blocks_for(st);
+    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks);
+    // beyond the fixed array: refuse, never spill into an allocation
+    if (d.B > kStaticMaxSeqs || nblocks > kStaticMaxBlocks || lay.stg_q > kStaticScratchBytes)
+        return DA_ERR_WORKSPACE;
+    if (!g_static_scratch_addr[dev]) {
+        // once per device, with that device current: the device address of the array
+        void *p = nullptr;
+        DA_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (!p) return cuda_fail(cudaErrorInvalidSymbol);
+        g_static_scratch_addr[dev] = static_cast<uint8_t *>(p);
+    }
+    uint8_t *ws = g_static_scratch_addr[dev];
+    // the array keeps the previous call's contents; only the status record has to start at zero
+    DA_CUDA(cudaMemsetAsync(ws + lay.status, 0, 16, stream));
+    if (d.B > 0) {
+        rc = launch_path(st, d, ws, lay, nblocks, q, k_pages, v_pages, block_table, seq_lens, window, scale, out, lse,
+                         stream);
+        if (rc != DA_OK) return rc;
+    }
+    if (dev_status4)
+        DA_CUDA(cudaMemcpyAsync(dev_status4, ws + lay.status, 16, cudaMemcpyDeviceToDevice, stream));
     return DA_OK;
 }
 
