@@ -16,11 +16,11 @@ namespace da {
 constexpr int HEAD_DIM = 128;
 constexpr int NCW = 4;                      // consumer warps per block; each owns 16 tokens of a tile
 constexpr int TILE_T = 16 * NCW;            // tokens per pipeline stage
-constexpr int PLANE_BYTES = TILE_T * 128;   // one 64-column half of a K or V tile, 128-B rows
-constexpr int KV_BYTES = 2 * PLANE_BYTES;   // a K (or V) tile
+constexpr int KV_BYTES = TILE_T * 256;      // a K (or V) tile: TILE_T rows of 128 bf16
 constexpr int STAGE_BYTES = 2 * KV_BYTES;   // K tile followed by V tile
 constexpr int NTHREADS = (NCW + 1) * 32;    // + one producer warp
 constexpr int PLAN_THREADS = 1024;
+constexpr int PLAN_SMEM_SEQS = 4096;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
@@ -108,6 +108,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
 {
     __shared__ int warp_tot[PLAN_THREADS / 32];
     __shared__ int running_s;
+    __shared__ int prefix_s[PLAN_SMEM_SEQS + 1];   // copy of the prefix for the searches below
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0)
         running_s = 0;
@@ -155,6 +156,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         if (b < p.B) {
             p.seq_info[b] = make_int4(lo, L, first, nt);
             p.prefix[b] = excl;
+            if (b < PLAN_SMEM_SEQS)
+                prefix_s[b] = excl;
         }
         __syncthreads();
         if (tid == PLAN_THREADS - 1)
@@ -162,9 +165,14 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         __syncthreads();
     }
     const int tiles_per_head = running_s;
-    if (tid == 0)
+    const bool in_smem = p.B <= PLAN_SMEM_SEQS;
+    if (tid == 0) {
         p.prefix[p.B] = tiles_per_head;
+        if (in_smem)
+            prefix_s[p.B] = tiles_per_head;
+    }
     __syncthreads();   // this block's global writes are visible to itself after the barrier
+    const int *prefix = in_smem ? prefix_s : p.prefix;
 
     const int64_t total = (int64_t)tiles_per_head * p.Hkv;
     for (int c = tid; c < p.nblocks; c += PLAN_THREADS) {
@@ -177,14 +185,14 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
             int lo_i = 0, hi_i = p.B;   // invariant: prefix[lo_i] <= x < prefix[hi_i]
             while (hi_i - lo_i > 1) {
                 const int mid = (lo_i + hi_i) >> 1;
-                if (p.prefix[mid] <= x)
+                if (prefix[mid] <= x)
                     lo_i = mid;
                 else
                     hi_i = mid;
             }
             const int b = lo_i;
-            const int nt = p.seq_info[b].w;
-            const int64_t rem = ws - (int64_t)p.prefix[b] * p.Hkv;
+            const int nt = prefix[b + 1] - prefix[b];
+            const int64_t rem = ws - (int64_t)prefix[b] * p.Hkv;
             bw = make_int4(b, (int)(rem / nt), (int)(rem % nt), (int)(we - ws));
         }
         p.block_work[c] = bw;
@@ -192,12 +200,14 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
 }
 
 // =====================================================================================  partition
-// Shared-memory address of the 16-byte chunk `chunk` (0..15 along head_dim) of token row `row`
-// inside a K or V tile that TMA wrote with the 128-byte swizzle: two 64-column planes of
-// 128-byte rows, chunk index XORed with the row's low three bits.
-__device__ __forceinline__ uint32_t tile_addr(uint32_t tile_base, int row, int chunk)
+// Layout of a K or V tile in shared memory.  One TMA box is box_rows token rows of one page, all
+// 128 columns, written as two 64-column planes of box_rows 128-byte rows with the 128-byte swizzle
+// (16-byte chunk index XORed with the row's low three bits).  A tile is TILE_T / box_rows such boxes
+// back to back.  Row `row` of the tile therefore starts at row_offset(); its chunk c (0..15 along
+// head_dim) is at  + (c >> 3) * plane_bytes + (((c & 7) ^ (row & 7)) << 4).
+__device__ __forceinline__ uint32_t row_offset(int row, int box_rows)
 {
-    return tile_base + (chunk >> 3) * PLANE_BYTES + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
+    return (uint32_t)((row / box_rows) * (box_rows * 256) + (row % box_rows) * 128);
 }
 
 template <int NT8>
@@ -241,11 +251,11 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
     if (warp == NCW) {
         // ------------------------------------------------------------------ producer warp
-        // Lane -> (box, K|V, 64-column plane).  A box is box_rows token rows of one page.
+        // Lane -> (box, K|V).  A box is box_rows token rows (all 128 columns) of one page.
         const int nboxes = TILE_T / p.box_rows;
-        const int box = lane >> 2, is_v = (lane >> 1) & 1, plane = lane & 1;
-        const bool active = lane < nboxes * 4;
-        const uint32_t box_bytes = (uint32_t)p.box_rows * 128u;
+        const int box = lane >> 1, is_v = lane & 1;
+        const bool active = lane < nboxes * 2;
+        const uint32_t box_bytes = (uint32_t)p.box_rows * 256u;
         const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
         uint32_t it = 0;
         bool aborted = false;
@@ -318,9 +328,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 mbar_arrive_expect_tx(bar_full + 8 * stage, (uint32_t)__popc(mask) * box_bytes);
             __syncwarp();
             if (need) {
-                const uint32_t dst = smem_base + stage * STAGE_BYTES + is_v * KV_BYTES + plane * PLANE_BYTES +
-                                     box * box_bytes;
-                tma_load_4d(dst, tm, plane * 64, row, gg, page, bar_full + 8 * stage);
+                const uint32_t dst = smem_base + stage * STAGE_BYTES + is_v * KV_BYTES + box * box_bytes;
+                tma_load_5d(dst, tm, 0, row, 0, gg, page, bar_full + 8 * stage);
             }
             ++it;
             have = n_have;
@@ -356,6 +365,9 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const int k_chunk = lane >> 4;                                      //    matrices 2,3 are chunk +1
     const int v_row = 16 * warp + (lane & 7) + (lane >> 4) * 8;         // V: matrices 2,3 are rows +8
     const int v_chunk = (lane >> 3) & 1;                                //    matrices 1,3 are chunk +1
+    const uint32_t plane_bytes = (uint32_t)p.box_rows * 128u;
+    const uint32_t k_off = row_offset(k_row, p.box_rows), v_off = row_offset(v_row, p.box_rows);
+    const uint32_t k_sw = (uint32_t)(k_row & 7), v_sw = (uint32_t)(v_row & 7);
 
     while (remaining > 0) {
         const int4 si = p.seq_info[b];
@@ -413,7 +425,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         const int rr = e >> 4, ch = e & 15;
                         const int t = a + rr;
                         if (t < v_lo || t >= v_hi) {
-                            const uint32_t addr = v_base + (ch >> 3) * PLANE_BYTES + (16 * warp + rr) * 128 + ((ch & 7) << 4);
+                            const uint32_t addr = v_base + row_offset(16 * warp + rr, p.box_rows) + (ch >> 3) * plane_bytes + ((ch & 7) << 4);
                             asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
                         }
                     }
@@ -431,7 +443,9 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         uint32_t af[4];
-                        ldmatrix_x4(af, tile_addr(k_base, k_row, 2 * kk + k_chunk));
+                        // chunk 2kk + k_chunk: plane kk >> 2, position ((2kk + k_chunk) & 7) ^ (row & 7)
+                        ldmatrix_x4(af, k_base + k_off + (kk >> 2) * plane_bytes +
+                                            ((((2 * kk + k_chunk) & 7) ^ k_sw) << 4));
 #pragma unroll
                         for (int n = 0; n < NT8; ++n)
                             mma_bf16_16816(acc[n][kk & 1], af, qf[n][kk][0], qf[n][kk][1]);
@@ -510,7 +524,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     uint32_t vf[4];
-                    ldmatrix_x4_trans(vf, tile_addr(v_base, v_row, 2 * j + v_chunk));
+                    ldmatrix_x4_trans(vf, v_base + v_off + (j >> 2) * plane_bytes + ((((2 * j + v_chunk) & 7) ^ v_sw) << 4));
 #pragma unroll
                     for (int n = 0; n < NT8; ++n) {
                         mma_bf16_16816(o[n][j], vf, ph[n][0], ph[n][1]);
@@ -598,34 +612,53 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 }
 
 // =====================================================================================  merge
-// One block per (sequence, KV head); thread = one head_dim column.  Pairs that a single thread
-// block covered were already written by the partition kernel; empty sequences get out = 0 and
-// lse = -inf; the rest are combined from their partial slots:
-//   M = max_s lse_s,  w_s = exp(lse_s - M),  out = sum_s w_s O_s / sum_s w_s,  lse = M + ln sum_s w_s.
-__global__ void __launch_bounds__(HEAD_DIM) merge_kernel(const MergeParams p)
+// One block per (sequence, KV head); thread = (head of the group, four head_dim columns).  Pairs
+// that a single thread block covered were already written by the partition kernel; empty sequences
+// get out = 0 and lse = -inf; the rest are combined from their partial slots, one split at a time:
+//   M' = max(M, lse_s);  acc = acc * exp(M - M') + exp(lse_s - M') * O_s;  den likewise;
+//   out = acc / den;  lse = M + ln den.
+constexpr int MERGE_LANES = HEAD_DIM / 4;
+
+__global__ void __launch_bounds__(16 * MERGE_LANES) merge_kernel(const MergeParams p)
 {
     const int b = blockIdx.x / p.Hkv, g = blockIdx.x % p.Hkv;
-    const int d = threadIdx.x;
+    const int head = threadIdx.x / MERGE_LANES, d = (threadIdx.x % MERGE_LANES) * 4;
+    if (head >= p.G)
+        return;
     const int4 si = p.seq_info[b];
+    const int tiles_before = p.prefix[b], tiles_all = p.prefix[p.B];
     const int nt = si.w;
+    const int h = g * p.G + head;
 
-    auto store = [&](int head, float val, float lse_val) {
-        const int h = g * p.G + head;
-        if (p.out_bf16)
-            reinterpret_cast<__nv_bfloat16 *>(p.out)[(int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d] = __float2bfloat16_rn(val);
-        else
-            reinterpret_cast<float *>(p.out)[(int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d] = val;
+    auto store = [&](float4 v, float lse_val) {
+        const int64_t at = (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d;
+        if (p.out_bf16) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+            __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
+            if ((reinterpret_cast<uintptr_t>(o) & 7u) == 0) {
+                uint2 pk = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+                *reinterpret_cast<uint2 *>(o) = pk;
+            } else {
+                o[0] = lo.x; o[1] = lo.y; o[2] = hi.x; o[3] = hi.y;
+            }
+        } else {
+            float *o = reinterpret_cast<float *>(p.out) + at;
+            if ((reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+                *reinterpret_cast<float4 *>(o) = v;
+            } else {
+                o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+            }
+        }
         if (d == 0 && p.lse)
             p.lse[(int64_t)b * p.l_sb + (int64_t)h * p.l_sh] = lse_val;
     };
 
     if (nt == 0) {
-        for (int head = 0; head < p.G; ++head)
-            store(head, 0.f, -INFINITY);
+        store(make_float4(0.f, 0.f, 0.f, 0.f), -INFINITY);
         return;
     }
-    const int64_t total = (int64_t)p.prefix[p.B] * p.Hkv;
-    const int64_t w0 = (int64_t)p.prefix[b] * p.Hkv + (int64_t)g * nt;
+    const int64_t total = (int64_t)tiles_all * p.Hkv;
+    const int64_t w0 = (int64_t)tiles_before * p.Hkv + (int64_t)g * nt;
     const int c_first = range_owner(total, p.nblocks, w0);
     const int c_last = range_owner(total, p.nblocks, w0 + nt - 1);
     if (c_first == c_last)
@@ -633,21 +666,25 @@ __global__ void __launch_bounds__(HEAD_DIM) merge_kernel(const MergeParams p)
     // the pair is the first item of every block but possibly c_first, where it is the first item
     // only if that block's range starts exactly at the pair
     const int slot_first = 2 * c_first + (range_start(total, p.nblocks, c_first) == w0 ? 0 : 1);
-    for (int head = 0; head < p.G; ++head) {
-        float M = -INFINITY;
-        for (int cc = c_first; cc <= c_last; ++cc) {
-            const int slot = (cc == c_first) ? slot_first : 2 * cc;
-            M = fmaxf(M, p.part_lse[(int64_t)slot * p.heads_pad + head]);
-        }
-        float den = 0.f, num = 0.f;
-        for (int cc = c_first; cc <= c_last; ++cc) {
-            const int slot = (cc == c_first) ? slot_first : 2 * cc;
-            const float w = __expf(p.part_lse[(int64_t)slot * p.heads_pad + head] - M);
-            den += w;
-            num += w * p.part_o[((int64_t)slot * p.heads_pad + head) * HEAD_DIM + d];
-        }
-        store(head, num / den, M + __logf(den));
+    float M = -INFINITY, den = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int cc = c_first; cc <= c_last; ++cc) {
+        const int slot = (cc == c_first) ? slot_first : 2 * cc;
+        const float l = p.part_lse[(int64_t)slot * p.heads_pad + head];
+        const float4 o = *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)slot * p.heads_pad + head) * HEAD_DIM + d);
+        const float m_new = fmaxf(M, l);
+        const float sc = (M == -INFINITY) ? 0.f : __expf(M - m_new);
+        const float w = __expf(l - m_new);
+        acc.x = acc.x * sc + w * o.x;
+        acc.y = acc.y * sc + w * o.y;
+        acc.z = acc.z * sc + w * o.z;
+        acc.w = acc.w * sc + w * o.w;
+        den = den * sc + w;
+        M = m_new;
     }
+    const float inv = 1.f / den;
+    store(make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv), M + __logf(den));
 }
 
 }  // namespace da

@@ -142,8 +142,10 @@ int get_encoder()
     return DA_OK;
 }
 
-// A 4-D view {d, token, kv head, page} of a K or V pool with box {64, box_rows, 1, 1} and the
-// 128-byte swizzle: one box is box_rows rows of 128 bytes, the unit tile_addr() indexes.
+// A 5-D view {d within a 64-column half, token, half, kv head, page} of a K or V pool, box
+// {64, box_rows, 2, 1, 1}, 128-byte swizzle.  Splitting head_dim into two halves keeps the inner box
+// extent at the swizzle span (128 bytes) while one TMA operation still brings all 128 columns of
+// box_rows tokens: in shared memory a box is two planes of box_rows 128-byte rows.
 int get_tmap(const da_tensor *t, int box_rows, CUtensorMap *out)
 {
     TmapKey key;
@@ -162,13 +164,12 @@ int get_tmap(const da_tensor *t, int box_rows, CUtensorMap *out)
     int rc = get_encoder();
     if (rc != DA_OK)
         return rc;
-    cuuint64_t gdim[4] = {(cuuint64_t)t->shape[3], (cuuint64_t)t->shape[2], (cuuint64_t)t->shape[1],
-                          (cuuint64_t)t->shape[0]};
-    cuuint64_t gstr[3] = {(cuuint64_t)t->stride[2] * 2, (cuuint64_t)t->stride[1] * 2, (cuuint64_t)t->stride[0] * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
+    cuuint64_t gdim[5] = {64, (cuuint64_t)t->shape[2], 2, (cuuint64_t)t->shape[1], (cuuint64_t)t->shape[0]};
+    cuuint64_t gstr[4] = {(cuuint64_t)t->stride[2] * 2, 128, (cuuint64_t)t->stride[1] * 2, (cuuint64_t)t->stride[0] * 2};
+    cuuint32_t box[5] = {64, (cuuint32_t)box_rows, 2, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     CUtensorMap m;
-    CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, t->data, gdim, gstr, box, estr,
+    CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, t->data, gdim, gstr, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -349,7 +350,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     mp.heads_pad = nt8 * 8;
     mp.nblocks = nblocks;
     mp.out_bf16 = pa.out_bf16;
-    merge_kernel<<<(unsigned)(d.B * d.Hkv), HEAD_DIM, 0, stream>>>(mp);
+    merge_kernel<<<(unsigned)(d.B * d.Hkv), (unsigned)(nt8 * 8 * MERGE_LANES), 0, stream>>>(mp);
     g_launches.fetch_add(1);
     DA_CUDA(cudaGetLastError());
     return DA_OK;
