@@ -138,7 +138,8 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
  *                copied on `stream` after the kernels.
  * Limits: B <= 4096 sequences and at most 320 thread blocks in the partition kernel (the default
  * of two per SM on a B200 is 296); beyond either, or if the layout would exceed the 6 MiB, the
- * call returns DA_ERR_WORKSPACE and launches nothing.
+ * call returns DA_ERR_WORKSPACE and launches nothing.  To keep the split partials inside the
+ * array, the work is cut into one static range per thread block only (as with "tail_units" 0).
  *
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  * that device current); make that first call outside any stream capture.  All calls on a device
@@ -173,24 +174,32 @@ int decode_attn_read_device_status(void *stream, int32_t *host_status4);
 /*
  * decode_attn_plan -- runs only the plan kernel (the split schedule of the partition kernel) and
  * copies it to HOST arrays, synchronising `stream`.  A debugging and test aid: it shows which
- * token ranges each thread block will cover.
+ * token ranges each work unit covers.  Units 0 .. num_static-1 are the ranges the thread blocks
+ * of the partition kernel start on; the others are handed out through a ticket counter as blocks
+ * finish.
  *   seq_lens        DEVICE i32 [B] view
  *   host_seq_info   HOST int32 [B][4]: {lo, L, first_tile, num_tiles}; a tile is tile_tokens
  *                   consecutive tokens starting at a multiple of tile_tokens
- *   host_block_work HOST int32 [*num_blocks][4]: {b, kv_head, first tile of that pair relative to
- *                   its first_tile, number of tiles}; a block walks forward from there through
+ *   host_unit_work  HOST int32 [capacity][4]: {b, kv_head, first tile of that pair relative to its
+ *                   first_tile, number of tiles}; a unit walks forward from there through
  *                   (b, kv_head) pairs in row-major order
- *   num_blocks      HOST in: capacity of host_block_work in rows; out: the grid size
+ *   num_units       HOST in: capacity of host_unit_work in rows (8192 always suffices);
+ *                   out: units in use
+ *   num_static      HOST out: the partition kernel's grid size
  *   tile_tokens     HOST out
  */
 int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int32_t P,
-                     int64_t max_pages, int32_t *host_seq_info, int32_t *host_block_work,
-                     int32_t *num_blocks, int32_t *tile_tokens, void *stream);
+                     int64_t max_pages, int32_t *host_seq_info, int32_t *host_unit_work,
+                     int32_t *num_units, int32_t *num_static, int32_t *tile_tokens, void *stream);
 
 /*
- * Launch options, for tests and tuning.  Names: "grid_blocks" (thread blocks of the partition
- * kernel; 0 = two per SM; every value gives the same result up to fp32 rounding and changes how
- * sequences are split).  Returns DA_ERR_UNSUPPORTED for an unknown name or a value out of range.
+ * Launch options, for tests and tuning.  Every setting gives the same result up to fp32 rounding;
+ * they change how sequences are split.
+ *   "grid_blocks"  thread blocks of the partition kernel (0 = two per SM, at most 4096)
+ *   "tail_units"   work units per thread block that are handed out by ticket after the static
+ *                  ranges (0 .. 64, default 6; 0 = static ranges only)
+ *   "static_frac"  share of the work, in 1/256, covered by the static ranges (default 192)
+ * Returns DA_ERR_UNSUPPORTED for an unknown name or a value out of range.
  */
 int decode_attn_set_option(const char *name, int64_t value);
 int64_t decode_attn_get_option(const char *name);

@@ -59,7 +59,7 @@ def lib() -> ctypes.CDLL:
             L.decode_attn_read_device_status.argtypes = [vp, ctypes.POINTER(i32)]
             L.decode_attn_plan.restype = ctypes.c_int
             L.decode_attn_plan.argtypes = [T, i32, i32, i32, i64, ctypes.POINTER(i32), ctypes.POINTER(i32),
-                                           ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
+                                           ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
             L.decode_attn_set_option.restype = ctypes.c_int
             L.decode_attn_set_option.argtypes = [ctypes.c_char_p, i64]
             L.decode_attn_get_option.restype = i64
@@ -212,20 +212,21 @@ def read_device_status(stream: Optional[torch.cuda.Stream] = None):
 
 def plan(seq_lens: torch.Tensor, window: int, Hkv: int, P: int, max_pages: int,
          stream: Optional[torch.cuda.Stream] = None):
-    """Run only the plan kernel; returns (seq_info [B,4], block_work [nblocks,4], tile_tokens) as
-    host int32 tensors: per sequence {lo, L, first_tile, num_tiles}; per thread block
-    {b, kv_head, first tile relative to the pair's first_tile, tiles}."""
+    """Run only the plan kernel; returns (seq_info [B,4], unit_work [units,4], num_static, tile_tokens)
+    as host values: per sequence {lo, L, first_tile, num_tiles}; per work unit
+    {b, kv_head, first tile relative to the pair's first_tile, tiles}.  Units below num_static are
+    the thread blocks' own ranges, the rest are handed out by ticket."""
     B = seq_lens.shape[0]
     with torch.cuda.device(seq_lens.device):
         ensure_workspace(B, 1, Hkv, 128, P, max_pages, seq_lens.device)
-        cap = 4096
+        cap = 8192
         seq_info = torch.zeros((max(B, 1), 4), dtype=torch.int32)
-        block_work = torch.zeros((cap, 4), dtype=torch.int32)
-        nb = ctypes.c_int32(cap)
-        tt = ctypes.c_int32(0)
+        unit_work = torch.zeros((cap, 4), dtype=torch.int32)
+        nu, ns, tt = ctypes.c_int32(cap), ctypes.c_int32(0), ctypes.c_int32(0)
         sv = _view(seq_lens)
+        i32p = ctypes.POINTER(ctypes.c_int32)
         _check(lib().decode_attn_plan(_ref(sv), int(window), int(Hkv), int(P), int(max_pages),
-                                      ctypes.cast(seq_info.data_ptr(), ctypes.POINTER(ctypes.c_int32)),
-                                      ctypes.cast(block_work.data_ptr(), ctypes.POINTER(ctypes.c_int32)),
-                                      ctypes.byref(nb), ctypes.byref(tt), _stream_ptr(stream)))
-    return seq_info[:B], block_work[:nb.value], tt.value
+                                      ctypes.cast(seq_info.data_ptr(), i32p),
+                                      ctypes.cast(unit_work.data_ptr(), i32p),
+                                      ctypes.byref(nu), ctypes.byref(ns), ctypes.byref(tt), _stream_ptr(stream)))
+    return seq_info[:B], unit_work[:nu.value], ns.value, tt.value

@@ -3,11 +3,14 @@
 //
 // Work model.  A "tile" is TILE_T consecutive tokens starting at a multiple of TILE_T.  Sequence b
 // contributes nt_b tiles (those that intersect its attended range [lo_b, L_b)) for each of its Hkv
-// KV heads.  All (b, kv head, tile) units are laid out in row-major order and cut into gridDim.x
-// equal contiguous ranges, one per thread block, so every block streams the same number of bytes
-// whatever the mix of sequence lengths.  A block's range covers a run of (b, kv head) pairs; the
-// pairs it covers completely are written straight to `out`, the (at most two) pairs it shares with
-// its neighbours go to a partial slot and are combined by the merge kernel.
+// KV heads.  All (b, kv head, tile) triples, in row-major order, form one line of `total` tiles.
+// The line is cut into work units: its first part into one large unit per thread block (each block
+// starts on its own, so no block waits for a ticket), the rest into many small units that the
+// blocks take from an atomic ticket counter as they finish -- thread blocks do not all stream at
+// the same speed, and the small units even out their finishing times.  A unit covers a run of
+// (b, kv head) pairs; the pairs it covers completely are written straight to `out`, the (at most
+// two) pairs it shares with neighbouring units go to a partial slot and are combined by the merge
+// kernel.
 #pragma once
 #include "da_ptx.cuh"
 
@@ -21,8 +24,15 @@ constexpr int STAGE_BYTES = 2 * KV_BYTES;   // K tile followed by V tile
 constexpr int NTHREADS = (NCW + 1) * 32;    // + one producer warp
 constexpr int PLAN_THREADS = 1024;
 constexpr int PLAN_SMEM_SEQS = 4096;
+constexpr int MIN_TAIL_UNIT_TILES = 4;      // a ticketed unit is never cut smaller than this
+constexpr int MERGE_BIG = 16;               // pairs cut into more splits are merged by a whole block
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
+
+// flags of a tile's descriptor (written by the producer warp, read by the consumer warps)
+constexpr int TILE_ITEM_END = 1;   // last tile this unit holds of its (b, kv head) pair
+constexpr int TILE_WHOLE = 2;      // the unit holds every tile of the pair: write `out` directly
+constexpr int TILE_STOP = 4;       // no more work for this block (carries no data)
 
 template <int NT8>
 struct PartCfg {
@@ -32,9 +42,26 @@ struct PartCfg {
     static constexpr int STATS_BYTES = 2 * NCW * HEADS * 4;              // (m, l) per warp and head
     static constexpr int OFF_XBUF = NSTAGES * STAGE_BYTES;
     static constexpr int OFF_STATS = OFF_XBUF + XBUF_BYTES;
-    static constexpr int OFF_BARS = OFF_STATS + STATS_BYTES;             // full[NSTAGES], empty[NSTAGES]
-    static constexpr int OFF_FLAGS = OFF_BARS + 2 * NSTAGES * 8;         // abort flag
+    static constexpr int OFF_META = OFF_STATS + STATS_BYTES;             // two int4 per stage
+    static constexpr int OFF_BARS = OFF_META + NSTAGES * 32;             // full[NSTAGES], empty[NSTAGES], epi[2]
+    static constexpr int OFF_FLAGS = OFF_BARS + (2 * NSTAGES + 2) * 8;   // abort flag
     static constexpr int SMEM_BYTES = OFF_FLAGS + 16;
+};
+
+// What the plan kernel decides, read by the other two kernels.  Units 0 .. n_static-1 cut
+// [0, static_w) into near-equal ranges (the first r_static of them one tile longer, q_static + 1);
+// units n_static .. n_static+n_tail-1 cut [static_w, total) the same way.
+struct PlanHeader {
+    long long total;      // tiles over all (b, kv head) pairs
+    long long static_w;   // tiles covered by the n_static large units (the rest: ticketed units)
+    long long q_static, q_tail;   // floor(range / units) of the two cuts
+    int r_static, r_tail;         // remainder of the two cuts
+    int n_static;         // = thread blocks of the partition kernel
+    int n_tail;           // ticketed units (0: none)
+    int ticket;           // next ticketed unit to hand out (reset by the plan kernel)
+    int n_merge_small;    // entries of the two merge lists (pairs cut into <= / > MERGE_BIG splits)
+    int n_merge_big;
+    int pad;
 };
 
 struct PartParams {
@@ -47,9 +74,10 @@ struct PartParams {
     float *lse;
     int64_t l_sb, l_sh;
     const int4 *seq_info;     // {lo, L, first_tile, num_tiles} per sequence
-    const int4 *block_work;   // {b, kv_head, first tile (relative), tiles} per thread block
-    float *part_o;            // [2*gridDim.x][HEADS][128]
-    float *part_lse;          // [2*gridDim.x][HEADS]
+    const int4 *unit_work;    // {b, kv_head, first tile (relative to the pair's first), tiles} per unit
+    PlanHeader *hdr;
+    float *part_o;            // [2 * units][HEADS][128]
+    float *part_lse;          // [2 * units][HEADS]
     int32_t *status;
     int32_t B, Hkv, G, P, box_rows, num_pages, out_bf16;
     float scale_log2;         // scale * log2(e)
@@ -60,22 +88,28 @@ struct PlanParams {
     int64_t sl_stride;
     int4 *seq_info;
     int32_t *prefix;          // [B+1] exclusive prefix of num_tiles
-    int4 *block_work;
+    int4 *unit_work;
+    int32_t *merge_small, *merge_big;   // lists of pair ids b * Hkv + g, one per split pair
+    PlanHeader *hdr;
     int32_t *status;
-    int32_t B, Hkv, P, window, nblocks;
+    int32_t B, Hkv, P, window;
+    int32_t n_static, n_tail_max, static_frac_q8;   // large units; most ticketed units; share of the
+                                                    // line given to the large units, in 1/256
     int64_t max_pages;
 };
 
 struct MergeParams {
     const int4 *seq_info;
     const int32_t *prefix;
+    const PlanHeader *hdr;
+    const int32_t *merge_small, *merge_big;
     const float *part_o;
     const float *part_lse;
     void *out;
     int64_t o_sb, o_sh;
     float *lse;
     int64_t l_sb, l_sh;
-    int32_t B, Hkv, G, heads_pad, nblocks, out_bf16;
+    int32_t B, Hkv, G, heads_pad, out_bf16;
 };
 
 __device__ __forceinline__ void report_status(int32_t *status, int code, int a, int b, int c)
@@ -87,29 +121,59 @@ __device__ __forceinline__ void report_status(int32_t *status, int code, int a, 
     }
 }
 
-// Start of block c's range when `total` units are cut into `n` contiguous near-equal ranges.
-__host__ __device__ __forceinline__ int64_t range_start(int64_t total, int n, int c)
+// Start of range c of a cut with quotient q and remainder r.
+__host__ __device__ __forceinline__ long long cut_start(long long q, int r, int c)
 {
-    const int64_t qq = total / n, rr = total % n;
-    return qq * c + (c < rr ? c : rr);
+    return q * c + (c < r ? c : r);
 }
-// The block whose range holds unit w.
-__host__ __device__ __forceinline__ int range_owner(int64_t total, int n, int64_t w)
+// The range of that cut that holds offset w.
+__host__ __device__ __forceinline__ int cut_owner(long long q, int r, long long w)
 {
-    const int64_t qq = total / n, rr = total % n;
-    const int64_t big = rr * (qq + 1);
-    return (w < big) ? (int)(w / (qq + 1)) : (int)(rr + (w - big) / qq);
+    const long long big = (long long)r * (q + 1);
+    if (w < big)
+        return (q + 1 < 0x7fffffffll && w < 0x7fffffffll) ? (int)((unsigned)w / (unsigned)(q + 1)) : (int)(w / (q + 1));
+    const long long x = w - big;
+    return r + ((q < 0x7fffffffll && x < 0x7fffffffll) ? (int)((unsigned)x / (unsigned)q) : (int)(x / q));
+}
+__host__ __device__ __forceinline__ long long unit_start(const PlanHeader &h, int u)
+{
+    if (u < h.n_static)
+        return cut_start(h.q_static, h.r_static, u);
+    if (u >= h.n_static + h.n_tail)
+        return h.total;
+    return h.static_w + cut_start(h.q_tail, h.r_tail, u - h.n_static);
+}
+__host__ __device__ __forceinline__ int unit_owner(const PlanHeader &h, long long w)
+{
+    if (w < h.static_w)
+        return cut_owner(h.q_static, h.r_static, w);
+    return h.n_static + cut_owner(h.q_tail, h.r_tail, w - h.static_w);
+}
+// Static units that hold tiles: with fewer tiles than thread blocks the last ones are empty.
+__host__ __device__ __forceinline__ int static_units_in_use(const PlanHeader &h)
+{
+    return (int)(h.static_w < h.n_static ? h.static_w : h.n_static);
+}
+// How many units hold a piece of the pair whose tiles are [w0, w0 + nt) (nt > 0), and the first.
+__host__ __device__ __forceinline__ int pair_splits(const PlanHeader &h, long long w0, int nt, int *u_first)
+{
+    const int uf = unit_owner(h, w0), ul = unit_owner(h, w0 + nt - 1);
+    const int n_full = static_units_in_use(h);
+    *u_first = uf;
+    return (ul - uf + 1) - ((uf < n_full && ul >= h.n_static) ? h.n_static - n_full : 0);
 }
 
 // =====================================================================================  plan
-// One block.  Per sequence: attended range, tiles, exclusive prefix of tiles; per thread block of
-// the partition kernel: where its range starts.
+// One block.  Per sequence: attended range, tiles, exclusive prefix of tiles; then the cut of the
+// line into units and, per unit, where it starts.
 __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
 {
     __shared__ int warp_tot[PLAN_THREADS / 32];
     __shared__ int running_s;
     __shared__ int prefix_s[PLAN_SMEM_SEQS + 1];   // copy of the prefix for the searches below
+    __shared__ PlanHeader hdr_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    grid_launch_dependents();   // the partition kernel may set up its blocks while the plan is made
     if (tid == 0)
         running_s = 0;
     __syncthreads();
@@ -170,33 +234,78 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         p.prefix[p.B] = tiles_per_head;
         if (in_smem)
             prefix_s[p.B] = tiles_per_head;
+        // the cut: a share of the line to the large units, the rest to ticketed units of at least
+        // MIN_TAIL_UNIT_TILES tiles each
+        PlanHeader h;
+        h.total = (long long)tiles_per_head * p.Hkv;
+        h.n_static = p.n_static;
+        long long tail_w = h.total * (256 - p.static_frac_q8) / 256;
+        long long n_tail = tail_w / MIN_TAIL_UNIT_TILES;
+        if (n_tail > p.n_tail_max)
+            n_tail = p.n_tail_max;
+        if (n_tail <= 0) {
+            n_tail = 0;
+            tail_w = 0;
+        }
+        h.n_tail = (int)n_tail;
+        h.static_w = h.total - tail_w;
+        h.q_static = h.static_w / h.n_static;
+        h.r_static = (int)(h.static_w % h.n_static);
+        h.q_tail = n_tail ? tail_w / n_tail : 0;
+        h.r_tail = n_tail ? (int)(tail_w % n_tail) : 0;
+        h.ticket = 0;
+        h.n_merge_small = 0;
+        h.n_merge_big = 0;
+        h.pad = 0;
+        hdr_s = h;
     }
     __syncthreads();   // this block's global writes are visible to itself after the barrier
     const int *prefix = in_smem ? prefix_s : p.prefix;
+    const PlanHeader h = hdr_s;
 
-    const int64_t total = (int64_t)tiles_per_head * p.Hkv;
-    for (int c = tid; c < p.nblocks; c += PLAN_THREADS) {
-        const int64_t ws = range_start(total, p.nblocks, c);
-        const int64_t we = range_start(total, p.nblocks, c + 1);
-        int4 bw = make_int4(0, 0, 0, 0);
-        if (we > ws) {
-            const int x = (int)(ws / p.Hkv);
-            // largest b with prefix[b] <= x; equal prefixes (empty sequences) resolve to the last
-            int lo_i = 0, hi_i = p.B;   // invariant: prefix[lo_i] <= x < prefix[hi_i]
-            while (hi_i - lo_i > 1) {
-                const int mid = (lo_i + hi_i) >> 1;
-                if (prefix[mid] <= x)
-                    lo_i = mid;
-                else
-                    hi_i = mid;
+    const int n_units = h.n_static + h.n_tail;
+    const int n_full = static_units_in_use(h);
+    for (int u = tid; u < p.n_static + p.n_tail_max; u += PLAN_THREADS) {
+        int4 uw = make_int4(0, 0, 0, 0);
+        if (u < n_units) {
+            const long long ws = unit_start(h, u), we = unit_start(h, u + 1);
+            if (we > ws) {
+                const long long xq = ws / p.Hkv;
+                const int x = (int)xq;
+                // largest b with prefix[b] <= x; equal prefixes (empty sequences) resolve to the last
+                int lo_i = 0, hi_i = p.B;   // invariant: prefix[lo_i] <= x < prefix[hi_i]
+                while (hi_i - lo_i > 1) {
+                    const int mid = (lo_i + hi_i) >> 1;
+                    if (prefix[mid] <= x)
+                        lo_i = mid;
+                    else
+                        hi_i = mid;
+                }
+                const int b = lo_i;
+                const int nt = prefix[b + 1] - prefix[b];
+                const int rem = (int)(ws - (long long)prefix[b] * p.Hkv);   // < Hkv * nt
+                const int g = rem / nt, rel = rem - g * nt;
+                uw = make_int4(b, g, rel, (int)(we - ws));
+                // A unit that starts inside a pair marks that pair as split.  The pair is listed once,
+                // by the first such unit: the one whose predecessor holds the pair's first tile.
+                if (rel > 0) {
+                    const int prev = (u == h.n_static) ? n_full - 1 : u - 1;
+                    if (unit_start(h, prev) <= ws - rel) {
+                        int uf;
+                        const int ns = pair_splits(h, ws - rel, nt, &uf);
+                        if (ns > MERGE_BIG)
+                            p.merge_big[atomicAdd(&hdr_s.n_merge_big, 1)] = b * p.Hkv + g;
+                        else
+                            p.merge_small[atomicAdd(&hdr_s.n_merge_small, 1)] = b * p.Hkv + g;
+                    }
+                }
             }
-            const int b = lo_i;
-            const int nt = prefix[b + 1] - prefix[b];
-            const int64_t rem = ws - (int64_t)prefix[b] * p.Hkv;
-            bw = make_int4(b, (int)(rem / nt), (int)(rem % nt), (int)(we - ws));
         }
-        p.block_work[c] = bw;
+        p.unit_work[u] = uw;
     }
+    __syncthreads();
+    if (tid == 0)
+        *p.hdr = hdr_s;
 }
 
 // =====================================================================================  partition
@@ -223,9 +332,11 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     float *xbuf = reinterpret_cast<float *>(smem + C::OFF_XBUF);
     float *st_m = reinterpret_cast<float *>(smem + C::OFF_STATS);
     float *st_l = st_m + NCW * HEADS;
+    int4 *meta = reinterpret_cast<int4 *>(smem + C::OFF_META);   // [stage][2]
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAGS);
     const uint32_t bar_full = smem_base + C::OFF_BARS;
     const uint32_t bar_empty = bar_full + NSTAGES * 8;
+    const uint32_t bar_epi = bar_empty + NSTAGES * 8;   // two barriers for the consumers' epilogue
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -240,14 +351,15 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, NCW);
         }
+        mbar_init(bar_epi, NCW);
+        mbar_init(bar_epi + 8, NCW);
         mbar_fence_init();
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
     }
+    grid_launch_dependents();   // lets the merge kernel's blocks become resident early
     __syncthreads();
-
-    const int4 bw = p.block_work[blockIdx.x];
-    int b = bw.x, g = bw.y, rel = bw.z, remaining = bw.w;
+    grid_dependency_wait();     // the plan (and everything before it in the stream) is complete
 
     if (warp == NCW) {
         // ------------------------------------------------------------------ producer warp
@@ -257,40 +369,68 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         const bool active = lane < nboxes * 2;
         const uint32_t box_bytes = (uint32_t)p.box_rows * 256u;
         const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
+        const int n_static = p.hdr->n_static, n_units = n_static + p.hdr->n_tail;
         uint32_t it = 0;
         bool aborted = false;
 
-        // state of the tile whose page id is being fetched ahead
+        // cursor over this block's tiles: unit u, pair (b, g), tile i of cnt
+        int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
+        int b = 0, g = 0, rel = 0, remaining = 0, cnt = 0, i = 0;
         int4 si = make_int4(0, 0, 0, 0);
-        int cnt = 0, i = 0;
-        auto open_pair = [&]() {   // position on the next (b, g) pair that has tiles; false at the end
-            while (remaining > 0) {
-                si = p.seq_info[b];
-                if (si.w > 0) {
-                    cnt = min(si.w - rel, remaining);
-                    i = 0;
+        bool first_item = true;
+        auto take_ticket = [&]() {
+            int t = 0;
+            if (lane == 0)
+                t = atomicAdd(&p.hdr->ticket, 1);
+            t = __shfl_sync(0xffffffffu, t, 0) + n_static;
+            return t < n_units ? t : -1;
+        };
+        auto open_unit = [&]() {   // make u a unit that has tiles, taking tickets past empty ones
+            while (u >= 0) {
+                const int4 uw = p.unit_work[u];
+                if (uw.w > 0) {
+                    b = uw.x; g = uw.y; rel = uw.z; remaining = uw.w;
+                    first_item = true;
                     return true;
                 }
-                ++b;   // an empty sequence (only reachable with g == 0)
+                u = take_ticket();
             }
             return false;
         };
-        auto fetch_page = [&](int &page, int &row, bool &need, int &t0_out, int &g_out, int &b_out) {
-            const int t0 = (si.z + rel + i) * TILE_T;
-            const int tok0 = t0 + box * p.box_rows;
-            need = active && tok0 < si.y && tok0 + p.box_rows > si.x;
-            page = 0;
-            row = tok0 % p.P;
-            if (need)
-                page = __ldg(p.block_table + (int64_t)b * p.bt_sb + tok0 / p.P);
-            t0_out = t0;
-            g_out = g;
-            b_out = b;
+        auto open_pair = [&]() {   // position on the next (b, g) pair that has tiles; false at the end
+            for (;;) {
+                while (remaining > 0) {
+                    si = p.seq_info[b];
+                    if (si.w > 0) {
+                        cnt = min(si.w - rel, remaining);
+                        i = 0;
+                        return true;
+                    }
+                    ++b;   // an empty sequence (only reachable with g == 0)
+                }
+                u = take_ticket();   // this unit is finished
+                if (!open_unit())
+                    return false;
+            }
         };
-        auto advance = [&]() {   // step to the next tile of this block's range
+        struct Tile { int page, row, t0, g, b, lo, L, flags, slot; bool need; };
+        auto fetch = [&](Tile &t) {   // describe the cursor's tile and start its block-table read
+            t.t0 = (si.z + rel + i) * TILE_T;
+            const int tok0 = t.t0 + box * p.box_rows;
+            t.need = active && tok0 < si.y && tok0 + p.box_rows > si.x;
+            t.page = 0;
+            t.row = tok0 % p.P;
+            if (t.need)
+                t.page = __ldg(p.block_table + (int64_t)b * p.bt_sb + tok0 / p.P);
+            t.g = g; t.b = b; t.lo = si.x; t.L = si.y;
+            t.flags = (i == cnt - 1 ? TILE_ITEM_END : 0) | (cnt == si.w ? TILE_WHOLE : 0);
+            t.slot = 2 * u + (first_item ? 0 : 1);
+        };
+        auto advance = [&]() {   // step to the next tile; false when the block has no more work
             if (++i == cnt) {
                 remaining -= cnt;
                 rel = 0;
+                first_item = false;
                 if (++g == p.Hkv) {
                     g = 0;
                     ++b;
@@ -300,40 +440,53 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             return true;
         };
 
-        bool have = open_pair();
-        int page = 0, row = 0, t0 = 0, gg = 0, bb = 0;
-        bool need = false;
+        Tile cur, nxt;
+        bool have = open_unit() && open_pair();
         if (have)
-            fetch_page(page, row, need, t0, gg, bb);
+            fetch(cur);
         while (have) {
             // issue the next tile's block-table read before waiting for a free stage
-            int n_page = 0, n_row = 0, n_t0 = 0, n_g = 0, n_b = 0;
-            bool n_need = false;
             const bool n_have = advance();
             if (n_have)
-                fetch_page(n_page, n_row, n_need, n_t0, n_g, n_b);
+                fetch(nxt);
 
             const int stage = it % NSTAGES;
             const uint32_t phase = (it / NSTAGES) & 1u;
-            if (need && (uint32_t)page >= (uint32_t)p.num_pages) {
-                report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, bb, (t0 + box * p.box_rows) / p.P, page);
-                need = false;   // skip the load; the rows keep whatever the stage held
+            if (cur.need && (uint32_t)cur.page >= (uint32_t)p.num_pages) {
+                report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, cur.b, (cur.t0 + box * p.box_rows) / p.P, cur.page);
+                cur.need = false;   // skip the load; the rows keep whatever the stage held
             }
-            const uint32_t mask = __ballot_sync(0xffffffffu, need);
+            const uint32_t mask = __ballot_sync(0xffffffffu, cur.need);
             if (!mbar_wait_bounded(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) {
                 aborted = true;
                 break;
             }
-            if (lane == 0)
+            if (lane == 0) {
+                meta[2 * stage] = make_int4(cur.b, cur.g, cur.t0, cur.flags);
+                meta[2 * stage + 1] = make_int4(cur.lo, cur.L, cur.slot, 0);
                 mbar_arrive_expect_tx(bar_full + 8 * stage, (uint32_t)__popc(mask) * box_bytes);
+            }
             __syncwarp();
-            if (need) {
+            if (cur.need) {
                 const uint32_t dst = smem_base + stage * STAGE_BYTES + is_v * KV_BYTES + box * box_bytes;
-                tma_load_5d(dst, tm, 0, row, 0, gg, page, bar_full + 8 * stage);
+                tma_load_5d(dst, tm, 0, cur.row, 0, cur.g, cur.page, bar_full + 8 * stage);
             }
             ++it;
             have = n_have;
-            page = n_page; row = n_row; need = n_need; t0 = n_t0; gg = n_g; bb = n_b;
+            cur = nxt;
+        }
+        if (!aborted) {
+            // tell the consumers that nothing follows
+            const int stage = it % NSTAGES;
+            const uint32_t phase = (it / NSTAGES) & 1u;
+            if (mbar_wait_bounded(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) {
+                if (lane == 0) {
+                    meta[2 * stage] = make_int4(0, 0, 0, TILE_STOP);
+                    mbar_arrive(bar_full + 8 * stage);
+                }
+            } else {
+                aborted = true;
+            }
         }
         if (aborted) {
             // Do not leave the block while copies may still land in its shared memory: wait (bounded)
@@ -343,8 +496,6 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -2, (int)blockIdx.x, (int)it);
                 for (uint32_t k = 0; k < (uint32_t)NSTAGES && k < it; ++k) {
                     const uint32_t j = it - 1 - k;
-                    const uint32_t t_start = 0;
-                    (void)t_start;
                     const uint64_t t_begin = globaltimer_ns();
                     while (!mbar_try_wait(bar_full + 8 * (j % NSTAGES), (j / NSTAGES) & 1u)) {
                         if (globaltimer_ns() - t_begin > 1000000000ull)
@@ -357,10 +508,11 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     }
 
     // ---------------------------------------------------------------------- consumer warps
+    // They follow the tile descriptors the producer leaves with each stage.  A failed (timed-out)
+    // wait raises the abort flag and leaves at once; every other wait then gives up quickly too.
     const int r = lane >> 2, c = lane & 3;
-    uint32_t it = 0;
-    bool first_item = true;
-    // per-lane byte offsets used by the ldmatrix address patterns
+    uint32_t it = 0, items = 0;
+    // per-lane offsets used by the ldmatrix address patterns
     const int k_row = 16 * warp + (lane & 7) + ((lane >> 3) & 1) * 8;   // K: matrices 1,3 are rows +8
     const int k_chunk = lane >> 4;                                      //    matrices 2,3 are chunk +1
     const int v_row = 16 * warp + (lane & 7) + (lane >> 4) * 8;         // V: matrices 2,3 are rows +8
@@ -369,18 +521,14 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const uint32_t k_off = row_offset(k_row, p.box_rows), v_off = row_offset(v_row, p.box_rows);
     const uint32_t k_sw = (uint32_t)(k_row & 7), v_sw = (uint32_t)(v_row & 7);
 
-    while (remaining > 0) {
-        const int4 si = p.seq_info[b];
-        if (si.w == 0) {
-            ++b;
-            continue;
+    auto give_up = [&](int where) {
+        if (*abort_flag == 0) {
+            *abort_flag = 1;
+            report_status(p.status, 3 /* DA_DEV_TIMEOUT */, where, (int)blockIdx.x, (int)it);
         }
-        const int lo = si.x, L = si.y;
-        const int cnt = min(si.w - rel, remaining);
-        const bool whole = (cnt == si.w);
-
-        // Q^T fragments (B operand of S^T = K Q^T): lane holds head r, dims 16kk + 2c + {0,1} (+8)
-        uint32_t qf[NT8][8][2];
+    };
+    // Q^T fragments (B operand of S^T = K Q^T): lane holds head r, dims 16kk + 2c + {0,1} (+8)
+    auto load_q = [&](uint32_t (&qf)[NT8][8][2], int b, int g) {
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
             const int head = n * 8 + r;
@@ -392,6 +540,21 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 qf[n][kk][1] = head < p.G ? __ldg(qrow + 8 * kk + 4 + c) : 0u;
             }
         }
+    };
+
+    if (!mbar_wait_bounded(bar_full, 0u, abort_flag)) {
+        give_up(-3);
+        return;
+    }
+    int4 m0 = meta[0], m1 = meta[1];
+    if (m0.w & TILE_STOP)
+        return;
+    uint32_t qf[NT8][8][2];
+    load_q(qf, m0.x, m0.y);
+
+    for (;;) {   // one (b, kv head) item per iteration
+        const int b = m0.x, g = m0.y, lo = m1.x, L = m1.y, slot = m1.z;
+        const bool whole = (m0.w & TILE_WHOLE) != 0;
         float m_run[NT8][2], l_run[NT8][2], o[NT8][8][4];
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
@@ -402,18 +565,11 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 o[n][j][0] = o[n][j][1] = o[n][j][2] = o[n][j][3] = 0.f;
         }
 
-        for (int i = 0; i < cnt; ++i, ++it) {
+        for (;;) {   // the item's tiles; (m0, m1) describe the tile in stage it % NSTAGES, already full
             const int stage = it % NSTAGES;
-            const uint32_t phase = (it / NSTAGES) & 1u;
-            const int a = (si.z + rel + i) * TILE_T + 16 * warp;   // first token of this warp's rows
+            const int a = m0.z + 16 * warp;   // first token of this warp's rows
             const int v_lo = max(a, lo), v_hi = min(a + 16, L);
-            if (!mbar_wait_bounded(bar_full + 8 * stage, phase, abort_flag)) {
-                // results are void from here on; keep walking so that every barrier below is still met
-                if (*abort_flag == 0) {
-                    *abort_flag = 1;
-                    report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -3, (int)blockIdx.x, (int)it);
-                }
-            }
+            const bool item_end = (m0.w & TILE_ITEM_END) != 0;
             if (v_lo < v_hi) {
                 const uint32_t k_base = smem_base + stage * STAGE_BYTES;
                 const uint32_t v_base = k_base + KV_BYTES;
@@ -425,7 +581,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         const int rr = e >> 4, ch = e & 15;
                         const int t = a + rr;
                         if (t < v_lo || t >= v_hi) {
-                            const uint32_t addr = v_base + row_offset(16 * warp + rr, p.box_rows) + (ch >> 3) * plane_bytes + ((ch & 7) << 4);
+                            const uint32_t addr = v_base + row_offset(16 * warp + rr, p.box_rows) +
+                                                  (ch >> 3) * plane_bytes + ((ch & 7) << 4);
                             asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
                         }
                     }
@@ -524,7 +681,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     uint32_t vf[4];
-                    ldmatrix_x4_trans(vf, v_base + v_off + (j >> 2) * plane_bytes + ((((2 * j + v_chunk) & 7) ^ v_sw) << 4));
+                    ldmatrix_x4_trans(vf, v_base + v_off + (j >> 2) * plane_bytes +
+                                              ((((2 * j + v_chunk) & 7) ^ v_sw) << 4));
 #pragma unroll
                     for (int n = 0; n < NT8; ++n) {
                         mma_bf16_16816(o[n][j], vf, ph[n][0], ph[n][1]);
@@ -537,9 +695,25 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_empty + 8 * stage);
+            ++it;
+            // the next tile (of this item, or the first of the next one, or the stop mark)
+            const int nstage = it % NSTAGES;
+            if (!mbar_wait_bounded(bar_full + 8 * nstage, (it / NSTAGES) & 1u, abort_flag)) {
+                give_up(-3);
+                return;
+            }
+            m0 = meta[2 * nstage];
+            m1 = meta[2 * nstage + 1];
+            if (item_end)
+                break;
         }
 
-        // ---- combine the four warps' (m, l, O) and write the pair's result or partial
+        // ---- the item is complete.  Start the next item's Q loads, then combine the four warps'
+        //      (m, l, O) and write the pair's result or partial.
+        const bool stop = (m0.w & TILE_STOP) != 0;
+        uint32_t qn[NT8][8][2];
+        if (!stop)
+            load_q(qn, m0.x, m0.y);
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
 #pragma unroll
@@ -564,10 +738,15 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 xb[HEAD_DIM + d1] = o[n][j][3];
             }
         }
-        named_barrier_sync(1, NCW * 32);
+        __syncwarp();
+        if (lane == 0)
+            mbar_arrive(bar_epi);
+        if (!mbar_wait_bounded(bar_epi, items & 1u, abort_flag)) {
+            give_up(-4);
+            return;
+        }
         {
             const int d = tid;   // 0..127
-            const int slot = 2 * (int)blockIdx.x + (first_item ? 0 : 1);
             for (int head = 0; head < p.G; ++head) {
                 float M = st_m[head];
 #pragma unroll
@@ -599,38 +778,67 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 }
             }
         }
-        named_barrier_sync(1, NCW * 32);
-
-        first_item = false;
-        remaining -= cnt;
-        rel = 0;
-        if (++g == p.Hkv) {
-            g = 0;
-            ++b;
+        __syncwarp();
+        if (lane == 0)
+            mbar_arrive(bar_epi + 8);
+        if (!mbar_wait_bounded(bar_epi + 8, items & 1u, abort_flag)) {
+            give_up(-5);
+            return;
         }
+        ++items;
+        if (stop)
+            return;
+#pragma unroll
+        for (int n = 0; n < NT8; ++n)
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                qf[n][kk][0] = qn[n][kk][0];
+                qf[n][kk][1] = qn[n][kk][1];
+            }
     }
 }
 
 // =====================================================================================  merge
-// One block per (sequence, KV head); thread = (head of the group, four head_dim columns).  Pairs
-// that a single thread block covered were already written by the partition kernel; empty sequences
-// get out = 0 and lse = -inf; the rest are combined from their partial slots, one split at a time:
+// A fixed, small grid.  Its work comes from the two lists of split pairs the plan kernel made
+// (pairs that one unit covered were already written by the partition kernel) and from the empty
+// sequences, which get out = 0 and lse = -inf.  Partials of a (pair, head) are folded one at a time,
 //   M' = max(M, lse_s);  acc = acc * exp(M - M') + exp(lse_s - M') * O_s;  den likewise;
-//   out = acc / den;  lse = M + ln den.
+//   out = acc / den;  lse = M + ln den,
+// by one warp for a pair of the "small" list (each lane owns four head_dim columns), by all eight
+// warps of a block for a pair of the "big" list (warp k folds splits k, k + 8, ..., then warp 0
+// folds the eight results through shared memory).
 constexpr int MERGE_LANES = HEAD_DIM / 4;
+constexpr int MERGE_WARPS = 8;
+constexpr int MERGE_THREADS = MERGE_WARPS * MERGE_LANES;
 
-__global__ void __launch_bounds__(16 * MERGE_LANES) merge_kernel(const MergeParams p)
+struct MergeAcc {
+    float M, den;
+    float4 acc;
+};
+__device__ __forceinline__ void merge_fold(MergeAcc &a, float l, float w_den, const float4 &o)
 {
-    const int b = blockIdx.x / p.Hkv, g = blockIdx.x % p.Hkv;
-    const int head = threadIdx.x / MERGE_LANES, d = (threadIdx.x % MERGE_LANES) * 4;
-    if (head >= p.G)
-        return;
-    const int4 si = p.seq_info[b];
-    const int tiles_before = p.prefix[b], tiles_all = p.prefix[p.B];
-    const int nt = si.w;
-    const int h = g * p.G + head;
+    const float m_new = fmaxf(a.M, l);
+    const float sc = (a.M == -INFINITY) ? 0.f : __expf(a.M - m_new);
+    const float w = __expf(l - m_new);
+    a.acc.x = a.acc.x * sc + w * o.x;
+    a.acc.y = a.acc.y * sc + w * o.y;
+    a.acc.z = a.acc.z * sc + w * o.z;
+    a.acc.w = a.acc.w * sc + w * o.w;
+    a.den = a.den * sc + w * w_den;
+    a.M = m_new;
+}
 
-    auto store = [&](float4 v, float lse_val) {
+__global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const MergeParams p)
+{
+    __shared__ float4 s_acc[MERGE_WARPS][MERGE_LANES];
+    __shared__ float s_m[MERGE_WARPS], s_den[MERGE_WARPS];
+    const int warp = threadIdx.x / MERGE_LANES, ln = threadIdx.x % MERGE_LANES, d = ln * 4;
+    grid_dependency_wait();     // partials and the plan are complete and visible
+    const PlanHeader hdr = *p.hdr;
+    const int n_full = static_units_in_use(hdr);
+    const int gap = hdr.n_static - n_full;
+
+    auto store = [&](int b, int h, float4 v, float lse_val) {
         const int64_t at = (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d;
         if (p.out_bf16) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
@@ -649,42 +857,70 @@ __global__ void __launch_bounds__(16 * MERGE_LANES) merge_kernel(const MergePara
                 o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
             }
         }
-        if (d == 0 && p.lse)
+        if (ln == 0 && p.lse)
             p.lse[(int64_t)b * p.l_sb + (int64_t)h * p.l_sh] = lse_val;
     };
-
-    if (nt == 0) {
-        store(make_float4(0.f, 0.f, 0.f, 0.f), -INFINITY);
-        return;
-    }
-    const int64_t total = (int64_t)tiles_all * p.Hkv;
-    const int64_t w0 = (int64_t)tiles_before * p.Hkv + (int64_t)g * nt;
-    const int c_first = range_owner(total, p.nblocks, w0);
-    const int c_last = range_owner(total, p.nblocks, w0 + nt - 1);
-    if (c_first == c_last)
-        return;
-    // the pair is the first item of every block but possibly c_first, where it is the first item
-    // only if that block's range starts exactly at the pair
-    const int slot_first = 2 * c_first + (range_start(total, p.nblocks, c_first) == w0 ? 0 : 1);
-    float M = -INFINITY, den = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    // fold splits first, first + stride, ... of (pair, head) into a
+    auto fold_splits = [&](MergeAcc &a, int pair, int head, int first, int stride, int *nsplit_out) {
+        const int b = pair / p.Hkv, g = pair % p.Hkv;
+        const int nt = p.seq_info[b].w;
+        const long long w0 = (long long)p.prefix[b] * p.Hkv + (long long)g * nt;
+        int u_first;
+        const int nsplit = pair_splits(hdr, w0, nt, &u_first);
+        *nsplit_out = nsplit;
+        // the pair is the first item of every unit but possibly u_first, where it is the first item
+        // only if that unit starts exactly at the pair
+        const int slot_first = 2 * u_first + (unit_start(hdr, u_first) == w0 ? 0 : 1);
 #pragma unroll 4
-    for (int cc = c_first; cc <= c_last; ++cc) {
-        const int slot = (cc == c_first) ? slot_first : 2 * cc;
-        const float l = p.part_lse[(int64_t)slot * p.heads_pad + head];
-        const float4 o = *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)slot * p.heads_pad + head) * HEAD_DIM + d);
-        const float m_new = fmaxf(M, l);
-        const float sc = (M == -INFINITY) ? 0.f : __expf(M - m_new);
-        const float w = __expf(l - m_new);
-        acc.x = acc.x * sc + w * o.x;
-        acc.y = acc.y * sc + w * o.y;
-        acc.z = acc.z * sc + w * o.z;
-        acc.w = acc.w * sc + w * o.w;
-        den = den * sc + w;
-        M = m_new;
+        for (int k = first; k < nsplit; k += stride) {
+            int uu = u_first + k;
+            if (u_first < n_full && uu >= n_full)
+                uu += gap;   // skip the static units that hold no tiles
+            const int slot = (k == 0) ? slot_first : 2 * uu;
+            const float l = p.part_lse[(int64_t)slot * p.heads_pad + head];
+            const float4 o = *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)slot * p.heads_pad + head) * HEAD_DIM + d);
+            merge_fold(a, l, 1.f, o);
+        }
+    };
+
+    // ---- pairs with many splits: one (pair, head) per block at a time
+    for (int item = blockIdx.x; item < hdr.n_merge_big * p.G; item += gridDim.x) {
+        const int pair = p.merge_big[item / p.G], head = item % p.G;
+        MergeAcc a = {-INFINITY, 0.f, make_float4(0.f, 0.f, 0.f, 0.f)};
+        int nsplit;
+        fold_splits(a, pair, head, warp, MERGE_WARPS, &nsplit);
+        s_acc[warp][ln] = a.acc;
+        if (ln == 0) {
+            s_m[warp] = a.M;
+            s_den[warp] = a.den;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            for (int k = 1; k < MERGE_WARPS && k < nsplit; ++k)
+                merge_fold(a, s_m[k], s_den[k], s_acc[k][ln]);
+            const float inv = 1.f / a.den;
+            store(pair / p.Hkv, (pair % p.Hkv) * p.G + head,
+                  make_float4(a.acc.x * inv, a.acc.y * inv, a.acc.z * inv, a.acc.w * inv), a.M + __logf(a.den));
+        }
+        __syncthreads();
     }
-    const float inv = 1.f / den;
-    store(make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv), M + __logf(den));
+    // ---- pairs with few splits: one (pair, head) per warp
+    for (int item = blockIdx.x * MERGE_WARPS + warp; item < hdr.n_merge_small * p.G; item += gridDim.x * MERGE_WARPS) {
+        const int pair = p.merge_small[item / p.G], head = item % p.G;
+        MergeAcc a = {-INFINITY, 0.f, make_float4(0.f, 0.f, 0.f, 0.f)};
+        int nsplit;
+        fold_splits(a, pair, head, 0, 1, &nsplit);
+        const float inv = 1.f / a.den;
+        store(pair / p.Hkv, (pair % p.Hkv) * p.G + head,
+              make_float4(a.acc.x * inv, a.acc.y * inv, a.acc.z * inv, a.acc.w * inv), a.M + __logf(a.den));
+    }
+    // ---- empty sequences
+    for (int b = blockIdx.x; b < p.B; b += gridDim.x) {
+        if (p.seq_info[b].w != 0)
+            continue;
+        for (int h = warp; h < p.Hkv * p.G; h += MERGE_WARPS)
+            store(b, h, make_float4(0.f, 0.f, 0.f, 0.f), -INFINITY);
+    }
 }
 
 }  // namespace da

@@ -129,6 +129,15 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may start while the
+// kernel before it in the stream is still running; it must not touch that kernel's results before
+// grid_dependency_wait() returns (which is when the earlier grid has completed and its writes are
+// visible).  The earlier kernel lets its successor start by calling grid_launch_dependents().
+// Both are no-ops when the launch has no such dependency.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- scalar helpers
 __device__ __forceinline__ float fast_exp2(float x)
 {

@@ -19,12 +19,15 @@ using namespace da;
 constexpr int kVersion = 100;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
+constexpr int kMaxUnits = 8192;
 constexpr int kMaxGroup = 16;
 
 std::mutex g_mu;
 std::atomic<int> g_last_cuda_error{0};
 std::atomic<int64_t> g_launches{0};
 int64_t g_opt_grid_blocks = 0;   // 0 = two blocks per SM
+int64_t g_opt_tail_units = 6;    // ticketed units per thread block (0: one static range per block only)
+int64_t g_opt_static_frac = 192; // share of the work given to the static ranges, in 1/256
 cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 struct DeviceState {
@@ -100,12 +103,21 @@ int grid_blocks_for(const DeviceState *st)
     return (int)n;
 }
 
+// Ticketed units for a grid of nblocks (all units together stay within kMaxUnits).
+int tail_units_for(int nblocks)
+{
+    int64_t t = g_opt_tail_units * (int64_t)nblocks;
+    if (t + nblocks > kMaxUnits) t = kMaxUnits - nblocks;
+    return t > 0 ? (int)t : 0;
+}
+
 struct WsLayout {
-    size_t status, seq_info, prefix, block_work, part_lse, part_o;
+    size_t status, hdr, seq_info, prefix, unit_work, merge_small, merge_big, part_lse, part_o;
     size_t stg_q, stg_bt, stg_sl, stg_out, stg_lse, total;
 };
 
-WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int nblocks)
+// `units` = thread blocks of the partition kernel x (1 + ticketed units per block)
+WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int units)
 {
     WsLayout w;
     size_t off = 0;
@@ -115,11 +127,14 @@ WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int nblo
         return at;
     };
     w.status = take(16);
+    w.hdr = take(sizeof(PlanHeader));
     w.seq_info = take((size_t)B * 16);
     w.prefix = take((size_t)(B + 1) * 4);
-    w.block_work = take((size_t)nblocks * 16);
-    w.part_lse = take((size_t)2 * nblocks * kMaxGroup * 4);
-    w.part_o = take((size_t)2 * nblocks * kMaxGroup * HEAD_DIM * 4);
+    w.unit_work = take((size_t)units * 16);
+    w.merge_small = take((size_t)units * 4);
+    w.merge_big = take((size_t)units * 4);
+    w.part_lse = take((size_t)2 * units * kMaxGroup * 4);
+    w.part_o = take((size_t)2 * units * kMaxGroup * HEAD_DIM * 4);
     w.stg_q = take((size_t)B * Hq * D * 2);
     w.stg_bt = take((size_t)B * max_pages * 4);
     w.stg_sl = take((size_t)B * 4);
@@ -252,20 +267,25 @@ int set_kernel_attrs()
 }
 
 int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws, const WsLayout &lay, int nblocks,
-                cudaStream_t stream)
+                int n_tail, cudaStream_t stream)
 {
     PlanParams pp;
     pp.seq_lens = static_cast<const int32_t *>(sl->data);
     pp.sl_stride = sl->stride[0];
     pp.seq_info = reinterpret_cast<int4 *>(ws + lay.seq_info);
     pp.prefix = reinterpret_cast<int32_t *>(ws + lay.prefix);
-    pp.block_work = reinterpret_cast<int4 *>(ws + lay.block_work);
+    pp.unit_work = reinterpret_cast<int4 *>(ws + lay.unit_work);
+    pp.merge_small = reinterpret_cast<int32_t *>(ws + lay.merge_small);
+    pp.merge_big = reinterpret_cast<int32_t *>(ws + lay.merge_big);
+    pp.hdr = reinterpret_cast<PlanHeader *>(ws + lay.hdr);
     pp.status = reinterpret_cast<int32_t *>(ws + lay.status);
     pp.B = (int32_t)d.B;
     pp.Hkv = (int32_t)d.Hkv;
     pp.P = (int32_t)d.P;
     pp.window = window;
-    pp.nblocks = nblocks;
+    pp.n_static = nblocks;
+    pp.n_tail_max = n_tail;
+    pp.static_frac_q8 = (int32_t)g_opt_static_frac;
     pp.max_pages = d.max_pages;
     plan_kernel<<<1, PLAN_THREADS, 0, stream>>>(pp);
     g_launches.fetch_add(1);
@@ -275,7 +295,8 @@ int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws,
 
 // The three launches of the hot path, with every scratch array taken from `ws` as laid out by `lay`.
 // Called with g_mu held.
-int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay, int nblocks, const da_tensor *q,
+int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay, int nblocks, int n_tail,
+                const da_tensor *q,
                 const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl, int32_t window,
                 float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream)
 {
@@ -294,7 +315,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     rc = get_tmap(v, box_rows, &tm_v);
     if (rc != DA_OK) return rc;
 
-    rc = launch_plan(sl, window, d, ws, lay, nblocks, stream);
+    rc = launch_plan(sl, window, d, ws, lay, nblocks, n_tail, stream);
     if (rc != DA_OK) return rc;
 
     PartParams pa;
@@ -310,7 +331,8 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pa.l_sb = lse ? lse->stride[0] : 0;
     pa.l_sh = lse ? lse->stride[1] : 0;
     pa.seq_info = reinterpret_cast<const int4 *>(ws + lay.seq_info);
-    pa.block_work = reinterpret_cast<const int4 *>(ws + lay.block_work);
+    pa.unit_work = reinterpret_cast<const int4 *>(ws + lay.unit_work);
+    pa.hdr = reinterpret_cast<PlanHeader *>(ws + lay.hdr);
     pa.part_o = reinterpret_cast<float *>(ws + lay.part_o);
     pa.part_lse = reinterpret_cast<float *>(ws + lay.part_lse);
     pa.status = reinterpret_cast<int32_t *>(ws + lay.status);
@@ -325,17 +347,35 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     const int nt8 = d.G <= 8 ? 1 : 2;
     const bool timed = g_ev_before && g_ev_after;
     if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
-    if (nt8 == 1)
-        partition_kernel<1><<<nblocks, NTHREADS, PartCfg<1>::SMEM_BYTES, stream>>>(tm_k, tm_v, pa);
-    else
-        partition_kernel<2><<<nblocks, NTHREADS, PartCfg<2>::SMEM_BYTES, stream>>>(tm_k, tm_v, pa);
+    // Both dependent kernels are launched with programmatic stream serialization: their blocks may
+    // become resident while the kernel before them still runs, and they wait on the device
+    // (griddepcontrol.wait) before touching its results.
+    cudaLaunchAttribute pdl;
+    pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((unsigned)nblocks);
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.stream = stream;
+    cfg.attrs = &pdl;
+    cfg.numAttrs = 1;
+    if (nt8 == 1) {
+        cfg.dynamicSmemBytes = PartCfg<1>::SMEM_BYTES;
+        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<1>, tm_k, tm_v, pa));
+    } else {
+        cfg.dynamicSmemBytes = PartCfg<2>::SMEM_BYTES;
+        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<2>, tm_k, tm_v, pa));
+    }
     g_launches.fetch_add(1);
-    DA_CUDA(cudaGetLastError());
     if (timed) DA_CUDA(cudaEventRecord(g_ev_after, stream));
 
     MergeParams mp;
     mp.seq_info = pa.seq_info;
     mp.prefix = reinterpret_cast<const int32_t *>(ws + lay.prefix);
+    mp.hdr = pa.hdr;
+    mp.merge_small = reinterpret_cast<const int32_t *>(ws + lay.merge_small);
+    mp.merge_big = reinterpret_cast<const int32_t *>(ws + lay.merge_big);
     mp.part_o = pa.part_o;
     mp.part_lse = pa.part_lse;
     mp.out = out->data;
@@ -348,11 +388,12 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     mp.Hkv = pa.Hkv;
     mp.G = pa.G;
     mp.heads_pad = nt8 * 8;
-    mp.nblocks = nblocks;
     mp.out_bf16 = pa.out_bf16;
-    merge_kernel<<<(unsigned)(d.B * d.Hkv), (unsigned)(nt8 * 8 * MERGE_LANES), 0, stream>>>(mp);
+    cfg.gridDim = dim3((unsigned)(4 * st->sm_count));
+    cfg.blockDim = dim3((unsigned)MERGE_THREADS);
+    cfg.dynamicSmemBytes = 0;
+    DA_CUDA(cudaLaunchKernelEx(&cfg, merge_kernel, mp));
     g_launches.fetch_add(1);
-    DA_CUDA(cudaGetLastError());
     return DA_OK;
 }
 
@@ -369,11 +410,12 @@ int run(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_ten
     rc = current_device(&dev, &st);
     if (rc != DA_OK) return rc;
     const int nblocks = grid_blocks_for(st);
-    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks);
+    const int n_tail = tail_units_for(nblocks);
+    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks + n_tail);
     if (!st->ws || st->ws_bytes < lay.stg_q) return DA_ERR_WORKSPACE;   // staging is only for host_io
     if (d.B == 0) return DA_OK;
-    return launch_path(st, d, static_cast<uint8_t *>(st->ws), lay, nblocks, q, k, v, bt, sl, window, scale, out, lse,
-                       stream);
+    return launch_path(st, d, static_cast<uint8_t *>(st->ws), lay, nblocks, n_tail, q, k, v, bt, sl, window, scale,
+                       out, lse, stream);
 }
 
 bool contiguous(const da_tensor *t)
@@ -415,7 +457,8 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
         DeviceState *st;
         rc = current_device(&dev, &st);
         if (rc != DA_OK) return rc;
-        lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, grid_blocks_for(st));
+        const int nb = grid_blocks_for(st);
+        lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nb + tail_units_for(nb));
         if (!st->ws || st->ws_bytes < lay.total) return DA_ERR_WORKSPACE;
         ws = static_cast<uint8_t *>(st->ws);
     }
@@ -471,8 +514,9 @@ int decode_attn_static_scratch(const da_tensor *q, const da_tensor *k_pages, con
     // the array keeps the previous call's contents; only the status record has to start at zero
     DA_CUDA(cudaMemsetAsync(ws + lay.status, 0, 16, stream));
     if (d.B > 0) {
-        rc = launch_path(st, d, ws, lay, nblocks, q, k_pages, v_pages, block_table, seq_lens, window, scale, out, lse,
-                         stream);
+        // one static range per thread block, no ticketed units: keeps the partial slots within the array
+        rc = launch_path(st, d, ws, lay, nblocks, 0, q, k_pages, v_pages, block_table, seq_lens, window, scale, out,
+                         lse, stream);
         if (rc != DA_OK) return rc;
     }
     if (dev_status4)
@@ -491,7 +535,7 @@ size_t decode_attn_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t D
     int nblocks = g_opt_grid_blocks > 0 ? (int)g_opt_grid_blocks : kMaxGridBlocks;
     if (g_opt_grid_blocks <= 0 && current_device(&dev, &st) == DA_OK)
         nblocks = grid_blocks_for(st);
-    return ws_layout(B, Hq, D, max_pages, nblocks).total;
+    return ws_layout(B, Hq, D, max_pages, nblocks + tail_units_for(nblocks)).total;
 }
 
 int decode_attn_set_workspace(void *dev_ptr, size_t bytes)
@@ -536,10 +580,10 @@ int decode_attn_read_device_status(void *stream_, int32_t *host_status4)
 }
 
 int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int32_t P, int64_t max_pages,
-                     int32_t *host_seq_info, int32_t *host_block_work, int32_t *num_blocks, int32_t *tile_tokens,
-                     void *stream_)
+                     int32_t *host_seq_info, int32_t *host_unit_work, int32_t *num_units, int32_t *num_static,
+                     int32_t *tile_tokens, void *stream_)
 {
-    if (!seq_lens || !seq_lens->data || !host_seq_info || !host_block_work || !num_blocks || !tile_tokens)
+    if (!seq_lens || !seq_lens->data || !host_seq_info || !host_unit_work || !num_units || !num_static || !tile_tokens)
         return DA_ERR_NULL;
     if (seq_lens->dtype != DA_I32) return DA_ERR_DTYPE;
     if (seq_lens->ndim != 1 || Hkv <= 0 || max_pages <= 0) return DA_ERR_SHAPE;
@@ -551,23 +595,29 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
     int rc = current_device(&dev, &st);
     if (rc != DA_OK) return rc;
     const int nblocks = grid_blocks_for(st);
+    const int n_tail = tail_units_for(nblocks);
     Dims d;
     d.B = seq_lens->shape[0];
     d.Hkv = Hkv;
     d.P = P;
     d.max_pages = max_pages;
-    const WsLayout lay = ws_layout(d.B, 1, HEAD_DIM, max_pages, nblocks);
+    const WsLayout lay = ws_layout(d.B, 1, HEAD_DIM, max_pages, nblocks + n_tail);
     if (!st->ws || st->ws_bytes < lay.part_lse) return DA_ERR_WORKSPACE;
-    if (*num_blocks < nblocks) return DA_ERR_SHAPE;
-    *num_blocks = nblocks;
+    if (*num_units < nblocks + n_tail) return DA_ERR_SHAPE;
+    *num_units = 0;
+    *num_static = nblocks;
     *tile_tokens = TILE_T;
     if (d.B == 0) return DA_OK;
     uint8_t *ws = static_cast<uint8_t *>(st->ws);
-    rc = launch_plan(seq_lens, window, d, ws, lay, nblocks, stream);
+    rc = launch_plan(seq_lens, window, d, ws, lay, nblocks, n_tail, stream);
     if (rc != DA_OK) return rc;
+    PlanHeader h;
+    DA_CUDA(cudaMemcpyAsync(&h, ws + lay.hdr, sizeof h, cudaMemcpyDeviceToHost, stream));
     DA_CUDA(cudaMemcpyAsync(host_seq_info, ws + lay.seq_info, (size_t)d.B * 16, cudaMemcpyDeviceToHost, stream));
-    DA_CUDA(cudaMemcpyAsync(host_block_work, ws + lay.block_work, (size_t)nblocks * 16, cudaMemcpyDeviceToHost, stream));
+    DA_CUDA(cudaMemcpyAsync(host_unit_work, ws + lay.unit_work, (size_t)(nblocks + n_tail) * 16, cudaMemcpyDeviceToHost,
+                            stream));
     DA_CUDA(cudaStreamSynchronize(stream));
+    *num_units = h.n_static + h.n_tail;
     return DA_OK;
 }
 
@@ -580,6 +630,16 @@ int decode_attn_set_option(const char *name, int64_t value)
         g_opt_grid_blocks = value;
         return DA_OK;
     }
+    if (std::strcmp(name, "tail_units") == 0) {
+        if (value < 0 || value > 64) return DA_ERR_UNSUPPORTED;
+        g_opt_tail_units = value;
+        return DA_OK;
+    }
+    if (std::strcmp(name, "static_frac") == 0) {
+        if (value < 0 || value > 256) return DA_ERR_UNSUPPORTED;
+        g_opt_static_frac = value;
+        return DA_OK;
+    }
     return DA_ERR_UNSUPPORTED;
 }
 
@@ -588,6 +648,8 @@ int64_t decode_attn_get_option(const char *name)
     if (!name) return -1;
     std::lock_guard<std::mutex> lock(g_mu);
     if (std::strcmp(name, "grid_blocks") == 0) return g_opt_grid_blocks;
+    if (std::strcmp(name, "tail_units") == 0) return g_opt_tail_units;
+    if (std::strcmp(name, "static_frac") == 0) return g_opt_static_frac;
     return -1;
 }
 

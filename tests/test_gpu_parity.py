@@ -21,6 +21,8 @@ def da():
     pkg.lib()
     yield pkg
     pkg.set_option("grid_blocks", 0)
+    pkg.set_option("tail_units", 6)
+    pkg.set_option("static_frac", 192)
 
 
 def oracle_of(case):
@@ -106,6 +108,21 @@ def test_any_split_schedule_gives_the_same_answer(da, grid):
     base, base_lse = gpu_of(da, case)
     np.testing.assert_allclose(got, base, atol=2e-5, rtol=1e-5)
     np.testing.assert_allclose(got_lse, base_lse, atol=2e-5, rtol=1e-5)
+
+
+@pytest.mark.parametrize("tail,frac", [(0, 192), (1, 128), (6, 0), (6, 256), (20, 64), (64, 200)])
+def test_any_mix_of_static_and_ticketed_units_gives_the_same_answer(da, tail, frac):
+    case = workloads.build_case("units", [2500, 3, 900, 0, 64, 4097, 130, 9000], 16, 13, "cpu", window=0)
+    try:
+        da.set_option("tail_units", tail)
+        da.set_option("static_frac", frac)
+        for grid in (0, 5, 64):
+            check(da, case, f"tail={tail} frac={frac} grid={grid}", grid)
+        case.window = 700
+        check(da, case, f"tail={tail} frac={frac} window", 0)
+    finally:
+        da.set_option("tail_units", 6)
+        da.set_option("static_frac", 192)
 
 
 @pytest.mark.parametrize("B", [1, 2, 3, 7])
@@ -266,11 +283,16 @@ def test_integer_mean_is_exact(da):
     vi = torch.randint(-8, 9, case.v_pages.shape, generator=torch.Generator().manual_seed(1)).to(torch.bfloat16)
     case.v_pages = torch.where(torch.isfinite(case.v_pages), vi, case.v_pages)
     ref, ref_lse = oracle_of(case)
-    da.set_option("grid_blocks", 1)
-    got, got_lse = gpu_of(da, case)
-    assert np.array_equal(got, ref)
-    np.testing.assert_allclose(got_lse, ref_lse, atol=1e-6)
-    da.set_option("grid_blocks", 0)
+    try:
+        # one thread block, one unit: no split, so every sum is a sum of small integers
+        da.set_option("grid_blocks", 1)
+        da.set_option("tail_units", 0)
+        got, got_lse = gpu_of(da, case)
+        assert np.array_equal(got, ref)
+        np.testing.assert_allclose(got_lse, ref_lse, atol=1e-6)
+    finally:
+        da.set_option("grid_blocks", 0)
+        da.set_option("tail_units", 6)
     got, _ = gpu_of(da, case)
     np.testing.assert_allclose(got, ref, atol=1e-6)
 
@@ -293,36 +315,47 @@ def test_nan_canaries(da):
 def test_plan_covers_every_attended_token_exactly_once(da, window):
     lens = np.concatenate([workloads.lengths_c2(1, 20), [0, 1, 64, 65]])
     sl = torch.tensor(lens, dtype=torch.int32, device="cuda")
-    for grid in (0, 1, 7, 1000):
-        da.set_option("grid_blocks", grid)
-        seq_info, block_work, T = da.plan(sl, window, 8, 16, 2048)
-        si = seq_info.numpy()
-        for b, L in enumerate(lens):
-            lo = L - window if 0 < window < L else 0
-            assert si[b, 0] == lo and si[b, 1] == L
-            if L > 0:
-                assert si[b, 2] == lo // T and si[b, 3] == (L - 1) // T - lo // T + 1
+    try:
+        for grid, tail in ((0, 6), (1, 0), (7, 3), (1000, 1), (0, 0)):
+            da.set_option("grid_blocks", grid)
+            da.set_option("tail_units", tail)
+            seq_info, unit_work, n_static, T = da.plan(sl, window, 8, 16, 2048)
+            si = seq_info.numpy()
+            for b, L in enumerate(lens):
+                lo = L - window if 0 < window < L else 0
+                assert si[b, 0] == lo and si[b, 1] == L
+                if L > 0:
+                    assert si[b, 2] == lo // T and si[b, 3] == (L - 1) // T - lo // T + 1
+                else:
+                    assert si[b, 3] == 0
+            covered = np.zeros((len(lens), 8, int(si[:, 3].max()) + 1), dtype=np.int32)
+            sizes = []
+            for b0, g0, rel0, n in unit_work.numpy():
+                sizes.append(int(n))
+                b, g, rel = int(b0), int(g0), int(rel0)
+                while n > 0:
+                    while si[b, 3] == 0:
+                        b += 1
+                    take = min(si[b, 3] - rel, n)
+                    covered[b, g, rel:rel + take] += 1
+                    n -= take
+                    rel = 0
+                    g += 1
+                    if g == 8:
+                        g, b = 0, b + 1
+            for b in range(len(lens)):
+                assert (covered[b, :, :si[b, 3]] == 1).all() and (covered[b, :, si[b, 3]:] == 0).all()
+            assert n_static == (grid if grid else 2 * torch.cuda.get_device_properties(0).multi_processor_count)
+            assert len(sizes) <= n_static * (1 + tail)
+            # equal work within the static ranges and within the ticketed units
+            assert max(sizes[:n_static]) - min(sizes[:n_static]) <= 1
+            if len(sizes) > n_static:
+                assert max(sizes[n_static:]) - min(sizes[n_static:]) <= 1 and min(sizes[n_static:]) >= 4
             else:
-                assert si[b, 3] == 0
-        covered = np.zeros((len(lens), 8, int(si[:, 3].max()) + 1), dtype=np.int32)
-        sizes = []
-        for b0, g0, rel0, n in block_work.numpy():
-            sizes.append(int(n))
-            b, g, rel = int(b0), int(g0), int(rel0)
-            while n > 0:
-                while si[b, 3] == 0:
-                    b += 1
-                take = min(si[b, 3] - rel, n)
-                covered[b, g, rel:rel + take] += 1
-                n -= take
-                rel = 0
-                g += 1
-                if g == 8:
-                    g, b = 0, b + 1
-        for b in range(len(lens)):
-            assert (covered[b, :, :si[b, 3]] == 1).all() and (covered[b, :, si[b, 3]:] == 0).all()
-        assert max(sizes) - min(sizes) <= 1
-    da.set_option("grid_blocks", 0)
+                assert tail == 0 or sum(sizes) < 4 * 256 // 64 + 64
+    finally:
+        da.set_option("grid_blocks", 0)
+        da.set_option("tail_units", 6)
 
 
 # ------------------------------------------------------------------ errors, on the host and on the device
