@@ -25,7 +25,8 @@ constexpr int NTHREADS = (NCW + 1) * 32;    // + one producer warp
 constexpr int PLAN_THREADS = 1024;
 constexpr int PLAN_SMEM_SEQS = 4096;
 constexpr int MIN_TAIL_UNIT_TILES = 4;      // a ticketed unit is never cut smaller than this
-constexpr int MERGE_BIG = 16;               // pairs cut into more splits are merged by a whole block
+constexpr int PLAN_BLOCKS = 8;              // the plan kernel's grid: each block cuts a slice of the units
+constexpr int MERGE_WARP_SPLITS = 32;       // pairs cut into more splits are merged by a whole block
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
@@ -59,9 +60,12 @@ struct PlanHeader {
     int n_static;         // = thread blocks of the partition kernel
     int n_tail;           // ticketed units (0: none)
     int ticket;           // next ticketed unit to hand out (reset by the plan kernel)
-    int n_merge_small;    // entries of the two merge lists (pairs cut into <= / > MERGE_BIG splits)
-    int n_merge_big;
-    int pad;
+    int pad[3];
+};
+// Split pairs found by plan block k: how many with <= MERGE_WARP_SPLITS splits, how many with more.
+struct MergeCounts {
+    int n_small[PLAN_BLOCKS];
+    int n_big[PLAN_BLOCKS];
 };
 
 struct PartParams {
@@ -89,7 +93,10 @@ struct PlanParams {
     int4 *seq_info;
     int32_t *prefix;          // [B+1] exclusive prefix of num_tiles
     int4 *unit_work;
-    int32_t *merge_small, *merge_big;   // lists of pair ids b * Hkv + g, one per split pair
+    int4 *merge_small, *merge_big;      // per split pair {pair id b * Hkv + g, first slot, first unit, splits};
+                                        // plan block k appends at [k * merge_seg, ...)
+    MergeCounts *merge_counts;
+    int32_t merge_seg;
     PlanHeader *hdr;
     int32_t *status;
     int32_t B, Hkv, P, window;
@@ -102,7 +109,9 @@ struct MergeParams {
     const int4 *seq_info;
     const int32_t *prefix;
     const PlanHeader *hdr;
-    const int32_t *merge_small, *merge_big;
+    const int4 *merge_small, *merge_big;
+    const MergeCounts *merge_counts;
+    int32_t merge_seg;
     const float *part_o;
     const float *part_lse;
     void *out;
@@ -164,18 +173,25 @@ __host__ __device__ __forceinline__ int pair_splits(const PlanHeader &h, long lo
 }
 
 // =====================================================================================  plan
-// One block.  Per sequence: attended range, tiles, exclusive prefix of tiles; then the cut of the
-// line into units and, per unit, where it starts.
+// PLAN_BLOCKS blocks.  Every block computes, per sequence, the attended range, its tiles and the
+// exclusive prefix of tiles (block 0 stores them), and the cut of the line into units; then each
+// block works out, for its slice of the units, where the unit starts and whether it is the unit
+// that makes a pair "split" (such pairs go to the merge lists).
 __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
 {
+    __shared__ int n_small_s, n_big_s;
     __shared__ int warp_tot[PLAN_THREADS / 32];
     __shared__ int running_s;
     __shared__ int prefix_s[PLAN_SMEM_SEQS + 1];   // copy of the prefix for the searches below
     __shared__ PlanHeader hdr_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     grid_launch_dependents();   // the partition kernel may set up its blocks while the plan is made
-    if (tid == 0)
+    const bool writer = blockIdx.x == 0;
+    if (tid == 0) {
         running_s = 0;
+        n_small_s = 0;
+        n_big_s = 0;
+    }
     __syncthreads();
 
     for (int base = 0; base < p.B; base += PLAN_THREADS) {
@@ -184,7 +200,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         if (b < p.B) {
             L = p.seq_lens[(int64_t)b * p.sl_stride];
             if (L < 0 || (int64_t)L > p.max_pages * (int64_t)p.P) {
-                report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
+                if (writer)
+                    report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
                 L = 0;
             }
             lo = (p.window > 0 && p.window < L) ? L - p.window : 0;
@@ -218,8 +235,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         const int run = running_s;
         const int excl = run + (warp ? warp_tot[warp - 1] : 0) + incl - nt;
         if (b < p.B) {
-            p.seq_info[b] = make_int4(lo, L, first, nt);
-            p.prefix[b] = excl;
+            if (writer) {
+                p.seq_info[b] = make_int4(lo, L, first, nt);
+                p.prefix[b] = excl;
+            }
             if (b < PLAN_SMEM_SEQS)
                 prefix_s[b] = excl;
         }
@@ -231,7 +250,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     const int tiles_per_head = running_s;
     const bool in_smem = p.B <= PLAN_SMEM_SEQS;
     if (tid == 0) {
-        p.prefix[p.B] = tiles_per_head;
+        if (writer)
+            p.prefix[p.B] = tiles_per_head;
         if (in_smem)
             prefix_s[p.B] = tiles_per_head;
         // the cut: a share of the line to the large units, the rest to ticketed units of at least
@@ -254,24 +274,31 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         h.q_tail = n_tail ? tail_w / n_tail : 0;
         h.r_tail = n_tail ? (int)(tail_w % n_tail) : 0;
         h.ticket = 0;
-        h.n_merge_small = 0;
-        h.n_merge_big = 0;
-        h.pad = 0;
+        h.pad[0] = h.pad[1] = h.pad[2] = 0;
         hdr_s = h;
+        if (writer)
+            *p.hdr = h;
     }
     __syncthreads();   // this block's global writes are visible to itself after the barrier
+    // With more sequences than fit in shared memory the searches read block 0's global copy.
+    // (Blocks cannot wait for one another, so in that case block 0 alone cuts all the units.)
     const int *prefix = in_smem ? prefix_s : p.prefix;
     const PlanHeader h = hdr_s;
-
     const int n_units = h.n_static + h.n_tail;
     const int n_full = static_units_in_use(h);
-    for (int u = tid; u < p.n_static + p.n_tail_max; u += PLAN_THREADS) {
+    const int units_max = p.n_static + p.n_tail_max;
+    const int nblk = in_smem ? (int)gridDim.x : 1;
+    const int slice = (units_max + nblk - 1) / nblk;
+    const int u_begin = (int)blockIdx.x * slice;
+    const int u_end = ((int)blockIdx.x < nblk) ? min(u_begin + slice, units_max) : u_begin;
+    int4 *my_small = p.merge_small + (size_t)blockIdx.x * p.merge_seg;
+    int4 *my_big = p.merge_big + (size_t)blockIdx.x * p.merge_seg;
+    for (int u = u_begin + tid; u < u_end; u += PLAN_THREADS) {
         int4 uw = make_int4(0, 0, 0, 0);
         if (u < n_units) {
             const long long ws = unit_start(h, u), we = unit_start(h, u + 1);
             if (we > ws) {
-                const long long xq = ws / p.Hkv;
-                const int x = (int)xq;
+                const int x = (ws < 0x7fffffffll) ? (int)((unsigned)ws / (unsigned)p.Hkv) : (int)(ws / p.Hkv);
                 // largest b with prefix[b] <= x; equal prefixes (empty sequences) resolve to the last
                 int lo_i = 0, hi_i = p.B;   // invariant: prefix[lo_i] <= x < prefix[hi_i]
                 while (hi_i - lo_i > 1) {
@@ -290,13 +317,16 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
                 // by the first such unit: the one whose predecessor holds the pair's first tile.
                 if (rel > 0) {
                     const int prev = (u == h.n_static) ? n_full - 1 : u - 1;
-                    if (unit_start(h, prev) <= ws - rel) {
+                    const long long w0 = ws - rel, prev_start = unit_start(h, prev);
+                    if (prev_start <= w0) {
                         int uf;
-                        const int ns = pair_splits(h, ws - rel, nt, &uf);
-                        if (ns > MERGE_BIG)
-                            p.merge_big[atomicAdd(&hdr_s.n_merge_big, 1)] = b * p.Hkv + g;
+                        const int ns = pair_splits(h, w0, nt, &uf);
+                        // the pair is the first item of unit `prev` only if that unit starts at it
+                        const int4 e = make_int4(b * p.Hkv + g, 2 * prev + (prev_start == w0 ? 0 : 1), prev, ns);
+                        if (ns > MERGE_WARP_SPLITS)
+                            my_big[atomicAdd(&n_big_s, 1)] = e;
                         else
-                            p.merge_small[atomicAdd(&hdr_s.n_merge_small, 1)] = b * p.Hkv + g;
+                            my_small[atomicAdd(&n_small_s, 1)] = e;
                     }
                 }
             }
@@ -304,8 +334,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         p.unit_work[u] = uw;
     }
     __syncthreads();
-    if (tid == 0)
-        *p.hdr = hdr_s;
+    if (tid == 0) {
+        p.merge_counts->n_small[blockIdx.x] = n_small_s;
+        p.merge_counts->n_big[blockIdx.x] = n_big_s;
+    }
 }
 
 // =====================================================================================  partition
@@ -799,14 +831,14 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 }
 
 // =====================================================================================  merge
-// A fixed, small grid.  Its work comes from the two lists of split pairs the plan kernel made
-// (pairs that one unit covered were already written by the partition kernel) and from the empty
-// sequences, which get out = 0 and lse = -inf.  Partials of a (pair, head) are folded one at a time,
-//   M' = max(M, lse_s);  acc = acc * exp(M - M') + exp(lse_s - M') * O_s;  den likewise;
-//   out = acc / den;  lse = M + ln den,
-// by one warp for a pair of the "small" list (each lane owns four head_dim columns), by all eight
-// warps of a block for a pair of the "big" list (warp k folds splits k, k + 8, ..., then warp 0
-// folds the eight results through shared memory).
+// A fixed, small grid.  Its work comes from the lists of split pairs the plan kernel made (pairs
+// that one unit covered were already written by the partition kernel) and from the empty
+// sequences, which get out = 0 and lse = -inf.  For one (pair, head) with partials (O_s, lse_s):
+//   M = max_s lse_s;  w_s = exp(lse_s - M);  out = sum_s w_s O_s / sum_s w_s;  lse = M + ln sum_s w_s.
+// A warp takes up to 32 splits at once: lane s reads lse_s, the maximum and the sum of weights come
+// from warp shuffles, then every lane accumulates its four head_dim columns over the splits (the
+// loads do not depend on one another).  Pairs with more than 32 splits are folded by the eight
+// warps of a block, 32 splits per warp and pass, and combined through shared memory.
 constexpr int MERGE_LANES = HEAD_DIM / 4;
 constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_THREADS = MERGE_WARPS * MERGE_LANES;
@@ -815,29 +847,48 @@ struct MergeAcc {
     float M, den;
     float4 acc;
 };
-__device__ __forceinline__ void merge_fold(MergeAcc &a, float l, float w_den, const float4 &o)
+// a <- a (+) b, both already weighted sums relative to their own maxima
+__device__ __forceinline__ void merge_fold(MergeAcc &a, const MergeAcc &b)
 {
-    const float m_new = fmaxf(a.M, l);
-    const float sc = (a.M == -INFINITY) ? 0.f : __expf(a.M - m_new);
-    const float w = __expf(l - m_new);
-    a.acc.x = a.acc.x * sc + w * o.x;
-    a.acc.y = a.acc.y * sc + w * o.y;
-    a.acc.z = a.acc.z * sc + w * o.z;
-    a.acc.w = a.acc.w * sc + w * o.w;
-    a.den = a.den * sc + w * w_den;
+    if (b.M == -INFINITY)
+        return;
+    const float m_new = fmaxf(a.M, b.M);
+    const float sa = (a.M == -INFINITY) ? 0.f : __expf(a.M - m_new);
+    const float sb = __expf(b.M - m_new);
+    a.acc.x = a.acc.x * sa + b.acc.x * sb;
+    a.acc.y = a.acc.y * sa + b.acc.y * sb;
+    a.acc.z = a.acc.z * sa + b.acc.z * sb;
+    a.acc.w = a.acc.w * sa + b.acc.w * sb;
+    a.den = a.den * sa + b.den * sb;
     a.M = m_new;
 }
 
 __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const MergeParams p)
 {
-    __shared__ float4 s_acc[MERGE_WARPS][MERGE_LANES];
-    __shared__ float s_m[MERGE_WARPS], s_den[MERGE_WARPS];
+    __shared__ MergeAcc s_part[MERGE_WARPS][MERGE_LANES];
     const int warp = threadIdx.x / MERGE_LANES, ln = threadIdx.x % MERGE_LANES, d = ln * 4;
     grid_dependency_wait();     // partials and the plan are complete and visible
     const PlanHeader hdr = *p.hdr;
+    const MergeCounts cnt = *p.merge_counts;
     const int n_full = static_units_in_use(hdr);
     const int gap = hdr.n_static - n_full;
-
+    int n_small = 0, n_big = 0;
+#pragma unroll
+    for (int k = 0; k < PLAN_BLOCKS; ++k) {
+        n_small += cnt.n_small[k];
+        n_big += cnt.n_big[k];
+    }
+    // i-th entry of a list that the plan blocks filled segment by segment
+    auto entry = [&](const int4 *list, const int (&per_block)[PLAN_BLOCKS], int i) {
+        int k = 0;
+#pragma unroll
+        for (int j = 0; j < PLAN_BLOCKS - 1; ++j)
+            if (k == j && i >= per_block[j]) {
+                i -= per_block[j];
+                ++k;
+            }
+        return list[(size_t)k * p.merge_seg + i];
+    };
     auto store = [&](int b, int h, float4 v, float lse_val) {
         const int64_t at = (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d;
         if (p.out_bf16) {
@@ -860,59 +911,67 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const MergeParams 
         if (ln == 0 && p.lse)
             p.lse[(int64_t)b * p.l_sb + (int64_t)h * p.l_sh] = lse_val;
     };
-    // fold splits first, first + stride, ... of (pair, head) into a
-    auto fold_splits = [&](MergeAcc &a, int pair, int head, int first, int stride, int *nsplit_out) {
-        const int b = pair / p.Hkv, g = pair % p.Hkv;
-        const int nt = p.seq_info[b].w;
-        const long long w0 = (long long)p.prefix[b] * p.Hkv + (long long)g * nt;
-        int u_first;
-        const int nsplit = pair_splits(hdr, w0, nt, &u_first);
-        *nsplit_out = nsplit;
-        // the pair is the first item of every unit but possibly u_first, where it is the first item
-        // only if that unit starts exactly at the pair
-        const int slot_first = 2 * u_first + (unit_start(hdr, u_first) == w0 ? 0 : 1);
-#pragma unroll 4
-        for (int k = first; k < nsplit; k += stride) {
-            int uu = u_first + k;
-            if (u_first < n_full && uu >= n_full)
-                uu += gap;   // skip the static units that hold no tiles
-            const int slot = (k == 0) ? slot_first : 2 * uu;
-            const float l = p.part_lse[(int64_t)slot * p.heads_pad + head];
-            const float4 o = *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)slot * p.heads_pad + head) * HEAD_DIM + d);
-            merge_fold(a, l, 1.f, o);
+    // splits [k0, k0 + 32) of entry e (pair id, first slot, first unit, splits), one head
+    auto warp_merge = [&](const int4 &e, int head, int k0) {
+        const int k = k0 + ln;
+        const bool valid = k < e.w;
+        int uu = e.z + k;
+        if (e.z < n_full && uu >= n_full)
+            uu += gap;   // skip the static units that hold no tiles
+        const int slot = (k == 0) ? e.y : 2 * uu;
+        const float l = valid ? p.part_lse[(int64_t)slot * p.heads_pad + head] : -INFINITY;
+        MergeAcc a;
+        a.M = l;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+            a.M = fmaxf(a.M, __shfl_xor_sync(0xffffffffu, a.M, o));
+        const float w = valid ? __expf(l - a.M) : 0.f;
+        a.den = w;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+            a.den += __shfl_xor_sync(0xffffffffu, a.den, o);
+        a.acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int n = min(e.w - k0, 32);
+#pragma unroll 8
+        for (int s2 = 0; s2 < n; ++s2) {
+            const float ws = __shfl_sync(0xffffffffu, w, s2);
+            const int sl = __shfl_sync(0xffffffffu, slot, s2);
+            const float4 o = *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)sl * p.heads_pad + head) * HEAD_DIM + d);
+            a.acc.x += ws * o.x;
+            a.acc.y += ws * o.y;
+            a.acc.z += ws * o.z;
+            a.acc.w += ws * o.w;
         }
+        return a;
+    };
+    auto finish = [&](const int4 &e, int head, const MergeAcc &a) {
+        const float inv = 1.f / a.den;
+        store(e.x / p.Hkv, (e.x % p.Hkv) * p.G + head,
+              make_float4(a.acc.x * inv, a.acc.y * inv, a.acc.z * inv, a.acc.w * inv), a.M + __logf(a.den));
     };
 
     // ---- pairs with many splits: one (pair, head) per block at a time
-    for (int item = blockIdx.x; item < hdr.n_merge_big * p.G; item += gridDim.x) {
-        const int pair = p.merge_big[item / p.G], head = item % p.G;
+    for (int item = blockIdx.x; item < n_big * p.G; item += gridDim.x) {
+        const int4 e = entry(p.merge_big, cnt.n_big, item / p.G);
+        const int head = item % p.G;
         MergeAcc a = {-INFINITY, 0.f, make_float4(0.f, 0.f, 0.f, 0.f)};
-        int nsplit;
-        fold_splits(a, pair, head, warp, MERGE_WARPS, &nsplit);
-        s_acc[warp][ln] = a.acc;
-        if (ln == 0) {
-            s_m[warp] = a.M;
-            s_den[warp] = a.den;
-        }
+        for (int k0 = warp * 32; k0 < e.w; k0 += MERGE_WARPS * 32)
+            merge_fold(a, warp_merge(e, head, k0));
+        s_part[warp][ln] = a;
         __syncthreads();
         if (warp == 0) {
-            for (int k = 1; k < MERGE_WARPS && k < nsplit; ++k)
-                merge_fold(a, s_m[k], s_den[k], s_acc[k][ln]);
-            const float inv = 1.f / a.den;
-            store(pair / p.Hkv, (pair % p.Hkv) * p.G + head,
-                  make_float4(a.acc.x * inv, a.acc.y * inv, a.acc.z * inv, a.acc.w * inv), a.M + __logf(a.den));
+#pragma unroll
+            for (int k = 1; k < MERGE_WARPS; ++k)
+                merge_fold(a, s_part[k][ln]);
+            finish(e, head, a);
         }
         __syncthreads();
     }
-    // ---- pairs with few splits: one (pair, head) per warp
-    for (int item = blockIdx.x * MERGE_WARPS + warp; item < hdr.n_merge_small * p.G; item += gridDim.x * MERGE_WARPS) {
-        const int pair = p.merge_small[item / p.G], head = item % p.G;
-        MergeAcc a = {-INFINITY, 0.f, make_float4(0.f, 0.f, 0.f, 0.f)};
-        int nsplit;
-        fold_splits(a, pair, head, 0, 1, &nsplit);
-        const float inv = 1.f / a.den;
-        store(pair / p.Hkv, (pair % p.Hkv) * p.G + head,
-              make_float4(a.acc.x * inv, a.acc.y * inv, a.acc.z * inv, a.acc.w * inv), a.M + __logf(a.den));
+    // ---- pairs with at most 32 splits: one (pair, head) per warp
+    for (int item = blockIdx.x * MERGE_WARPS + warp; item < n_small * p.G; item += gridDim.x * MERGE_WARPS) {
+        const int4 e = entry(p.merge_small, cnt.n_small, item / p.G);
+        const int head = item % p.G;
+        finish(e, head, warp_merge(e, head, 0));
     }
     // ---- empty sequences
     for (int b = blockIdx.x; b < p.B; b += gridDim.x) {

@@ -112,7 +112,8 @@ int tail_units_for(int nblocks)
 }
 
 struct WsLayout {
-    size_t status, hdr, seq_info, prefix, unit_work, merge_small, merge_big, part_lse, part_o;
+    size_t status, hdr, merge_counts, seq_info, prefix, unit_work, merge_small, merge_big, part_lse, part_o;
+    int merge_seg;
     size_t stg_q, stg_bt, stg_sl, stg_out, stg_lse, total;
 };
 
@@ -128,11 +129,13 @@ WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int unit
     };
     w.status = take(16);
     w.hdr = take(sizeof(PlanHeader));
+    w.merge_counts = take(sizeof(MergeCounts));
+    w.merge_seg = (units + PLAN_BLOCKS - 1) / PLAN_BLOCKS;   // a plan block lists at most one pair per unit it cuts
     w.seq_info = take((size_t)B * 16);
     w.prefix = take((size_t)(B + 1) * 4);
     w.unit_work = take((size_t)units * 16);
-    w.merge_small = take((size_t)units * 4);
-    w.merge_big = take((size_t)units * 4);
+    w.merge_small = take((size_t)w.merge_seg * PLAN_BLOCKS * 16);
+    w.merge_big = take((size_t)w.merge_seg * PLAN_BLOCKS * 16);
     w.part_lse = take((size_t)2 * units * kMaxGroup * 4);
     w.part_o = take((size_t)2 * units * kMaxGroup * HEAD_DIM * 4);
     w.stg_q = take((size_t)B * Hq * D * 2);
@@ -275,8 +278,10 @@ int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws,
     pp.seq_info = reinterpret_cast<int4 *>(ws + lay.seq_info);
     pp.prefix = reinterpret_cast<int32_t *>(ws + lay.prefix);
     pp.unit_work = reinterpret_cast<int4 *>(ws + lay.unit_work);
-    pp.merge_small = reinterpret_cast<int32_t *>(ws + lay.merge_small);
-    pp.merge_big = reinterpret_cast<int32_t *>(ws + lay.merge_big);
+    pp.merge_small = reinterpret_cast<int4 *>(ws + lay.merge_small);
+    pp.merge_big = reinterpret_cast<int4 *>(ws + lay.merge_big);
+    pp.merge_counts = reinterpret_cast<MergeCounts *>(ws + lay.merge_counts);
+    pp.merge_seg = lay.merge_seg;
     pp.hdr = reinterpret_cast<PlanHeader *>(ws + lay.hdr);
     pp.status = reinterpret_cast<int32_t *>(ws + lay.status);
     pp.B = (int32_t)d.B;
@@ -287,7 +292,7 @@ int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws,
     pp.n_tail_max = n_tail;
     pp.static_frac_q8 = (int32_t)g_opt_static_frac;
     pp.max_pages = d.max_pages;
-    plan_kernel<<<1, PLAN_THREADS, 0, stream>>>(pp);
+    plan_kernel<<<PLAN_BLOCKS, PLAN_THREADS, 0, stream>>>(pp);
     g_launches.fetch_add(1);
     DA_CUDA(cudaGetLastError());
     return DA_OK;
@@ -374,8 +379,10 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     mp.seq_info = pa.seq_info;
     mp.prefix = reinterpret_cast<const int32_t *>(ws + lay.prefix);
     mp.hdr = pa.hdr;
-    mp.merge_small = reinterpret_cast<const int32_t *>(ws + lay.merge_small);
-    mp.merge_big = reinterpret_cast<const int32_t *>(ws + lay.merge_big);
+    mp.merge_small = reinterpret_cast<const int4 *>(ws + lay.merge_small);
+    mp.merge_big = reinterpret_cast<const int4 *>(ws + lay.merge_big);
+    mp.merge_counts = reinterpret_cast<const MergeCounts *>(ws + lay.merge_counts);
+    mp.merge_seg = lay.merge_seg;
     mp.part_o = pa.part_o;
     mp.part_lse = pa.part_lse;
     mp.out = out->data;
