@@ -34,6 +34,9 @@ import workloads  # noqa: E402
 METRIC = "decode-attn KV-cache GB/s (fraction of 8 TB/s HBM); sequences/s per layer"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the partition kernel, from the ncu
+# capture summarised in profiles/partition_kernel_<workload>.md; valid for that library version only.
+NCU_TRAFFIC = {("c2", 101): 2223268000 + 8050000}
 WORKLOAD_TEXT = {
     "c1": "c1: 1 seq x 512 tok, page 16, contiguous, seed 0, 3 keys x20",
     "c2": "c2: 64 seqs, len U[1024,16384], 48q/8kv heads, d128, page 16, permuted pool, seed 1",
@@ -291,7 +294,7 @@ def run_ours(args):
         "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
         "roofline": {"bound": "hbm", "kernel": "partition_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                     "kernel_ms": kms, "traffic": None},
+                     "kernel_ms": kms, "traffic": NCU_TRAFFIC.get((args.workload, da.version()))},
         "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms_max,
                 "note": "q, block_table, seq_lens from pinned host memory and out, lse back to it every step; "

@@ -197,8 +197,8 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
  * they change how sequences are split.
  *   "grid_blocks"  thread blocks of the partition kernel (0 = two per SM, at most 4096)
  *   "tail_units"   work units per thread block that are handed out by ticket after the static
- *                  ranges (0 .. 64, default 6; 0 = static ranges only)
- *   "static_frac"  share of the work, in 1/256, covered by the static ranges (default 192)
+ *                  ranges (0 .. 64, default 4; 0 = static ranges only)
+ *   "static_frac"  share of the work, in 1/256, covered by the static ranges (default 224)
  * Returns DA_ERR_UNSUPPORTED for an unknown name or a value out of range.
  */
 int decode_attn_set_option(const char *name, int64_t value);

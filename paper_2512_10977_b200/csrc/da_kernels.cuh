@@ -863,7 +863,7 @@ __device__ __forceinline__ void merge_fold(MergeAcc &a, const MergeAcc &b)
     a.M = m_new;
 }
 
-__global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const MergeParams p)
+__global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergeParams p)
 {
     __shared__ MergeAcc s_part[MERGE_WARPS][MERGE_LANES];
     const int warp = threadIdx.x / MERGE_LANES, ln = threadIdx.x % MERGE_LANES, d = ln * 4;
@@ -932,15 +932,28 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const MergeParams 
             a.den += __shfl_xor_sync(0xffffffffu, a.den, o);
         a.acc = make_float4(0.f, 0.f, 0.f, 0.f);
         const int n = min(e.w - k0, 32);
-#pragma unroll 8
-        for (int s2 = 0; s2 < n; ++s2) {
-            const float ws = __shfl_sync(0xffffffffu, w, s2);
-            const int sl = __shfl_sync(0xffffffffu, slot, s2);
-            const float4 o = *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)sl * p.heads_pad + head) * HEAD_DIM + d);
-            a.acc.x += ws * o.x;
-            a.acc.y += ws * o.y;
-            a.acc.z += ws * o.z;
-            a.acc.w += ws * o.w;
+        // 8 independent loads in flight per lane and pass
+        for (int s0 = 0; s0 < n; s0 += 8) {
+            float4 o[8];
+            float ws[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int s2 = s0 + j;
+                ws[j] = __shfl_sync(0xffffffffu, w, s2 & 31);
+                const int sl = __shfl_sync(0xffffffffu, slot, s2 & 31);
+                o[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (s2 < n)
+                    o[j] = *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)sl * p.heads_pad + head) * HEAD_DIM + d);
+                else
+                    ws[j] = 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                a.acc.x += ws[j] * o[j].x;
+                a.acc.y += ws[j] * o[j].y;
+                a.acc.z += ws[j] * o[j].z;
+                a.acc.w += ws[j] * o[j].w;
+            }
         }
         return a;
     };
@@ -950,8 +963,9 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const MergeParams 
               make_float4(a.acc.x * inv, a.acc.y * inv, a.acc.z * inv, a.acc.w * inv), a.M + __logf(a.den));
     };
 
-    // ---- pairs with many splits: one (pair, head) per block at a time
-    for (int item = blockIdx.x; item < n_big * p.G; item += gridDim.x) {
+    // ---- pairs with many splits: one (pair, head) per block at a time, handed out from the last
+    //      block down so that they rarely meet the warp-sized items below in the same block
+    for (int item = (int)(gridDim.x - 1 - blockIdx.x); item < n_big * p.G; item += gridDim.x) {
         const int4 e = entry(p.merge_big, cnt.n_big, item / p.G);
         const int head = item % p.G;
         MergeAcc a = {-INFINITY, 0.f, make_float4(0.f, 0.f, 0.f, 0.f)};

@@ -16,7 +16,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 100;
+constexpr int kVersion = 101;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -26,8 +26,8 @@ std::mutex g_mu;
 std::atomic<int> g_last_cuda_error{0};
 std::atomic<int64_t> g_launches{0};
 int64_t g_opt_grid_blocks = 0;   // 0 = two blocks per SM
-int64_t g_opt_tail_units = 6;    // ticketed units per thread block (0: one static range per block only)
-int64_t g_opt_static_frac = 192; // share of the work given to the static ranges, in 1/256
+int64_t g_opt_tail_units = 4;    // ticketed units per thread block (0: one static range per block only)
+int64_t g_opt_static_frac = 224; // share of the work given to the static ranges, in 1/256
 cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 struct DeviceState {

@@ -53,10 +53,10 @@ def test_options(pkg):
     with pytest.raises(pkg.DecodeAttnError) as e:
         pkg.set_option("grid_blocks", 10 ** 6)
     assert e.value.status == 5
-    assert pkg.get_option("tail_units") == 6 and pkg.get_option("static_frac") == 192
+    assert pkg.get_option("tail_units") == 4 and pkg.get_option("static_frac") == 224
     pkg.set_option("tail_units", 0)
     assert pkg.get_option("tail_units") == 0
-    pkg.set_option("tail_units", 6)
+    pkg.set_option("tail_units", 4)
     for name, bad in (("tail_units", 65), ("tail_units", -1), ("static_frac", 257)):
         with pytest.raises(pkg.DecodeAttnError) as e:
             pkg.set_option(name, bad)

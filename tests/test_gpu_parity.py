@@ -21,8 +21,8 @@ def da():
     pkg.lib()
     yield pkg
     pkg.set_option("grid_blocks", 0)
-    pkg.set_option("tail_units", 6)
-    pkg.set_option("static_frac", 192)
+    pkg.set_option("tail_units", 4)
+    pkg.set_option("static_frac", 224)
 
 
 def oracle_of(case):
@@ -121,8 +121,8 @@ def test_any_mix_of_static_and_ticketed_units_gives_the_same_answer(da, tail, fr
         case.window = 700
         check(da, case, f"tail={tail} frac={frac} window", 0)
     finally:
-        da.set_option("tail_units", 6)
-        da.set_option("static_frac", 192)
+        da.set_option("tail_units", 4)
+        da.set_option("static_frac", 224)
 
 
 @pytest.mark.parametrize("B", [1, 2, 3, 7])
@@ -292,7 +292,7 @@ def test_integer_mean_is_exact(da):
         np.testing.assert_allclose(got_lse, ref_lse, atol=1e-6)
     finally:
         da.set_option("grid_blocks", 0)
-        da.set_option("tail_units", 6)
+        da.set_option("tail_units", 4)
     got, _ = gpu_of(da, case)
     np.testing.assert_allclose(got, ref, atol=1e-6)
 
@@ -316,7 +316,7 @@ def test_plan_covers_every_attended_token_exactly_once(da, window):
     lens = np.concatenate([workloads.lengths_c2(1, 20), [0, 1, 64, 65]])
     sl = torch.tensor(lens, dtype=torch.int32, device="cuda")
     try:
-        for grid, tail in ((0, 6), (1, 0), (7, 3), (1000, 1), (0, 0)):
+        for grid, tail in ((0, 4), (1, 0), (7, 3), (1000, 1), (0, 0)):
             da.set_option("grid_blocks", grid)
             da.set_option("tail_units", tail)
             seq_info, unit_work, n_static, T = da.plan(sl, window, 8, 16, 2048)
@@ -355,7 +355,7 @@ def test_plan_covers_every_attended_token_exactly_once(da, window):
                 assert tail == 0 or sum(sizes) < 4 * 256 // 64 + 64
     finally:
         da.set_option("grid_blocks", 0)
-        da.set_option("tail_units", 6)
+        da.set_option("tail_units", 4)
 
 
 # ------------------------------------------------------------------ errors, on the host and on the device
