@@ -108,6 +108,29 @@ int decode_attn(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
                 da_tensor *out, da_tensor *lse, void *stream);
 
 /*
+ * decode_attn_cascade -- decode_attn() (full attention, no window) for a batch whose sequences all
+ * START WITH THE SAME PAGES: entries 0 .. shared_prefix_tokens / P - 1 are identical in every row of
+ * the block table (the sessions of the paper's agent share one long initial prompt: task rules,
+ * output format and three reference kernels; Sec. 3.2 "Generate Kernel" and App. B).  The result
+ * is the same as decode_attn's; only the schedule differs.  The prefix is not streamed once per
+ * sequence: all B * Hq query vectors attend it together, as a (B * Hq/Hkv) x prefix score matrix
+ * per KV head on the tcgen05 tensor cores (the prefix kernel), each sequence's own tokens past the
+ * prefix go through the plan / partition / merge kernels as usual, and a last kernel folds the two
+ * with the log-sum-exp rule.
+ *
+ *   shared_prefix_tokens  a multiple of 128, at most max_pages * P; <= 0 means no shared prefix
+ *                         (plain decode_attn).  Every seq_lens[b] must be >= shared_prefix_tokens
+ *                         (a shorter one sets DA_DEV_BAD_SEQLEN in the device status).
+ *   The page ids of the prefix are read from row 0 of the block table; that the other rows agree
+ *   is the caller's promise and is not checked.
+ * Other arguments, results, workspace and error conventions: as decode_attn().
+ */
+int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                        const da_tensor *block_table, const da_tensor *seq_lens,
+                        int32_t shared_prefix_tokens, float scale, da_tensor *out, da_tensor *lse,
+                        void *stream);
+
+/*
  * decode_attn_host_io -- the same call for a caller whose per-step tensors are in HOST memory.
  * q, block_table, seq_lens, out and lse are HOST views (pinned memory makes the copies
  * asynchronous; they must stay valid until the stream reaches the end of the call); k_pages and

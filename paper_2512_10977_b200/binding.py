@@ -47,6 +47,8 @@ def lib() -> ctypes.CDLL:
             vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
             L.decode_attn.restype = ctypes.c_int
             L.decode_attn.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_cascade.restype = ctypes.c_int
+            L.decode_attn_cascade.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_host_io.restype = ctypes.c_int
             L.decode_attn_host_io.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_static_scratch.restype = ctypes.c_int
@@ -168,6 +170,25 @@ def decode_attn(q, k_pages, v_pages, block_table, seq_lens, window: int, scale: 
         tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
         _check(lib().decode_attn(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
                                  int(window), float(scale), _ref(tv[5]), _ref(tv[6]), _stream_ptr(stream)))
+    return out, lse
+
+
+def decode_attn_cascade(q, k_pages, v_pages, block_table, seq_lens, shared_prefix_tokens: int, scale: float,
+                        out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                        stream: Optional[torch.cuda.Stream] = None, out_dtype=torch.float32):
+    """decode_attn (no window) for sequences whose first ``shared_prefix_tokens`` tokens are the same
+    physical pages in every block-table row; the prefix is attended once for the whole batch on the
+    tensor cores.  Same result as ``decode_attn``.  Returns (out, lse)."""
+    if out is None:
+        out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+    with torch.cuda.device(k_pages.device):
+        _auto_workspace(q, k_pages, block_table)
+        tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
+        _check(lib().decode_attn_cascade(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
+                                         int(shared_prefix_tokens), float(scale), _ref(tv[5]), _ref(tv[6]),
+                                         _stream_ptr(stream)))
     return out, lse
 
 

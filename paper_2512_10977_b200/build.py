@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libdecode_attn.so")
 SOURCES = ["decode_attn.cu"]
-HEADERS = ["da_ptx.cuh", "da_kernels.cuh", os.path.join("..", "..", "include", "decode_attn.h")]
+HEADERS = ["da_ptx.cuh", "da_kernels.cuh", "da_prefix.cuh", os.path.join("..", "..", "include", "decode_attn.h")]
 
 
 def _stale() -> bool:

@@ -100,6 +100,7 @@ struct PlanParams {
     PlanHeader *hdr;
     int32_t *status;
     int32_t B, Hkv, P, window;
+    int32_t first_token;      // tokens before this one are not attended (the cascade's suffix pass)
     int32_t n_static, n_tail_max, static_frac_q8;   // large units; most ticketed units; share of the
                                                     // line given to the large units, in 1/256
     int64_t max_pages;
@@ -204,8 +205,14 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
                     report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
                 L = 0;
             }
+            if (L > 0 && L < p.first_token) {
+                if (writer)
+                    report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 1, L);
+                L = 0;
+            }
             lo = (p.window > 0 && p.window < L) ? L - p.window : 0;
-            if (L > 0) {
+            lo = max(lo, min(p.first_token, L));
+            if (L > lo) {
                 first = lo / TILE_T;
                 nt = (L - 1) / TILE_T - first + 1;
             }

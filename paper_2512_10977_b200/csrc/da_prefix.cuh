@@ -1,0 +1,475 @@
+// Shared-prefix ("cascade") decode: when every sequence of the batch starts with the same pages --
+// the agent sessions all begin with one long initial prompt -- the attention of all B * Hq query
+// vectors over that prefix is one dense contraction per KV head: a (B*G) x T score matrix against
+// K, softmax, times V.  That is tensor-core work, done here with tcgen05 (operands in shared memory
+// by TMA, accumulators in tensor memory), instead of streaming the same pages once per sequence.
+//
+// prefix_kernel: one block = 128 query rows (row = b * G + head-in-group) of one KV head and one
+// range of 128-token KV tiles.  Per tile:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in TMEM)
+// -> the four softmax warps read their rows of S (one thread per row), keep running max / sum in
+// the log2 domain, write P = exp2(S - m) as bf16 high and low parts into swizzled shared memory
+// -> O_tile = P_hi V + P_lo V (two more tcgen05.mma into a second TMEM region) -> the softmax
+// threads add O_tile into their fp32 row accumulators (rescaled when the max moved).  A fifth warp
+// drives TMA and issues the MMAs.  Result: a normalised partial (O / l, lse) per (split, b, h),
+// combined with the per-sequence suffix attention by cascade_merge_kernel.
+#pragma once
+#include "da_kernels.cuh"
+
+namespace da {
+
+constexpr int PF_ROWS = 128;                 // query rows per block (UMMA M)
+constexpr int PF_TOK = 128;                  // tokens per KV tile (UMMA N for S, K for PV)
+constexpr int PF_PLANE = PF_TOK * 128;       // one 64-column half of a 128-row tile: 128-byte rows
+constexpr int PF_TILE = 2 * PF_PLANE;        // 32 KB: Q, a K tile, a V tile, P_hi, P_lo
+constexpr int PF_THREADS = 160;              // 4 softmax warps + 1 driver warp
+constexpr int PF_OFF_Q = 0;
+constexpr int PF_OFF_K = PF_TILE;            // two K buffers
+constexpr int PF_OFF_V = 3 * PF_TILE;        // two V buffers
+constexpr int PF_OFF_PH = 5 * PF_TILE;
+constexpr int PF_OFF_PL = 6 * PF_TILE;
+constexpr int PF_OFF_BARS = 7 * PF_TILE;     // kfull[2], vfull[2], s, o, p
+constexpr int PF_OFF_MISC = PF_OFF_BARS + 64;   // TMEM base address, abort flag
+constexpr int PF_SMEM_BYTES = PF_OFF_MISC + 16;
+constexpr int PF_TMEM_COLS = 256;            // S in columns [0,128), O_tile in [128,256)
+
+struct PrefixParams {
+    const __nv_bfloat16 *q;
+    int64_t q_sb, q_sh;
+    const int32_t *block_table;   // row 0 names the shared pages
+    float *pre_o;                 // [splits][B*Hq][128] normalised partials
+    float *pre_lse;               // [splits][B*Hq]
+    int32_t *status;
+    int32_t B, Hkv, G, P, box_rows, num_pages;
+    int32_t prefix_tiles;         // shared prefix length / PF_TOK
+    int32_t splits;               // KV ranges per (row tile, head)
+    int32_t row_tiles;            // ceil(B*G / 128)
+    float scale_log2;
+};
+
+// ---------------------------------------------------------------- tcgen05 wrappers
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Shared-memory matrix descriptor: start address, leading / stride byte offsets (all >> 4),
+// descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B, A K-major, B K- or
+// MN-major, N and M in units of 8 and 16.
+__device__ __forceinline__ uint32_t umma_idesc(int m, int n, bool b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+// Arrive on `bar` once every tcgen05 operation this thread issued so far has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane (lane = 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
+        "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        v[i] = __uint_as_float(r[i]);
+}
+// The K/V pools are read here through a 4-D tiled map {d, token, head, page} with box {64, box_rows, 1, 1}:
+// one box is one 64-column plane of box_rows token rows, so a plane of a tile is contiguous and
+// its 8-row groups are 1024 bytes apart, which is what the matrix descriptors above assume.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, int c2, int c3, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(PF_THREADS, 1)
+prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const PrefixParams p)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];   // no static shared memory: keeps the base 1024-B aligned
+    uint32_t &tmem_base_s = *reinterpret_cast<uint32_t *>(smem + PF_OFF_MISC);
+    int &abort_s = *reinterpret_cast<int *>(smem + PF_OFF_MISC + 4);
+    const uint32_t sb = smem_u32(smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t bar_kfull = sb + PF_OFF_BARS, bar_vfull = bar_kfull + 16, bar_s = bar_kfull + 32, bar_o = bar_kfull + 40,
+                   bar_p = bar_kfull + 48;
+    volatile int *abort_flag = &abort_s;
+
+    // block -> (row tile, kv head, split)
+    const int rt = blockIdx.x % p.row_tiles;
+    const int g = (blockIdx.x / p.row_tiles) % p.Hkv;
+    const int split = blockIdx.x / (p.row_tiles * p.Hkv);
+    const int t_begin = (int)((long long)p.prefix_tiles * split / p.splits);
+    const int t_end = (int)((long long)p.prefix_tiles * (split + 1) / p.splits);
+    const int ntiles = t_end - t_begin;
+    const int R = p.B * p.G;
+
+    if ((sb & 1023u) != 0) {
+        if (tid == 0)
+            report_status(p.status, 3, -6, (int)blockIdx.x, (int)sb);
+        return;
+    }
+    if (tid == 0) {
+        abort_s = 0;
+        mbar_init(bar_kfull, 1);
+        mbar_init(bar_kfull + 8, 1);
+        mbar_init(bar_vfull, 1);
+        mbar_init(bar_vfull + 8, 1);
+        mbar_init(bar_s, 1);
+        mbar_init(bar_o, 1);
+        mbar_init(bar_p, 128);
+        mbar_fence_init();
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    if (warp == 4)
+        tmem_alloc(smem_u32(&tmem_base_s), PF_TMEM_COLS);
+    // Q rows of this block into the swizzled K-major layout: row r, 16-byte chunk c (0..15 along d)
+    // -> plane c >> 3, byte r * 128 + (((c & 7) ^ (r & 7)) << 4).  Rows past B * G are zero.
+    for (int e = tid; e < PF_ROWS * 16; e += PF_THREADS) {
+        const int r = e >> 4, c = e & 15;
+        const int row = rt * PF_ROWS + r;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (row < R) {
+            const int b = row / p.G, hi = row % p.G;
+            const __nv_bfloat16 *src = p.q + (int64_t)b * p.q_sb + (int64_t)(g * p.G + hi) * p.q_sh + c * 8;
+            if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+                val = *reinterpret_cast<const uint4 *>(src);
+            } else {
+                const uint32_t *s32p = reinterpret_cast<const uint32_t *>(src);
+                val = make_uint4(s32p[0], s32p[1], s32p[2], s32p[3]);
+            }
+        }
+        *reinterpret_cast<uint4 *>(smem + PF_OFF_Q + (c >> 3) * PF_PLANE + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = val;
+    }
+    fence_proxy_async_smem();   // Q is read by the tensor core through the async proxy
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ driver: TMA + MMA issue
+        if (lane == 0 && ntiles > 0) {
+            const int boxes = PF_TOK / p.box_rows;
+            const uint32_t tile_bytes = (uint32_t)PF_TILE;
+            bool ok = true;
+            int issued = 0;   // tiles whose loads were issued
+            auto load_tile = [&](int j) {   // K and V of tile j into buffer j & 1
+                const int buf = j & 1;
+                issued = j + 1;
+                const int tok0 = (t_begin + j) * PF_TOK;
+                mbar_arrive_expect_tx(bar_kfull + 8 * buf, tile_bytes);
+                mbar_arrive_expect_tx(bar_vfull + 8 * buf, tile_bytes);
+                for (int bx = 0; bx < boxes; ++bx) {
+                    const int t = tok0 + bx * p.box_rows;
+                    int page = __ldg(p.block_table + t / p.P);
+                    if ((uint32_t)page >= (uint32_t)p.num_pages) {
+                        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, 0, t / p.P, page);
+                        page = p.num_pages;   // out of range: TMA fills zeros and still counts the bytes
+                    }
+                    const int row = t % p.P;
+                    for (int pl = 0; pl < 2; ++pl) {
+                        const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + bx * p.box_rows * 128);
+                        tma_load_4d(sb + PF_OFF_K + off, &tm_k, pl * 64, row, g, page, bar_kfull + 8 * buf);
+                        tma_load_4d(sb + PF_OFF_V + off, &tm_v, pl * 64, row, g, page, bar_vfull + 8 * buf);
+                    }
+                }
+            };
+            auto mma_s = [&](int j) {   // S = Q K^T for tile j
+                const uint32_t kb = sb + PF_OFF_K + (j & 1) * PF_TILE;
+                const uint32_t idesc = umma_idesc(PF_ROWS, PF_TOK, false);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (kk >> 2) * PF_PLANE + (kk & 3) * 32;
+                    umma_bf16(tmem_s, umma_desc(sb + PF_OFF_Q + off, 16, 1024), umma_desc(kb + off, 16, 1024), idesc, kk > 0);
+                }
+                umma_commit(bar_s);
+            };
+            auto mma_o = [&](int j) {   // O_tile = P_hi V + P_lo V for tile j
+                const uint32_t vb = sb + PF_OFF_V + (j & 1) * PF_TILE;
+                const uint32_t idesc = umma_idesc(PF_ROWS, HEAD_DIM, true);
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const uint32_t pb = sb + (half ? PF_OFF_PL : PF_OFF_PH);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        // A = P (K-major over tokens), B = V stored [token][d]: MN-major, planes are the
+                        // two halves of d (leading offset = plane), 8-token groups 1024 B apart
+                        umma_bf16(tmem_o, umma_desc(pb + (kk >> 2) * PF_PLANE + (kk & 3) * 32, 16, 1024),
+                                  umma_desc(vb + kk * 2048, PF_PLANE, 1024), idesc, half > 0 || kk > 0);
+                    }
+                }
+                umma_commit(bar_o);
+            };
+
+            load_tile(0);
+            if (ntiles > 1)
+                load_tile(1);
+            ok = mbar_wait_bounded(bar_kfull, 0u, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                mma_s(0);
+            }
+            for (int j = 0; ok && j < ntiles; ++j) {
+                const uint32_t ph = (uint32_t)(j & 1), ph2 = (uint32_t)((j >> 1) & 1);
+                ok = mbar_wait_bounded(bar_p, ph, abort_flag) && mbar_wait_bounded(bar_vfull + 8 * (j & 1), ph2, abort_flag);
+                if (!ok)
+                    break;
+                tc_fence_after();
+                mma_o(j);
+                if (j + 1 < ntiles) {
+                    ok = mbar_wait_bounded(bar_kfull + 8 * ((j + 1) & 1), (uint32_t)(((j + 1) >> 1) & 1), abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    mma_s(j + 1);
+                }
+                if (j + 2 < ntiles) {
+                    // both buffers j & 1 are free once O_tile(j) is complete (S(j) completed long before)
+                    ok = mbar_wait_bounded(bar_o, ph, abort_flag);
+                    if (!ok)
+                        break;
+                    load_tile(j + 2);
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -7, (int)blockIdx.x, 0);
+                // do not leave while copies may still land in shared memory: bounded wait for the
+                // latest fill of each buffer
+                for (int j = ntiles - 1, seen = 0; j >= 0 && seen < 2; --j) {
+                    if (j >= issued)
+                        continue;
+                    ++seen;
+                    const uint64_t t0 = globaltimer_ns();
+                    while (!(mbar_try_wait(bar_kfull + 8 * (j & 1), (uint32_t)((j >> 1) & 1)) &&
+                             mbar_try_wait(bar_vfull + 8 * (j & 1), (uint32_t)((j >> 1) & 1)))) {
+                        if (globaltimer_ns() - t0 > 1000000000ull)
+                            break;
+                    }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax warps: thread = row
+        const int r = tid;                               // row of the tile = TMEM lane
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float m_run = -INFINITY, l_run = 0.f, alpha_prev = 1.f;
+        float o_acc[HEAD_DIM];
+#pragma unroll
+        for (int i = 0; i < HEAD_DIM; ++i)
+            o_acc[i] = 0.f;
+        bool ok = true;
+        auto add_o_tile = [&](float alpha) {
+#pragma unroll
+            for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
+                float v[32];
+                tmem_ld32(tmem_o + lane_base + c0, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    o_acc[c0 + i] = o_acc[c0 + i] * alpha + v[i];
+            }
+        };
+        for (int j = 0; j < ntiles; ++j) {
+            const uint32_t ph = (uint32_t)(j & 1);
+            if (!mbar_wait_bounded(bar_s, ph, abort_flag)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            // pass 1: the row maximum of this tile's scaled scores
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c0 = 0; c0 < PF_TOK; c0 += 32) {
+                float v[32];
+                tmem_ld32(tmem_s + lane_base + c0, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    mx = fmaxf(mx, v[i] * p.scale_log2);
+            }
+            const float m_new = fmaxf(m_run, mx);
+            const float alpha = (m_run == -INFINITY) ? 0.f : fast_exp2(m_run - m_new);
+            // the previous tile's PV product must be folded in before its P buffer is overwritten
+            if (j > 0) {
+                if (!mbar_wait_bounded(bar_o, (uint32_t)((j - 1) & 1), abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                add_o_tile(alpha_prev);
+            }
+            // pass 2: weights, their sum, and P as bf16 high + low parts in the swizzled K-major layout
+            float lsum = 0.f;
+#pragma unroll
+            for (int c0 = 0; c0 < PF_TOK; c0 += 32) {
+                float v[32];
+                tmem_ld32(tmem_s + lane_base + c0, v);
+#pragma unroll
+                for (int q8 = 0; q8 < 4; ++q8) {   // 8 tokens = one 16-byte chunk
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float p0 = fast_exp2(v[q8 * 8 + 2 * e] * p.scale_log2 - m_new);
+                        const float p1 = fast_exp2(v[q8 * 8 + 2 * e + 1] * p.scale_log2 - m_new);
+                        lsum += p0 + p1;
+                        hi[e] = pack_bf16(p0, p1);
+                        lo[e] = pack_bf16(p0 - bf16_lo_to_float(hi[e]), p1 - bf16_hi_to_float(hi[e]));
+                    }
+                    const int chunk = (c0 >> 3) + q8;   // 0..15 along tokens
+                    const uint32_t off = (uint32_t)((chunk >> 3) * PF_PLANE + r * 128 + (((chunk & 7) ^ (r & 7)) << 4));
+                    *reinterpret_cast<uint4 *>(smem + PF_OFF_PH + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4 *>(smem + PF_OFF_PL + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                }
+            }
+            l_run = l_run * alpha + lsum;
+            m_run = m_new;
+            alpha_prev = alpha;
+            fence_proxy_async_smem();   // P is read by the tensor core through the async proxy
+            tc_fence_before();          // and this thread's TMEM reads precede the MMAs that follow
+            mbar_arrive(bar_p);
+        }
+        if (ok && ntiles > 0) {
+            if (mbar_wait_bounded(bar_o, (uint32_t)((ntiles - 1) & 1), abort_flag)) {
+                tc_fence_after();
+                add_o_tile(alpha_prev);
+            } else {
+                ok = false;
+            }
+        }
+        if (!ok) {
+            if (*abort_flag == 0) {
+                *abort_flag = 1;
+                report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -8, (int)blockIdx.x, 0);
+            }
+        } else {
+            const int row = rt * PF_ROWS + r;
+            if (row < R) {
+                const int b = row / p.G, hi = row % p.G;
+                const int64_t bh = (int64_t)b * (p.Hkv * p.G) + g * p.G + hi;
+                const int64_t at = (int64_t)split * p.B * (p.Hkv * p.G) + bh;
+                float *dst = p.pre_o + at * HEAD_DIM;
+                if (ntiles > 0) {
+                    const float inv = 1.f / l_run;
+#pragma unroll
+                    for (int i = 0; i < HEAD_DIM; i += 4)
+                        *reinterpret_cast<float4 *>(dst + i) =
+                            make_float4(o_acc[i] * inv, o_acc[i + 1] * inv, o_acc[i + 2] * inv, o_acc[i + 3] * inv);
+                    p.pre_lse[at] = (m_run + fast_log2(l_run)) * LN2;
+                } else {
+#pragma unroll
+                    for (int i = 0; i < HEAD_DIM; i += 4)
+                        *reinterpret_cast<float4 *>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+                    p.pre_lse[at] = -INFINITY;
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4)
+        tmem_dealloc(tmem, PF_TMEM_COLS);
+}
+
+// =====================================================================================  cascade merge
+// One warp per (b, h): fold the prefix partials (one per KV split) and the suffix result (computed
+// by the plan / partition / merge kernels over tokens >= prefix into fp32 scratch) and write `out`
+// and `lse`.  lse = -inf marks "no tokens" and contributes nothing.
+struct CascadeMergeParams {
+    const float *pre_o, *pre_lse;   // [splits][B*Hq][128], [splits][B*Hq]
+    const float *suf_o, *suf_lse;   // [B*Hq][128], [B*Hq]
+    void *out;
+    int64_t o_sb, o_sh;
+    float *lse;
+    int64_t l_sb, l_sh;
+    int32_t B, Hq, splits, out_bf16;
+};
+
+__global__ void __launch_bounds__(256) cascade_merge_kernel(const CascadeMergeParams p)
+{
+    const int warp = threadIdx.x >> 5, ln = threadIdx.x & 31, d = ln * 4;
+    const int64_t bh = (int64_t)blockIdx.x * 8 + warp;
+    const int64_t n = (int64_t)p.B * p.Hq;
+    if (bh >= n)
+        return;
+    float M = p.suf_lse[bh];
+    for (int s = 0; s < p.splits; ++s)
+        M = fmaxf(M, p.pre_lse[(int64_t)s * n + bh]);
+    float den = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto fold = [&](float l, const float *o) {
+        if (l == -INFINITY)
+            return;
+        const float w = __expf(l - M);
+        const float4 v = *reinterpret_cast<const float4 *>(o + d);
+        acc.x += w * v.x;
+        acc.y += w * v.y;
+        acc.z += w * v.z;
+        acc.w += w * v.w;
+        den += w;
+    };
+    fold(p.suf_lse[bh], p.suf_o + bh * HEAD_DIM);
+    for (int s = 0; s < p.splits; ++s)
+        fold(p.pre_lse[(int64_t)s * n + bh], p.pre_o + ((int64_t)s * n + bh) * HEAD_DIM);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    float lse_val = -INFINITY;
+    if (den > 0.f) {
+        const float inv = 1.f / den;
+        v = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+        lse_val = M + __logf(den);
+    }
+    const int b = (int)(bh / p.Hq), h = (int)(bh % p.Hq);
+    const int64_t at = (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d;
+    if (p.out_bf16) {
+        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
+        o[0] = __float2bfloat16_rn(v.x);
+        o[1] = __float2bfloat16_rn(v.y);
+        o[2] = __float2bfloat16_rn(v.z);
+        o[3] = __float2bfloat16_rn(v.w);
+    } else {
+        float *o = reinterpret_cast<float *>(p.out) + at;
+        o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+    }
+    if (ln == 0 && p.lse)
+        p.lse[(int64_t)b * p.l_sb + (int64_t)h * p.l_sh] = lse_val;
+}
+
+}  // namespace da

@@ -10,7 +10,7 @@
 #include <cstring>
 #include <mutex>
 
-#include "da_kernels.cuh"
+#include "da_prefix.cuh"
 
 namespace {
 
@@ -20,6 +20,7 @@ constexpr int kVersion = 101;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
+constexpr int kMaxPrefixSplits = 4;
 constexpr int kMaxGroup = 16;
 
 std::mutex g_mu;
@@ -43,6 +44,7 @@ struct TmapKey {
     int64_t shape[4];
     int64_t stride[4];
     int box_rows;
+    int planes;   // 2: 5-D view, one box = both 64-column halves; 1: 4-D view, one box = one half
 };
 struct TmapEntry {
     TmapKey key;
@@ -114,7 +116,8 @@ int tail_units_for(int nblocks)
 struct WsLayout {
     size_t status, hdr, merge_counts, seq_info, prefix, unit_work, merge_small, merge_big, part_lse, part_o;
     int merge_seg;
-    size_t stg_q, stg_bt, stg_sl, stg_out, stg_lse, total;
+    size_t stg_q, stg_bt, stg_sl, stg_out, stg_lse;
+    size_t pre_o, pre_lse, suf_o, suf_lse, total;   // cascade scratch
 };
 
 // `units` = thread blocks of the partition kernel x (1 + ticketed units per block)
@@ -143,6 +146,10 @@ WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int unit
     w.stg_sl = take((size_t)B * 4);
     w.stg_out = take((size_t)B * Hq * D * 4);
     w.stg_lse = take((size_t)B * Hq * 4);
+    w.pre_o = take((size_t)kMaxPrefixSplits * B * Hq * D * 4);
+    w.pre_lse = take((size_t)kMaxPrefixSplits * B * Hq * 4);
+    w.suf_o = take((size_t)B * Hq * D * 4);
+    w.suf_lse = take((size_t)B * Hq * 4);
     w.total = off;
     return w;
 }
@@ -164,7 +171,10 @@ int get_encoder()
 // {64, box_rows, 2, 1, 1}, 128-byte swizzle.  Splitting head_dim into two halves keeps the inner box
 // extent at the swizzle span (128 bytes) while one TMA operation still brings all 128 columns of
 // box_rows tokens: in shared memory a box is two planes of box_rows 128-byte rows.
-int get_tmap(const da_tensor *t, int box_rows, CUtensorMap *out)
+// planes = 2: the partition kernel's view.  planes = 1: a 4-D view {d, token, kv head, page} with
+// box {64, box_rows, 1, 1} (one 64-column half per box), used by the prefix kernel, whose matrix
+// descriptors want each half of a tile contiguous.
+int get_tmap(const da_tensor *t, int box_rows, int planes, CUtensorMap *out)
 {
     TmapKey key;
     std::memset(&key, 0, sizeof key);
@@ -174,6 +184,7 @@ int get_tmap(const da_tensor *t, int box_rows, CUtensorMap *out)
         key.stride[i] = t->stride[i];
     }
     key.box_rows = box_rows;
+    key.planes = planes;
     for (int i = 0; i < kTmapCache; ++i)
         if (g_tmaps[i].used && std::memcmp(&g_tmaps[i].key, &key, sizeof key) == 0) {
             *out = g_tmaps[i].map;
@@ -182,14 +193,23 @@ int get_tmap(const da_tensor *t, int box_rows, CUtensorMap *out)
     int rc = get_encoder();
     if (rc != DA_OK)
         return rc;
-    cuuint64_t gdim[5] = {64, (cuuint64_t)t->shape[2], 2, (cuuint64_t)t->shape[1], (cuuint64_t)t->shape[0]};
-    cuuint64_t gstr[4] = {(cuuint64_t)t->stride[2] * 2, 128, (cuuint64_t)t->stride[1] * 2, (cuuint64_t)t->stride[0] * 2};
-    cuuint32_t box[5] = {64, (cuuint32_t)box_rows, 2, 1, 1};
-    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     CUtensorMap m;
-    CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, t->data, gdim, gstr, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r;
+    if (planes == 2) {
+        cuuint64_t gdim[5] = {64, (cuuint64_t)t->shape[2], 2, (cuuint64_t)t->shape[1], (cuuint64_t)t->shape[0]};
+        cuuint64_t gstr[4] = {(cuuint64_t)t->stride[2] * 2, 128, (cuuint64_t)t->stride[1] * 2, (cuuint64_t)t->stride[0] * 2};
+        cuuint32_t box[5] = {64, (cuuint32_t)box_rows, 2, 1, 1};
+        cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, t->data, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        cuuint64_t gdim[4] = {(cuuint64_t)t->shape[3], (cuuint64_t)t->shape[2], (cuuint64_t)t->shape[1], (cuuint64_t)t->shape[0]};
+        cuuint64_t gstr[3] = {(cuuint64_t)t->stride[2] * 2, (cuuint64_t)t->stride[1] * 2, (cuuint64_t)t->stride[0] * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, t->data, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
     if (r != CUDA_SUCCESS) {
         g_last_cuda_error.store((int)cudaErrorInvalidValue);
         return DA_ERR_CUDA;
@@ -269,8 +289,8 @@ int set_kernel_attrs()
     return DA_OK;
 }
 
-int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws, const WsLayout &lay, int nblocks,
-                int n_tail, cudaStream_t stream)
+int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const Dims &d, uint8_t *ws,
+                const WsLayout &lay, int nblocks, int n_tail, cudaStream_t stream)
 {
     PlanParams pp;
     pp.seq_lens = static_cast<const int32_t *>(sl->data);
@@ -288,6 +308,7 @@ int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws,
     pp.Hkv = (int32_t)d.Hkv;
     pp.P = (int32_t)d.P;
     pp.window = window;
+    pp.first_token = first_token;
     pp.n_static = nblocks;
     pp.n_tail_max = n_tail;
     pp.static_frac_q8 = (int32_t)g_opt_static_frac;
@@ -303,7 +324,7 @@ int launch_plan(const da_tensor *sl, int32_t window, const Dims &d, uint8_t *ws,
 int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay, int nblocks, int n_tail,
                 const da_tensor *q,
                 const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl, int32_t window,
-                float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream)
+                float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, int32_t first_token = 0)
 {
     int rc;
     if (!st->attrs_set) {
@@ -311,16 +332,17 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
         if (rc != DA_OK) return rc;
         rc = set_kernel_attrs<2>();
         if (rc != DA_OK) return rc;
+        DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
         st->attrs_set = true;
     }
     const int box_rows = d.P < TILE_T ? (int)d.P : TILE_T;
     CUtensorMap tm_k, tm_v;
-    rc = get_tmap(k, box_rows, &tm_k);
+    rc = get_tmap(k, box_rows, 2, &tm_k);
     if (rc != DA_OK) return rc;
-    rc = get_tmap(v, box_rows, &tm_v);
+    rc = get_tmap(v, box_rows, 2, &tm_v);
     if (rc != DA_OK) return rc;
 
-    rc = launch_plan(sl, window, d, ws, lay, nblocks, n_tail, stream);
+    rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream);
     if (rc != DA_OK) return rc;
 
     PartParams pa;
@@ -443,6 +465,104 @@ int decode_attn(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
                 const da_tensor *seq_lens, int32_t window, float scale, da_tensor *out, da_tensor *lse, void *stream)
 {
     return run(q, k_pages, v_pages, block_table, seq_lens, window, scale, out, lse, static_cast<cudaStream_t>(stream));
+}
+
+int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                        const da_tensor *block_table, const da_tensor *seq_lens, int32_t shared_prefix_tokens, float scale,
+                        da_tensor *out, da_tensor *lse, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (shared_prefix_tokens <= 0)
+        return run(q, k_pages, v_pages, block_table, seq_lens, 0, scale, out, lse, stream);
+    Dims d;
+    int rc = validate(q, k_pages, v_pages, block_table, seq_lens, out, lse, &d);
+    if (rc != DA_OK) return rc;
+    if (shared_prefix_tokens % PF_TOK != 0 || (int64_t)shared_prefix_tokens > d.max_pages * d.P) return DA_ERR_SHAPE;
+    if (d.B * d.Hq > 0x7fffffffll / HEAD_DIM) return DA_ERR_UNSUPPORTED;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    rc = current_device(&dev, &st);
+    if (rc != DA_OK) return rc;
+    const int nblocks = grid_blocks_for(st);
+    const int n_tail = tail_units_for(nblocks);
+    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks + n_tail);
+    if (!st->ws || st->ws_bytes < lay.total) return DA_ERR_WORKSPACE;
+    if (d.B == 0) return DA_OK;
+    uint8_t *ws = static_cast<uint8_t *>(st->ws);
+
+    // 1. attention over the tokens past the prefix, per sequence, into fp32 scratch
+    da_tensor so, sl;
+    so.data = ws + lay.suf_o;
+    so.dtype = DA_F32;
+    so.ndim = 3;
+    so.shape[0] = d.B; so.shape[1] = d.Hq; so.shape[2] = HEAD_DIM; so.shape[3] = 0;
+    so.stride[0] = d.Hq * HEAD_DIM; so.stride[1] = HEAD_DIM; so.stride[2] = 1; so.stride[3] = 0;
+    sl.data = ws + lay.suf_lse;
+    sl.dtype = DA_F32;
+    sl.ndim = 2;
+    sl.shape[0] = d.B; sl.shape[1] = d.Hq; sl.shape[2] = sl.shape[3] = 0;
+    sl.stride[0] = d.Hq; sl.stride[1] = 1; sl.stride[2] = sl.stride[3] = 0;
+    rc = launch_path(st, d, ws, lay, nblocks, n_tail, q, k_pages, v_pages, block_table, seq_lens, 0, scale, &so, &sl, stream,
+                     shared_prefix_tokens);
+    if (rc != DA_OK) return rc;
+
+    // 2. attention of every query row over the shared prefix, on the tensor cores
+    const int box_rows = d.P < PF_TOK ? (int)d.P : PF_TOK;
+    CUtensorMap tm_k, tm_v;
+    rc = get_tmap(k_pages, box_rows, 1, &tm_k);
+    if (rc != DA_OK) return rc;
+    rc = get_tmap(v_pages, box_rows, 1, &tm_v);
+    if (rc != DA_OK) return rc;
+    PrefixParams pf;
+    pf.q = static_cast<const __nv_bfloat16 *>(q->data);
+    pf.q_sb = q->stride[0];
+    pf.q_sh = q->stride[1];
+    pf.block_table = static_cast<const int32_t *>(block_table->data);
+    pf.pre_o = reinterpret_cast<float *>(ws + lay.pre_o);
+    pf.pre_lse = reinterpret_cast<float *>(ws + lay.pre_lse);
+    pf.status = reinterpret_cast<int32_t *>(ws + lay.status);
+    pf.B = (int32_t)d.B;
+    pf.Hkv = (int32_t)d.Hkv;
+    pf.G = (int32_t)d.G;
+    pf.P = (int32_t)d.P;
+    pf.box_rows = box_rows;
+    pf.num_pages = (int32_t)d.num_pages;
+    pf.prefix_tiles = shared_prefix_tokens / PF_TOK;
+    pf.row_tiles = (int32_t)((d.B * d.G + PF_ROWS - 1) / PF_ROWS);
+    int splits = (st->sm_count + pf.row_tiles * pf.Hkv - 1) / (pf.row_tiles * pf.Hkv);
+    if (splits > kMaxPrefixSplits) splits = kMaxPrefixSplits;
+    if (splits > pf.prefix_tiles) splits = pf.prefix_tiles;
+    if (splits < 1) splits = 1;
+    pf.splits = splits;
+    pf.scale_log2 = scale * LOG2E;
+    const long long grid = (long long)pf.row_tiles * pf.Hkv * splits;
+    if (grid > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+    prefix_kernel<<<(unsigned)grid, PF_THREADS, PF_SMEM_BYTES, stream>>>(tm_k, tm_v, pf);
+    g_launches.fetch_add(1);
+    DA_CUDA(cudaGetLastError());
+
+    // 3. fold prefix partials and suffix result
+    CascadeMergeParams cm;
+    cm.pre_o = pf.pre_o;
+    cm.pre_lse = pf.pre_lse;
+    cm.suf_o = reinterpret_cast<const float *>(ws + lay.suf_o);
+    cm.suf_lse = reinterpret_cast<const float *>(ws + lay.suf_lse);
+    cm.out = out->data;
+    cm.o_sb = out->stride[0];
+    cm.o_sh = out->stride[1];
+    cm.lse = lse ? static_cast<float *>(lse->data) : nullptr;
+    cm.l_sb = lse ? lse->stride[0] : 0;
+    cm.l_sh = lse ? lse->stride[1] : 0;
+    cm.B = (int32_t)d.B;
+    cm.Hq = (int32_t)d.Hq;
+    cm.splits = splits;
+    cm.out_bf16 = out->dtype == DA_BF16;
+    cascade_merge_kernel<<<(unsigned)((d.B * d.Hq + 7) / 8), 256, 0, stream>>>(cm);
+    g_launches.fetch_add(1);
+    DA_CUDA(cudaGetLastError());
+    return DA_OK;
 }
 
 int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tensor *v_pages,
@@ -616,7 +736,7 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
     *tile_tokens = TILE_T;
     if (d.B == 0) return DA_OK;
     uint8_t *ws = static_cast<uint8_t *>(st->ws);
-    rc = launch_plan(seq_lens, window, d, ws, lay, nblocks, n_tail, stream);
+    rc = launch_plan(seq_lens, window, 0, d, ws, lay, nblocks, n_tail, stream);
     if (rc != DA_OK) return rc;
     PlanHeader h;
     DA_CUDA(cudaMemcpyAsync(&h, ws + lay.hdr, sizeof h, cudaMemcpyDeviceToHost, stream));
