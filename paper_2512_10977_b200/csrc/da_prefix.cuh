@@ -27,10 +27,10 @@ constexpr int PF_OFF_K = PF_TILE;            // two K buffers
 constexpr int PF_OFF_V = 3 * PF_TILE;        // two V buffers
 constexpr int PF_OFF_PH = 5 * PF_TILE;
 constexpr int PF_OFF_PL = 6 * PF_TILE;
-constexpr int PF_OFF_BARS = 7 * PF_TILE;     // kfull[2], vfull[2], s, o, p
+constexpr int PF_OFF_BARS = 7 * PF_TILE;     // kfull[2], vfull[2], s[2], o, p
 constexpr int PF_OFF_MISC = PF_OFF_BARS + 64;   // TMEM base address, abort flag
 constexpr int PF_SMEM_BYTES = PF_OFF_MISC + 16;
-constexpr int PF_TMEM_COLS = 256;            // S in columns [0,128), O_tile in [128,256)
+constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O_tile in [256,384)
 
 struct PrefixParams {
     const __nv_bfloat16 *q;
@@ -128,8 +128,8 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     int &abort_s = *reinterpret_cast<int *>(smem + PF_OFF_MISC + 4);
     const uint32_t sb = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t bar_kfull = sb + PF_OFF_BARS, bar_vfull = bar_kfull + 16, bar_s = bar_kfull + 32, bar_o = bar_kfull + 40,
-                   bar_p = bar_kfull + 48;
+    const uint32_t bar_kfull = sb + PF_OFF_BARS, bar_vfull = bar_kfull + 16, bar_s = bar_kfull + 32, bar_o = bar_kfull + 48,
+                   bar_p = bar_kfull + 56;
     volatile int *abort_flag = &abort_s;
 
     // block -> (row tile, kv head, split)
@@ -153,6 +153,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         mbar_init(bar_vfull, 1);
         mbar_init(bar_vfull + 8, 1);
         mbar_init(bar_s, 1);
+        mbar_init(bar_s + 8, 1);
         mbar_init(bar_o, 1);
         mbar_init(bar_p, 128);
         mbar_fence_init();
@@ -184,33 +185,43 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
-    const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
+    const uint32_t tmem_s = tmem, tmem_o = tmem + 256;   // S(j) lives at tmem_s + 128 * (j & 1)
 
     if (warp == 4) {
-        // ------------------------------------------------------------------ driver: TMA + MMA issue
-        if (lane == 0 && ntiles > 0) {
+        // ------------------------------------------------------------------ driver warp: TMA + MMA issue
+        // All lanes walk the same control flow (waits included); lane bx < boxes reads the page id of
+        // box bx of a tile and issues its four loads; lane 0 alone arms barriers and issues the MMAs.
+        if (ntiles > 0) {
             const int boxes = PF_TOK / p.box_rows;
             const uint32_t tile_bytes = (uint32_t)PF_TILE;
             bool ok = true;
             int issued = 0;   // tiles whose loads were issued
-            auto load_tile = [&](int j) {   // K and V of tile j into buffer j & 1
+            auto read_page = [&](int j) {   // page id of this lane's box of tile j (0 for idle lanes)
+                if (lane >= boxes || j >= ntiles)
+                    return 0;
+                const int t = (t_begin + j) * PF_TOK + lane * p.box_rows;
+                return __ldg(p.block_table + t / p.P);
+            };
+            auto load_kv = [&](int j, int page, bool is_v) {   // K or V of tile j into buffer j & 1
                 const int buf = j & 1;
-                issued = j + 1;
-                const int tok0 = (t_begin + j) * PF_TOK;
-                mbar_arrive_expect_tx(bar_kfull + 8 * buf, tile_bytes);
-                mbar_arrive_expect_tx(bar_vfull + 8 * buf, tile_bytes);
-                for (int bx = 0; bx < boxes; ++bx) {
-                    const int t = tok0 + bx * p.box_rows;
-                    int page = __ldg(p.block_table + t / p.P);
+                const uint32_t bar = (is_v ? bar_vfull : bar_kfull) + 8 * buf;
+                if (is_v)
+                    issued = j + 1;
+                if (lane == 0)
+                    mbar_arrive_expect_tx(bar, tile_bytes);
+                __syncwarp();
+                if (lane < boxes) {
+                    const int t = (t_begin + j) * PF_TOK + lane * p.box_rows;
                     if ((uint32_t)page >= (uint32_t)p.num_pages) {
-                        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, 0, t / p.P, page);
+                        if (!is_v)
+                            report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, 0, t / p.P, page);
                         page = p.num_pages;   // out of range: TMA fills zeros and still counts the bytes
                     }
                     const int row = t % p.P;
+#pragma unroll
                     for (int pl = 0; pl < 2; ++pl) {
-                        const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + bx * p.box_rows * 128);
-                        tma_load_4d(sb + PF_OFF_K + off, &tm_k, pl * 64, row, g, page, bar_kfull + 8 * buf);
-                        tma_load_4d(sb + PF_OFF_V + off, &tm_v, pl * 64, row, g, page, bar_vfull + 8 * buf);
+                        const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + lane * p.box_rows * 128);
+                        tma_load_4d(sb + (is_v ? PF_OFF_V : PF_OFF_K) + off, is_v ? &tm_v : &tm_k, pl * 64, row, g, page, bar);
                     }
                 }
             };
@@ -220,9 +231,10 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint32_t off = (kk >> 2) * PF_PLANE + (kk & 3) * 32;
-                    umma_bf16(tmem_s, umma_desc(sb + PF_OFF_Q + off, 16, 1024), umma_desc(kb + off, 16, 1024), idesc, kk > 0);
+                    umma_bf16(tmem_s + 128 * (j & 1), umma_desc(sb + PF_OFF_Q + off, 16, 1024), umma_desc(kb + off, 16, 1024),
+                              idesc, kk > 0);
                 }
-                umma_commit(bar_s);
+                umma_commit(bar_s + 8 * (j & 1));
             };
             auto mma_o = [&](int j) {   // O_tile = P_hi V + P_lo V for tile j
                 const uint32_t vb = sb + PF_OFF_V + (j & 1) * PF_TILE;
@@ -241,13 +253,25 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 umma_commit(bar_o);
             };
 
-            load_tile(0);
-            if (ntiles > 1)
-                load_tile(1);
-            ok = mbar_wait_bounded(bar_kfull, 0u, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                mma_s(0);
+            // Order of events for tile j:  P(j) ready -> PV product of j; K(j+2) requested; once the
+            // product is done, V(j+2) requested; once K(j+2) is there, S(j+2) into the S buffer that
+            // the softmax of j has just finished with.  The scores of tile j+1 were computed while the
+            // softmax of j ran, so the softmax warps never wait for the tensor core.
+            int page0 = read_page(0), page1 = read_page(1);
+            load_kv(0, page0, false);
+            load_kv(0, page0, true);
+            if (ntiles > 1) {
+                load_kv(1, page1, false);
+                load_kv(1, page1, true);
+            }
+            int page_next = read_page(2);   // fetched ahead of its use
+            for (int j = 0; ok && j < 2 && j < ntiles; ++j) {
+                ok = mbar_wait_bounded(bar_kfull + 8 * j, 0u, abort_flag);
+                if (ok) {
+                    tc_fence_after();
+                    if (lane == 0)
+                        mma_s(j);
+                }
             }
             for (int j = 0; ok && j < ntiles; ++j) {
                 const uint32_t ph = (uint32_t)(j & 1), ph2 = (uint32_t)((j >> 1) & 1);
@@ -255,23 +279,25 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 if (!ok)
                     break;
                 tc_fence_after();
-                mma_o(j);
-                if (j + 1 < ntiles) {
-                    ok = mbar_wait_bounded(bar_kfull + 8 * ((j + 1) & 1), (uint32_t)(((j + 1) >> 1) & 1), abort_flag);
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-                    mma_s(j + 1);
-                }
+                if (lane == 0)
+                    mma_o(j);
                 if (j + 2 < ntiles) {
-                    // both buffers j & 1 are free once O_tile(j) is complete (S(j) completed long before)
+                    const int page = page_next;
+                    page_next = read_page(j + 3);
+                    load_kv(j + 2, page, false);   // K buffer j & 1: S(j) was complete before the softmax of j began
                     ok = mbar_wait_bounded(bar_o, ph, abort_flag);
                     if (!ok)
                         break;
-                    load_tile(j + 2);
+                    load_kv(j + 2, page, true);    // V buffer j & 1: free once the PV product of j is complete
+                    ok = mbar_wait_bounded(bar_kfull + 8 * (j & 1), ph2 ^ 1u, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    if (lane == 0)
+                        mma_s(j + 2);
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 *abort_flag = 1;
                 report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -7, (int)blockIdx.x, 0);
                 // do not leave while copies may still land in shared memory: bounded wait for the
@@ -310,8 +336,8 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         };
         for (int j = 0; j < ntiles; ++j) {
-            const uint32_t ph = (uint32_t)(j & 1);
-            if (!mbar_wait_bounded(bar_s, ph, abort_flag)) {
+            const uint32_t tmem_sj = tmem_s + 128 * (j & 1);
+            if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag)) {
                 ok = false;
                 break;
             }
@@ -321,7 +347,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 #pragma unroll
             for (int c0 = 0; c0 < PF_TOK; c0 += 32) {
                 float v[32];
-                tmem_ld32(tmem_s + lane_base + c0, v);
+                tmem_ld32(tmem_sj + lane_base + c0, v);
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
                     mx = fmaxf(mx, v[i] * p.scale_log2);
@@ -342,7 +368,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 #pragma unroll
             for (int c0 = 0; c0 < PF_TOK; c0 += 32) {
                 float v[32];
-                tmem_ld32(tmem_s + lane_base + c0, v);
+                tmem_ld32(tmem_sj + lane_base + c0, v);
 #pragma unroll
                 for (int q8 = 0; q8 < 4; ++q8) {   // 8 tokens = one 16-byte chunk
                     uint32_t hi[4], lo[4];

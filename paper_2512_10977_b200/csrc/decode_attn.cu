@@ -531,7 +531,8 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     pf.num_pages = (int32_t)d.num_pages;
     pf.prefix_tiles = shared_prefix_tokens / PF_TOK;
     pf.row_tiles = (int32_t)((d.B * d.G + PF_ROWS - 1) / PF_ROWS);
-    int splits = (st->sm_count + pf.row_tiles * pf.Hkv - 1) / (pf.row_tiles * pf.Hkv);
+    // one block per SM at a time (its shared memory fills an SM): as many KV ranges as fit one wave
+    int splits = st->sm_count / (pf.row_tiles * pf.Hkv);
     if (splits > kMaxPrefixSplits) splits = kMaxPrefixSplits;
     if (splits > pf.prefix_tiles) splits = pf.prefix_tiles;
     if (splits < 1) splits = 1;
