@@ -6,10 +6,10 @@
 //
 // prefix_kernel: one block = 128 query rows (row = b * G + head-in-group) of one KV head and one
 // range of 128-token KV tiles.  Per tile:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in TMEM)
-// -> the four softmax warps read their rows of S (one thread per row), keep running max / sum in
-// the log2 domain, write P = exp2(S - m) as bf16 high and low parts into swizzled shared memory
+// -> the eight softmax warps read their rows of S (two threads per row, 64 columns each), keep running
+// max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts into swizzled shared memory
 // -> O_tile = P_hi V + P_lo V (two more tcgen05.mma into a second TMEM region) -> the softmax
-// threads add O_tile into their fp32 row accumulators (rescaled when the max moved).  A fifth warp
+// threads add O_tile into their fp32 row accumulators (rescaled when the max moved).  A ninth warp
 // drives TMA and issues the MMAs.  Result: a normalised partial (O / l, lse) per (split, b, h),
 // combined with the per-sequence suffix attention by cascade_merge_kernel.
 #pragma once
@@ -21,15 +21,17 @@ constexpr int PF_ROWS = 128;                 // query rows per block (UMMA M)
 constexpr int PF_TOK = 128;                  // tokens per KV tile (UMMA N for S, K for PV)
 constexpr int PF_PLANE = PF_TOK * 128;       // one 64-column half of a 128-row tile: 128-byte rows
 constexpr int PF_TILE = 2 * PF_PLANE;        // 32 KB: Q, a K tile, a V tile, P_hi, P_lo
-constexpr int PF_THREADS = 160;              // 4 softmax warps + 1 driver warp
+constexpr int PF_DRV = 8;                    // warps 0..7: softmax (two threads per row); warp 8: driver
+constexpr int PF_THREADS = (PF_DRV + 1) * 32;
 constexpr int PF_OFF_Q = 0;
 constexpr int PF_OFF_K = PF_TILE;            // two K buffers
 constexpr int PF_OFF_V = 3 * PF_TILE;        // two V buffers
 constexpr int PF_OFF_PH = 5 * PF_TILE;
 constexpr int PF_OFF_PL = 6 * PF_TILE;
-constexpr int PF_OFF_BARS = 7 * PF_TILE;     // kfull[2], vfull[2], s[2], o, p
-constexpr int PF_OFF_MISC = PF_OFF_BARS + 64;   // TMEM base address, abort flag
-constexpr int PF_SMEM_BYTES = PF_OFF_MISC + 16;
+constexpr int PF_OFF_BARS = 7 * PF_TILE;     // kfull[2], vfull[2], s[2], o[2], p, x
+constexpr int PF_OFF_MISC = PF_OFF_BARS + 96;   // TMEM base address, abort flag
+constexpr int PF_OFF_XCHG = PF_OFF_MISC + 16;   // row maxima / sums swapped between a row's two threads
+constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + 2 * 2 * 128 * 4;
 constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O_tile in [256,384)
 
 struct PrefixParams {
@@ -108,6 +110,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
     for (int i = 0; i < 32; ++i)
         v[i] = __uint_as_float(r[i]);
 }
+// The same load without the wait, so that several can be in flight; tmem_ld_wait() ends them all.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
+        "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // The K/V pools are read here through a 4-D tiled map {d, token, head, page} with box {64, box_rows, 1, 1}:
 // one box is one 64-column plane of box_rows token rows, so a plane of a tile is contiguous and
 // its 8-row groups are 1024 bytes apart, which is what the matrix descriptors above assume.
@@ -129,7 +145,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const uint32_t sb = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t bar_kfull = sb + PF_OFF_BARS, bar_vfull = bar_kfull + 16, bar_s = bar_kfull + 32, bar_o = bar_kfull + 48,
-                   bar_p = bar_kfull + 56;
+                   bar_p = bar_kfull + 64, bar_x = bar_kfull + 72;   // bar_o is a pair: tile t uses bar_o + 8 * (t & 1)
     volatile int *abort_flag = &abort_s;
 
     // block -> (row tile, kv head, split)
@@ -155,12 +171,14 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         mbar_init(bar_s, 1);
         mbar_init(bar_s + 8, 1);
         mbar_init(bar_o, 1);
-        mbar_init(bar_p, 128);
+        mbar_init(bar_o + 8, 1);
+        mbar_init(bar_p, 2 * PF_ROWS);
+        mbar_init(bar_x, PF_DRV);
         mbar_fence_init();
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
     }
-    if (warp == 4)
+    if (warp == PF_DRV)
         tmem_alloc(smem_u32(&tmem_base_s), PF_TMEM_COLS);
     // Q rows of this block into the swizzled K-major layout: row r, 16-byte chunk c (0..15 along d)
     // -> plane c >> 3, byte r * 128 + (((c & 7) ^ (r & 7)) << 4).  Rows past B * G are zero.
@@ -187,7 +205,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const uint32_t tmem = tmem_base_s;
     const uint32_t tmem_s = tmem, tmem_o = tmem + 256;   // S(j) lives at tmem_s + 128 * (j & 1)
 
-    if (warp == 4) {
+    if (warp == PF_DRV) {
         // ------------------------------------------------------------------ driver warp: TMA + MMA issue
         // All lanes walk the same control flow (waits included); lane bx < boxes reads the page id of
         // box bx of a tile and issues its four loads; lane 0 alone arms barriers and issues the MMAs.
@@ -250,13 +268,16 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                                   umma_desc(vb + kk * 2048, PF_PLANE, 1024), idesc, half > 0 || kk > 0);
                     }
                 }
-                umma_commit(bar_o);
+                umma_commit(bar_o + 8 * (j & 1));
             };
 
-            // Order of events for tile j:  P(j) ready -> PV product of j; K(j+2) requested; once the
-            // product is done, V(j+2) requested; once K(j+2) is there, S(j+2) into the S buffer that
-            // the softmax of j has just finished with.  The scores of tile j+1 were computed while the
-            // softmax of j ran, so the softmax warps never wait for the tensor core.
+            // The driver is an event loop: whichever of its four jobs has its inputs ready goes next.
+            //   PV product of tile t : P(t) written (bar_p) and V(t) loaded
+            //   K load of tile t     : K buffer t & 1 free = S(t-2) consumed, known once P(t-2) was seen
+            //   V load of tile t     : V buffer t & 1 free = PV product of t-2 complete (bar_o)
+            //   scores of tile t     : K(t) loaded and S buffer t & 1 free (P(t-2) seen)
+            // so the scores of tile j+1 are computed while the softmax of tile j runs, and a slow load
+            // never delays a PV product whose inputs are ready.
             int page0 = read_page(0), page1 = read_page(1);
             load_kv(0, page0, false);
             load_kv(0, page0, true);
@@ -264,37 +285,46 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 load_kv(1, page1, false);
                 load_kv(1, page1, true);
             }
-            int page_next = read_page(2);   // fetched ahead of its use
-            for (int j = 0; ok && j < 2 && j < ntiles; ++j) {
-                ok = mbar_wait_bounded(bar_kfull + 8 * j, 0u, abort_flag);
-                if (ok) {
+            int next_o = 0, next_s = 0, next_k = min(2, ntiles), next_v = min(2, ntiles);
+            int page_k = read_page(2), page_v = page_k;   // page ids are fetched ahead of their use
+            uint64_t t_last = globaltimer_ns();
+            auto ready = [&](uint32_t bar, int n) {   // has the n-th completion of `bar` happened? (warp-uniform)
+                return __all_sync(0xffffffffu, mbar_test_wait(bar, (uint32_t)(n & 1)));
+            };
+            while (next_o < ntiles) {
+                bool progress = false;
+                if (next_s < ntiles && next_s < next_k && next_o > next_s - 2 &&
+                    ready(bar_kfull + 8 * (next_s & 1), next_s >> 1)) {
                     tc_fence_after();
                     if (lane == 0)
-                        mma_s(j);
+                        mma_s(next_s);
+                    ++next_s;
+                    progress = true;
                 }
-            }
-            for (int j = 0; ok && j < ntiles; ++j) {
-                const uint32_t ph = (uint32_t)(j & 1), ph2 = (uint32_t)((j >> 1) & 1);
-                ok = mbar_wait_bounded(bar_p, ph, abort_flag) && mbar_wait_bounded(bar_vfull + 8 * (j & 1), ph2, abort_flag);
-                if (!ok)
-                    break;
-                tc_fence_after();
-                if (lane == 0)
-                    mma_o(j);
-                if (j + 2 < ntiles) {
-                    const int page = page_next;
-                    page_next = read_page(j + 3);
-                    load_kv(j + 2, page, false);   // K buffer j & 1: S(j) was complete before the softmax of j began
-                    ok = mbar_wait_bounded(bar_o, ph, abort_flag);
-                    if (!ok)
-                        break;
-                    load_kv(j + 2, page, true);    // V buffer j & 1: free once the PV product of j is complete
-                    ok = mbar_wait_bounded(bar_kfull + 8 * (j & 1), ph2 ^ 1u, abort_flag);
-                    if (!ok)
-                        break;
+                if (ready(bar_p, next_o) && ready(bar_vfull + 8 * (next_o & 1), next_o >> 1)) {
                     tc_fence_after();
                     if (lane == 0)
-                        mma_s(j + 2);
+                        mma_o(next_o);
+                    ++next_o;
+                    progress = true;
+                }
+                if (next_k < ntiles && next_o > next_k - 2 && next_s > next_k - 2) {
+                    load_kv(next_k, page_k, false);
+                    ++next_k;
+                    page_k = read_page(next_k);
+                    progress = true;
+                }
+                if (next_v < ntiles && next_o > next_v - 2 && ready(bar_o + 8 * (next_v & 1), (next_v - 2) >> 1)) {
+                    load_kv(next_v, page_v, true);
+                    ++next_v;
+                    page_v = read_page(next_v);
+                    progress = true;
+                }
+                if (progress) {
+                    t_last = globaltimer_ns();
+                } else if (*abort_flag || globaltimer_ns() - t_last > 2000000000ull) {
+                    ok = false;
+                    break;
                 }
             }
             if (!ok && lane == 0) {
@@ -316,75 +346,92 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         }
     } else {
-        // ------------------------------------------------------------------ softmax warps: thread = row
-        const int r = tid;                               // row of the tile = TMEM lane
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        // ------------------------------------------------------------------ softmax warps
+        // Two threads per row: warp w and warp w + 4 read the same TMEM lanes (32 * (w % 4) ...), the
+        // first the tile's columns 0..63, the second 64..127 -- of S (tokens) and of O_tile (head_dim).
+        const int r = 32 * (warp & 3) + lane;            // row of the tile = TMEM lane
+        const int half = warp >> 2;
+        const uint32_t lane_base = ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(half * 64);
+        float *xchg = reinterpret_cast<float *>(smem + PF_OFF_XCHG);   // [2 buffers][2 halves][128 rows]
         float m_run = -INFINITY, l_run = 0.f, alpha_prev = 1.f;
-        float o_acc[HEAD_DIM];
+        float o_acc[64];
 #pragma unroll
-        for (int i = 0; i < HEAD_DIM; ++i)
+        for (int i = 0; i < 64; ++i)
             o_acc[i] = 0.f;
         bool ok = true;
         auto add_o_tile = [&](float alpha) {
+            uint32_t v[2][32];
+            tmem_ld32_issue(tmem_o + lane_base, v[0]);
+            tmem_ld32_issue(tmem_o + lane_base + 32, v[1]);
+            tmem_ld_wait();
 #pragma unroll
-            for (int c0 = 0; c0 < HEAD_DIM; c0 += 32) {
-                float v[32];
-                tmem_ld32(tmem_o + lane_base + c0, v);
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    o_acc[c0 + i] = o_acc[c0 + i] * alpha + v[i];
-            }
+            for (int i = 0; i < 64; ++i)
+                o_acc[i] = o_acc[i] * alpha + __uint_as_float(v[i >> 5][i & 31]);
         };
         for (int j = 0; j < ntiles; ++j) {
-            const uint32_t tmem_sj = tmem_s + 128 * (j & 1);
             if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
-            // pass 1: the row maximum of this tile's scaled scores
-            float mx = -INFINITY;
+            // this thread's 64 scores, scaled into the log2 domain, and their maximum
+            float sv[64];
+            {
+                uint32_t v[2][32];
+                tmem_ld32_issue(tmem_s + 128 * (j & 1) + lane_base, v[0]);
+                tmem_ld32_issue(tmem_s + 128 * (j & 1) + lane_base + 32, v[1]);
+                tmem_ld_wait();
 #pragma unroll
-            for (int c0 = 0; c0 < PF_TOK; c0 += 32) {
-                float v[32];
-                tmem_ld32(tmem_sj + lane_base + c0, v);
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    mx = fmaxf(mx, v[i] * p.scale_log2);
+                for (int i = 0; i < 64; ++i)
+                    sv[i] = __uint_as_float(v[i >> 5][i & 31]) * p.scale_log2;
             }
+            float mx = sv[0];
+#pragma unroll
+            for (int i = 1; i < 64; ++i)
+                mx = fmaxf(mx, sv[i]);
+            // the row's two halves must use one maximum: swap through shared memory
+            float *xb = xchg + (j & 1) * 256;
+            xb[half * 128 + r] = mx;
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(bar_x);
+            if (!mbar_wait_bounded(bar_x, (uint32_t)(j & 1), abort_flag)) {
+                ok = false;
+                break;
+            }
+            mx = fmaxf(mx, xb[(half ^ 1) * 128 + r]);
             const float m_new = fmaxf(m_run, mx);
             const float alpha = (m_run == -INFINITY) ? 0.f : fast_exp2(m_run - m_new);
-            // the previous tile's PV product must be folded in before its P buffer is overwritten
+            // weights, their sum, and P as bf16 high + low parts (kept in registers for now)
+            float lsum = 0.f;
+            uint32_t phi[32], plo[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+                const float p0 = fast_exp2(sv[2 * e] - m_new);
+                const float p1 = fast_exp2(sv[2 * e + 1] - m_new);
+                lsum += p0 + p1;
+                phi[e] = pack_bf16(p0, p1);
+                plo[e] = pack_bf16(p0 - bf16_lo_to_float(phi[e]), p1 - bf16_hi_to_float(phi[e]));
+            }
+            // the previous tile's PV product must be complete before its P buffer is overwritten; fold
+            // it into the row accumulators while we are at it
             if (j > 0) {
-                if (!mbar_wait_bounded(bar_o, (uint32_t)((j - 1) & 1), abort_flag)) {
+                if (!mbar_wait_bounded(bar_o + 8 * ((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1), abort_flag)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
                 add_o_tile(alpha_prev);
             }
-            // pass 2: weights, their sum, and P as bf16 high + low parts in the swizzled K-major layout
-            float lsum = 0.f;
+            // P into the swizzled K-major layout: token chunk c of 8 -> plane c >> 3 = this thread's
+            // half, position (c & 7) ^ (r & 7)
 #pragma unroll
-            for (int c0 = 0; c0 < PF_TOK; c0 += 32) {
-                float v[32];
-                tmem_ld32(tmem_sj + lane_base + c0, v);
-#pragma unroll
-                for (int q8 = 0; q8 < 4; ++q8) {   // 8 tokens = one 16-byte chunk
-                    uint32_t hi[4], lo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float p0 = fast_exp2(v[q8 * 8 + 2 * e] * p.scale_log2 - m_new);
-                        const float p1 = fast_exp2(v[q8 * 8 + 2 * e + 1] * p.scale_log2 - m_new);
-                        lsum += p0 + p1;
-                        hi[e] = pack_bf16(p0, p1);
-                        lo[e] = pack_bf16(p0 - bf16_lo_to_float(hi[e]), p1 - bf16_hi_to_float(hi[e]));
-                    }
-                    const int chunk = (c0 >> 3) + q8;   // 0..15 along tokens
-                    const uint32_t off = (uint32_t)((chunk >> 3) * PF_PLANE + r * 128 + (((chunk & 7) ^ (r & 7)) << 4));
-                    *reinterpret_cast<uint4 *>(smem + PF_OFF_PH + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<uint4 *>(smem + PF_OFF_PL + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                }
+            for (int q8 = 0; q8 < 8; ++q8) {
+                const uint32_t off = (uint32_t)(half * PF_PLANE + r * 128 + ((q8 ^ (r & 7)) << 4));
+                *reinterpret_cast<uint4 *>(smem + PF_OFF_PH + off) =
+                    make_uint4(phi[4 * q8], phi[4 * q8 + 1], phi[4 * q8 + 2], phi[4 * q8 + 3]);
+                *reinterpret_cast<uint4 *>(smem + PF_OFF_PL + off) =
+                    make_uint4(plo[4 * q8], plo[4 * q8 + 1], plo[4 * q8 + 2], plo[4 * q8 + 3]);
             }
             l_run = l_run * alpha + lsum;
             m_run = m_new;
@@ -394,12 +441,25 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             mbar_arrive(bar_p);
         }
         if (ok && ntiles > 0) {
-            if (mbar_wait_bounded(bar_o, (uint32_t)((ntiles - 1) & 1), abort_flag)) {
+            if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) & 1), (uint32_t)(((ntiles - 1) >> 1) & 1), abort_flag)) {
                 tc_fence_after();
                 add_o_tile(alpha_prev);
             } else {
                 ok = false;
             }
+        }
+        // the row's sum of weights is the sum of its two halves' sums (both relative to m_run)
+        float l_row = l_run;
+        if (ok && ntiles > 0) {
+            float *xb = xchg + (ntiles & 1) * 256;
+            xb[half * 128 + r] = l_run;
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(bar_x);
+            if (mbar_wait_bounded(bar_x, (uint32_t)(ntiles & 1), abort_flag))
+                l_row += xb[(half ^ 1) * 128 + r];
+            else
+                ok = false;
         }
         if (!ok) {
             if (*abort_flag == 0) {
@@ -412,26 +472,20 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 const int b = row / p.G, hi = row % p.G;
                 const int64_t bh = (int64_t)b * (p.Hkv * p.G) + g * p.G + hi;
                 const int64_t at = (int64_t)split * p.B * (p.Hkv * p.G) + bh;
-                float *dst = p.pre_o + at * HEAD_DIM;
-                if (ntiles > 0) {
-                    const float inv = 1.f / l_run;
+                float *dst = p.pre_o + at * HEAD_DIM + half * 64;
+                const float inv = ntiles > 0 ? 1.f / l_row : 0.f;
 #pragma unroll
-                    for (int i = 0; i < HEAD_DIM; i += 4)
-                        *reinterpret_cast<float4 *>(dst + i) =
-                            make_float4(o_acc[i] * inv, o_acc[i + 1] * inv, o_acc[i + 2] * inv, o_acc[i + 3] * inv);
-                    p.pre_lse[at] = (m_run + fast_log2(l_run)) * LN2;
-                } else {
-#pragma unroll
-                    for (int i = 0; i < HEAD_DIM; i += 4)
-                        *reinterpret_cast<float4 *>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
-                    p.pre_lse[at] = -INFINITY;
-                }
+                for (int i = 0; i < 64; i += 4)
+                    *reinterpret_cast<float4 *>(dst + i) =
+                        make_float4(o_acc[i] * inv, o_acc[i + 1] * inv, o_acc[i + 2] * inv, o_acc[i + 3] * inv);
+                if (half == 0)
+                    p.pre_lse[at] = ntiles > 0 ? (m_run + fast_log2(l_row)) * LN2 : -INFINITY;
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4)
+    if (warp == PF_DRV)
         tmem_dealloc(tmem, PF_TMEM_COLS);
 }
 
