@@ -273,7 +273,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 
             // The driver is an event loop: whichever of its four jobs has its inputs ready goes next.
             //   PV product of tile t : P(t) written (bar_p) and V(t) loaded
-            //   K load of tile t     : K buffer t & 1 free = S(t-2) consumed, known once P(t-2) was seen
+            //   K load of tile t     : K buffer t & 1 free = scores of tile t-2 complete (bar_s)
             //   V load of tile t     : V buffer t & 1 free = PV product of t-2 complete (bar_o)
             //   scores of tile t     : K(t) loaded and S buffer t & 1 free (P(t-2) seen)
             // so the scores of tile j+1 are computed while the softmax of tile j runs, and a slow load
@@ -293,6 +293,19 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             };
             while (next_o < ntiles) {
                 bool progress = false;
+                // loads first: issuing a batch of MMAs can stall this thread on the tensor queue
+                if (next_k < ntiles && next_s > next_k - 2 && ready(bar_s + 8 * (next_k & 1), (next_k - 2) >> 1)) {
+                    load_kv(next_k, page_k, false);   // the scores of tile next_k - 2 are complete: its K is dead
+                    ++next_k;
+                    page_k = read_page(next_k);
+                    progress = true;
+                }
+                if (next_v < ntiles && next_o > next_v - 2 && ready(bar_o + 8 * (next_v & 1), (next_v - 2) >> 1)) {
+                    load_kv(next_v, page_v, true);
+                    ++next_v;
+                    page_v = read_page(next_v);
+                    progress = true;
+                }
                 if (next_s < ntiles && next_s < next_k && next_o > next_s - 2 &&
                     ready(bar_kfull + 8 * (next_s & 1), next_s >> 1)) {
                     tc_fence_after();
@@ -306,18 +319,6 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     if (lane == 0)
                         mma_o(next_o);
                     ++next_o;
-                    progress = true;
-                }
-                if (next_k < ntiles && next_o > next_k - 2 && next_s > next_k - 2) {
-                    load_kv(next_k, page_k, false);
-                    ++next_k;
-                    page_k = read_page(next_k);
-                    progress = true;
-                }
-                if (next_v < ntiles && next_o > next_v - 2 && ready(bar_o + 8 * (next_v & 1), (next_v - 2) >> 1)) {
-                    load_kv(next_v, page_v, true);
-                    ++next_v;
-                    page_v = read_page(next_v);
                     progress = true;
                 }
                 if (progress) {
