@@ -7,8 +7,8 @@
 // prefix_kernel: one block = 128 query rows (row = b * G + head-in-group) of one KV head and one
 // range of 128-token KV tiles.  Per tile:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in TMEM)
 // -> the eight softmax warps read their rows of S (two threads per row, 64 columns each), keep running
-// max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts into swizzled shared memory
-// -> O_tile = P_hi V + P_lo V (two more tcgen05.mma into a second TMEM region) -> the softmax
+// max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts into tensor memory
+// -> O_tile = P_hi V + P_lo V (tcgen05.mma with the A operand in TMEM, into another TMEM region) -> the softmax
 // threads add O_tile into their fp32 row accumulators (rescaled when the max moved).  A ninth warp
 // drives TMA and issues the MMAs.  Result: a normalised partial (O / l, lse) per (split, b, h),
 // combined with the per-sequence suffix attention by cascade_merge_kernel.
@@ -20,19 +20,19 @@ namespace da {
 constexpr int PF_ROWS = 128;                 // query rows per block (UMMA M)
 constexpr int PF_TOK = 128;                  // tokens per KV tile (UMMA N for S, K for PV)
 constexpr int PF_PLANE = PF_TOK * 128;       // one 64-column half of a 128-row tile: 128-byte rows
-constexpr int PF_TILE = 2 * PF_PLANE;        // 32 KB: Q, a K tile, a V tile, P_hi, P_lo
+constexpr int PF_TILE = 2 * PF_PLANE;        // 32 KB: Q, a K tile, a V tile
 constexpr int PF_DRV = 8;                    // warps 0..7: softmax (two threads per row); warp 8: driver
 constexpr int PF_THREADS = (PF_DRV + 1) * 32;
 constexpr int PF_OFF_Q = 0;
 constexpr int PF_OFF_K = PF_TILE;            // two K buffers
 constexpr int PF_OFF_V = 3 * PF_TILE;        // two V buffers
-constexpr int PF_OFF_PH = 5 * PF_TILE;
-constexpr int PF_OFF_PL = 6 * PF_TILE;
-constexpr int PF_OFF_BARS = 7 * PF_TILE;     // kfull[2], vfull[2], s[2], o[2], p, x
+constexpr int PF_OFF_BARS = 5 * PF_TILE;     // kfull[2], vfull[2], s[2], o[2], p, x
 constexpr int PF_OFF_MISC = PF_OFF_BARS + 96;   // TMEM base address, abort flag
 constexpr int PF_OFF_XCHG = PF_OFF_MISC + 16;   // row maxima / sums swapped between a row's two threads
 constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + 2 * 2 * 128 * 4;
-constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O_tile in [256,384)
+constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O_tile in [256,384),
+constexpr int PF_TMEM_PH = 384;              // P high parts in [384,448), low parts in [448,512): 128 tokens as
+constexpr int PF_TMEM_PL = 448;              // 64 columns of bf16 pairs, the A operand of the PV product
 
 struct PrefixParams {
     const __nv_bfloat16 *q;
@@ -124,6 +124,28 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 32 consecutive 32-bit columns of this thread's TMEM lane, written from registers.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,"
+        "%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// D += A * B with the A operand in tensor memory (row i in lane i, two bf16 of K per column).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
 // The K/V pools are read here through a 4-D tiled map {d, token, head, page} with box {64, box_rows, 1, 1}:
 // one box is one 64-column plane of box_rows token rows, so a plane of a tile is contiguous and
 // its 8-row groups are 1024 bytes apart, which is what the matrix descriptors above assume.
@@ -259,13 +281,13 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 const uint32_t idesc = umma_idesc(PF_ROWS, HEAD_DIM, true);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    const uint32_t pb = sb + (half ? PF_OFF_PL : PF_OFF_PH);
+                    const uint32_t pa = tmem + (half ? PF_TMEM_PL : PF_TMEM_PH);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
-                        // A = P (K-major over tokens), B = V stored [token][d]: MN-major, planes are the
-                        // two halves of d (leading offset = plane), 8-token groups 1024 B apart
-                        umma_bf16(tmem_o, umma_desc(pb + (kk >> 2) * PF_PLANE + (kk & 3) * 32, 16, 1024),
-                                  umma_desc(vb + kk * 2048, PF_PLANE, 1024), idesc, half > 0 || kk > 0);
+                        // A = P from tensor memory (16 tokens = 8 columns per step); B = V stored
+                        // [token][d]: MN-major, planes are the two halves of d (leading offset = plane),
+                        // 8-token groups 1024 B apart
+                        umma_bf16_ts(tmem_o, pa + kk * 8, umma_desc(vb + kk * 2048, PF_PLANE, 1024), idesc, half > 0 || kk > 0);
                     }
                 }
                 umma_commit(bar_o + 8 * (j & 1));
@@ -424,21 +446,14 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 tc_fence_after();
                 add_o_tile(alpha_prev);
             }
-            // P into the swizzled K-major layout: token chunk c of 8 -> plane c >> 3 = this thread's
-            // half, position (c & 7) ^ (r & 7)
-#pragma unroll
-            for (int q8 = 0; q8 < 8; ++q8) {
-                const uint32_t off = (uint32_t)(half * PF_PLANE + r * 128 + ((q8 ^ (r & 7)) << 4));
-                *reinterpret_cast<uint4 *>(smem + PF_OFF_PH + off) =
-                    make_uint4(phi[4 * q8], phi[4 * q8 + 1], phi[4 * q8 + 2], phi[4 * q8 + 3]);
-                *reinterpret_cast<uint4 *>(smem + PF_OFF_PL + off) =
-                    make_uint4(plo[4 * q8], plo[4 * q8 + 1], plo[4 * q8 + 2], plo[4 * q8 + 3]);
-            }
+            // P into tensor memory: this thread's 64 tokens are 32 columns of bf16 pairs
+            tmem_st32(tmem + PF_TMEM_PH + ((uint32_t)(32 * (warp & 3)) << 16) + half * 32, phi);
+            tmem_st32(tmem + PF_TMEM_PL + ((uint32_t)(32 * (warp & 3)) << 16) + half * 32, plo);
+            tmem_st_wait();
             l_run = l_run * alpha + lsum;
             m_run = m_new;
             alpha_prev = alpha;
-            fence_proxy_async_smem();   // P is read by the tensor core through the async proxy
-            tc_fence_before();          // and this thread's TMEM reads precede the MMAs that follow
+            tc_fence_before();          // this thread's TMEM reads and writes precede the MMAs that follow
             mbar_arrive(bar_p);
         }
         if (ok && ntiles > 0) {
