@@ -10,7 +10,7 @@
 // max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts into tensor memory
 // -> O_tile = P_hi V + P_lo V (tcgen05.mma with the A operand in TMEM, into another TMEM region) -> the softmax
 // threads add O_tile into their fp32 row accumulators (rescaled when the max moved).  A ninth warp
-// drives TMA and issues the MMAs.  Result: a normalised partial (O / l, lse) per (split, b, h),
+// issues the MMAs and a tenth the TMA loads (one warp doing both spent most of a tile's time issuing).  Result: a normalised partial (O / l, lse) per (split, b, h),
 // combined with the per-sequence suffix attention by cascade_merge_kernel.
 #pragma once
 #include "da_kernels.cuh"
@@ -21,13 +21,16 @@ constexpr int PF_ROWS = 128;                 // query rows per block (UMMA M)
 constexpr int PF_TOK = 128;                  // tokens per KV tile (UMMA N for S, K for PV)
 constexpr int PF_PLANE = PF_TOK * 128;       // one 64-column half of a 128-row tile: 128-byte rows
 constexpr int PF_TILE = 2 * PF_PLANE;        // 32 KB: Q, a K tile, a V tile
-constexpr int PF_DRV = 8;                    // warps 0..7: softmax (two threads per row); warp 8: driver
-constexpr int PF_THREADS = (PF_DRV + 1) * 32;
+constexpr int PF_DRV = 8;                    // warps 0..7: softmax (two threads per row); warp 8: issues the
+constexpr int PF_LOADER = 9;                 // MMAs (and owns the TMEM allocation); warp 9: issues the TMA loads
+constexpr int PF_THREADS = (PF_LOADER + 1) * 32;
 constexpr int PF_OFF_Q = 0;
-constexpr int PF_OFF_K = PF_TILE;            // two K buffers
-constexpr int PF_OFF_V = 3 * PF_TILE;        // two V buffers
-constexpr int PF_OFF_BARS = 5 * PF_TILE;     // kfull[2], vfull[2], s[2], o[2], p, x
-constexpr int PF_OFF_MISC = PF_OFF_BARS + 96;   // TMEM base address, abort flag
+constexpr uint32_t PF_WAIT_SLEEP_NS = 64;     // softmax warps yield while they wait: the driver warp shares their schedulers
+constexpr int PF_NB = 3;                     // K and V buffers (tiles in flight)
+constexpr int PF_OFF_K = PF_TILE;
+constexpr int PF_OFF_V = (1 + PF_NB) * PF_TILE;
+constexpr int PF_OFF_BARS = (1 + 2 * PF_NB) * PF_TILE;   // kfull[3], vfull[3], kfree[3], o[3], s[2], p, x
+constexpr int PF_OFF_MISC = PF_OFF_BARS + 128;  // TMEM base address, abort flag
 constexpr int PF_OFF_XCHG = PF_OFF_MISC + 16;   // row maxima / sums swapped between a row's two threads
 constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + 2 * 2 * 128 * 4;
 constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O_tile in [256,384),
@@ -166,8 +169,10 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     int &abort_s = *reinterpret_cast<int *>(smem + PF_OFF_MISC + 4);
     const uint32_t sb = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t bar_kfull = sb + PF_OFF_BARS, bar_vfull = bar_kfull + 16, bar_s = bar_kfull + 32, bar_o = bar_kfull + 48,
-                   bar_p = bar_kfull + 64, bar_x = bar_kfull + 72;   // bar_o is a pair: tile t uses bar_o + 8 * (t & 1)
+    // per K/V buffer (tile t uses buffer t % 3): K loaded, V loaded, K no longer needed (scores complete),
+    // PV product complete; per S buffer (t & 1): scores complete; P written; row-maximum exchange
+    const uint32_t bar_kfull = sb + PF_OFF_BARS, bar_vfull = bar_kfull + 24, bar_kfree = bar_kfull + 48, bar_o = bar_kfull + 72,
+                   bar_s = bar_kfull + 96, bar_p = bar_kfull + 112, bar_x = bar_kfull + 120;
     volatile int *abort_flag = &abort_s;
 
     // block -> (row tile, kv head, split)
@@ -186,14 +191,14 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     }
     if (tid == 0) {
         abort_s = 0;
-        mbar_init(bar_kfull, 1);
-        mbar_init(bar_kfull + 8, 1);
-        mbar_init(bar_vfull, 1);
-        mbar_init(bar_vfull + 8, 1);
+        for (int i = 0; i < PF_NB; ++i) {
+            mbar_init(bar_kfull + 8 * i, 1);
+            mbar_init(bar_vfull + 8 * i, 1);
+            mbar_init(bar_kfree + 8 * i, 1);
+            mbar_init(bar_o + 8 * i, 1);
+        }
         mbar_init(bar_s, 1);
         mbar_init(bar_s + 8, 1);
-        mbar_init(bar_o, 1);
-        mbar_init(bar_o + 8, 1);
         mbar_init(bar_p, 2 * PF_ROWS);
         mbar_init(bar_x, PF_DRV);
         mbar_fence_init();
@@ -227,46 +232,100 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const uint32_t tmem = tmem_base_s;
     const uint32_t tmem_s = tmem, tmem_o = tmem + 256;   // S(j) lives at tmem_s + 128 * (j & 1)
 
-    if (warp == PF_DRV) {
-        // ------------------------------------------------------------------ driver warp: TMA + MMA issue
-        // All lanes walk the same control flow (waits included); lane bx < boxes reads the page id of
-        // box bx of a tile and issues its four loads; lane 0 alone arms barriers and issues the MMAs.
+    if (warp == PF_LOADER) {
+        // ------------------------------------------------------------------ loader warp: TMA
+        // Lane l < 2 * boxes issues one load per call: box l >> 1 (box_rows tokens of one page), plane
+        // l & 1.  Tiles 0..2 fill the three buffers; after that K(t) follows the completion of the
+        // scores of tile t-3 (bar_kfree) and V(t) the completion of the PV product of tile t-3
+        // (bar_o).  The tensor core finishes S(t-2) before PV(t-3), so the order is K(t), V(t-1).
         if (ntiles > 0) {
             const int boxes = PF_TOK / p.box_rows;
-            const uint32_t tile_bytes = (uint32_t)PF_TILE;
+            const int box = lane >> 1, pl = lane & 1;
+            const bool active = lane < 2 * boxes;
             bool ok = true;
-            int issued = 0;   // tiles whose loads were issued
+            int issued_k = 0, issued_v = 0;
             auto read_page = [&](int j) {   // page id of this lane's box of tile j (0 for idle lanes)
-                if (lane >= boxes || j >= ntiles)
+                if (!active || j >= ntiles)
                     return 0;
-                const int t = (t_begin + j) * PF_TOK + lane * p.box_rows;
-                return __ldg(p.block_table + t / p.P);
+                return __ldg(p.block_table + ((t_begin + j) * PF_TOK + box * p.box_rows) / p.P);
             };
-            auto load_kv = [&](int j, int page, bool is_v) {   // K or V of tile j into buffer j & 1
-                const int buf = j & 1;
+            auto load_kv = [&](int j, int page, bool is_v) {   // K or V of tile j into buffer j % 3
+                const int buf = j % PF_NB;
                 const uint32_t bar = (is_v ? bar_vfull : bar_kfull) + 8 * buf;
-                if (is_v)
-                    issued = j + 1;
                 if (lane == 0)
-                    mbar_arrive_expect_tx(bar, tile_bytes);
+                    mbar_arrive_expect_tx(bar, (uint32_t)PF_TILE);
                 __syncwarp();
-                if (lane < boxes) {
-                    const int t = (t_begin + j) * PF_TOK + lane * p.box_rows;
+                if (active) {
+                    const int t = (t_begin + j) * PF_TOK + box * p.box_rows;
                     if ((uint32_t)page >= (uint32_t)p.num_pages) {
-                        if (!is_v)
+                        if (!is_v && pl == 0)
                             report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, 0, t / p.P, page);
                         page = p.num_pages;   // out of range: TMA fills zeros and still counts the bytes
                     }
-                    const int row = t % p.P;
-#pragma unroll
-                    for (int pl = 0; pl < 2; ++pl) {
-                        const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + lane * p.box_rows * 128);
-                        tma_load_4d(sb + (is_v ? PF_OFF_V : PF_OFF_K) + off, is_v ? &tm_v : &tm_k, pl * 64, row, g, page, bar);
+                    const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + box * p.box_rows * 128);
+                    tma_load_4d(sb + (is_v ? PF_OFF_V : PF_OFF_K) + off, is_v ? &tm_v : &tm_k, pl * 64, t % p.P, g, page, bar);
+                }
+                if (is_v)
+                    issued_v = j + 1;
+                else
+                    issued_k = j + 1;
+            };
+            int pg_k = read_page(0);
+            for (int j = 0; j < PF_NB && j < ntiles; ++j) {
+                const int pg = pg_k;
+                pg_k = read_page(j + 1);
+                load_kv(j, pg, false);
+                load_kv(j, pg, true);
+            }
+            int pg_v = pg_k;   // page ids of tile 3, fetched ahead
+            for (int t = PF_NB; ok && t <= ntiles; ++t) {
+                if (t < ntiles) {
+                    ok = mbar_wait_bounded(bar_kfree + 8 * (t % PF_NB), (uint32_t)(((t - PF_NB) / PF_NB) & 1), abort_flag);
+                    if (!ok)
+                        break;
+                    const int pg = pg_k;
+                    pg_k = read_page(t + 1);
+                    load_kv(t, pg, false);
+                }
+                const int tv = t - 1;   // V of the tile before
+                if (tv >= PF_NB) {
+                    ok = mbar_wait_bounded(bar_o + 8 * (tv % PF_NB), (uint32_t)(((tv - PF_NB) / PF_NB) & 1), abort_flag);
+                    if (!ok)
+                        break;
+                    const int pg = pg_v;
+                    pg_v = read_page(tv + 1);
+                    load_kv(tv, pg, true);
+                }
+            }
+            if (!ok && lane == 0) {
+                if (*abort_flag == 0) {
+                    *abort_flag = 1;
+                    report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -9, (int)blockIdx.x, 0);
+                }
+            }
+            if (*abort_flag && lane == 0) {
+                // do not leave while copies may still land in shared memory: bounded wait for the
+                // latest fill of each buffer
+                for (int k = 0; k < PF_NB; ++k) {
+                    const int jk = issued_k - 1 - k, jv = issued_v - 1 - k;
+                    const uint64_t t0 = globaltimer_ns();
+                    while ((jk >= 0 && !mbar_try_wait(bar_kfull + 8 * (jk % PF_NB), (uint32_t)((jk / PF_NB) & 1))) ||
+                           (jv >= 0 && !mbar_try_wait(bar_vfull + 8 * (jv % PF_NB), (uint32_t)((jv / PF_NB) & 1)))) {
+                        if (globaltimer_ns() - t0 > 1000000000ull)
+                            break;
                     }
                 }
-            };
+            }
+        }
+    } else if (warp == PF_DRV) {
+        // ------------------------------------------------------------------ MMA warp
+        // All lanes wait together; lane 0 issues.  Order on the tensor core: S(0), S(1), then for every
+        // tile j: PV(j) as soon as P(j) is written, and S(j+2) into the S buffer the softmax of j has
+        // just released -- so the scores of tile j+1 are ready before the softmax of j ends.
+        if (ntiles > 0) {
+            bool ok = true;
             auto mma_s = [&](int j) {   // S = Q K^T for tile j
-                const uint32_t kb = sb + PF_OFF_K + (j & 1) * PF_TILE;
+                const uint32_t kb = sb + PF_OFF_K + (j % PF_NB) * PF_TILE;
                 const uint32_t idesc = umma_idesc(PF_ROWS, PF_TOK, false);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
@@ -275,9 +334,10 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                               idesc, kk > 0);
                 }
                 umma_commit(bar_s + 8 * (j & 1));
+                umma_commit(bar_kfree + 8 * (j % PF_NB));
             };
             auto mma_o = [&](int j) {   // O_tile = P_hi V + P_lo V for tile j
-                const uint32_t vb = sb + PF_OFF_V + (j & 1) * PF_TILE;
+                const uint32_t vb = sb + PF_OFF_V + (j % PF_NB) * PF_TILE;
                 const uint32_t idesc = umma_idesc(PF_ROWS, HEAD_DIM, true);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
@@ -290,82 +350,42 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         umma_bf16_ts(tmem_o, pa + kk * 8, umma_desc(vb + kk * 2048, PF_PLANE, 1024), idesc, half > 0 || kk > 0);
                     }
                 }
-                umma_commit(bar_o + 8 * (j & 1));
+                umma_commit(bar_o + 8 * (j % PF_NB));
             };
-
-            // The driver is an event loop: whichever of its four jobs has its inputs ready goes next.
-            //   PV product of tile t : P(t) written (bar_p) and V(t) loaded
-            //   K load of tile t     : K buffer t & 1 free = scores of tile t-2 complete (bar_s)
-            //   V load of tile t     : V buffer t & 1 free = PV product of t-2 complete (bar_o)
-            //   scores of tile t     : K(t) loaded and S buffer t & 1 free (P(t-2) seen)
-            // so the scores of tile j+1 are computed while the softmax of tile j runs, and a slow load
-            // never delays a PV product whose inputs are ready.
-            int page0 = read_page(0), page1 = read_page(1);
-            load_kv(0, page0, false);
-            load_kv(0, page0, true);
-            if (ntiles > 1) {
-                load_kv(1, page1, false);
-                load_kv(1, page1, true);
+            auto kfull = [&](int j) {
+                return mbar_wait_bounded(bar_kfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag);
+            };
+            for (int j = 0; ok && j < 2 && j < ntiles; ++j) {
+                ok = kfull(j);
+                if (ok) {
+                    tc_fence_after();
+                    if (lane == 0)
+                        mma_s(j);
+                    __syncwarp();
+                }
             }
-            int next_o = 0, next_s = 0, next_k = min(2, ntiles), next_v = min(2, ntiles);
-            int page_k = read_page(2), page_v = page_k;   // page ids are fetched ahead of their use
-            uint64_t t_last = globaltimer_ns();
-            auto ready = [&](uint32_t bar, int n) {   // has the n-th completion of `bar` happened? (warp-uniform)
-                return __all_sync(0xffffffffu, mbar_test_wait(bar, (uint32_t)(n & 1)));
-            };
-            while (next_o < ntiles) {
-                bool progress = false;
-                // loads first: issuing a batch of MMAs can stall this thread on the tensor queue
-                if (next_k < ntiles && next_s > next_k - 2 && ready(bar_s + 8 * (next_k & 1), (next_k - 2) >> 1)) {
-                    load_kv(next_k, page_k, false);   // the scores of tile next_k - 2 are complete: its K is dead
-                    ++next_k;
-                    page_k = read_page(next_k);
-                    progress = true;
-                }
-                if (next_v < ntiles && next_o > next_v - 2 && ready(bar_o + 8 * (next_v & 1), (next_v - 2) >> 1)) {
-                    load_kv(next_v, page_v, true);
-                    ++next_v;
-                    page_v = read_page(next_v);
-                    progress = true;
-                }
-                if (next_s < ntiles && next_s < next_k && next_o > next_s - 2 &&
-                    ready(bar_kfull + 8 * (next_s & 1), next_s >> 1)) {
-                    tc_fence_after();
-                    if (lane == 0)
-                        mma_s(next_s);
-                    ++next_s;
-                    progress = true;
-                }
-                if (ready(bar_p, next_o) && ready(bar_vfull + 8 * (next_o & 1), next_o >> 1)) {
-                    tc_fence_after();
-                    if (lane == 0)
-                        mma_o(next_o);
-                    ++next_o;
-                    progress = true;
-                }
-                if (progress) {
-                    t_last = globaltimer_ns();
-                } else if (*abort_flag || globaltimer_ns() - t_last > 2000000000ull) {
-                    ok = false;
+            for (int j = 0; ok && j < ntiles; ++j) {
+                ok = mbar_wait_bounded(bar_p, (uint32_t)(j & 1), abort_flag) &&
+                     mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag);
+                if (!ok)
                     break;
+                tc_fence_after();
+                if (lane == 0)
+                    mma_o(j);
+                __syncwarp();
+                if (j + 2 < ntiles) {
+                    ok = kfull(j + 2);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    if (lane == 0)
+                        mma_s(j + 2);
+                    __syncwarp();
                 }
             }
-            if (!ok && lane == 0) {
+            if (!ok && lane == 0 && *abort_flag == 0) {
                 *abort_flag = 1;
                 report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -7, (int)blockIdx.x, 0);
-                // do not leave while copies may still land in shared memory: bounded wait for the
-                // latest fill of each buffer
-                for (int j = ntiles - 1, seen = 0; j >= 0 && seen < 2; --j) {
-                    if (j >= issued)
-                        continue;
-                    ++seen;
-                    const uint64_t t0 = globaltimer_ns();
-                    while (!(mbar_try_wait(bar_kfull + 8 * (j & 1), (uint32_t)((j >> 1) & 1)) &&
-                             mbar_try_wait(bar_vfull + 8 * (j & 1), (uint32_t)((j >> 1) & 1)))) {
-                        if (globaltimer_ns() - t0 > 1000000000ull)
-                            break;
-                    }
-                }
             }
         }
     } else {
@@ -392,7 +412,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 o_acc[i] = o_acc[i] * alpha + __uint_as_float(v[i >> 5][i & 31]);
         };
         for (int j = 0; j < ntiles; ++j) {
-            if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag)) {
+            if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                 ok = false;
                 break;
             }
@@ -418,7 +438,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_x);
-            if (!mbar_wait_bounded(bar_x, (uint32_t)(j & 1), abort_flag)) {
+            if (!mbar_wait_bounded(bar_x, (uint32_t)(j & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                 ok = false;
                 break;
             }
@@ -439,7 +459,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             // the previous tile's PV product must be complete before its P buffer is overwritten; fold
             // it into the row accumulators while we are at it
             if (j > 0) {
-                if (!mbar_wait_bounded(bar_o + 8 * ((j - 1) & 1), (uint32_t)(((j - 1) >> 1) & 1), abort_flag)) {
+                if (!mbar_wait_bounded(bar_o + 8 * ((j - 1) % PF_NB), (uint32_t)(((j - 1) / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                     ok = false;
                     break;
                 }
@@ -457,7 +477,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             mbar_arrive(bar_p);
         }
         if (ok && ntiles > 0) {
-            if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) & 1), (uint32_t)(((ntiles - 1) >> 1) & 1), abort_flag)) {
+            if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) % PF_NB), (uint32_t)(((ntiles - 1) / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                 tc_fence_after();
                 add_o_tile(alpha_prev);
             } else {
@@ -472,7 +492,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_x);
-            if (mbar_wait_bounded(bar_x, (uint32_t)(ntiles & 1), abort_flag))
+            if (mbar_wait_bounded(bar_x, (uint32_t)(ntiles & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS))
                 l_row += xb[(half ^ 1) * 128 + r];
             else
                 ok = false;

@@ -66,8 +66,10 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
 // Waits until the phase with the given parity has completed.  Every wait is bounded: after
 // `limit_ns` without completion, or as soon as another thread of the block has raised the
 // abort flag, it gives up and returns false, so a pipeline bug cannot hang the device.
+// `sleep_ns` > 0 makes a waiting warp yield its issue slots between probes (for waits whose
+// outcome depends on another warp of the same scheduler getting to run).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                                  uint64_t limit_ns = 2000000000ull)
+                                                  uint64_t limit_ns = 2000000000ull, uint32_t sleep_ns = 0)
 {
     if (mbar_try_wait(bar, parity))
         return true;
@@ -78,6 +80,8 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     for (;;) {
         if (mbar_try_wait(bar, parity))
             return true;
+        if (sleep_ns)
+            __nanosleep(sleep_ns);
         if (((++spins) & 0x3F) == 0) {
             if (*abort_flag)
                 return false;
