@@ -8,8 +8,8 @@
 // range of 128-token KV tiles.  Per tile:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in TMEM)
 // -> the eight softmax warps read their rows of S (two threads per row, 64 columns each), keep running
 // max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts into tensor memory
-// -> O_tile = P_hi V + P_lo V (tcgen05.mma with the A operand in TMEM, into another TMEM region) -> the softmax
-// threads add O_tile into their fp32 row accumulators (rescaled when the max moved).  A ninth warp
+// -> O += P_hi V + P_lo V (tcgen05.mma with the A operand in TMEM, accumulating in another TMEM region) -> the softmax
+// threads rescale a row of O in TMEM only when its maximum has grown by more than 2^8 (rare).  A ninth warp
 // issues the MMAs and a tenth the TMA loads (one warp doing both spent most of a tile's time issuing).  Result: a normalised partial (O / l, lse) per (split, b, h),
 // combined with the per-sequence suffix attention by cascade_merge_kernel.
 #pragma once
@@ -25,6 +25,7 @@ constexpr int PF_DRV = 8;                    // warps 0..7: softmax (two threads
 constexpr int PF_LOADER = 9;                 // MMAs (and owns the TMEM allocation); warp 9: issues the TMA loads
 constexpr int PF_THREADS = (PF_LOADER + 1) * 32;
 constexpr int PF_OFF_Q = 0;
+constexpr float PF_RESCALE_LOG2 = 8.f;       // a row's reference maximum moves only when the maximum grew by more
 constexpr uint32_t PF_WAIT_SLEEP_NS = 64;     // softmax warps yield while they wait: the driver warp shares their schedulers
 constexpr int PF_NB = 3;                     // K and V buffers (tiles in flight)
 constexpr int PF_OFF_K = PF_TILE;
@@ -347,7 +348,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         // A = P from tensor memory (16 tokens = 8 columns per step); B = V stored
                         // [token][d]: MN-major, planes are the two halves of d (leading offset = plane),
                         // 8-token groups 1024 B apart
-                        umma_bf16_ts(tmem_o, pa + kk * 8, umma_desc(vb + kk * 2048, PF_PLANE, 1024), idesc, half > 0 || kk > 0);
+                        umma_bf16_ts(tmem_o, pa + kk * 8, umma_desc(vb + kk * 2048, PF_PLANE, 1024), idesc, j > 0 || half > 0 || kk > 0);
                     }
                 }
                 umma_commit(bar_o + 8 * (j % PF_NB));
@@ -396,21 +397,12 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         const int half = warp >> 2;
         const uint32_t lane_base = ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(half * 64);
         float *xchg = reinterpret_cast<float *>(smem + PF_OFF_XCHG);   // [2 buffers][2 halves][128 rows]
-        float m_run = -INFINITY, l_run = 0.f, alpha_prev = 1.f;
-        float o_acc[64];
-#pragma unroll
-        for (int i = 0; i < 64; ++i)
-            o_acc[i] = 0.f;
+        // O accumulates in tensor memory across tiles, relative to a reference maximum m_run that is
+        // moved only when a row's maximum has grown by more than PF_RESCALE_LOG2 (weights then stay
+        // below 2^PF_RESCALE_LOG2, well inside what the bf16 high + low pair carries); moving it
+        // means scaling that row of O, which after the first few tiles is rare.
+        float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;
-        auto add_o_tile = [&](float alpha) {
-            uint32_t v[2][32];
-            tmem_ld32_issue(tmem_o + lane_base, v[0]);
-            tmem_ld32_issue(tmem_o + lane_base + 32, v[1]);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 64; ++i)
-                o_acc[i] = o_acc[i] * alpha + __uint_as_float(v[i >> 5][i & 31]);
-        };
         for (int j = 0; j < ntiles; ++j) {
             if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                 ok = false;
@@ -443,8 +435,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 break;
             }
             mx = fmaxf(mx, xb[(half ^ 1) * 128 + r]);
-            const float m_new = fmaxf(m_run, mx);
-            const float alpha = (m_run == -INFINITY) ? 0.f : fast_exp2(m_run - m_new);
+            const bool moved = (m_run == -INFINITY) || (mx > m_run + PF_RESCALE_LOG2);
+            const float m_new = moved ? mx : m_run;
+            const float alpha = !moved ? 1.f : (m_run == -INFINITY ? 0.f : fast_exp2(m_run - m_new));
             // weights, their sum, and P as bf16 high + low parts (kept in registers for now)
             float lsum = 0.f;
             uint32_t phi[32], plo[32];
@@ -456,15 +449,25 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 phi[e] = pack_bf16(p0, p1);
                 plo[e] = pack_bf16(p0 - bf16_lo_to_float(phi[e]), p1 - bf16_hi_to_float(phi[e]));
             }
-            // the previous tile's PV product must be complete before its P buffer is overwritten; fold
-            // it into the row accumulators while we are at it
+            // the previous tile's PV product must be complete before its P buffer is overwritten, and
+            // before a row of O is rescaled
             if (j > 0) {
                 if (!mbar_wait_bounded(bar_o + 8 * ((j - 1) % PF_NB), (uint32_t)(((j - 1) / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                add_o_tile(alpha_prev);
+                if (__any_sync(0xffffffffu, moved)) {   // tcgen05.ld / .st are warp-wide: all lanes go
+                    uint32_t v[2][32];
+                    tmem_ld32_issue(tmem_o + lane_base, v[0]);
+                    tmem_ld32_issue(tmem_o + lane_base + 32, v[1]);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 64; ++i)
+                        v[i >> 5][i & 31] = __float_as_uint(__uint_as_float(v[i >> 5][i & 31]) * alpha);
+                    tmem_st32(tmem_o + lane_base, v[0]);
+                    tmem_st32(tmem_o + lane_base + 32, v[1]);
+                }
             }
             // P into tensor memory: this thread's 64 tokens are 32 columns of bf16 pairs
             tmem_st32(tmem + PF_TMEM_PH + ((uint32_t)(32 * (warp & 3)) << 16) + half * 32, phi);
@@ -472,14 +475,16 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             tmem_st_wait();
             l_run = l_run * alpha + lsum;
             m_run = m_new;
-            alpha_prev = alpha;
             tc_fence_before();          // this thread's TMEM reads and writes precede the MMAs that follow
             mbar_arrive(bar_p);
         }
+        uint32_t o_raw[2][32];
         if (ok && ntiles > 0) {
             if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) % PF_NB), (uint32_t)(((ntiles - 1) / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                 tc_fence_after();
-                add_o_tile(alpha_prev);
+                tmem_ld32_issue(tmem_o + lane_base, o_raw[0]);
+                tmem_ld32_issue(tmem_o + lane_base + 32, o_raw[1]);
+                tmem_ld_wait();
             } else {
                 ok = false;
             }
@@ -511,9 +516,13 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 float *dst = p.pre_o + at * HEAD_DIM + half * 64;
                 const float inv = ntiles > 0 ? 1.f / l_row : 0.f;
 #pragma unroll
-                for (int i = 0; i < 64; i += 4)
-                    *reinterpret_cast<float4 *>(dst + i) =
-                        make_float4(o_acc[i] * inv, o_acc[i + 1] * inv, o_acc[i + 2] * inv, o_acc[i + 3] * inv);
+                for (int i = 0; i < 64; i += 4) {
+                    float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (ntiles > 0)
+                        v4 = make_float4(__uint_as_float(o_raw[i >> 5][i & 31]) * inv, __uint_as_float(o_raw[i >> 5][(i + 1) & 31]) * inv,
+                                         __uint_as_float(o_raw[i >> 5][(i + 2) & 31]) * inv, __uint_as_float(o_raw[i >> 5][(i + 3) & 31]) * inv);
+                    *reinterpret_cast<float4 *>(dst + i) = v4;
+                }
                 if (half == 0)
                     p.pre_lse[at] = ntiles > 0 ? (m_run + fast_log2(l_row)) * LN2 : -INFINITY;
             }
