@@ -230,7 +230,8 @@ int64_t decode_attn_get_option(const char *name);
 /*
  * decode_attn_set_profile_events -- timing aid.  While both handles are non-NULL, every
  * decode_attn() call records `before` (a cudaEvent_t) on its stream just before the partition
- * kernel's launch and `after` just after it, so that a benchmark can time that kernel alone.
+ * kernel's launch and `after` just after it, so that a benchmark can time that kernel alone
+ * (decode_attn_cascade() brackets its prefix kernel instead).
  * Pass NULL, NULL to stop.  The events stay owned by the caller.
  */
 int decode_attn_set_profile_events(void *before, void *after);

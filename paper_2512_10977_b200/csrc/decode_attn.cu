@@ -16,7 +16,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 101;
+constexpr int kVersion = 102;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -504,8 +504,13 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     sl.ndim = 2;
     sl.shape[0] = d.B; sl.shape[1] = d.Hq; sl.shape[2] = sl.shape[3] = 0;
     sl.stride[0] = d.Hq; sl.stride[1] = 1; sl.stride[2] = sl.stride[3] = 0;
+    // (profile events, if set, bracket the prefix kernel in this entry point, not the partition kernel)
+    cudaEvent_t ev_before = g_ev_before, ev_after = g_ev_after;
+    g_ev_before = g_ev_after = nullptr;
     rc = launch_path(st, d, ws, lay, nblocks, n_tail, q, k_pages, v_pages, block_table, seq_lens, 0, scale, &so, &sl, stream,
                      shared_prefix_tokens);
+    g_ev_before = ev_before;
+    g_ev_after = ev_after;
     if (rc != DA_OK) return rc;
 
     // 2. attention of every query row over the shared prefix, on the tensor cores
@@ -540,9 +545,12 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     pf.scale_log2 = scale * LOG2E;
     const long long grid = (long long)pf.row_tiles * pf.Hkv * splits;
     if (grid > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+    const bool timed = ev_before && ev_after;
+    if (timed) DA_CUDA(cudaEventRecord(ev_before, stream));
     prefix_kernel<<<(unsigned)grid, PF_THREADS, PF_SMEM_BYTES, stream>>>(tm_k, tm_v, pf);
     g_launches.fetch_add(1);
     DA_CUDA(cudaGetLastError());
+    if (timed) DA_CUDA(cudaEventRecord(ev_after, stream));
 
     // 3. fold prefix partials and suffix result
     CascadeMergeParams cm;
