@@ -131,6 +131,22 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
                         void *stream);
 
 /*
+ * decode_attn_append -- the step that precedes decode_attn() in each layer of a decoding loop:
+ * writes the new token's key and value vectors into the paged cache (the per-token growth of the
+ * sessions' contexts; paper Sec. 3.2, the dialog that every FSM iteration extends).
+ *
+ *   k_new, v_new  bf16 [B, Hkv, 128], last dim contiguous, base and strides multiples of 16 bytes
+ *   k_pages, v_pages, block_table, seq_lens   as in decode_attn(); the pools are WRITTEN
+ * seq_lens already counts the new token: its rows go to position L-1, i.e. page
+ * block_table[b][(L-1)/P], row (L-1) % P, of every KV head.  L <= 0 writes nothing; L < 0 or a
+ * position beyond the block-table row sets DA_DEV_BAD_SEQLEN, a page id outside the pool sets
+ * DA_DEV_BAD_PAGE, and that sequence is skipped.  Needs a registered workspace (for the status
+ * record).  One kernel on `stream`; no RoPE or other transform is applied to the vectors.
+ */
+int decode_attn_append(const da_tensor *k_new, const da_tensor *v_new, da_tensor *k_pages, da_tensor *v_pages,
+                       const da_tensor *block_table, const da_tensor *seq_lens, void *stream);
+
+/*
  * decode_attn_host_io -- the same call for a caller whose per-step tensors are in HOST memory.
  * q, block_table, seq_lens, out and lse are HOST views (pinned memory makes the copies
  * asynchronous; they must stay valid until the stream reaches the end of the call); k_pages and

@@ -50,6 +50,8 @@ def _load():
                 i32, ctypes.c_double,        # window, scale
                 p, p, i32,                   # out, lse, num_threads
             ]
+            lib.kv_append_oracle.restype = ctypes.c_int
+            lib.kv_append_oracle.argtypes = [p, p, i64, i64, i64, p, p, i64, i64, i64, i64, i64, p, i64, p]
             lib.decode_attn_oracle_max_threads.restype = ctypes.c_int
             _lib = lib
     return _lib
@@ -114,3 +116,25 @@ def decode_attn_oracle(q, k_pages, v_pages, block_table, seq_lens, window: int, 
     if rc != 0:
         raise RuntimeError(f"decode_attn_oracle failed with code {rc}")
     return out, lse
+
+
+def kv_append_oracle(k_new, v_new, k_pages, v_pages, block_table, seq_lens) -> None:
+    """Write each sequence's new K/V rows (bf16 [B, Hkv, D]) into position seq_lens[b]-1 of the paged
+    cache, IN PLACE in ``k_pages`` / ``v_pages`` (CPU torch bf16 tensors or uint16 arrays)."""
+    lib = _load()
+    kn = np.ascontiguousarray(_bf16_bits(k_new))
+    vn = np.ascontiguousarray(_bf16_bits(v_new))
+    kb, vb = _bf16_bits(k_pages), _bf16_bits(v_pages)
+    if kb.shape != vb.shape or kb.strides != vb.strides or kb.ndim != 4 or kb.strides[3] != 2:
+        raise ValueError("k_pages and v_pages must share shape and strides, contiguous last dim")
+    B, Hkv, D = kn.shape
+    num_pages, Hk, P, Dk = kb.shape
+    if Hk != Hkv or Dk != D or vn.shape != kn.shape:
+        raise ValueError("shape mismatch")
+    bt = np.ascontiguousarray(np.asarray(block_table, dtype=np.int32))
+    sl = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32))
+    st = [x // 2 for x in kb.strides]
+    rc = lib.kv_append_oracle(kn.ctypes.data, vn.ctypes.data, B, Hkv, D, kb.ctypes.data, vb.ctypes.data,
+                              num_pages, P, st[0], st[1], st[2], bt.ctypes.data, bt.shape[1], sl.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"kv_append_oracle failed with code {rc}")

@@ -174,3 +174,41 @@ int decode_attn_oracle_max_threads(void)
     return 1;
 #endif
 }
+
+/*
+ * kv_append_oracle -- the step that precedes decode attention in each layer of a decoding loop:
+ * the new token's key and value rows are written into the paged cache.  seq_lens already counts
+ * the new token (the reading taken for decode attention), so the rows go to position L-1:
+ * page block_table[b][(L-1)/P], row (L-1) % P, for every KV head.  Sequences with L <= 0 are
+ * skipped.  Pure byte moves; HOST pointers; same layout conventions as decode_attn_oracle.
+ *   k_new, v_new   bf16 bits [B, Hkv, D] contiguous
+ * Returns ORACLE_BAD_PAGE / ORACLE_BAD_ARG if a sequence points outside the pool or its table.
+ */
+int kv_append_oracle(const uint16_t *k_new, const uint16_t *v_new, int64_t B, int64_t Hkv, int64_t D,
+                     uint16_t *k_pages, uint16_t *v_pages, int64_t num_pages, int64_t P,
+                     int64_t stride_page, int64_t stride_head, int64_t stride_tok,
+                     const int32_t *block_table, int64_t max_pages, const int32_t *seq_lens)
+{
+    if (!k_new || !v_new || !k_pages || !v_pages || !block_table || !seq_lens)
+        return ORACLE_BAD_ARG;
+    for (int64_t b = 0; b < B; ++b) {
+        const int64_t L = seq_lens[b];
+        if (L <= 0)
+            continue;
+        const int64_t t = L - 1;
+        if (t / P >= max_pages)
+            return ORACLE_BAD_ARG;
+        const int64_t page = block_table[b * max_pages + t / P];
+        if (page < 0 || page >= num_pages)
+            return ORACLE_BAD_PAGE;
+        for (int64_t g = 0; g < Hkv; ++g) {
+            const int64_t dst = page * stride_page + g * stride_head + (t % P) * stride_tok;
+            const int64_t src = (b * Hkv + g) * D;
+            for (int64_t d = 0; d < D; ++d) {
+                k_pages[dst + d] = k_new[src + d];
+                v_pages[dst + d] = v_new[src + d];
+            }
+        }
+    }
+    return ORACLE_OK;
+}

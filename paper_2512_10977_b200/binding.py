@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
             L.decode_attn.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_cascade.restype = ctypes.c_int
             L.decode_attn_cascade.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_append.restype = ctypes.c_int
+            L.decode_attn_append.argtypes = [T, T, T, T, T, T, vp]
             L.decode_attn_host_io.restype = ctypes.c_int
             L.decode_attn_host_io.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_static_scratch.restype = ctypes.c_int
@@ -190,6 +192,17 @@ def decode_attn_cascade(q, k_pages, v_pages, block_table, seq_lens, shared_prefi
                                          int(shared_prefix_tokens), float(scale), _ref(tv[5]), _ref(tv[6]),
                                          _stream_ptr(stream)))
     return out, lse
+
+
+def decode_attn_append(k_new, v_new, k_pages, v_pages, block_table, seq_lens,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Write the new token's K/V rows (bf16 [B, Hkv, 128]) into position seq_lens[b]-1 of the paged
+    cache, in place (the step before ``decode_attn`` in a decoding loop)."""
+    with torch.cuda.device(k_pages.device):
+        ensure_workspace(k_new.shape[0], k_new.shape[1], k_pages.shape[1], 128, k_pages.shape[2],
+                         block_table.shape[1], k_pages.device)
+        tv = [_view(t) for t in (k_new, v_new, k_pages, v_pages, block_table, seq_lens)]
+        _check(lib().decode_attn_append(*[_ref(t) for t in tv], _stream_ptr(stream)))
 
 
 def decode_attn_host_io(q_host, k_pages, v_pages, block_table_host, seq_lens_host, window: int, scale: float,

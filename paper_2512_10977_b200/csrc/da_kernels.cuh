@@ -1003,4 +1003,54 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
     }
 }
 
+// =====================================================================================  append
+// The step before decode attention in a layer: the new token's K and V rows go into the paged cache
+// at position L-1 (seq_lens already counts the new token).  One block per sequence; thread ->
+// (K or V, kv head, 16-byte chunk of the row).  Pure byte moves, 16-byte vectors both ways.
+struct AppendParams {
+    const __nv_bfloat16 *k_new, *v_new;   // [B, Hkv, 128]
+    int64_t kn_sb, kn_sh, vn_sb, vn_sh;
+    __nv_bfloat16 *k_pages, *v_pages;     // strides in elements: page, head, token
+    int64_t k_sp, k_sh, k_st, v_sp, v_sh, v_st;
+    const int32_t *block_table;
+    int64_t bt_sb;
+    const int32_t *seq_lens;
+    int64_t sl_stride;
+    int32_t *status;
+    int32_t B, Hkv, P, num_pages;
+    int64_t max_pages;
+};
+
+__global__ void __launch_bounds__(256) append_kernel(const AppendParams p)
+{
+    const int b = blockIdx.x;
+    const int L = p.seq_lens[(int64_t)b * p.sl_stride];
+    if (L <= 0) {
+        if (L < 0 && threadIdx.x == 0)
+            report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
+        return;
+    }
+    const int t = L - 1;
+    if ((int64_t)(t / p.P) >= p.max_pages) {
+        if (threadIdx.x == 0)
+            report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
+        return;
+    }
+    const int page = __ldg(p.block_table + (int64_t)b * p.bt_sb + t / p.P);
+    if ((uint32_t)page >= (uint32_t)p.num_pages) {
+        if (threadIdx.x == 0)
+            report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, b, t / p.P, page);
+        return;
+    }
+    const int row = t % p.P;
+    for (int e = threadIdx.x; e < 2 * p.Hkv * 16; e += blockDim.x) {
+        const int c = e & 15, g = (e >> 4) % p.Hkv, is_v = e / (16 * p.Hkv);
+        const __nv_bfloat16 *src = is_v ? p.v_new + (int64_t)b * p.vn_sb + (int64_t)g * p.vn_sh
+                                        : p.k_new + (int64_t)b * p.kn_sb + (int64_t)g * p.kn_sh;
+        __nv_bfloat16 *dst = is_v ? p.v_pages + (int64_t)page * p.v_sp + (int64_t)g * p.v_sh + (int64_t)row * p.v_st
+                                  : p.k_pages + (int64_t)page * p.k_sp + (int64_t)g * p.k_sh + (int64_t)row * p.k_st;
+        *reinterpret_cast<uint4 *>(dst + c * 8) = *reinterpret_cast<const uint4 *>(src + c * 8);
+    }
+}
+
 }  // namespace da

@@ -358,3 +358,33 @@ def test_pins_catch_planted_mistakes():
     assert not np.allclose(variant(lo_shift=-1)[0], good, atol=1e-6)
     assert not np.allclose(variant(head_map=lambda h: h % 2)[0], good, atol=1e-6)  # interleaved GQA
     assert not np.allclose(variant(drop_scale=True)[1], good_lse, atol=1e-6)
+
+
+# --------------------------------------------------------------------- KV append
+
+@pytest.mark.parametrize("layout", ["head_major", "token_major"])
+def test_kv_append_writes_exactly_the_new_rows(layout):
+    """Pinned by plain indexing: after the call the row (page of token L-1, L-1 mod P) of every KV
+    head holds the new vectors and every other element of the pools is untouched."""
+    lens = [5, 8, 0, 13, 1]
+    case = tiny(lens, P=4, seed=41, Hq=6, Hkv=2, Dh=8, layout=layout, pool_pages=12, poison=False)
+    k0, v0 = case.k_pages.clone(), case.v_pages.clone()
+    gen = torch.Generator().manual_seed(3)
+    k_new = torch.randn((5, 2, 8), generator=gen).to(torch.bfloat16)
+    v_new = torch.randn((5, 2, 8), generator=gen).to(torch.bfloat16)
+    oracle.kv_append_oracle(k_new, v_new, case.k_pages, case.v_pages, case.block_table, case.seq_lens)
+    want_k, want_v = k0.clone(), v0.clone()
+    bt = case.block_table.numpy()
+    for b, L in enumerate(lens):
+        if L > 0:
+            pg, r = int(bt[b, (L - 1) // 4]), (L - 1) % 4
+            want_k[pg, :, r] = k_new[b]
+            want_v[pg, :, r] = v_new[b]
+    assert torch.equal(case.k_pages.view(torch.int16), want_k.view(torch.int16))
+    assert torch.equal(case.v_pages.view(torch.int16), want_v.view(torch.int16))
+    # and decode attention over the updated cache sees the new token: with window 1 it returns v_new
+    out, _ = run(case, window=1)
+    for b, L in enumerate(lens):
+        if L > 0:
+            for h in range(6):
+                assert np.array_equal(out[b, h], f64(v_new[b, h // 3]))
