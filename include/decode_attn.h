@@ -147,6 +147,29 @@ int decode_attn_append(const da_tensor *k_new, const da_tensor *v_new, da_tensor
                        const da_tensor *block_table, const da_tensor *seq_lens, void *stream);
 
 /*
+ * decode_attn_extend -- attention for Lq NEW tokens per sequence at once, causal among them, over
+ * the same paged cache: the step that ingests a multi-thousand-token feedback prompt (compiler
+ * log, tensor summary; paper Sec. 3.2 "Feedback") into an existing context, or verifies a few
+ * speculated tokens.  The new tokens' K/V are already in the cache (seq_lens counts them); query
+ * qi of sequence b sits at position L_b - Lq + qi and attends tokens 0 .. L_b - Lq + qi:
+ *
+ *     out[b,qi,h,:] = sum_{t <= L_b-Lq+qi} softmax(scale * <q[b,qi,h], K[.., t]>)_t V[.., t]
+ *
+ * which for Lq = 1 is decode_attn() without a window.  Runs on the tcgen05 tensor cores (the same
+ * kernel as the cascade's prefix pass: 128 (query, head) rows of one KV group per thread block).
+ *
+ *   q      bf16 [B, Lq, Hq, 128], last dim contiguous
+ *   out    f32 or bf16 [B, Lq, Hq, 128], last dim contiguous
+ *   lse    f32 [B, Lq, Hq] or NULL
+ *   every seq_lens[b] must be >= Lq, or 0 (then out = 0, lse = -inf); otherwise DA_DEV_BAD_SEQLEN
+ *   is set and the sequence is treated as empty.  No window.  Other arguments, workspace and
+ *   conventions as decode_attn().
+ */
+int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                       const da_tensor *block_table, const da_tensor *seq_lens, float scale, da_tensor *out,
+                       da_tensor *lse, void *stream);
+
+/*
  * decode_attn_host_io -- the same call for a caller whose per-step tensors are in HOST memory.
  * q, block_table, seq_lens, out and lse are HOST views (pinned memory makes the copies
  * asynchronous; they must stay valid until the stream reaches the end of the call); k_pages and

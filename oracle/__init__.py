@@ -138,3 +138,20 @@ def kv_append_oracle(k_new, v_new, k_pages, v_pages, block_table, seq_lens) -> N
                               num_pages, P, st[0], st[1], st[2], bt.ctypes.data, bt.shape[1], sl.ctypes.data)
     if rc != 0:
         raise RuntimeError(f"kv_append_oracle failed with code {rc}")
+
+
+def extend_attn_oracle(q, k_pages, v_pages, block_table, seq_lens, scale: float, num_threads: int = 0):
+    """Causal attention of Lq new tokens per sequence, by its definition in terms of the single-token
+    oracle: query qi of sequence b sits at position L_b - Lq + qi, so it is decode attention over a
+    cache cut to L_b - Lq + qi + 1 tokens.  q: bf16 [B, Lq, Hq, D]; ``seq_lens`` counts the new
+    tokens.  Returns (out float64 [B, Lq, Hq, D], lse float64 [B, Lq, Hq])."""
+    import torch
+    B, Lq, Hq, D = q.shape
+    sl = np.asarray(seq_lens, dtype=np.int64)
+    out = np.zeros((B, Lq, Hq, D))
+    lse = np.full((B, Lq, Hq), -np.inf)
+    for qi in range(Lq):
+        cut = np.where(sl > 0, sl - Lq + qi + 1, 0).astype(np.int32)
+        o, l = decode_attn_oracle(q[:, qi].contiguous(), k_pages, v_pages, block_table, cut, 0, scale, num_threads)
+        out[:, qi], lse[:, qi] = o, l
+    return out, lse

@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
             L.decode_attn_cascade.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_append.restype = ctypes.c_int
             L.decode_attn_append.argtypes = [T, T, T, T, T, T, vp]
+            L.decode_attn_extend.restype = ctypes.c_int
+            L.decode_attn_extend.argtypes = [T, T, T, T, T, ctypes.c_float, T, T, vp]
             L.decode_attn_host_io.restype = ctypes.c_int
             L.decode_attn_host_io.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_static_scratch.restype = ctypes.c_int
@@ -203,6 +205,24 @@ def decode_attn_append(k_new, v_new, k_pages, v_pages, block_table, seq_lens,
                          block_table.shape[1], k_pages.device)
         tv = [_view(t) for t in (k_new, v_new, k_pages, v_pages, block_table, seq_lens)]
         _check(lib().decode_attn_append(*[_ref(t) for t in tv], _stream_ptr(stream)))
+
+
+def decode_attn_extend(q, k_pages, v_pages, block_table, seq_lens, scale: float,
+                       out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                       stream: Optional[torch.cuda.Stream] = None, out_dtype=torch.float32):
+    """Causal attention of Lq new tokens per sequence (q: bf16 [B, Lq, Hq, 128]) over the paged cache,
+    which already holds their K/V (``seq_lens`` counts them).  Returns (out [B,Lq,Hq,128], lse [B,Lq,Hq])."""
+    if out is None:
+        out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    with torch.cuda.device(k_pages.device):
+        ensure_workspace(q.shape[0], q.shape[2], k_pages.shape[1], q.shape[3], k_pages.shape[2],
+                         block_table.shape[1], k_pages.device)
+        tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
+        _check(lib().decode_attn_extend(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
+                                        float(scale), _ref(tv[5]), _ref(tv[6]), _stream_ptr(stream)))
+    return out, lse
 
 
 def decode_attn_host_io(q_host, k_pages, v_pages, block_table_host, seq_lens_host, window: int, scale: float,

@@ -38,17 +38,32 @@ constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and
 constexpr int PF_TMEM_PH = 384;              // P high parts in [384,448), low parts in [448,512): 128 tokens as
 constexpr int PF_TMEM_PL = 448;              // 64 columns of bf16 pairs, the A operand of the PV product
 
+// The kernel serves two callers.
+//  * cascade (ext = 0): rows = all sequences' heads of one KV group, row = b * G + head; keys = the
+//    shared prefix, named by row 0 of the block table; every row attends every prefix token.
+//  * extend (ext = 1): one sequence per block; rows = its Lq new query tokens' heads of one KV
+//    group, row = qi * G + head; keys = that sequence's own pages; query qi sits at position
+//    L - Lq + qi and attends tokens 0 .. L - Lq + qi (causal).
 struct PrefixParams {
     const __nv_bfloat16 *q;
-    int64_t q_sb, q_sh;
-    const int32_t *block_table;   // row 0 names the shared pages
-    float *pre_o;                 // [splits][B*Hq][128] normalised partials
-    float *pre_lse;               // [splits][B*Hq]
+    int64_t q_sb, q_sq, q_sh;     // strides of sequence, query token (extend), head
+    const int32_t *block_table;
+    int64_t bt_sb;
+    const int32_t *seq_lens;      // extend only
+    int64_t sl_stride;
+    float *pre_o;                 // [splits][rows_total * Hkv][128] normalised partials (rows_total = B*Lq*G)
+    float *pre_lse;               // [splits][rows_total * Hkv]
+    void *out;                    // extend with one split writes the result directly
+    int64_t o_sb, o_sq, o_sh;
+    float *lse;
+    int64_t l_sb, l_sq, l_sh;
     int32_t *status;
-    int32_t B, Hkv, G, P, box_rows, num_pages;
-    int32_t prefix_tiles;         // shared prefix length / PF_TOK
+    int32_t B, Hkv, G, P, box_rows, num_pages, out_bf16;
+    int32_t ext, Lq;
+    int64_t max_pages;
+    int32_t prefix_tiles;         // cascade: shared prefix length / PF_TOK
     int32_t splits;               // KV ranges per (row tile, head)
-    int32_t row_tiles;            // ceil(B*G / 128)
+    int32_t row_tiles;            // cascade: ceil(B*G / 128); extend: ceil(Lq*G / 128)
     float scale_log2;
 };
 
@@ -176,14 +191,33 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                    bar_s = bar_kfull + 96, bar_p = bar_kfull + 112, bar_x = bar_kfull + 120;
     volatile int *abort_flag = &abort_s;
 
-    // block -> (row tile, kv head, split)
+    // block -> (row tile, kv head, [sequence,] split)
     const int rt = blockIdx.x % p.row_tiles;
     const int g = (blockIdx.x / p.row_tiles) % p.Hkv;
-    const int split = blockIdx.x / (p.row_tiles * p.Hkv);
-    const int t_begin = (int)((long long)p.prefix_tiles * split / p.splits);
-    const int t_end = (int)((long long)p.prefix_tiles * (split + 1) / p.splits);
+    int split = blockIdx.x / (p.row_tiles * p.Hkv);
+    int bseq = 0, L = 0, kv_tiles = p.prefix_tiles;
+    int R = p.B * p.G;               // rows in this block's row space
+    if (p.ext) {
+        bseq = split % p.B;
+        split /= p.B;
+        R = p.Lq * p.G;
+        L = p.seq_lens[(int64_t)bseq * p.sl_stride];
+        if (L < 0 || (L > 0 && L < p.Lq) || (int64_t)L > p.max_pages * (int64_t)p.P) {
+            if (tid == 0)
+                report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, bseq, 2, L);
+            L = 0;
+        }
+        // causal: the block's last row attends tokens below L - Lq + qi_max + 1
+        const int qi_max = min(p.Lq - 1, (rt * PF_ROWS + PF_ROWS - 1) / p.G);
+        const int lim_max = L > 0 ? L - p.Lq + qi_max + 1 : 0;
+        kv_tiles = (lim_max + PF_TOK - 1) / PF_TOK;
+    }
+    const int t_begin = (int)((long long)kv_tiles * split / p.splits);
+    const int t_end = (int)((long long)kv_tiles * (split + 1) / p.splits);
     const int ntiles = t_end - t_begin;
-    const int R = p.B * p.G;
+    const int32_t *bt_row = p.block_table + (int64_t)bseq * p.bt_sb;
+    // extend: from this token on some row of the block is masked (the first query's limit)
+    const int mask_from = p.ext ? L - p.Lq + 1 : 0x7fffffff;
 
     if ((sb & 1023u) != 0) {
         if (tid == 0)
@@ -215,8 +249,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         const int row = rt * PF_ROWS + r;
         uint4 val = make_uint4(0, 0, 0, 0);
         if (row < R) {
-            const int b = row / p.G, hi = row % p.G;
-            const __nv_bfloat16 *src = p.q + (int64_t)b * p.q_sb + (int64_t)(g * p.G + hi) * p.q_sh + c * 8;
+            const int outer = row / p.G, hi = row % p.G;   // sequence (cascade) or query token (extend)
+            const __nv_bfloat16 *src = p.q + (p.ext ? (int64_t)bseq * p.q_sb + (int64_t)outer * p.q_sq : (int64_t)outer * p.q_sb) +
+                                       (int64_t)(g * p.G + hi) * p.q_sh + c * 8;
             if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
                 val = *reinterpret_cast<const uint4 *>(src);
             } else {
@@ -248,19 +283,25 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             auto read_page = [&](int j) {   // page id of this lane's box of tile j (0 for idle lanes)
                 if (!active || j >= ntiles)
                     return 0;
-                return __ldg(p.block_table + ((t_begin + j) * PF_TOK + box * p.box_rows) / p.P);
+                const int t = (t_begin + j) * PF_TOK + box * p.box_rows;
+                if (p.ext && t >= L)
+                    return 0;   // past the sequence's last page: the block table has no entry
+                return __ldg(bt_row + t / p.P);
             };
             auto load_kv = [&](int j, int page, bool is_v) {   // K or V of tile j into buffer j % 3
                 const int buf = j % PF_NB;
                 const uint32_t bar = (is_v ? bar_vfull : bar_kfull) + 8 * buf;
+                // extend: boxes wholly past the sequence's end are not loaded (their rows are masked)
+                const int t_tile = (t_begin + j) * PF_TOK;
+                const int nbox = p.ext ? min(boxes, (L - t_tile + p.box_rows - 1) / p.box_rows) : boxes;
                 if (lane == 0)
-                    mbar_arrive_expect_tx(bar, (uint32_t)PF_TILE);
+                    mbar_arrive_expect_tx(bar, (uint32_t)(nbox * p.box_rows * 256));
                 __syncwarp();
-                if (active) {
-                    const int t = (t_begin + j) * PF_TOK + box * p.box_rows;
+                if (active && box < nbox) {
+                    const int t = t_tile + box * p.box_rows;
                     if ((uint32_t)page >= (uint32_t)p.num_pages) {
                         if (!is_v && pl == 0)
-                            report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, 0, t / p.P, page);
+                            report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, bseq, t / p.P, page);
                         page = p.num_pages;   // out of range: TMA fills zeros and still counts the bytes
                     }
                     const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + box * p.box_rows * 128);
@@ -403,6 +444,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         // means scaling that row of O, which after the first few tiles is rare.
         float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;
+        // extend: this row's query attends tokens below `limit` (0 for padding rows: nothing)
+        const int rr = rt * PF_ROWS + r;
+        const int limit = (p.ext && rr < R && L > 0) ? L - p.Lq + rr / p.G + 1 : 0;
         for (int j = 0; j < ntiles; ++j) {
             if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                 ok = false;
@@ -419,6 +463,14 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 #pragma unroll
                 for (int i = 0; i < 64; ++i)
                     sv[i] = __uint_as_float(v[i >> 5][i & 31]) * p.scale_log2;
+            }
+            const int t_tile = (t_begin + j) * PF_TOK;
+            if (t_tile + PF_TOK > mask_from) {   // extend, near the end: causal mask by select (K rows past
+                const int t_mine = t_tile + half * 64;   // the sequence's end may hold anything)
+#pragma unroll
+                for (int i = 0; i < 64; ++i)
+                    if (t_mine + i >= limit)
+                        sv[i] = -INFINITY;
             }
             float mx = sv[0];
 #pragma unroll
@@ -441,10 +493,11 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             // weights, their sum, and P as bf16 high + low parts (kept in registers for now)
             float lsum = 0.f;
             uint32_t phi[32], plo[32];
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // a row with nothing to attend yet
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-                const float p0 = fast_exp2(sv[2 * e] - m_new);
-                const float p1 = fast_exp2(sv[2 * e + 1] - m_new);
+                const float p0 = fast_exp2(sv[2 * e] - m_use);
+                const float p1 = fast_exp2(sv[2 * e + 1] - m_use);
                 lsum += p0 + p1;
                 phi[e] = pack_bf16(p0, p1);
                 plo[e] = pack_bf16(p0 - bf16_lo_to_float(phi[e]), p1 - bf16_hi_to_float(phi[e]));
@@ -468,6 +521,22 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     tmem_st32(tmem_o + lane_base, v[0]);
                     tmem_st32(tmem_o + lane_base + 32, v[1]);
                 }
+            }
+            if (p.ext && t_tile + PF_TOK > L) {
+                // The tile reaches past the sequence's end: those V rows were not loaded, or are a page's
+                // unused tail, and may hold NaN, which a zero weight would not hide.  Clear them (both
+                // planes, 128 bytes a row) once V has landed, before the PV product reads them.
+                if (!mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
+                    ok = false;
+                    break;
+                }
+                const int first_bad = max(L - t_tile, 0);
+                uint8_t *vb = smem + PF_OFF_V + (j % PF_NB) * PF_TILE;
+                for (int e = tid; e < (PF_TOK - first_bad) * 16; e += 2 * PF_ROWS) {
+                    const int row = first_bad + (e >> 4), ch = e & 15;
+                    *reinterpret_cast<uint4 *>(vb + (ch >> 3) * PF_PLANE + row * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                }
+                fence_proxy_async_smem();
             }
             // P into tensor memory: this thread's 64 tokens are 32 columns of bf16 pairs
             tmem_st32(tmem + PF_TMEM_PH + ((uint32_t)(32 * (warp & 3)) << 16) + half * 32, phi);
@@ -508,23 +577,43 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -8, (int)blockIdx.x, 0);
             }
         } else {
-            const int row = rt * PF_ROWS + r;
-            if (row < R) {
-                const int b = row / p.G, hi = row % p.G;
-                const int64_t bh = (int64_t)b * (p.Hkv * p.G) + g * p.G + hi;
-                const int64_t at = (int64_t)split * p.B * (p.Hkv * p.G) + bh;
-                float *dst = p.pre_o + at * HEAD_DIM + half * 64;
-                const float inv = ntiles > 0 ? 1.f / l_row : 0.f;
+            if (rr < R) {
+                const int outer = rr / p.G, hd = rr % p.G;   // sequence (cascade) or query token (extend)
+                const bool any = ntiles > 0 && l_row > 0.f;
+                const float inv = any ? 1.f / l_row : 0.f;
+                const float lse_val = any ? (m_run + fast_log2(l_row)) * LN2 : -INFINITY;
+                float vals[64];
 #pragma unroll
-                for (int i = 0; i < 64; i += 4) {
-                    float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (ntiles > 0)
-                        v4 = make_float4(__uint_as_float(o_raw[i >> 5][i & 31]) * inv, __uint_as_float(o_raw[i >> 5][(i + 1) & 31]) * inv,
-                                         __uint_as_float(o_raw[i >> 5][(i + 2) & 31]) * inv, __uint_as_float(o_raw[i >> 5][(i + 3) & 31]) * inv);
-                    *reinterpret_cast<float4 *>(dst + i) = v4;
+                for (int i = 0; i < 64; ++i)
+                    vals[i] = any ? __uint_as_float(o_raw[i >> 5][i & 31]) * inv : 0.f;
+                const int h = g * p.G + hd;
+                if (p.ext && p.splits == 1) {
+                    const int64_t at = (int64_t)bseq * p.o_sb + (int64_t)outer * p.o_sq + (int64_t)h * p.o_sh + half * 64;
+                    if (p.out_bf16) {
+                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
+#pragma unroll
+                        for (int i = 0; i < 64; ++i)
+                            dst[i] = __float2bfloat16_rn(vals[i]);
+                    } else {
+                        float *dst = reinterpret_cast<float *>(p.out) + at;
+#pragma unroll
+                        for (int i = 0; i < 64; ++i)
+                            dst[i] = vals[i];
+                    }
+                    if (half == 0 && p.lse)
+                        p.lse[(int64_t)bseq * p.l_sb + (int64_t)outer * p.l_sq + (int64_t)h * p.l_sh] = lse_val;
+                } else {
+                    const int Hq = p.Hkv * p.G;
+                    const int64_t n_rows = (int64_t)p.B * (p.ext ? p.Lq : 1) * Hq;
+                    const int64_t idx = p.ext ? ((int64_t)bseq * p.Lq + outer) * Hq + h : (int64_t)outer * Hq + h;
+                    const int64_t at = (int64_t)split * n_rows + idx;
+                    float *dst = p.pre_o + at * HEAD_DIM + half * 64;
+#pragma unroll
+                    for (int i = 0; i < 64; i += 4)
+                        *reinterpret_cast<float4 *>(dst + i) = make_float4(vals[i], vals[i + 1], vals[i + 2], vals[i + 3]);
+                    if (half == 0)
+                        p.pre_lse[at] = lse_val;
                 }
-                if (half == 0)
-                    p.pre_lse[at] = ntiles > 0 ? (m_run + fast_log2(l_row)) * LN2 : -INFINITY;
             }
         }
     }
@@ -539,25 +628,25 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 // by the plan / partition / merge kernels over tokens >= prefix into fp32 scratch) and write `out`
 // and `lse`.  lse = -inf marks "no tokens" and contributes nothing.
 struct CascadeMergeParams {
-    const float *pre_o, *pre_lse;   // [splits][B*Hq][128], [splits][B*Hq]
-    const float *suf_o, *suf_lse;   // [B*Hq][128], [B*Hq]
+    const float *pre_o, *pre_lse;   // [splits][n][128], [splits][n]   with n = B * Lq * Hq
+    const float *suf_o, *suf_lse;   // [n][128], [n]; may be NULL (extend: no separate suffix pass)
     void *out;
-    int64_t o_sb, o_sh;
+    int64_t o_sb, o_sq, o_sh;
     float *lse;
-    int64_t l_sb, l_sh;
-    int32_t B, Hq, splits, out_bf16;
+    int64_t l_sb, l_sq, l_sh;
+    int32_t B, Lq, Hq, splits, out_bf16;
 };
 
 __global__ void __launch_bounds__(256) cascade_merge_kernel(const CascadeMergeParams p)
 {
     const int warp = threadIdx.x >> 5, ln = threadIdx.x & 31, d = ln * 4;
-    const int64_t bh = (int64_t)blockIdx.x * 8 + warp;
-    const int64_t n = (int64_t)p.B * p.Hq;
-    if (bh >= n)
+    const int64_t idx = (int64_t)blockIdx.x * 8 + warp;
+    const int64_t n = (int64_t)p.B * p.Lq * p.Hq;
+    if (idx >= n)
         return;
-    float M = p.suf_lse[bh];
+    float M = p.suf_lse ? p.suf_lse[idx] : -INFINITY;
     for (int s = 0; s < p.splits; ++s)
-        M = fmaxf(M, p.pre_lse[(int64_t)s * n + bh]);
+        M = fmaxf(M, p.pre_lse[(int64_t)s * n + idx]);
     float den = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     auto fold = [&](float l, const float *o) {
@@ -571,9 +660,10 @@ __global__ void __launch_bounds__(256) cascade_merge_kernel(const CascadeMergePa
         acc.w += w * v.w;
         den += w;
     };
-    fold(p.suf_lse[bh], p.suf_o + bh * HEAD_DIM);
+    if (p.suf_lse)
+        fold(p.suf_lse[idx], p.suf_o + idx * HEAD_DIM);
     for (int s = 0; s < p.splits; ++s)
-        fold(p.pre_lse[(int64_t)s * n + bh], p.pre_o + ((int64_t)s * n + bh) * HEAD_DIM);
+        fold(p.pre_lse[(int64_t)s * n + idx], p.pre_o + ((int64_t)s * n + idx) * HEAD_DIM);
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     float lse_val = -INFINITY;
     if (den > 0.f) {
@@ -581,8 +671,8 @@ __global__ void __launch_bounds__(256) cascade_merge_kernel(const CascadeMergePa
         v = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
         lse_val = M + __logf(den);
     }
-    const int b = (int)(bh / p.Hq), h = (int)(bh % p.Hq);
-    const int64_t at = (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d;
+    const int h = (int)(idx % p.Hq), qi = (int)((idx / p.Hq) % p.Lq), b = (int)(idx / ((int64_t)p.Hq * p.Lq));
+    const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h * p.o_sh + d;
     if (p.out_bf16) {
         __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
         o[0] = __float2bfloat16_rn(v.x);
@@ -594,7 +684,7 @@ __global__ void __launch_bounds__(256) cascade_merge_kernel(const CascadeMergePa
         o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
     }
     if (ln == 0 && p.lse)
-        p.lse[(int64_t)b * p.l_sb + (int64_t)h * p.l_sh] = lse_val;
+        p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h * p.l_sh] = lse_val;
 }
 
 }  // namespace da

@@ -523,8 +523,20 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     PrefixParams pf;
     pf.q = static_cast<const __nv_bfloat16 *>(q->data);
     pf.q_sb = q->stride[0];
+    pf.q_sq = 0;
     pf.q_sh = q->stride[1];
     pf.block_table = static_cast<const int32_t *>(block_table->data);
+    pf.bt_sb = block_table->stride[0];
+    pf.seq_lens = nullptr;
+    pf.sl_stride = 0;
+    pf.out = nullptr;
+    pf.o_sb = pf.o_sq = pf.o_sh = 0;
+    pf.lse = nullptr;
+    pf.l_sb = pf.l_sq = pf.l_sh = 0;
+    pf.out_bf16 = 0;
+    pf.ext = 0;
+    pf.Lq = 1;
+    pf.max_pages = d.max_pages;
     pf.pre_o = reinterpret_cast<float *>(ws + lay.pre_o);
     pf.pre_lse = reinterpret_cast<float *>(ws + lay.pre_lse);
     pf.status = reinterpret_cast<int32_t *>(ws + lay.status);
@@ -560,11 +572,14 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     cm.suf_lse = reinterpret_cast<const float *>(ws + lay.suf_lse);
     cm.out = out->data;
     cm.o_sb = out->stride[0];
+    cm.o_sq = 0;
     cm.o_sh = out->stride[1];
     cm.lse = lse ? static_cast<float *>(lse->data) : nullptr;
     cm.l_sb = lse ? lse->stride[0] : 0;
+    cm.l_sq = 0;
     cm.l_sh = lse ? lse->stride[1] : 0;
     cm.B = (int32_t)d.B;
+    cm.Lq = 1;
     cm.Hq = (int32_t)d.Hq;
     cm.splits = splits;
     cm.out_bf16 = out->dtype == DA_BF16;
@@ -638,6 +653,137 @@ int decode_attn_append(const da_tensor *k_new, const da_tensor *v_new, da_tensor
     append_kernel<<<(unsigned)B, 256, 0, stream>>>(ap);
     g_launches.fetch_add(1);
     DA_CUDA(cudaGetLastError());
+    return DA_OK;
+}
+
+int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
+                       const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return DA_ERR_NULL;
+    if (!q->data || !block_table->data || !seq_lens->data || !out->data || (lse && !lse->data)) return DA_ERR_NULL;
+    if (q->dtype != DA_BF16 || block_table->dtype != DA_I32 || seq_lens->dtype != DA_I32) return DA_ERR_DTYPE;
+    if (out->dtype != DA_F32 && out->dtype != DA_BF16) return DA_ERR_DTYPE;
+    if (lse && lse->dtype != DA_F32) return DA_ERR_DTYPE;
+    if (q->ndim != 4 || out->ndim != 4 || block_table->ndim != 2 || seq_lens->ndim != 1 || (lse && lse->ndim != 3))
+        return DA_ERR_SHAPE;
+    int rc = check_pool(k_pages);
+    if (rc != DA_OK) return rc;
+    rc = check_pool(v_pages);
+    if (rc != DA_OK) return rc;
+    for (int i = 0; i < 4; ++i)
+        if (k_pages->shape[i] != v_pages->shape[i]) return DA_ERR_SHAPE;
+    const int64_t B = q->shape[0], Lq = q->shape[1], Hq = q->shape[2];
+    const int64_t Hkv = k_pages->shape[1], P = k_pages->shape[2], max_pages = block_table->shape[1];
+    if (q->shape[3] != HEAD_DIM) return DA_ERR_UNSUPPORTED;
+    if (B < 0 || Lq <= 0 || Hq <= 0 || max_pages <= 0 || Hq % Hkv != 0) return DA_ERR_SHAPE;
+    if (P != 16 && P != 32 && P != 64 && P != 128) return DA_ERR_UNSUPPORTED;
+    if (B > (1 << 20) || Lq > (1 << 20) || k_pages->shape[0] > 0x7fffffffll || max_pages * P > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+    for (int i = 0; i < 4; ++i)
+        if (out->shape[i] != q->shape[i]) return DA_ERR_SHAPE;
+    if (lse && (lse->shape[0] != B || lse->shape[1] != Lq || lse->shape[2] != Hq)) return DA_ERR_SHAPE;
+    if (block_table->shape[0] != B || seq_lens->shape[0] != B) return DA_ERR_SHAPE;
+    if (q->stride[3] != 1 || out->stride[3] != 1 || block_table->stride[1] != 1) return DA_ERR_STRIDE_ALIGN;
+    if ((q->stride[0] | q->stride[1] | q->stride[2]) & 1 || (reinterpret_cast<uintptr_t>(q->data) & 3u)) return DA_ERR_STRIDE_ALIGN;
+    const int64_t G = Hq / Hkv;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    rc = current_device(&dev, &st);
+    if (rc != DA_OK) return rc;
+    const int nblocks = grid_blocks_for(st);
+    const WsLayout lay = ws_layout(B, Hq, HEAD_DIM, max_pages, nblocks + tail_units_for(nblocks));
+    if (!st->ws || st->ws_bytes < lay.total) return DA_ERR_WORKSPACE;
+    if (B == 0) return DA_OK;
+    uint8_t *ws = static_cast<uint8_t *>(st->ws);
+    if (!st->attrs_set) {
+        rc = set_kernel_attrs<1>();
+        if (rc != DA_OK) return rc;
+        rc = set_kernel_attrs<2>();
+        if (rc != DA_OK) return rc;
+        DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
+        st->attrs_set = true;
+    }
+    const int box_rows = P < PF_TOK ? (int)P : PF_TOK;
+    CUtensorMap tm_k, tm_v;
+    rc = get_tmap(k_pages, box_rows, 1, &tm_k);
+    if (rc != DA_OK) return rc;
+    rc = get_tmap(v_pages, box_rows, 1, &tm_v);
+    if (rc != DA_OK) return rc;
+
+    PrefixParams pf;
+    pf.q = static_cast<const __nv_bfloat16 *>(q->data);
+    pf.q_sb = q->stride[0];
+    pf.q_sq = q->stride[1];
+    pf.q_sh = q->stride[2];
+    pf.block_table = static_cast<const int32_t *>(block_table->data);
+    pf.bt_sb = block_table->stride[0];
+    pf.seq_lens = static_cast<const int32_t *>(seq_lens->data);
+    pf.sl_stride = seq_lens->stride[0];
+    pf.pre_o = reinterpret_cast<float *>(ws + lay.pre_o);
+    pf.pre_lse = reinterpret_cast<float *>(ws + lay.pre_lse);
+    pf.out = out->data;
+    pf.o_sb = out->stride[0];
+    pf.o_sq = out->stride[1];
+    pf.o_sh = out->stride[2];
+    pf.lse = lse ? static_cast<float *>(lse->data) : nullptr;
+    pf.l_sb = lse ? lse->stride[0] : 0;
+    pf.l_sq = lse ? lse->stride[1] : 0;
+    pf.l_sh = lse ? lse->stride[2] : 0;
+    pf.status = reinterpret_cast<int32_t *>(ws + lay.status);
+    pf.B = (int32_t)B;
+    pf.Hkv = (int32_t)Hkv;
+    pf.G = (int32_t)G;
+    pf.P = (int32_t)P;
+    pf.box_rows = box_rows;
+    pf.num_pages = (int32_t)k_pages->shape[0];
+    pf.out_bf16 = out->dtype == DA_BF16;
+    pf.ext = 1;
+    pf.Lq = (int32_t)Lq;
+    pf.max_pages = max_pages;
+    pf.prefix_tiles = 0;
+    pf.row_tiles = (int32_t)((Lq * G + PF_ROWS - 1) / PF_ROWS);
+    // KV ranges: as many as fill one wave, if their partials fit the scratch sized for the cascade
+    // (kMaxPrefixSplits x B x Hq rows); long query blocks have enough thread blocks anyway.
+    const long long base = (long long)B * Hkv * pf.row_tiles;
+    int splits = (int)(st->sm_count / base);
+    if (splits > kMaxPrefixSplits) splits = kMaxPrefixSplits;
+    if ((long long)splits * Lq > kMaxPrefixSplits) splits = (int)(kMaxPrefixSplits / Lq);
+    if (splits < 1) splits = 1;
+    pf.splits = splits;
+    pf.scale_log2 = scale * LOG2E;
+    const long long grid = base * splits;
+    if (grid > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+    const bool timed = g_ev_before && g_ev_after;
+    if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
+    prefix_kernel<<<(unsigned)grid, PF_THREADS, PF_SMEM_BYTES, stream>>>(tm_k, tm_v, pf);
+    g_launches.fetch_add(1);
+    DA_CUDA(cudaGetLastError());
+    if (timed) DA_CUDA(cudaEventRecord(g_ev_after, stream));
+    if (splits > 1) {
+        CascadeMergeParams cm;
+        cm.pre_o = pf.pre_o;
+        cm.pre_lse = pf.pre_lse;
+        cm.suf_o = nullptr;
+        cm.suf_lse = nullptr;
+        cm.out = out->data;
+        cm.o_sb = pf.o_sb;
+        cm.o_sq = pf.o_sq;
+        cm.o_sh = pf.o_sh;
+        cm.lse = pf.lse;
+        cm.l_sb = pf.l_sb;
+        cm.l_sq = pf.l_sq;
+        cm.l_sh = pf.l_sh;
+        cm.B = (int32_t)B;
+        cm.Lq = (int32_t)Lq;
+        cm.Hq = (int32_t)Hq;
+        cm.splits = splits;
+        cm.out_bf16 = pf.out_bf16;
+        cascade_merge_kernel<<<(unsigned)((B * Lq * Hq + 7) / 8), 256, 0, stream>>>(cm);
+        g_launches.fetch_add(1);
+        DA_CUDA(cudaGetLastError());
+    }
     return DA_OK;
 }
 

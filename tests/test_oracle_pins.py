@@ -388,3 +388,33 @@ def test_kv_append_writes_exactly_the_new_rows(layout):
         if L > 0:
             for h in range(6):
                 assert np.array_equal(out[b, h], f64(v_new[b, h // 3]))
+
+
+# --------------------------------------------------------------------- multi-token (extend) attention
+
+@pytest.mark.parametrize("P,Lq", [(4, 1), (4, 3), (16, 7)])
+def test_extend_oracle_agrees_with_dense_causal_bruteforce(P, Lq):
+    """Independent restatement: gather dense K, V per sequence, build the causal mask explicitly
+    (query qi sees tokens <= L - Lq + qi), scipy softmax."""
+    lens = [Lq, Lq + 5, 40, 23]
+    case = workloads.build_case("ext", lens, P, 50 + P + Lq, "cpu", Hq=6, Hkv=2, Dh=8)
+    gen = torch.Generator().manual_seed(Lq)
+    q = torch.randn((4, Lq, 6, 8), generator=gen).to(torch.bfloat16)
+    out, lse = oracle.extend_attn_oracle(q, case.k_pages, case.v_pages, case.block_table, case.seq_lens, case.scale)
+    K, V, bt = f64(case.k_pages), f64(case.v_pages), case.block_table.numpy()
+    qd = f64(q)
+    sc = float(np.float32(case.scale))
+    for b, L in enumerate(lens):
+        t = np.arange(L)
+        for h in range(6):
+            Kd, Vd = K[bt[b, t // P], h // 3, t % P], V[bt[b, t // P], h // 3, t % P]
+            s = sc * (qd[b, :, h] @ Kd.T)                                  # [Lq, L]
+            mask = t[None, :] <= (L - Lq + np.arange(Lq))[:, None]
+            s = np.where(mask, s, -np.inf)
+            np.testing.assert_allclose(out[b, :, h], softmax(s, axis=1) @ Vd, atol=1e-12)
+            np.testing.assert_allclose(lse[b, :, h], logsumexp(s, axis=1), atol=1e-12)
+    # Lq = 1 is plain decode attention
+    if Lq == 1:
+        o1, l1 = run(case)
+        o2, l2 = oracle.extend_attn_oracle(case.q[:, None], case.k_pages, case.v_pages, case.block_table, case.seq_lens, case.scale)
+        assert np.array_equal(o1, o2[:, 0]) and np.array_equal(l1, l2[:, 0])
