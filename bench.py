@@ -200,8 +200,24 @@ def run_ours(args):
             raise SystemExit("--cascade applies to the shared-prefix workload c5a (full attention)")
         prefix = 16384
 
+    Lq = int(args.extend)
+    if Lq:
+        if prefix or case.window:
+            raise SystemExit("--extend takes a workload without window, and not --cascade")
+        if int(case.lens.min()) < Lq:
+            raise SystemExit("--extend: every sequence must hold at least that many tokens")
+        q_ext = torch.randn((case.B, Lq) + tuple(case.q.shape[1:]), device=device,
+                            generator=torch.Generator(device=device).manual_seed(7)).to(torch.bfloat16)
+        out = torch.empty(q_ext.shape, dtype=torch.float32, device=device)
+        lse = torch.empty(q_ext.shape[:3], dtype=torch.float32, device=device)
+        Hq_, Dh_ = case.q.shape[1], case.q.shape[2]
+        nbytes += case.B * (Lq - 1) * (Hq_ * Dh_ * 2 + Hq_ * Dh_ * 4 + Hq_ * 4)   # the extra queries' q, out, lse
+
     def step():
-        if prefix:
+        if Lq:
+            da.decode_attn_extend(q_ext, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
+                                  case.scale, out=out, lse=lse, stream=stream)
+        elif prefix:
             da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
                                    prefix, case.scale, out=out, lse=lse, stream=stream)
         else:
@@ -262,16 +278,21 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
 
     # ---- end to end: per-step inputs from pinned host memory, result read back to the host
-    q_h, bt_h, sl_h = (t.cpu().pin_memory() for t in (case.q, case.block_table, case.seq_lens))
-    out_h = torch.empty(case.q.shape, dtype=torch.float32).pin_memory()
-    lse_h = torch.empty(case.q.shape[:2], dtype=torch.float32).pin_memory()
+    q_src = q_ext if Lq else case.q
+    q_h, bt_h, sl_h = (t.cpu().pin_memory() for t in (q_src, case.block_table, case.seq_lens))
+    out_h = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
     h2d = q_h.numel() * 2 + bt_h.numel() * 4 + sl_h.numel() * 4
     d2h = out_h.numel() * 4 + lse_h.numel() * 4
 
     q_d, bt_d, sl_d = (torch.empty_like(t, device=device) for t in (q_h, bt_h, sl_h))
 
     def e2e_step():
-        if prefix:   # the cascade has no host-io entry point: same copies, made here on the same stream
+        if Lq:
+            q_d.copy_(q_h, non_blocking=True); bt_d.copy_(bt_h, non_blocking=True); sl_d.copy_(sl_h, non_blocking=True)
+            da.decode_attn_extend(q_d, case.k_pages, case.v_pages, bt_d, sl_d, case.scale, out=out, lse=lse, stream=stream)
+            out_h.copy_(out, non_blocking=True); lse_h.copy_(lse, non_blocking=True)
+        elif prefix:   # the cascade has no host-io entry point: same copies, made here on the same stream
             q_d.copy_(q_h, non_blocking=True); bt_d.copy_(bt_h, non_blocking=True); sl_d.copy_(sl_h, non_blocking=True)
             da.decode_attn_cascade(q_d, case.k_pages, case.v_pages, bt_d, sl_d, prefix, case.scale,
                                    out=out, lse=lse, stream=stream)
@@ -303,6 +324,19 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "partition_kernel", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                 "kernel_ms": kms, "traffic": NCU_TRAFFIC.get((args.workload, da.version()))}
+    if Lq:
+        # one kernel, a dense causal contraction: algorithmic flops = QK^T and PV over each query's keys
+        Hq, Dh = case.q.shape[1], case.q.shape[2]
+        keys = sum(float(L - Lq) * Lq + Lq * (Lq + 1) / 2.0 for L in case.lens)
+        flops = 4.0 * Hq * Dh * keys
+        try:
+            with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+                tpeak, tsrc = float(json.load(f)["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops, burst)"
+        except Exception:
+            tpeak, tsrc = 1590.0, "fallback (1.59 PFLOP/s, earlier measurement on this pool)"
+        tf = flops / (kms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "prefix_kernel (extend mode)", "achieved": tf, "peak": tpeak,
+                    "unit": "TFLOP/s", "frac": tf / tpeak, "peak_source": tsrc, "kernel_ms": kms, "traffic": None}
     if prefix:
         # the profile events bracket the prefix kernel: a dense contraction, measured against the
         # bf16 tensor peak.  Algorithmic flops: QK^T and PV once each over the shared prefix.
@@ -326,7 +360,8 @@ def run_ours(args):
                    "l2": "inputs exceed L2 (no flush)" if nbytes > 4 * 126e6 else "inputs fit L2; not flushed",
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "grid_blocks": da.get_option("grid_blocks"),
-                   "path": "cascade (shared prefix on tcgen05)" if prefix else "decode_attn"},
+                   "path": f"decode_attn_extend, {Lq} new tokens per sequence (causal, tcgen05)" if Lq else
+                           ("cascade (shared prefix on tcgen05)" if prefix else "decode_attn")},
         "frac_of_8TBs": gbs / world / NOMINAL_HBM_GBS, "seq_per_s": seqs,
         "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
         "roofline": roofline,
@@ -355,6 +390,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-every", type=int, default=1, help="oracle sample: every n-th sequence")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extend", type=int, default=0, metavar="LQ",
+                    help="time decode_attn_extend with LQ new (causal) query tokens per sequence instead of decode_attn")
     ap.add_argument("--cascade", action="store_true",
                     help="c5a only: attend the shared 16384-token prefix once for the batch (decode_attn_cascade)")
     args = ap.parse_args()
