@@ -53,6 +53,24 @@ def _load():
             lib.kv_append_oracle.restype = ctypes.c_int
             lib.kv_append_oracle.argtypes = [p, p, i64, i64, i64, p, p, i64, i64, i64, i64, i64, p, i64, p]
             lib.decode_attn_oracle_max_threads.restype = ctypes.c_int
+            lib.e4m3_bits_to_double.restype = ctypes.c_double
+            lib.e4m3_bits_to_double.argtypes = [ctypes.c_uint8]
+            lib.e4m3_nearest_code.restype = ctypes.c_uint8
+            lib.e4m3_nearest_code.argtypes = [ctypes.c_double]
+            lib.e4m3_quantize_oracle.restype = None
+            lib.e4m3_quantize_oracle.argtypes = [p, i64, ctypes.c_float, p]
+            lib.decode_attn_fp8kv_oracle.restype = ctypes.c_int
+            lib.decode_attn_fp8kv_oracle.argtypes = [
+                p, i64, i64, i64,            # q, B, Hq, D
+                p, p, i64, i64, i64,         # k codes, v codes, num_pages, Hkv, P
+                i64, i64, i64,               # strides (bytes): page, head, token
+                p, p,                        # k_scale, v_scale (float [Hkv] or NULL)
+                p, i64, p,                   # block_table, max_pages, seq_lens
+                i32, ctypes.c_double,        # window, scale
+                p, p, i32,                   # out, lse, num_threads
+            ]
+            lib.kv_append_fp8_oracle.restype = ctypes.c_int
+            lib.kv_append_fp8_oracle.argtypes = [p, p, i64, i64, i64, p, p, i64, i64, i64, i64, i64, p, p, p, i64, p]
             _lib = lib
     return _lib
 
@@ -155,3 +173,110 @@ def extend_attn_oracle(q, k_pages, v_pages, block_table, seq_lens, scale: float,
         o, l = decode_attn_oracle(q[:, qi].contiguous(), k_pages, v_pages, block_table, cut, 0, scale, num_threads)
         out[:, qi], lse[:, qi] = o, l
     return out, lse
+
+
+# ----------------------------------------------------------------------------- 8-bit (E4M3) cache
+
+def _u8_codes(x) -> np.ndarray:
+    """View a cache of E4M3 codes (torch CPU uint8 / float8_e4m3fn, or numpy uint8) as uint8."""
+    if isinstance(x, np.ndarray):
+        if x.dtype != np.uint8:
+            raise TypeError("numpy inputs must hold E4M3 codes as uint8")
+        return x
+    import torch  # only to reinterpret a CPU tensor's storage
+
+    if x.device.type != "cpu":
+        raise TypeError("expected a CPU tensor")
+    if x.dtype == torch.float8_e4m3fn:
+        x = x.view(torch.uint8)
+    if x.dtype != torch.uint8:
+        raise TypeError("expected uint8 or float8_e4m3fn codes")
+    return x.numpy()
+
+
+def _scales(x, Hkv):
+    if x is None:
+        return None
+    a = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
+    if a.shape != (Hkv,):
+        raise ValueError("a scale array must be [Hkv]")
+    return a
+
+
+def e4m3_value(code: int) -> float:
+    """Value of one E4M3 code (NaN for 0x7F / 0xFF)."""
+    return float(_load().e4m3_bits_to_double(int(code) & 0xFF))
+
+
+def e4m3_nearest_code(x: float) -> int:
+    """The E4M3 code nearest to x: ties to even, saturating at +-448, NaN -> 0x7F."""
+    return int(_load().e4m3_nearest_code(float(x)))
+
+
+def e4m3_quantize(x_bf16, scale: float) -> np.ndarray:
+    """Codes of nearest_e4m3(x / scale) with the quotient taken in fp32; x: bf16 (any shape)."""
+    xb = np.ascontiguousarray(_bf16_bits(x_bf16))
+    out = np.empty(xb.shape, dtype=np.uint8)
+    _load().e4m3_quantize_oracle(xb.ctypes.data, xb.size, float(np.float32(scale)), out.ctypes.data)
+    return out
+
+
+def decode_attn_fp8kv_oracle(q, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens, window: int,
+                             scale: float, num_threads: int = 0):
+    """fp64 decode attention over a paged cache of E4M3 codes with per-KV-head fp32 factors.
+
+    q                 bf16 [B, Hq, D]
+    k_pages, v_pages  E4M3 codes [num_pages, Hkv, P, D], any strides with a contiguous last dim
+    k_scale, v_scale  float32 [Hkv] or None (all 1): K = k_scale[g] * e4m3(code)
+    other arguments and the result as decode_attn_oracle
+    """
+    lib = _load()
+    qb = np.ascontiguousarray(_bf16_bits(q))
+    kb, vb = _u8_codes(k_pages), _u8_codes(v_pages)
+    if kb.shape != vb.shape or kb.strides != vb.strides or kb.ndim != 4 or qb.ndim != 3:
+        raise ValueError("pools must share shape and strides; q must be [B,Hq,D]")
+    B, Hq, D = qb.shape
+    num_pages, Hkv, P, Dk = kb.shape
+    if Dk != D or kb.strides[3] != 1:
+        raise ValueError("head_dim mismatch or non-contiguous last dim")
+    ks, vs = _scales(k_scale, Hkv), _scales(v_scale, Hkv)
+    bt = np.ascontiguousarray(np.asarray(block_table, dtype=np.int32))
+    sl = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32))
+    if bt.ndim != 2 or bt.shape[0] != B or sl.shape != (B,):
+        raise ValueError("block_table must be [B,max_pages] and seq_lens [B]")
+    out = np.empty((B, Hq, D), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    rc = lib.decode_attn_fp8kv_oracle(
+        qb.ctypes.data, B, Hq, D, kb.ctypes.data, vb.ctypes.data, num_pages, Hkv, P,
+        kb.strides[0], kb.strides[1], kb.strides[2],
+        ks.ctypes.data if ks is not None else None, vs.ctypes.data if vs is not None else None,
+        bt.ctypes.data, bt.shape[1], sl.ctypes.data, int(window), float(np.float32(scale)),
+        out.ctypes.data, lse.ctypes.data, int(num_threads))
+    if rc != 0:
+        raise RuntimeError(f"decode_attn_fp8kv_oracle failed with code {rc}")
+    return out, lse
+
+
+def kv_append_fp8_oracle(k_new, v_new, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens) -> None:
+    """Quantise each sequence's new bf16 K/V rows [B, Hkv, D] per KV head and write the codes into
+    position seq_lens[b]-1 of the 8-bit cache, IN PLACE."""
+    lib = _load()
+    kn = np.ascontiguousarray(_bf16_bits(k_new))
+    vn = np.ascontiguousarray(_bf16_bits(v_new))
+    kb, vb = _u8_codes(k_pages), _u8_codes(v_pages)
+    if kb.shape != vb.shape or kb.strides != vb.strides or kb.ndim != 4 or kb.strides[3] != 1:
+        raise ValueError("k_pages and v_pages must share shape and strides, contiguous last dim")
+    B, Hkv, D = kn.shape
+    num_pages, Hk, P, Dk = kb.shape
+    if Hk != Hkv or Dk != D or vn.shape != kn.shape:
+        raise ValueError("shape mismatch")
+    ks, vs = _scales(k_scale, Hkv), _scales(v_scale, Hkv)
+    bt = np.ascontiguousarray(np.asarray(block_table, dtype=np.int32))
+    sl = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32))
+    rc = lib.kv_append_fp8_oracle(kn.ctypes.data, vn.ctypes.data, B, Hkv, D, kb.ctypes.data, vb.ctypes.data,
+                                  num_pages, P, kb.strides[0], kb.strides[1], kb.strides[2],
+                                  ks.ctypes.data if ks is not None else None,
+                                  vs.ctypes.data if vs is not None else None,
+                                  bt.ctypes.data, bt.shape[1], sl.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"kv_append_fp8_oracle failed with code {rc}")

@@ -35,6 +35,10 @@ class Case:
     window: int
     scale: float
     lens: np.ndarray = field(repr=False, default=None)  # host copy of seq_lens (int64)
+    # 8-bit cache only: the pools then hold E4M3 codes (torch.uint8) and these are the fp32 [Hkv]
+    # dequantisation factors (K = k_scale[g] * e4m3(code)); None for a bf16 cache
+    k_scale: Optional[torch.Tensor] = None
+    v_scale: Optional[torch.Tensor] = None
 
     @property
     def B(self) -> int:
@@ -62,13 +66,32 @@ class Case:
         lo = L - n
         P = self.P
         pages_touched = np.where(n > 0, (L - 1) // P - lo // P + 1, 0)
-        per_seq = (n * (2 * Hkv * Dh * 2) + pages_touched * 4 + 4
+        per_seq = (n * (2 * Hkv * Dh * self.k_pages.element_size()) + pages_touched * 4 + 4
                    + Hq * Dh * 2 + Hq * Dh * out_itemsize + Hq * 4)
-        return int(per_seq.sum())
+        scales = 2 * Hkv * 4 if self.k_scale is not None else 0
+        return int(per_seq.sum()) + scales
 
 
 def _randn_bf16(shape, gen: torch.Generator, device) -> torch.Tensor:
     return torch.randn(shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
+
+
+E4M3_NAN = 0x7F
+
+
+def _randn_e4m3(shape, gen: torch.Generator, device, inv_scale: torch.Tensor) -> torch.Tensor:
+    """Random E4M3 codes (uint8): N(0,1) draws times ``inv_scale`` (broadcast), cast by torch.  This
+    only makes inputs: both the CUDA path and the oracle take the codes as given."""
+    x = torch.randn(shape, generator=gen, device=device, dtype=torch.float32) * inv_scale
+    return x.clamp_(-448.0, 448.0).to(torch.float8_e4m3fn).view(torch.uint8)
+
+
+def default_kv_scales(Hkv: int):
+    """The fixed, deliberately not power-of-two factors the 8-bit workloads use: with them the
+    dequantised cache is again ~N(0,1) and the stored magnitudes stay below 448."""
+    g = np.arange(Hkv, dtype=np.float32)
+    return (np.float32(0.02) + np.float32(0.003) * g).astype(np.float32), \
+           (np.float32(0.025) - np.float32(0.001) * g).astype(np.float32)
 
 
 def build_case(name: str, lens: Sequence[int], P: int, seed: int, device="cpu", *,
@@ -76,7 +99,8 @@ def build_case(name: str, lens: Sequence[int], P: int, seed: int, device="cpu", 
                scale: Optional[float] = None, shuffle: bool = True,
                pool_pages: Optional[int] = None, shared_prefix_tokens: int = 0,
                layout: str = "head_major", poison: bool = True,
-               pad_table_to: Optional[int] = None, fill_chunk_pages: int = 16384) -> Case:
+               pad_table_to: Optional[int] = None, fill_chunk_pages: int = 16384,
+               kv_dtype: str = "bf16") -> Case:
     """Build one problem.
 
     lens                  context length of each sequence (current token included)
@@ -91,6 +115,8 @@ def build_case(name: str, lens: Sequence[int], P: int, seed: int, device="cpu", 
                           (same logical shape, different strides)
     poison                NaN in page tails past each sequence's end, in unused
                           pool pages; block-table padding is -1 either way
+    kv_dtype              "bf16", or "fp8": pools of E4M3 codes (uint8) with the per-KV-head
+                          factors of default_kv_scales(); NaN is then the code 0x7F
     """
     rng = np.random.default_rng(seed)
     gen = torch.Generator(device=device)
@@ -131,17 +157,29 @@ def build_case(name: str, lens: Sequence[int], P: int, seed: int, device="cpu", 
     else:
         raise ValueError(layout)
 
-    nan = float("nan")
+    if kv_dtype not in ("bf16", "fp8"):
+        raise ValueError(kv_dtype)
+    fp8 = kv_dtype == "fp8"
+    nan = E4M3_NAN if fp8 else float("nan")
+    pool_dtype = torch.uint8 if fp8 else torch.bfloat16
+    k_scale = v_scale = None
+    if fp8:
+        k_scale, v_scale = (torch.from_numpy(a).to(device) for a in default_kv_scales(Hkv))
+    head_shape = (1, Hkv, 1, 1) if layout == "head_major" else (1, 1, Hkv, 1)
     pools = []
-    for _ in range(2):
+    for which in range(2):
         if poison and pool > referenced:
-            t = torch.full(phys, nan, dtype=torch.bfloat16, device=device)
+            t = torch.full(phys, nan, dtype=pool_dtype, device=device)
         else:
-            t = torch.empty(phys, dtype=torch.bfloat16, device=device)
+            t = torch.empty(phys, dtype=pool_dtype, device=device)
         ids_t = torch.from_numpy(np.ascontiguousarray(ids)).to(device)
         for s in range(0, referenced, fill_chunk_pages):
             sel = ids_t[s:s + fill_chunk_pages]
-            t[sel] = _randn_bf16((len(sel),) + phys[1:], gen, device)
+            if fp8:
+                inv = (1.0 / (k_scale if which == 0 else v_scale)).reshape(head_shape)
+                t[sel] = _randn_e4m3((len(sel),) + phys[1:], gen, device, inv)
+            else:
+                t[sel] = _randn_bf16((len(sel),) + phys[1:], gen, device)
         pools.append(t)
     k_pages, v_pages = (to_logical(t) for t in pools)
 
@@ -160,7 +198,7 @@ def build_case(name: str, lens: Sequence[int], P: int, seed: int, device="cpu", 
         block_table=torch.from_numpy(bt).to(device),
         seq_lens=torch.from_numpy(lens.astype(np.int32)).to(device),
         window=int(window), scale=float(scale if scale is not None else 1.0 / math.sqrt(Dh)),
-        lens=lens.copy())
+        lens=lens.copy(), k_scale=k_scale, v_scale=v_scale)
 
 
 # ----------------------------------------------------------------------------
@@ -192,38 +230,38 @@ def c1(device="cpu") -> Case:
     return case
 
 
-def c2(device="cpu", B: int = 64) -> Case:
+def c2(device="cpu", B: int = 64, kv_dtype: str = "bf16") -> Case:
     """64 sequences, lengths uniform in [1024, 16384], page 16, block tables dealt
     from one random permutation of an exact-size pool, seed 1."""
-    return build_case("c2", lengths_c2(1, B), 16, 1, device)
+    return build_case("c2", lengths_c2(1, B), 16, 1, device, kv_dtype=kv_dtype)
 
 
-def c3(device="cpu", B: int = 256, pool_bytes: float = 20e9) -> Case:
+def c3(device="cpu", B: int = 256, pool_bytes: float = 20e9, kv_dtype: str = "bf16") -> Case:
     """256 sequences, lengths log-uniform in [512, 32768], page 16, referenced pages
     scattered through a ~20 GB pool (K + V) whose other pages are NaN, seed 2."""
     lens = lengths_c3(2, B)
-    page_bytes = 2 * HKV * 16 * D * 2
+    page_bytes = 2 * HKV * 16 * D * 2   # the pool keeps its page count when the cache is 8-bit
     referenced = int(((lens + 15) // 16).sum())
     pool = max(int(pool_bytes // page_bytes), referenced)
-    return build_case("c3", lens, 16, 2, device, pool_pages=pool)
+    return build_case("c3", lens, 16, 2, device, pool_pages=pool, kv_dtype=kv_dtype)
 
 
-def c4(device="cpu", B: int = 8, L: int = 131072) -> Case:
+def c4(device="cpu", B: int = 8, L: int = 131072, kv_dtype: str = "bf16") -> Case:
     """8 sequences x 131,072 tokens, page 64, shuffled pool, seed 3."""
-    return build_case("c4", [L] * B, 64, 3, device)
+    return build_case("c4", [L] * B, 64, 3, device, kv_dtype=kv_dtype)
 
 
-def c5(device="cpu", window: int = 0, B: int = 128) -> Case:
+def c5(device="cpu", window: int = 0, B: int = 128, kv_dtype: str = "bf16") -> Case:
     """128 sequences sharing a 16,384-token prefix (same physical pages in every
     block table) plus unique suffixes uniform in [0, 8192], page 16, seed 4;
     window = 0 (full) or 8192."""
     return build_case("c5b" if window else "c5a", lengths_c5(4, B), 16, 4, device,
-                      shared_prefix_tokens=16384, window=window)
+                      shared_prefix_tokens=16384, window=window, kv_dtype=kv_dtype)
 
 
 RECIPES = {"c1": c1, "c2": c2, "c3": c3, "c4": c4,
-           "c5a": lambda device="cpu": c5(device, 0),
-           "c5b": lambda device="cpu": c5(device, 8192)}
+           "c5a": lambda device="cpu", **kw: c5(device, 0, **kw),
+           "c5b": lambda device="cpu", **kw: c5(device, 8192, **kw)}
 
 
 # ----------------------------------------------------------------------------
@@ -252,7 +290,9 @@ def host_subcase(case: Case, seq_ids: Sequence[int]) -> Case:
     v = case.v_pages.index_select(0, sel).contiguous().cpu()
     return Case(name=case.name + "/sub", q=case.q[seq_ids].cpu(), k_pages=k, v_pages=v,
                 block_table=torch.from_numpy(new_bt), seq_lens=torch.from_numpy(lens.astype(np.int32)),
-                window=case.window, scale=case.scale, lens=lens.copy())
+                window=case.window, scale=case.scale, lens=lens.copy(),
+                k_scale=None if case.k_scale is None else case.k_scale.cpu(),
+                v_scale=None if case.v_scale is None else case.v_scale.cpu())
 
 
 def to_device(case: Case, device) -> Case:
@@ -267,4 +307,6 @@ def to_device(case: Case, device) -> Case:
         return dense.permute(inv)
     return Case(name=case.name, q=case.q.to(device), k_pages=mv(case.k_pages), v_pages=mv(case.v_pages),
                 block_table=case.block_table.to(device), seq_lens=case.seq_lens.to(device),
-                window=case.window, scale=case.scale, lens=case.lens.copy())
+                window=case.window, scale=case.scale, lens=case.lens.copy(),
+                k_scale=None if case.k_scale is None else case.k_scale.to(device),
+                v_scale=None if case.v_scale is None else case.v_scale.to(device))
