@@ -135,14 +135,30 @@ def oracle_sample(case, every: int):
     sub = workloads.host_subcase(case, ids)
     threads = oracle.max_threads()
     t0 = time.perf_counter()
-    oracle.decode_attn_oracle(sub.q, sub.k_pages, sub.v_pages, sub.block_table, sub.seq_lens,
-                              sub.window, sub.scale, 0)
+    if sub.k_scale is not None:   # 8-bit cache
+        oracle.decode_attn_fp8kv_oracle(sub.q, sub.k_pages, sub.v_pages, sub.k_scale, sub.v_scale, sub.block_table,
+                                        sub.seq_lens, sub.window, sub.scale, 0)
+    else:
+        oracle.decode_attn_oracle(sub.q, sub.k_pages, sub.v_pages, sub.block_table, sub.seq_lens,
+                                  sub.window, sub.scale, 0)
     dt = time.perf_counter() - t0
     nbytes = sub.algorithmic_bytes(4)
     return {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
             "sample": f"every {every}th sequence of {case.name} ({len(ids)} of {case.B} sequences, "
                       f"{int(sub.attended_tokens().sum())} attended tokens, {dt:.2f} s wall)",
             "seconds": dt, "seq_per_s": len(ids) / dt}
+
+
+def kv_text(args) -> str:
+    return "; KV cache as FP8 E4M3 codes with per-KV-head fp32 factors" if args.kv == "fp8" else ""
+
+
+def make_case(args, device):
+    if args.kv == "fp8":
+        if args.workload == "c1":
+            raise SystemExit("--kv fp8: c1 is a bf16 parity configuration")
+        return workloads.RECIPES[args.workload](device, kv_dtype="fp8")
+    return workloads.RECIPES[args.workload](device)
 
 
 # ----------------------------------------------------------------------------- reference arm
@@ -152,7 +168,7 @@ def run_reference(args):
     if rank != 0:
         return 0
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    case = workloads.RECIPES[args.workload](dev)
+    case = make_case(args, dev)
     every = max(args.ref_every, 1)
     for _ in range(args.warmup if args.warmup < 2 else 1):
         oracle_sample(case, every * 4)
@@ -163,7 +179,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": best["value"], "unit": "GB/s", "n_gpus": args.gpus,
         "steps": len(res), "warmup": 1, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD_TEXT[args.workload], "sample": best["sample"]},
+        "config": {"workload": WORKLOAD_TEXT[args.workload] + kv_text(args), "sample": best["sample"]},
         "seq_per_s": best["seq_per_s"], "frac_of_8TBs": best["value"] / NOMINAL_HBM_GBS,
         "cpu_baseline": {k: best[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": best["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -187,7 +203,10 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
-    case = workloads.RECIPES[args.workload](device)
+    case = make_case(args, device)
+    kv8 = args.kv == "fp8"
+    if kv8 and (args.cascade or args.extend):
+        raise SystemExit("--kv fp8 applies to decode_attn only")
     out = torch.empty(case.q.shape, dtype=torch.float32, device=device)
     lse = torch.empty(case.q.shape[:2], dtype=torch.float32, device=device)
     nbytes = case.algorithmic_bytes(4)
@@ -220,6 +239,9 @@ def run_ours(args):
         elif prefix:
             da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
                                    prefix, case.scale, out=out, lse=lse, stream=stream)
+        elif kv8:
+            da.decode_attn_fp8kv(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table,
+                                 case.seq_lens, case.window, case.scale, out=out, lse=lse, stream=stream)
         else:
             da.decode_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
                            case.window, case.scale, out=out, lse=lse, stream=stream)
@@ -297,6 +319,11 @@ def run_ours(args):
             da.decode_attn_cascade(q_d, case.k_pages, case.v_pages, bt_d, sl_d, prefix, case.scale,
                                    out=out, lse=lse, stream=stream)
             out_h.copy_(out, non_blocking=True); lse_h.copy_(lse, non_blocking=True)
+        elif kv8:   # no host-io entry point for the 8-bit cache: same copies, made here on the same stream
+            q_d.copy_(q_h, non_blocking=True); bt_d.copy_(bt_h, non_blocking=True); sl_d.copy_(sl_h, non_blocking=True)
+            da.decode_attn_fp8kv(q_d, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt_d, sl_d,
+                                 case.window, case.scale, out=out, lse=lse, stream=stream)
+            out_h.copy_(out, non_blocking=True); lse_h.copy_(lse, non_blocking=True)
         else:
             da.decode_attn_host_io(q_h, case.k_pages, case.v_pages, bt_h, sl_h, case.window, case.scale,
                                    out_h, lse_h, stream=stream)
@@ -321,9 +348,10 @@ def run_ours(args):
     peak, peak_src = measured_peak()
     kms = kernel_ms if kernel_ms is not None else ms_per_step
     achieved = nbytes / (kms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "partition_kernel", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "partition_kernel (8-bit cache)" if kv8 else "partition_kernel",
+                "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                "kernel_ms": kms, "traffic": NCU_TRAFFIC.get((args.workload, da.version()))}
+                "kernel_ms": kms, "traffic": None if kv8 else NCU_TRAFFIC.get((args.workload, da.version()))}
     if Lq:
         # one kernel, a dense causal contraction: algorithmic flops = QK^T and PV over each query's keys
         Hq, Dh = case.q.shape[1], case.q.shape[2]
@@ -354,14 +382,15 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD_TEXT[args.workload], "sequences": case.B,
+        "dtype": "fp8 e4m3 (f32 accumulate)" if kv8 else "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD_TEXT[args.workload] + kv_text(args), "sequences": case.B,
                    "attended_tokens": int(case.attended_tokens().sum()), "algorithmic_bytes": nbytes,
                    "l2": "inputs exceed L2 (no flush)" if nbytes > 4 * 126e6 else "inputs fit L2; not flushed",
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "grid_blocks": da.get_option("grid_blocks"),
                    "path": f"decode_attn_extend, {Lq} new tokens per sequence (causal, tcgen05)" if Lq else
-                           ("cascade (shared prefix on tcgen05)" if prefix else "decode_attn")},
+                           ("cascade (shared prefix on tcgen05)" if prefix else
+                            ("decode_attn_fp8kv" if kv8 else "decode_attn"))},
         "frac_of_8TBs": gbs / world / NOMINAL_HBM_GBS, "seq_per_s": seqs,
         "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
         "roofline": roofline,
@@ -392,6 +421,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extend", type=int, default=0, metavar="LQ",
                     help="time decode_attn_extend with LQ new (causal) query tokens per sequence instead of decode_attn")
+    ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
+                    help="cache element type: bf16 (decode_attn, the headline) or fp8 (decode_attn_fp8kv)")
     ap.add_argument("--cascade", action="store_true",
                     help="c5a only: attend the shared 16384-token prefix once for the batch (decode_attn_cascade)")
     args = ap.parse_args()

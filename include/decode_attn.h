@@ -59,7 +59,7 @@ typedef enum {
     DA_ERR_CUDA = 7          /* a CUDA call failed; see decode_attn_last_cuda_error()   */
 } da_status;
 
-typedef enum { DA_BF16 = 1, DA_F32 = 2, DA_I32 = 3 } da_dtype;
+typedef enum { DA_BF16 = 1, DA_F32 = 2, DA_I32 = 3, DA_FP8_E4M3 = 4 /* one byte per element */ } da_dtype;
 
 /* Device-side status codes (first word of the status record). */
 typedef enum {
@@ -106,6 +106,33 @@ typedef struct da_tensor {
 int decode_attn(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
                 const da_tensor *block_table, const da_tensor *seq_lens, int32_t window, float scale,
                 da_tensor *out, da_tensor *lse, void *stream);
+
+/*
+ * decode_attn_fp8kv -- decode_attn() over a cache stored in 8 bits per element: half the bytes per
+ * attended token, which is the only way past the HBM roofline of the bf16 cache.  The paper does
+ * not fix a cache precision; the reading taken is the usual serving one: K and V hold FP8 E4M3
+ * codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, S.1111.111 = NaN,
+ * largest finite value 448; "FP8 Formats for Deep Learning", Sec. 3) with one fp32 factor per KV
+ * head:  K[page,g,r,:] = k_scale[g] * e4m3(k_pages[page,g,r,:]),  V likewise with v_scale[g].
+ * The result is the attention of decode_attn() over those dequantised values.
+ *
+ *   k_pages, v_pages  DA_FP8_E4M3 [num_pages, Hkv, P, 128]; last dim contiguous, base and every
+ *                     stride a multiple of 16 bytes; P in {16, 32, 64, 128}
+ *   k_scale, v_scale  DEVICE float[Hkv]; NULL means all factors are 1
+ *   q                 bf16, finite (a head's query is rescaled by a power of two and split exactly
+ *                     into two E4M3 terms; elements below 2^-13 of the head's largest magnitude
+ *                     are carried to within 2^-21 of that largest)
+ *   other arguments, workspace, status and error conventions: as decode_attn().
+ *
+ * Arithmetic: both products run on the FP8 tensor-core path (mma m16n8k32, fp32 accumulation) with
+ * no conversion of the cache: softmax in fp32 as in decode_attn(); every softmax weight enters the
+ * PV product as four E5M2 terms, i.e. to 2^-12 of itself down to 2^-31 of the row's largest weight.
+ * Output error is therefore about 2^-12 * max|V| in the worst case (observed: ~1e-5 on N(0,1) data).
+ */
+int decode_attn_fp8kv(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                      const float *k_scale, const float *v_scale, const da_tensor *block_table,
+                      const da_tensor *seq_lens, int32_t window, float scale, da_tensor *out,
+                      da_tensor *lse, void *stream);
 
 /*
  * decode_attn_cascade -- decode_attn() (full attention, no window) for a batch whose sequences all

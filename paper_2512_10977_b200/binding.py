@@ -19,8 +19,10 @@ _lock = threading.Lock()
 _lib = None
 _workspaces = {}   # device index -> torch uint8 tensor kept alive while registered
 
-DA_BF16, DA_F32, DA_I32 = 1, 2, 3
-_DTYPES = {torch.bfloat16: DA_BF16, torch.float32: DA_F32, torch.int32: DA_I32}
+DA_BF16, DA_F32, DA_I32, DA_FP8_E4M3 = 1, 2, 3, 4
+# E4M3 codes may be handed over as torch.uint8 or torch.float8_e4m3fn storage
+_DTYPES = {torch.bfloat16: DA_BF16, torch.float32: DA_F32, torch.int32: DA_I32,
+           torch.uint8: DA_FP8_E4M3, torch.float8_e4m3fn: DA_FP8_E4M3}
 
 
 class DecodeAttnError(RuntimeError):
@@ -47,6 +49,8 @@ def lib() -> ctypes.CDLL:
             vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
             L.decode_attn.restype = ctypes.c_int
             L.decode_attn.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_fp8kv.restype = ctypes.c_int
+            L.decode_attn_fp8kv.argtypes = [T, T, T, vp, vp, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_cascade.restype = ctypes.c_int
             L.decode_attn_cascade.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_append.restype = ctypes.c_int
@@ -174,6 +178,30 @@ def decode_attn(q, k_pages, v_pages, block_table, seq_lens, window: int, scale: 
         tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
         _check(lib().decode_attn(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
                                  int(window), float(scale), _ref(tv[5]), _ref(tv[6]), _stream_ptr(stream)))
+    return out, lse
+
+
+def decode_attn_fp8kv(q, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens, window: int, scale: float,
+                      out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None, out_dtype=torch.float32, want_lse: bool = True):
+    """``decode_attn`` over a cache of FP8 E4M3 codes (torch.uint8 or float8_e4m3fn pools) with fp32
+    per-KV-head factors ``k_scale`` / ``v_scale`` (device tensors [Hkv], or None for 1).  Returns (out, lse)."""
+    if out is None:
+        out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+    for sc in (k_scale, v_scale):
+        if sc is not None and (sc.dtype != torch.float32 or not sc.is_contiguous() or sc.device != k_pages.device
+                               or sc.numel() != k_pages.shape[1]):
+            raise ValueError("scales must be contiguous float32 [Hkv] tensors on the cache's device")
+    with torch.cuda.device(k_pages.device):
+        _auto_workspace(q, k_pages, block_table)
+        tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
+        _check(lib().decode_attn_fp8kv(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]),
+                                       k_scale.data_ptr() if k_scale is not None else None,
+                                       v_scale.data_ptr() if v_scale is not None else None,
+                                       _ref(tv[3]), _ref(tv[4]), int(window), float(scale), _ref(tv[5]), _ref(tv[6]),
+                                       _stream_ptr(stream)))
     return out, lse
 
 

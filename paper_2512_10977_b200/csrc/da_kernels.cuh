@@ -18,8 +18,11 @@ namespace da {
 
 constexpr int HEAD_DIM = 128;
 constexpr int NCW = 4;                      // consumer warps per block; each owns 16 tokens of a tile
-constexpr int TILE_T = 16 * NCW;            // tokens per pipeline stage
-constexpr int KV_BYTES = TILE_T * 256;      // a K (or V) tile: TILE_T rows of 128 bf16
+constexpr int TILE_T = 16 * NCW;            // tokens per pipeline stage, bf16 cache
+constexpr int TILE_T8 = 32 * NCW;           // tokens per pipeline stage, 8-bit cache (a warp owns 32)
+constexpr int KV_BYTES = TILE_T * 256;      // a K (or V) tile: TILE_T rows of 128 bf16, or TILE_T8 rows of 128 bytes
+static_assert(TILE_T8 * 128 == KV_BYTES, "both cache types fill a stage");
+constexpr float P8_SHIFT = 15.f;            // 8-bit cache: softmax weights are carried as 2^15 * p (E5M2 terms)
 constexpr int STAGE_BYTES = 2 * KV_BYTES;   // K tile followed by V tile
 constexpr int NTHREADS = (NCW + 1) * 32;    // + one producer warp
 constexpr int PLAN_THREADS = 1024;
@@ -85,6 +88,7 @@ struct PartParams {
     int32_t *status;
     int32_t B, Hkv, G, P, box_rows, num_pages, out_bf16;
     float scale_log2;         // scale * log2(e)
+    const float *k_scale, *v_scale;   // 8-bit cache: per-KV-head factors (NULL: 1)
 };
 
 struct PlanParams {
@@ -100,6 +104,7 @@ struct PlanParams {
     PlanHeader *hdr;
     int32_t *status;
     int32_t B, Hkv, P, window;
+    int32_t tile_t;           // tokens per tile (TILE_T or TILE_T8)
     int32_t first_token;      // tokens before this one are not attended (the cascade's suffix pass)
     int32_t n_static, n_tail_max, static_frac_q8;   // large units; most ticketed units; share of the
                                                     // line given to the large units, in 1/256
@@ -213,8 +218,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
             lo = (p.window > 0 && p.window < L) ? L - p.window : 0;
             lo = max(lo, min(p.first_token, L));
             if (L > lo) {
-                first = lo / TILE_T;
-                nt = (L - 1) / TILE_T - first + 1;
+                first = lo / p.tile_t;
+                nt = (L - 1) / p.tile_t - first + 1;
             }
         }
         // block-wide exclusive scan of nt
@@ -358,12 +363,14 @@ __device__ __forceinline__ uint32_t row_offset(int row, int box_rows)
     return (uint32_t)((row / box_rows) * (box_rows * 256) + (row % box_rows) * 128);
 }
 
-template <int NT8>
+template <int NT8, bool KV8>
 __global__ void __launch_bounds__(NTHREADS, 2)
 partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const PartParams p)
 {
     using C = PartCfg<NT8>;
+    constexpr int TT = KV8 ? TILE_T8 : TILE_T;        // tokens per tile
+    constexpr uint32_t ROW_BYTES = KV8 ? 128u : 256u;  // one token row of one KV head
     constexpr int NSTAGES = C::NSTAGES;
     constexpr int HEADS = C::HEADS;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -403,10 +410,10 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     if (warp == NCW) {
         // ------------------------------------------------------------------ producer warp
         // Lane -> (box, K|V).  A box is box_rows token rows (all 128 columns) of one page.
-        const int nboxes = TILE_T / p.box_rows;
+        const int nboxes = TT / p.box_rows;
         const int box = lane >> 1, is_v = lane & 1;
         const bool active = lane < nboxes * 2;
-        const uint32_t box_bytes = (uint32_t)p.box_rows * 256u;
+        const uint32_t box_bytes = (uint32_t)p.box_rows * ROW_BYTES;
         const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
         const int n_static = p.hdr->n_static, n_units = n_static + p.hdr->n_tail;
         uint32_t it = 0;
@@ -454,7 +461,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         };
         struct Tile { int page, row, t0, g, b, lo, L, flags, slot; bool need; };
         auto fetch = [&](Tile &t) {   // describe the cursor's tile and start its block-table read
-            t.t0 = (si.z + rel + i) * TILE_T;
+            t.t0 = (si.z + rel + i) * TT;
             const int tok0 = t.t0 + box * p.box_rows;
             t.need = active && tok0 < si.y && tok0 + p.box_rows > si.x;
             t.page = 0;
@@ -508,7 +515,10 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             __syncwarp();
             if (cur.need) {
                 const uint32_t dst = smem_base + stage * STAGE_BYTES + is_v * KV_BYTES + box * box_bytes;
-                tma_load_5d(dst, tm, 0, cur.row, 0, cur.g, cur.page, bar_full + 8 * stage);
+                if constexpr (KV8)
+                    tma_load_4d(dst, tm, 0, cur.row, cur.g, cur.page, bar_full + 8 * stage);
+                else
+                    tma_load_5d(dst, tm, 0, cur.row, 0, cur.g, cur.page, bar_full + 8 * stage);
             }
             ++it;
             have = n_have;
@@ -560,6 +570,27 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const uint32_t k_off = row_offset(k_row, p.box_rows), v_off = row_offset(v_row, p.box_rows);
     const uint32_t k_sw = (uint32_t)(k_row & 7), v_sw = (uint32_t)(v_row & 7);
 
+    // ---- 8-bit cache: a warp owns 32 tokens of a 128-token tile (rows of 128 bytes, 16-byte chunk index
+    // XORed with the row's low three bits).  Its scores form two 16-row tiles A and B (mma m16n8k32,
+    // K rows as the A operand); row x of tile A is warp-local token tok_a(x), of tile B tok_b(x).  The
+    // maps are chosen so that (1) the eight rows of every ldmatrix phase differ in their low three bits
+    // (no bank conflicts) and (2) the PV product can take the weights of BOTH tiles as one k = 32
+    // operand: packing the codes of (A row x, B row x) into one 16-bit element and transposing with
+    // movmatrix puts, in k slot 4c+i of the B fragment, A row 2c (i=0), B row 2c (1), A row 2c+1 (2),
+    // B row 2c+1 (3), and rows +8 in slots 16..31; V's transposed ldmatrix takes one row address per k
+    // slot, so it is simply pointed at the token each slot holds.
+    auto tok_a = [](int x) { return x < 4 ? x : (x < 12 ? x + 8 : x + 16); };
+    auto tok_b = [](int x) { return x < 8 ? x + 4 : x + 12; };
+    const int x8 = (lane & 7) + ((lane >> 3) & 1) * 8;          // QK ldmatrix: row of the 16-row tile
+    const int k8_chunk = lane >> 4;                             //              16-byte half of the 32-byte k step
+    const int row_a8 = 32 * warp + tok_a(x8), row_b8 = 32 * warp + tok_b(x8);
+    const uint32_t ka8_off = (uint32_t)row_a8 * 128u, kb8_off = (uint32_t)row_b8 * 128u;
+    const uint32_t ka8_sw = (uint32_t)(row_a8 & 7), kb8_sw = (uint32_t)(row_b8 & 7);
+    const int slot_x = 2 * ((lane & 15) >> 2) + ((lane & 3) >> 1) + 8 * (lane >> 4);   // PV: k slot `lane`
+    const int row_v8 = 32 * warp + ((lane & 1) ? tok_b(slot_x) : tok_a(slot_x));
+    const uint32_t v8_off = (uint32_t)row_v8 * 128u, v8_sw = (uint32_t)(row_v8 & 7);
+    const int t_a0 = tok_a(r), t_a1 = tok_a(r + 8), t_b0 = tok_b(r), t_b1 = tok_b(r + 8);   // tokens of this lane's scores
+
     auto give_up = [&](int where) {
         if (*abort_flag == 0) {
             *abort_flag = 1;
@@ -581,6 +612,62 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
     };
 
+    // 8-bit cache: Q^T as E4M3 B fragments of S^T = K Q^T (mma m16n8k32).  A head's query vector is
+    // scaled by a power of two so that its largest magnitude lies in [128, 256), then split into two
+    // E4M3 terms q * f = t1 + t2 / 16 (t1 = nearest code, t2 = nearest code of 16 x the remainder): a
+    // bf16 has 8 significant bits, each term carries 4, so the split is exact for every element within
+    // 2^-13 of the head's largest and loses at most 2^-21 of that largest below.  qf[n][2 * kk + term]
+    // is the fragment of k step kk (32 dims); lane (r, c) holds head r, dims 32kk + 4c .. +3 and
+    // 32kk + 16 + 4c .. +3.  fh[n][e]: what turns the raw products of head 2c + e into log2-domain scores.
+    auto load_q8 = [&](uint32_t (&qf)[NT8][8][2], float (&fh)[NT8][2], int b, int g) {
+        const float ks = p.k_scale ? __ldg(p.k_scale + g) : 1.f;
+#pragma unroll
+        for (int n = 0; n < NT8; ++n) {
+            const int head = n * 8 + r;
+            const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
+                p.q + (int64_t)b * p.q_sb + (int64_t)(g * p.G + (head < p.G ? head : 0)) * p.q_sh);
+            float qv[4][2][4];
+            float amax = 0.f;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const uint32_t w0 = head < p.G ? __ldg(qrow + 16 * kk + 8 * hf + 2 * c) : 0u;
+                    const uint32_t w1 = head < p.G ? __ldg(qrow + 16 * kk + 8 * hf + 2 * c + 1) : 0u;
+                    qv[kk][hf][0] = bf16_lo_to_float(w0);
+                    qv[kk][hf][1] = bf16_hi_to_float(w0);
+                    qv[kk][hf][2] = bf16_lo_to_float(w1);
+                    qv[kk][hf][3] = bf16_hi_to_float(w1);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        amax = fmaxf(amax, fabsf(qv[kk][hf][e]));
+                }
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+            // f = 2^(7 - exponent of amax), kept inside the normal fp32 range
+            int fexp = 261 - (int)((__float_as_uint(amax) >> 23) & 0xffu);
+            fexp = min(max(fexp, 1), 254);
+            const float f = __uint_as_float((uint32_t)fexp << 23);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    float x[4], t[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        x[e] = qv[kk][hf][e] * f;
+                    const uint32_t t1 = pack_e4m3x4(x[0], x[1], x[2], x[3]);
+                    unpack_e4m3x4(t1, t);
+                    qf[n][2 * kk][hf] = t1;
+                    qf[n][2 * kk + 1][hf] = pack_e4m3x4((x[0] - t[0]) * 16.f, (x[1] - t[1]) * 16.f,
+                                                        (x[2] - t[2]) * 16.f, (x[3] - t[3]) * 16.f);
+                }
+            const float fin = (1.f / f) * ks * p.scale_log2;   // the same in all four lanes of head r
+            fh[n][0] = __shfl_sync(0xffffffffu, fin, 8 * c);
+            fh[n][1] = __shfl_sync(0xffffffffu, fin, 8 * c + 4);
+        }
+    };
+
     if (!mbar_wait_bounded(bar_full, 0u, abort_flag)) {
         give_up(-3);
         return;
@@ -589,7 +676,15 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     if (m0.w & TILE_STOP)
         return;
     uint32_t qf[NT8][8][2];
-    load_q(qf, m0.x, m0.y);
+    float fh[NT8][2];
+    if constexpr (KV8) {
+        load_q8(qf, fh, m0.x, m0.y);
+    } else {
+        load_q(qf, m0.x, m0.y);
+#pragma unroll
+        for (int n = 0; n < NT8; ++n)
+            fh[n][0] = fh[n][1] = 0.f;
+    }
 
     for (;;) {   // one (b, kv head) item per iteration
         const int b = m0.x, g = m0.y, lo = m1.x, L = m1.y, slot = m1.z;
@@ -606,9 +701,152 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
         for (;;) {   // the item's tiles; (m0, m1) describe the tile in stage it % NSTAGES, already full
             const int stage = it % NSTAGES;
-            const int a = m0.z + 16 * warp;   // first token of this warp's rows
-            const int v_lo = max(a, lo), v_hi = min(a + 16, L);
+            constexpr int WT = KV8 ? 32 : 16;   // tokens of a tile that one warp owns
+            const int a = m0.z + WT * warp;     // first token of this warp's rows
+            const int v_lo = max(a, lo), v_hi = min(a + WT, L);
             const bool item_end = (m0.w & TILE_ITEM_END) != 0;
+            if constexpr (KV8) {
+              if (v_lo < v_hi) {
+                const uint32_t k_base = smem_base + stage * STAGE_BYTES;
+                const uint32_t v_base = k_base + KV_BYTES;
+                const bool ragged = (v_lo > a) || (v_hi < a + 32);
+                if (ragged) {
+                    // rows outside the attended range may hold NaN codes: clear those V rows (8 chunks each)
+                    for (int e = lane; e < 256; e += 32) {
+                        const int rr = e >> 3, ch = e & 7;
+                        const int t = a + rr;
+                        if (t < v_lo || t >= v_hi) {
+                            const uint32_t addr = v_base + (uint32_t)(32 * warp + rr) * 128u + (ch << 4);
+                            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+                        }
+                    }
+                    __syncwarp();
+                }
+                // ---- S^T = K Q^T for the two 16-token tiles, Q's two terms in separate accumulators
+                float sa[NT8][4], sb[NT8][4];
+                {
+                    float ah[NT8][4], al[NT8][4], bh[NT8][4], bl[NT8][4];
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            ah[n][e] = al[n][e] = bh[n][e] = bl[n][e] = 0.f;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        uint32_t fa[4], fb[4];
+                        ldmatrix_x4(fa, k_base + ka8_off + ((((uint32_t)(2 * kk + k8_chunk)) ^ ka8_sw) << 4));
+                        ldmatrix_x4(fb, k_base + kb8_off + ((((uint32_t)(2 * kk + k8_chunk)) ^ kb8_sw) << 4));
+#pragma unroll
+                        for (int n = 0; n < NT8; ++n) {
+                            mma_e4m3_e4m3_16832(ah[n], fa, qf[n][2 * kk][0], qf[n][2 * kk][1]);
+                            mma_e4m3_e4m3_16832(bh[n], fb, qf[n][2 * kk][0], qf[n][2 * kk][1]);
+                            mma_e4m3_e4m3_16832(al[n], fa, qf[n][2 * kk + 1][0], qf[n][2 * kk + 1][1]);
+                            mma_e4m3_e4m3_16832(bl[n], fb, qf[n][2 * kk + 1][0], qf[n][2 * kk + 1][1]);
+                        }
+                    }
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            sa[n][e] = fmaf(al[n][e], 0.0625f, ah[n][e]) * fh[n][e & 1];
+                            sb[n][e] = fmaf(bl[n][e], 0.0625f, bh[n][e]) * fh[n][e & 1];
+                        }
+                }
+                // sa[n][0]: (token a + t_a0, head 2c) [1]: (t_a0, 2c+1) [2]: (t_a1, 2c) [3]: (t_a1, 2c+1); sb: t_b0, t_b1
+                if (ragged) {
+                    const bool oa0 = (a + t_a0 >= v_lo) && (a + t_a0 < v_hi), oa1 = (a + t_a1 >= v_lo) && (a + t_a1 < v_hi);
+                    const bool ob0 = (a + t_b0 >= v_lo) && (a + t_b0 < v_hi), ob1 = (a + t_b1 >= v_lo) && (a + t_b1 < v_hi);
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n) {
+                        if (!oa0) sa[n][0] = sa[n][1] = -INFINITY;
+                        if (!oa1) sa[n][2] = sa[n][3] = -INFINITY;
+                        if (!ob0) sb[n][0] = sb[n][1] = -INFINITY;
+                        if (!ob1) sb[n][2] = sb[n][3] = -INFINITY;
+                    }
+                }
+                // ---- online softmax in the log2 domain: column (head) maxima over the 32 tokens
+                float mx[NT8][2];
+                bool grew = false;
+#pragma unroll
+                for (int n = 0; n < NT8; ++n) {
+                    mx[n][0] = fmaxf(fmaxf(sa[n][0], sa[n][2]), fmaxf(sb[n][0], sb[n][2]));
+                    mx[n][1] = fmaxf(fmaxf(sa[n][1], sa[n][3]), fmaxf(sb[n][1], sb[n][3]));
+#pragma unroll
+                    for (int o_ = 4; o_ < 32; o_ <<= 1) {
+                        mx[n][0] = fmaxf(mx[n][0], __shfl_xor_sync(0xffffffffu, mx[n][0], o_));
+                        mx[n][1] = fmaxf(mx[n][1], __shfl_xor_sync(0xffffffffu, mx[n][1], o_));
+                    }
+                    grew |= (mx[n][0] > m_run[n][0]) | (mx[n][1] > m_run[n][1]);
+                }
+                if (__any_sync(0xffffffffu, grew)) {
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n) {
+                        float al[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float m_new = fmaxf(m_run[n][e], mx[n][e]);
+                            al[e] = (m_run[n][e] == -INFINITY) ? 0.f : fast_exp2(m_run[n][e] - m_new);
+                            m_run[n][e] = m_new;
+                            l_run[n][e] *= al[e];
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            o[n][j][0] *= al[0];
+                            o[n][j][1] *= al[1];
+                            o[n][j][2] *= al[0];
+                            o[n][j][3] *= al[1];
+                        }
+                    }
+                }
+                // ---- weights w = 2^15 * exp2(s - m), each split into four E5M2 terms (three significant
+                //      bits apiece: the first three by truncation, the last by rounding, so a weight is
+                //      carried to 2^-12 of itself down to 2^-31 of the largest), packed and transposed
+                //      into the B operand of O^T += V^T P^T (k = 32 tokens)
+                uint32_t pb[4][NT8][2];
+#pragma unroll
+                for (int n = 0; n < NT8; ++n) {
+                    float wa[4], wb[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        wa[e] = fast_exp2(sa[n][e] - m_run[n][e & 1] + P8_SHIFT);
+                        wb[e] = fast_exp2(sb[n][e] - m_run[n][e & 1] + P8_SHIFT);
+                    }
+                    l_run[n][0] += (wa[0] + wa[2]) + (wb[0] + wb[2]);
+                    l_run[n][1] += (wa[1] + wa[3]) + (wb[1] + wb[3]);
+#pragma unroll
+                    for (int term = 0; term < 4; ++term) {
+                        float ta[4], tb[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if (term < 3) {
+                                ta[e] = __uint_as_float(__float_as_uint(wa[e]) & 0xFFE00000u);
+                                tb[e] = __uint_as_float(__float_as_uint(wb[e]) & 0xFFE00000u);
+                                wa[e] -= ta[e];
+                                wb[e] -= tb[e];
+                            } else {
+                                ta[e] = wa[e];
+                                tb[e] = wb[e];
+                            }
+                        }
+                        // 16-bit element (row, head) = {code of tile A, code of tile B}
+                        pb[term][n][0] = movmatrix_trans(pack_e5m2x4(ta[0], tb[0], ta[1], tb[1]));   // rows r
+                        pb[term][n][1] = movmatrix_trans(pack_e5m2x4(ta[2], tb[2], ta[3], tb[3]));   // rows r + 8
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t vf[4];
+                    ldmatrix_b8_x2_trans(vf, v_base + v8_off + ((((uint32_t)j) ^ v8_sw) << 4));
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n)
+#pragma unroll
+                        for (int term = 0; term < 4; ++term)
+                            mma_e4m3_e5m2_16832(o[n][j], vf, pb[term][n][0], pb[term][n][1]);
+                }
+                if (ragged)
+                    fence_proxy_async_smem();   // the zeroed rows will be overwritten by a later TMA load
+              }
+            } else
             if (v_lo < v_hi) {
                 const uint32_t k_base = smem_base + stage * STAGE_BYTES;
                 const uint32_t v_base = k_base + KV_BYTES;
@@ -751,8 +989,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         //      (m, l, O) and write the pair's result or partial.
         const bool stop = (m0.w & TILE_STOP) != 0;
         uint32_t qn[NT8][8][2];
-        if (!stop)
-            load_q(qn, m0.x, m0.y);
+        float fn[NT8][2];
+        if (!stop) {
+            if constexpr (KV8)
+                load_q8(qn, fn, m0.x, m0.y);
+            else
+                load_q(qn, m0.x, m0.y);
+        }
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
 #pragma unroll
@@ -762,7 +1005,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 l += __shfl_xor_sync(0xffffffffu, l, 8);
                 l += __shfl_xor_sync(0xffffffffu, l, 16);
                 if (r == 0) {
-                    st_m[warp * HEADS + n * 8 + 2 * c + e] = m_run[n][e];
+                    // (8-bit cache: the weights were carried times 2^15, i.e. relative to m - 15)
+                    st_m[warp * HEADS + n * 8 + 2 * c + e] = KV8 ? m_run[n][e] - P8_SHIFT : m_run[n][e];
                     st_l[warp * HEADS + n * 8 + 2 * c + e] = l;
                 }
             }
@@ -786,6 +1030,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
         {
             const int d = tid;   // 0..127
+            const float vmul = (KV8 && p.v_scale) ? __ldg(p.v_scale + g) : 1.f;
             for (int head = 0; head < p.G; ++head) {
                 float M = st_m[head];
 #pragma unroll
@@ -799,7 +1044,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     den += st_l[w * HEADS + head] * f;
                     num += xbuf[(w * HEADS + head) * HEAD_DIM + dx] * f;
                 }
-                const float val = num / den;
+                const float val = KV8 ? (num / den) * vmul : num / den;
                 const float lse_nat = (M + fast_log2(den)) * LN2;
                 if (whole) {
                     const int h = g * p.G + head;
@@ -834,6 +1079,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 qf[n][kk][0] = qn[n][kk][0];
                 qf[n][kk][1] = qn[n][kk][1];
             }
+        if constexpr (KV8) {
+#pragma unroll
+            for (int n = 0; n < NT8; ++n) {
+                fh[n][0] = fn[n][0];
+                fh[n][1] = fn[n][1];
+            }
+        }
     }
 }
 

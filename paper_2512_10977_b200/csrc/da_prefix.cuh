@@ -168,14 +168,7 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
 // The K/V pools are read here through a 4-D tiled map {d, token, head, page} with box {64, box_rows, 1, 1}:
 // one box is one 64-column plane of box_rows token rows, so a plane of a tile is contiguous and
 // its 8-row groups are 1024 bytes apart, which is what the matrix descriptors above assume.
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, int c2, int c3, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
-        "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
-        : "memory");
-}
+// (tma_load_4d itself is in da_ptx.cuh.)
 
 __global__ void __launch_bounds__(PF_THREADS, 1)
 prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const PrefixParams p)

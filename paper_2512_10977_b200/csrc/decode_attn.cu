@@ -16,7 +16,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 102;
+constexpr int kVersion = 103;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -44,7 +44,8 @@ struct TmapKey {
     int64_t shape[4];
     int64_t stride[4];
     int box_rows;
-    int planes;   // 2: 5-D view, one box = both 64-column halves; 1: 4-D view, one box = one half
+    int planes;   // 2: 5-D view, one box = both 64-column halves; 1: 4-D view, one box = one half;
+                  // 0: 8-bit pool, 4-D view, one box = whole 128-byte rows
 };
 struct TmapEntry {
     TmapKey key;
@@ -195,7 +196,16 @@ int get_tmap(const da_tensor *t, int box_rows, int planes, CUtensorMap *out)
         return rc;
     CUtensorMap m;
     CUresult r;
-    if (planes == 2) {
+    if (planes == 0) {
+        // 8-bit codes: {d, token, kv head, page}, strides in bytes, box {128, box_rows, 1, 1}: a row is
+        // exactly the 128-byte swizzle span
+        cuuint64_t gdim[4] = {(cuuint64_t)t->shape[3], (cuuint64_t)t->shape[2], (cuuint64_t)t->shape[1], (cuuint64_t)t->shape[0]};
+        cuuint64_t gstr[3] = {(cuuint64_t)t->stride[2], (cuuint64_t)t->stride[1], (cuuint64_t)t->stride[0]};
+        cuuint32_t box[4] = {128, (cuuint32_t)box_rows, 1, 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, t->data, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else if (planes == 2) {
         cuuint64_t gdim[5] = {64, (cuuint64_t)t->shape[2], 2, (cuuint64_t)t->shape[1], (cuuint64_t)t->shape[0]};
         cuuint64_t gstr[4] = {(cuuint64_t)t->stride[2] * 2, 128, (cuuint64_t)t->stride[1] * 2, (cuuint64_t)t->stride[0] * 2};
         cuuint32_t box[5] = {64, (cuuint32_t)box_rows, 2, 1, 1};
@@ -229,21 +239,22 @@ struct Dims {
     int64_t B, Hq, Hkv, G, P, num_pages, max_pages;
 };
 
-int check_pool(const da_tensor *t)
+int check_pool(const da_tensor *t, int32_t dtype = DA_BF16)
 {
     if (!t->data) return DA_ERR_NULL;
-    if (t->dtype != DA_BF16) return DA_ERR_DTYPE;
+    if (t->dtype != dtype) return DA_ERR_DTYPE;
     if (t->ndim != 4) return DA_ERR_SHAPE;
     if (t->shape[3] != HEAD_DIM) return DA_ERR_UNSUPPORTED;
     if (t->stride[3] != 1 || !aligned16(t->data)) return DA_ERR_STRIDE_ALIGN;
+    const int64_t item = dtype == DA_FP8_E4M3 ? 1 : 2;
     for (int i = 0; i < 3; ++i)
-        if (t->stride[i] <= 0 || (t->stride[i] * 2) % 16 != 0 || t->stride[i] * 2 >= (1ll << 40))
+        if (t->stride[i] <= 0 || (t->stride[i] * item) % 16 != 0 || t->stride[i] * item >= (1ll << 40))
             return DA_ERR_STRIDE_ALIGN;
     return DA_OK;
 }
 
 int validate(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl,
-             const da_tensor *out, const da_tensor *lse, Dims *d)
+             const da_tensor *out, const da_tensor *lse, Dims *d, int32_t pool_dtype = DA_BF16)
 {
     if (!q || !k || !v || !bt || !sl || !out) return DA_ERR_NULL;
     if (!q->data || !bt->data || !sl->data || !out->data) return DA_ERR_NULL;
@@ -253,9 +264,9 @@ int validate(const da_tensor *q, const da_tensor *k, const da_tensor *v, const d
     if (lse && lse->dtype != DA_F32) return DA_ERR_DTYPE;
     if (q->ndim != 3 || bt->ndim != 2 || sl->ndim != 1 || out->ndim != 3) return DA_ERR_SHAPE;
     if (lse && lse->ndim != 2) return DA_ERR_SHAPE;
-    int rc = check_pool(k);
+    int rc = check_pool(k, pool_dtype);
     if (rc != DA_OK) return rc;
-    rc = check_pool(v);
+    rc = check_pool(v, pool_dtype);
     if (rc != DA_OK) return rc;
     for (int i = 0; i < 4; ++i)
         if (k->shape[i] != v->shape[i]) return DA_ERR_SHAPE;
@@ -284,13 +295,15 @@ int validate(const da_tensor *q, const da_tensor *k, const da_tensor *v, const d
 template <int NT8>
 int set_kernel_attrs()
 {
-    DA_CUDA(cudaFuncSetAttribute(partition_kernel<NT8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    DA_CUDA(cudaFuncSetAttribute(partition_kernel<NT8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PartCfg<NT8>::SMEM_BYTES));
+    DA_CUDA(cudaFuncSetAttribute(partition_kernel<NT8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  PartCfg<NT8>::SMEM_BYTES));
     return DA_OK;
 }
 
 int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const Dims &d, uint8_t *ws,
-                const WsLayout &lay, int nblocks, int n_tail, cudaStream_t stream)
+                const WsLayout &lay, int nblocks, int n_tail, cudaStream_t stream, int tile_t = TILE_T)
 {
     PlanParams pp;
     pp.seq_lens = static_cast<const int32_t *>(sl->data);
@@ -308,6 +321,7 @@ int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const 
     pp.Hkv = (int32_t)d.Hkv;
     pp.P = (int32_t)d.P;
     pp.window = window;
+    pp.tile_t = tile_t;
     pp.first_token = first_token;
     pp.n_static = nblocks;
     pp.n_tail_max = n_tail;
@@ -324,7 +338,8 @@ int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const 
 int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay, int nblocks, int n_tail,
                 const da_tensor *q,
                 const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl, int32_t window,
-                float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, int32_t first_token = 0)
+                float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, int32_t first_token = 0,
+                bool kv8 = false, const float *k_scale = nullptr, const float *v_scale = nullptr)
 {
     int rc;
     if (!st->attrs_set) {
@@ -335,14 +350,15 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
         DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
         st->attrs_set = true;
     }
-    const int box_rows = d.P < TILE_T ? (int)d.P : TILE_T;
+    const int tile_t = kv8 ? TILE_T8 : TILE_T;
+    const int box_rows = d.P < tile_t ? (int)d.P : tile_t;
     CUtensorMap tm_k, tm_v;
-    rc = get_tmap(k, box_rows, 2, &tm_k);
+    rc = get_tmap(k, box_rows, kv8 ? 0 : 2, &tm_k);
     if (rc != DA_OK) return rc;
-    rc = get_tmap(v, box_rows, 2, &tm_v);
+    rc = get_tmap(v, box_rows, kv8 ? 0 : 2, &tm_v);
     if (rc != DA_OK) return rc;
 
-    rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream);
+    rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream, tile_t);
     if (rc != DA_OK) return rc;
 
     PartParams pa;
@@ -371,6 +387,8 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pa.num_pages = (int32_t)d.num_pages;
     pa.out_bf16 = out->dtype == DA_BF16;
     pa.scale_log2 = scale * LOG2E;
+    pa.k_scale = k_scale;
+    pa.v_scale = v_scale;
     const int nt8 = d.G <= 8 ? 1 : 2;
     const bool timed = g_ev_before && g_ev_after;
     if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
@@ -387,13 +405,15 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     cfg.stream = stream;
     cfg.attrs = &pdl;
     cfg.numAttrs = 1;
-    if (nt8 == 1) {
-        cfg.dynamicSmemBytes = PartCfg<1>::SMEM_BYTES;
-        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<1>, tm_k, tm_v, pa));
-    } else {
-        cfg.dynamicSmemBytes = PartCfg<2>::SMEM_BYTES;
-        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<2>, tm_k, tm_v, pa));
-    }
+    cfg.dynamicSmemBytes = nt8 == 1 ? PartCfg<1>::SMEM_BYTES : PartCfg<2>::SMEM_BYTES;
+    if (nt8 == 1 && !kv8)
+        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<1, false>, tm_k, tm_v, pa));
+    else if (nt8 == 1)
+        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<1, true>, tm_k, tm_v, pa));
+    else if (!kv8)
+        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<2, false>, tm_k, tm_v, pa));
+    else
+        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<2, true>, tm_k, tm_v, pa));
     g_launches.fetch_add(1);
     if (timed) DA_CUDA(cudaEventRecord(g_ev_after, stream));
 
@@ -427,10 +447,11 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
 }
 
 int run(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl,
-        int32_t window, float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream)
+        int32_t window, float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, bool kv8 = false,
+        const float *k_scale = nullptr, const float *v_scale = nullptr)
 {
     Dims d;
-    int rc = validate(q, k, v, bt, sl, out, lse, &d);
+    int rc = validate(q, k, v, bt, sl, out, lse, &d, kv8 ? DA_FP8_E4M3 : DA_BF16);
     if (rc != DA_OK) return rc;
 
     std::lock_guard<std::mutex> lock(g_mu);
@@ -444,7 +465,7 @@ int run(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_ten
     if (!st->ws || st->ws_bytes < lay.stg_q) return DA_ERR_WORKSPACE;   // staging is only for host_io
     if (d.B == 0) return DA_OK;
     return launch_path(st, d, static_cast<uint8_t *>(st->ws), lay, nblocks, n_tail, q, k, v, bt, sl, window, scale,
-                       out, lse, stream);
+                       out, lse, stream, 0, kv8, k_scale, v_scale);
 }
 
 bool contiguous(const da_tensor *t)
@@ -465,6 +486,14 @@ int decode_attn(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
                 const da_tensor *seq_lens, int32_t window, float scale, da_tensor *out, da_tensor *lse, void *stream)
 {
     return run(q, k_pages, v_pages, block_table, seq_lens, window, scale, out, lse, static_cast<cudaStream_t>(stream));
+}
+
+int decode_attn_fp8kv(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const float *k_scale,
+                      const float *v_scale, const da_tensor *block_table, const da_tensor *seq_lens, int32_t window,
+                      float scale, da_tensor *out, da_tensor *lse, void *stream)
+{
+    return run(q, k_pages, v_pages, block_table, seq_lens, window, scale, out, lse, static_cast<cudaStream_t>(stream),
+               true, k_scale, v_scale);
 }
 
 int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,

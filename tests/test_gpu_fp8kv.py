@@ -1,0 +1,319 @@
+"""GPU parity of decode_attn_fp8kv (8-bit E4M3 cache with per-KV-head factors), through the C ABI,
+against the fp64 oracle of the same operation on the same seeded codes.  Tolerance as for the bf16
+cache: fp32 out and lse |d| <= 1e-3 + 1e-3*|ref|; bf16 out |d| <= 8e-3; indexing checks bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+
+pytestmark = pytest.mark.gpu
+
+ATOL, RTOL = 1e-3, 1e-3
+
+
+@pytest.fixture(scope="module")
+def da():
+    import paper_2512_10977_b200 as pkg
+    pkg.lib()
+    yield pkg
+    pkg.set_option("grid_blocks", 0)
+    pkg.set_option("tail_units", 4)
+    pkg.set_option("static_frac", 224)
+
+
+def oracle_of(case):
+    return oracle.decode_attn_fp8kv_oracle(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
+                                           case.block_table, case.seq_lens, case.window, case.scale)
+
+
+def gpu_of(da, case, out_dtype=torch.float32):
+    dev = workloads.to_device(case, "cuda")
+    out, lse = da.decode_attn_fp8kv(dev.q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, dev.block_table,
+                                    dev.seq_lens, dev.window, dev.scale, out_dtype=out_dtype)
+    st = da.read_device_status()
+    assert st == (0, 0, 0, 0), f"device status {st}"
+    return out.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+
+
+def assert_close(got, ref, what, atol=ATOL, rtol=RTOL):
+    got, ref = np.asarray(got), np.asarray(ref)
+    both_ninf = np.isneginf(got) & np.isneginf(ref)
+    with np.errstate(invalid="ignore"):
+        err = np.where(both_ninf, 0.0, np.abs(got - ref))
+    lim = atol + rtol * np.abs(np.where(both_ninf, 0.0, ref))
+    bad = ~(err <= lim)
+    if bad.any():
+        i = np.unravel_index(np.argmax(np.where(bad, err, -1)), err.shape)
+        raise AssertionError(f"{what}: {bad.sum()} of {bad.size} outside tolerance; worst at {i}: "
+                             f"got {got[i]!r} want {ref[i]!r}")
+
+
+def check(da, case, what, grid=0, out_dtype=torch.float32):
+    da.set_option("grid_blocks", grid)
+    ref, ref_lse = oracle_of(case)
+    got, got_lse = gpu_of(da, case, out_dtype)
+    if out_dtype == torch.float32:
+        assert_close(got, ref, what + " out")
+    else:
+        assert (np.abs(got - ref) <= 8e-3).all(), what + " out(bf16)"
+    assert_close(got_lse, ref_lse, what + " lse")
+    return got, got_lse, ref, ref_lse
+
+
+def fp8_case(name, lens, P, seed, **kw):
+    return workloads.build_case(name, lens, P, seed, "cpu", kv_dtype="fp8", **kw)
+
+
+LENS = [1, 2, 15, 16, 17, 31, 33, 63, 64, 65, 127, 128, 129, 255, 257, 1000]
+
+
+@pytest.mark.parametrize("P", [16, 32, 64, 128])
+def test_lengths_around_tile_and_page_edges(da, P):
+    case = fp8_case("edges8", LENS, P, 200 + P, pad_table_to=40)
+    for grid in (0, 1, 5):
+        got, _, ref, _ = check(da, case, f"P={P} grid={grid}", grid)
+    # how close the path really is on N(0,1)-like data (the bar above is much wider)
+    assert np.abs(got - ref).max() < 2e-4
+
+
+@pytest.mark.parametrize("window", [1, 5, 16, 17, 63, 64, 65, 127, 128, 129, 200, 257, 100000])
+def test_sliding_window(da, window):
+    lens = [1, 17, 64, 65, 200, 257, 258, 700]
+    case = fp8_case("win8", lens, 16, 7, window=window)
+    check(da, case, f"W={window}")
+    check(da, case, f"W={window} one block", 1)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(8, 8), (32, 8), (48, 8), (64, 8), (24, 2), (16, 1), (40, 4)])
+def test_group_sizes(da, Hq, Hkv):
+    case = fp8_case("gqa8", [300, 77, 1, 129], 16, Hq, Hq=Hq, Hkv=Hkv)
+    check(da, case, f"Hq={Hq} Hkv={Hkv}")
+    check(da, case, f"Hq={Hq} Hkv={Hkv} grid 3", 3)
+
+
+@pytest.mark.parametrize("grid", [1, 2, 3, 7, 64, 148, 296, 1000, 4096])
+def test_any_split_schedule_gives_the_same_answer(da, grid):
+    case = fp8_case("splits8", [2500, 3, 900, 64, 4097, 130], 16, 11)
+    check(da, case, f"grid={grid}", grid)
+
+
+@pytest.mark.parametrize("tail,frac", [(0, 192), (1, 128), (6, 0), (6, 256), (64, 200)])
+def test_any_mix_of_static_and_ticketed_units_gives_the_same_answer(da, tail, frac):
+    case = fp8_case("units8", [2500, 3, 900, 0, 64, 4097, 130, 9000], 16, 13)
+    try:
+        da.set_option("tail_units", tail)
+        da.set_option("static_frac", frac)
+        for grid in (0, 5, 64):
+            check(da, case, f"tail={tail} frac={frac} grid={grid}", grid)
+        case.window = 700
+        check(da, case, f"tail={tail} frac={frac} window", 0)
+    finally:
+        da.set_option("tail_units", 4)
+        da.set_option("static_frac", 224)
+
+
+def test_empty_sequences(da):
+    case = fp8_case("empty8", [0, 130, 0, 0, 5, 2049, 0], 16, 3)
+    got, got_lse, _, _ = check(da, case, "empties")
+    for b in (0, 2, 3, 6):
+        assert (got[b] == 0).all() and np.isneginf(got_lse[b]).all()
+    case = fp8_case("allempty8", [0, 0], 16, 5)
+    got, got_lse, _, _ = check(da, case, "all empty")
+    assert (got == 0).all() and np.isneginf(got_lse).all()
+
+
+def test_token_major_layout(da):
+    case = fp8_case("tm8", [513, 40, 1300], 16, 21, layout="token_major")
+    assert case.k_pages.stride(1) < case.k_pages.stride(2)
+    check(da, case, "token-major")
+
+
+def test_bf16_output_and_unit_factors(da):
+    case = fp8_case("bf16o8", [700, 33, 2100, 1], 16, 23)
+    check(da, case, "bf16 out", 0, torch.bfloat16)
+    case.k_scale = None
+    case.scale = 0.002          # raw K codes reach ~200: keep the scores O(1)
+    check(da, case, "no K factors")
+
+
+def test_float8_dtype_pools_are_accepted(da):
+    case = fp8_case("f8dtype", [300, 64], 16, 25)
+    ref, ref_lse = oracle_of(case)
+    dev = workloads.to_device(case, "cuda")
+    out, lse = da.decode_attn_fp8kv(dev.q, dev.k_pages.view(torch.float8_e4m3fn), dev.v_pages.view(torch.float8_e4m3fn),
+                                    dev.k_scale, dev.v_scale, dev.block_table, dev.seq_lens, 0, dev.scale)
+    assert_close(out.cpu().numpy(), ref, "float8 view")
+
+
+def test_wide_range_of_query_magnitudes(da):
+    """Heads whose queries are tiny, huge or span many binades: the power-of-two rescaling and the
+    two-term split of q must not lose them."""
+    case = fp8_case("qrange8", [600, 90], 16, 27)
+    q = case.q.float()
+    q[:, 0] *= 2.0 ** -20
+    q[:, 1] *= 2.0 ** 12
+    q[:, 2, ::2] *= 2.0 ** -9          # elements far below the head's largest
+    q[:, 3] = 0
+    case.q = q.to(torch.bfloat16)
+    case.scale = 1.0 / 64
+    check(da, case, "q magnitudes")
+
+
+def test_sharp_and_flat_softmax(da):
+    """One dominant key (weights collapse) and scale 0 (all weights equal)."""
+    case = fp8_case("sharp8", [900, 130], 16, 29)
+    check(da, case, "flat", 0)
+    case.scale = 0.0
+    got, got_lse, ref, _ = check(da, case, "scale 0")
+    case.scale = 4.0
+    check(da, case, "sharp")
+
+
+# ------------------------------------------------------------------ indexing, bit-exact
+
+def _probe_case(P, lens, window, seed):
+    """K codes 0 everywhere; V rows carry (token, physical page, kv head) as small integers (exact in
+    E4M3 up to 16); factors 1."""
+    case = fp8_case("probe8", lens, P, seed, window=window, poison=True)
+    case.k_scale = case.v_scale = None
+    nan = workloads.E4M3_NAN
+    case.k_pages[case.k_pages != nan] = 0
+    bt = case.block_table.numpy()
+    for b, L in enumerate(lens):
+        for t in range(L):
+            pg = int(bt[b, t // P])
+            for g in range(case.k_pages.shape[1]):
+                v = torch.zeros(128)
+                v[0], v[1], v[2], v[3] = t % 16, (t // 16) % 16, t // 256, pg % 16
+                v[4], v[5], v[6] = (pg // 16) % 16, g, b
+                case.v_pages[pg, g, t % P] = v.to(torch.float8_e4m3fn).view(torch.uint8)
+    return case
+
+
+@pytest.mark.parametrize("P", [16, 64])
+def test_probe_token_is_returned_bit_for_bit(da, P):
+    lens, W = [300, 77, 1025], 100
+    base = _probe_case(P, lens, W, 41)
+    dev = workloads.to_device(base, "cuda")
+    bt = base.block_table.numpy()
+    # queries: +-2 patterns (exact in two E4M3 terms); the probe key is 4 * q, others 0: gap = 16 * 128 * scale
+    sign = torch.where(torch.rand((len(lens), 8, 128), generator=torch.Generator().manual_seed(3)) < 0.5, -1.0, 1.0)
+    q = (2 * sign).repeat_interleave(6, dim=1).to(torch.bfloat16).cuda()
+    for grid in (0, 1):
+        da.set_option("grid_blocks", grid)
+        for b, L in enumerate(lens):
+            lo = max(L - W, 0)
+            cand = [lo, lo + 1, L - 1, (lo // P + 1) * P - 1, (lo // P + 1) * P,
+                    (lo // 128 + 1) * 128 - 1, (lo // 128 + 1) * 128, (L - 1) // 128 * 128 - 1, (L - 1) // 128 * 128,
+                    (lo // 32 + 1) * 32 - 1, (lo // 32 + 1) * 32]
+            for t_star in sorted({t for t in cand if lo <= t < L}):
+                pg = int(bt[b, t_star // P])
+                saved = dev.k_pages[pg, :, t_star % P].clone()
+                kstar = (4 * sign[b]).to(torch.float8_e4m3fn).view(torch.uint8).cuda()      # [8, 128]
+                dev.k_pages[pg, :, t_star % P] = kstar
+                out, _ = da.decode_attn_fp8kv(q, dev.k_pages, dev.v_pages, None, None, dev.block_table, dev.seq_lens, W, 1.0)
+                want = dev.v_pages[pg, :, t_star % P].view(torch.float8_e4m3fn).float()     # [8, 128]
+                got = out[b].view(8, 6, 128)
+                assert torch.equal(got, want[:, None, :].expand(8, 6, 128)), (P, grid, b, t_star)
+                assert got[0, 0, 0].item() == t_star % 16 and got[0, 0, 2].item() == t_star // 256
+                assert got[3, 2, 5].item() == 3 and got[0, 0, 6].item() == b
+                dev.k_pages[pg, :, t_star % P] = saved
+    assert da.read_device_status() == (0, 0, 0, 0)
+
+
+def test_integer_mean_is_exact(da):
+    """K = 0 and V small integers over a power-of-two number of tokens: the mean is exact in fp32."""
+    lens = [256, 1024, 128]
+    case = fp8_case("int8", lens, 16, 47)
+    case.k_scale = case.v_scale = None
+    nan = workloads.E4M3_NAN
+    case.k_pages[case.k_pages != nan] = 0
+    vi = torch.randint(-8, 9, case.v_pages.shape, generator=torch.Generator().manual_seed(1)).float()
+    vi = vi.to(torch.float8_e4m3fn).view(torch.uint8)
+    case.v_pages = torch.where(case.v_pages != nan, vi, case.v_pages)
+    ref, ref_lse = oracle_of(case)
+    try:
+        da.set_option("grid_blocks", 1)
+        da.set_option("tail_units", 0)
+        got, got_lse = gpu_of(da, case)
+        assert np.array_equal(got, ref)
+        np.testing.assert_allclose(got_lse, ref_lse, atol=1e-6)
+    finally:
+        da.set_option("grid_blocks", 0)
+        da.set_option("tail_units", 4)
+
+
+def test_nan_canaries(da):
+    lens = [5, 17, 300, 1029, 64, 128]
+    dirty = fp8_case("dirty8", lens, 16, 53, poison=True, pool_pages=400, pad_table_to=90)
+    assert (dirty.k_pages == workloads.E4M3_NAN).sum() > 1000 and (dirty.block_table == -1).any()
+    for grid in (0, 1, 9):
+        got, got_lse, _, _ = check(da, dirty, f"canary grid={grid}", grid)
+        assert np.isfinite(got).all() and np.isfinite(got_lse).all()
+    check(da, fp8_case("dirtyw8", lens, 16, 53, poison=True, pool_pages=400, window=20), "canary window")
+
+
+def test_host_side_argument_errors(da):
+    case = workloads.to_device(fp8_case("err8", [100], 16, 59), "cuda")
+    bf = workloads.to_device(workloads.build_case("errbf", [100], 16, 59, "cpu"), "cuda")
+    with pytest.raises(da.DecodeAttnError) as e:      # a bf16 pool handed to the 8-bit entry point
+        da.decode_attn_fp8kv(case.q, bf.k_pages, bf.v_pages, None, None, case.block_table, case.seq_lens, 0, 1.0)
+    assert e.value.status == 3
+    with pytest.raises(da.DecodeAttnError) as e:      # and the reverse
+        da.decode_attn(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens, 0, 1.0)
+    assert e.value.status == 3
+    with pytest.raises(da.DecodeAttnError) as e:
+        da.decode_attn_fp8kv(case.q, case.k_pages[:, :, :8], case.v_pages[:, :, :8], None, None, case.block_table,
+                             case.seq_lens, 0, 1.0)
+    assert e.value.status == 5
+    with pytest.raises(ValueError):
+        da.decode_attn_fp8kv(case.q, case.k_pages, case.v_pages, case.k_scale[:4], None, case.block_table,
+                             case.seq_lens, 0, 1.0)
+    assert da.read_device_status() == (0, 0, 0, 0)
+
+
+def test_device_side_errors_set_the_status_word_without_faulting(da):
+    good = fp8_case("bad8", [100, 200, 40], 16, 61)
+    ref, _ = oracle_of(good)
+    dev = workloads.to_device(good, "cuda")
+    bt = good.block_table.clone()
+    bt[1, 3] = 10 ** 6
+    out, lse = da.decode_attn_fp8kv(dev.q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, bt.cuda(), dev.seq_lens,
+                                    0, dev.scale)
+    st = da.read_device_status()
+    assert st[0] == 1 and st[1] == 1 and st[3] == 10 ** 6
+    assert_close(out[0].cpu().numpy(), ref[0], "other sequences are unaffected")
+    check(da, good, "after errors")
+
+
+# ------------------------------------------------------------------ the workloads at full size
+
+def _sampled_full_size(da, case, ids, what):
+    out, lse = da.decode_attn_fp8kv(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table,
+                                    case.seq_lens, case.window, case.scale)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    assert torch.isfinite(out).all() and torch.isfinite(lse).all()
+    sub = workloads.host_subcase(case, ids)
+    ref, ref_lse = oracle_of(sub)
+    assert_close(out[ids].cpu().numpy(), ref, what + " out")
+    assert_close(lse[ids].cpu().numpy(), ref_lse, what + " lse")
+
+
+def test_c2_full_size_sampled(da):
+    da.set_option("grid_blocks", 0)
+    case = workloads.c2("cuda", kv_dtype="fp8")
+    ids = sorted({int(np.argmin(case.lens)), int(np.argmax(case.lens)), 0, 31, 63})
+    _sampled_full_size(da, case, ids, "c2 fp8")
+
+
+def test_c4_long_context_page64_sampled(da):
+    da.set_option("grid_blocks", 0)
+    _sampled_full_size(da, workloads.c4("cuda", kv_dtype="fp8"), [0, 7], "c4 fp8")
+
+
+def test_c5b_window_sampled(da):
+    da.set_option("grid_blocks", 0)
+    case = workloads.c5("cuda", 8192, kv_dtype="fp8")
+    _sampled_full_size(da, case, [0, int(np.argmax(case.lens))], "c5b fp8")
