@@ -22,7 +22,7 @@ constexpr int TILE_T = 16 * NCW;            // tokens per pipeline stage, bf16 c
 constexpr int TILE_T8 = 32 * NCW;           // tokens per pipeline stage, 8-bit cache (a warp owns 32)
 constexpr int KV_BYTES = TILE_T * 256;      // a K (or V) tile: TILE_T rows of 128 bf16, or TILE_T8 rows of 128 bytes
 static_assert(TILE_T8 * 128 == KV_BYTES, "both cache types fill a stage");
-constexpr float P8_SHIFT = 15.f;            // 8-bit cache: softmax weights are carried as 2^15 * p (E5M2 terms)
+constexpr float P8_SHIFT = 15.f;            // 8-bit cache: softmax weights are carried as 2^15 * p (f16 high + low)
 constexpr int STAGE_BYTES = 2 * KV_BYTES;   // K tile followed by V tile
 constexpr int NTHREADS = (NCW + 1) * 32;    // + one producer warp
 constexpr int PLAN_THREADS = 1024;
@@ -571,25 +571,28 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const uint32_t k_sw = (uint32_t)(k_row & 7), v_sw = (uint32_t)(v_row & 7);
 
     // ---- 8-bit cache: a warp owns 32 tokens of a 128-token tile (rows of 128 bytes, 16-byte chunk index
-    // XORed with the row's low three bits).  Its scores form two 16-row tiles A and B (mma m16n8k32,
-    // K rows as the A operand); row x of tile A is warp-local token tok_a(x), of tile B tok_b(x).  The
-    // maps are chosen so that (1) the eight rows of every ldmatrix phase differ in their low three bits
-    // (no bank conflicts) and (2) the PV product can take the weights of BOTH tiles as one k = 32
-    // operand: packing the codes of (A row x, B row x) into one 16-bit element and transposing with
-    // movmatrix puts, in k slot 4c+i of the B fragment, A row 2c (i=0), B row 2c (1), A row 2c+1 (2),
-    // B row 2c+1 (3), and rows +8 in slots 16..31; V's transposed ldmatrix takes one row address per k
-    // slot, so it is simply pointed at the token each slot holds.
-    auto tok_a = [](int x) { return x < 4 ? x : (x < 12 ? x + 8 : x + 16); };
-    auto tok_b = [](int x) { return x < 8 ? x + 4 : x + 12; };
+    // XORed with the row's low three bits).  The codes are widened to f16 in registers (exactly: every
+    // E4M3 value is an f16 value) and both products run as f16 mma with fp32 accumulation.  The warp's
+    // scores form two 16-row tiles A and B; row x of tile A is warp-local token tok8(x), of tile B
+    // 16 + tok8(x).  tok8 swaps rows 8-11 with 12-15 so that the eight rows of every ldmatrix phase,
+    // for K and for the transposed V reads below, differ in their low three bits (no bank conflicts).
+    //   K: one ldmatrix.x4 brings 16 rows x 32 dims as four registers of four codes (dims 4c..4c+3 of
+    //      rows r / r+8, first and second 16 dims).  The low halves widen to the (k = 2c, 2c+1)
+    //      fragment registers of one m16n8k16 step and the high halves to its (k = 2c+8, 2c+9)
+    //      registers; Q's fragments are loaded in the same dim order, so the order does not matter.
+    //   V: the transposed 8-bit ldmatrix takes one row address per k slot: lane j points slot j at the
+    //      token whose weight sits in that slot of P's fragment (slots 4c+e <- block row 2c+e of the
+    //      rows 0-7 block, 4c+2+e <- of the rows 8-15 block; tile A in slots 0-15, tile B in 16-31).
+    auto tok8 = [](int x) { return x < 8 ? x : 8 + ((x + 4) & 7); };
     const int x8 = (lane & 7) + ((lane >> 3) & 1) * 8;          // QK ldmatrix: row of the 16-row tile
-    const int k8_chunk = lane >> 4;                             //              16-byte half of the 32-byte k step
-    const int row_a8 = 32 * warp + tok_a(x8), row_b8 = 32 * warp + tok_b(x8);
+    const int k8_chunk = lane >> 4;                             //              16-byte half of the 32-dim step
+    const int row_a8 = 32 * warp + tok8(x8), row_b8 = row_a8 + 16;
     const uint32_t ka8_off = (uint32_t)row_a8 * 128u, kb8_off = (uint32_t)row_b8 * 128u;
     const uint32_t ka8_sw = (uint32_t)(row_a8 & 7), kb8_sw = (uint32_t)(row_b8 & 7);
-    const int slot_x = 2 * ((lane & 15) >> 2) + ((lane & 3) >> 1) + 8 * (lane >> 4);   // PV: k slot `lane`
-    const int row_v8 = 32 * warp + ((lane & 1) ? tok_b(slot_x) : tok_a(slot_x));
+    const int slot_row = 8 * ((lane >> 1) & 1) + 2 * ((lane & 15) >> 2) + (lane & 1);   // PV: tile row of k slot `lane`
+    const int row_v8 = 32 * warp + tok8(slot_row) + 16 * (lane >> 4);
     const uint32_t v8_off = (uint32_t)row_v8 * 128u, v8_sw = (uint32_t)(row_v8 & 7);
-    const int t_a0 = tok_a(r), t_a1 = tok_a(r + 8), t_b0 = tok_b(r), t_b1 = tok_b(r + 8);   // tokens of this lane's scores
+    const int t_a0 = tok8(r), t_a1 = tok8(r + 8);               // tokens of this lane's scores (tile B: + 16)
 
     auto give_up = [&](int where) {
         if (*abort_flag == 0) {
@@ -612,13 +615,12 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
     };
 
-    // 8-bit cache: Q^T as E4M3 B fragments of S^T = K Q^T (mma m16n8k32).  A head's query vector is
-    // scaled by a power of two so that its largest magnitude lies in [128, 256), then split into two
-    // E4M3 terms q * f = t1 + t2 / 16 (t1 = nearest code, t2 = nearest code of 16 x the remainder): a
-    // bf16 has 8 significant bits, each term carries 4, so the split is exact for every element within
-    // 2^-13 of the head's largest and loses at most 2^-21 of that largest below.  qf[n][2 * kk + term]
-    // is the fragment of k step kk (32 dims); lane (r, c) holds head r, dims 32kk + 4c .. +3 and
-    // 32kk + 16 + 4c .. +3.  fh[n][e]: what turns the raw products of head 2c + e into log2-domain scores.
+    // 8-bit cache: Q^T as f16 B fragments of S^T = K Q^T.  A head's query vector is scaled by a power
+    // of two so that its largest magnitude lies in [2^14, 2^15) and rounded to f16; a bf16 has 8
+    // significant bits and f16 carries 11 down to 2^-14, so the conversion is exact for every element
+    // within 2^-28 of the head's largest (smaller ones are off by at most 2^-25 of the scaled value).
+    // qf[n][i] is the fragment of k step i (16 dims): lane (r, c) holds head r, dims 16i + 4c .. + 3.
+    // fh[n][e]: what turns the raw products of head 2c + e into log2-domain scores.
     auto load_q8 = [&](uint32_t (&qf)[NT8][8][2], float (&fh)[NT8][2], int b, int g) {
         const float ks = p.k_scale ? __ldg(p.k_scale + g) : 1.f;
 #pragma unroll
@@ -626,42 +628,26 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             const int head = n * 8 + r;
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
                 p.q + (int64_t)b * p.q_sb + (int64_t)(g * p.G + (head < p.G ? head : 0)) * p.q_sh);
-            float qv[4][2][4];
+            uint32_t w[8][2];
             float amax = 0.f;
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
+            for (int i = 0; i < 8; ++i)
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
-                    const uint32_t w0 = head < p.G ? __ldg(qrow + 16 * kk + 8 * hf + 2 * c) : 0u;
-                    const uint32_t w1 = head < p.G ? __ldg(qrow + 16 * kk + 8 * hf + 2 * c + 1) : 0u;
-                    qv[kk][hf][0] = bf16_lo_to_float(w0);
-                    qv[kk][hf][1] = bf16_hi_to_float(w0);
-                    qv[kk][hf][2] = bf16_lo_to_float(w1);
-                    qv[kk][hf][3] = bf16_hi_to_float(w1);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        amax = fmaxf(amax, fabsf(qv[kk][hf][e]));
+                    w[i][hf] = head < p.G ? __ldg(qrow + 8 * i + 2 * c + hf) : 0u;
+                    amax = fmaxf(amax, fmaxf(fabsf(bf16_lo_to_float(w[i][hf])), fabsf(bf16_hi_to_float(w[i][hf]))));
                 }
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-            // f = 2^(7 - exponent of amax), kept inside the normal fp32 range
-            int fexp = 261 - (int)((__float_as_uint(amax) >> 23) & 0xffu);
+            // f = 2^(14 - exponent of amax), kept inside the normal fp32 range
+            int fexp = 268 - (int)((__float_as_uint(amax) >> 23) & 0xffu);
             fexp = min(max(fexp, 1), 254);
             const float f = __uint_as_float((uint32_t)fexp << 23);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
+            for (int i = 0; i < 8; ++i)
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    float x[4], t[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        x[e] = qv[kk][hf][e] * f;
-                    const uint32_t t1 = pack_e4m3x4(x[0], x[1], x[2], x[3]);
-                    unpack_e4m3x4(t1, t);
-                    qf[n][2 * kk][hf] = t1;
-                    qf[n][2 * kk + 1][hf] = pack_e4m3x4((x[0] - t[0]) * 16.f, (x[1] - t[1]) * 16.f,
-                                                        (x[2] - t[2]) * 16.f, (x[3] - t[3]) * 16.f);
-                }
+                for (int hf = 0; hf < 2; ++hf)
+                    qf[n][i][hf] = pack_f16(bf16_lo_to_float(w[i][hf]) * f, bf16_hi_to_float(w[i][hf]) * f);
             const float fin = (1.f / f) * ks * p.scale_log2;   // the same in all four lanes of head r
             fh[n][0] = __shfl_sync(0xffffffffu, fin, 8 * c);
             fh[n][1] = __shfl_sync(0xffffffffu, fin, 8 * c + 4);
@@ -722,40 +708,51 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     }
                     __syncwarp();
                 }
-                // ---- S^T = K Q^T for the two 16-token tiles, Q's two terms in separate accumulators
+                // ---- S^T = K Q^T for the two 16-token tiles; two accumulators each to shorten the chains
                 float sa[NT8][4], sb[NT8][4];
                 {
-                    float ah[NT8][4], al[NT8][4], bh[NT8][4], bl[NT8][4];
+                    float aa[NT8][2][4], ab[NT8][2][4];
 #pragma unroll
                     for (int n = 0; n < NT8; ++n)
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
-                            ah[n][e] = al[n][e] = bh[n][e] = bl[n][e] = 0.f;
+                            aa[n][0][e] = aa[n][1][e] = ab[n][0][e] = ab[n][1][e] = 0.f;
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        uint32_t fa[4], fb[4];
-                        ldmatrix_x4(fa, k_base + ka8_off + ((((uint32_t)(2 * kk + k8_chunk)) ^ ka8_sw) << 4));
-                        ldmatrix_x4(fb, k_base + kb8_off + ((((uint32_t)(2 * kk + k8_chunk)) ^ kb8_sw) << 4));
+                        uint32_t ca[4], cb[4];
+                        ldmatrix_x4(ca, k_base + ka8_off + ((((uint32_t)(2 * kk + k8_chunk)) ^ ka8_sw) << 4));
+                        ldmatrix_x4(cb, k_base + kb8_off + ((((uint32_t)(2 * kk + k8_chunk)) ^ kb8_sw) << 4));
 #pragma unroll
-                        for (int n = 0; n < NT8; ++n) {
-                            mma_e4m3_e4m3_16832(ah[n], fa, qf[n][2 * kk][0], qf[n][2 * kk][1]);
-                            mma_e4m3_e4m3_16832(bh[n], fb, qf[n][2 * kk][0], qf[n][2 * kk][1]);
-                            mma_e4m3_e4m3_16832(al[n], fa, qf[n][2 * kk + 1][0], qf[n][2 * kk + 1][1]);
-                            mma_e4m3_e4m3_16832(bl[n], fb, qf[n][2 * kk + 1][0], qf[n][2 * kk + 1][1]);
+                        for (int hf = 0; hf < 2; ++hf) {   // the two 16-dim steps of this 32-dim load
+                            uint32_t fa[4], fb[4];
+                            fa[0] = e4m3x2_lo_to_f16x2(ca[2 * hf]);
+                            fa[1] = e4m3x2_lo_to_f16x2(ca[2 * hf + 1]);
+                            fa[2] = e4m3x2_hi_to_f16x2(ca[2 * hf]);
+                            fa[3] = e4m3x2_hi_to_f16x2(ca[2 * hf + 1]);
+                            fb[0] = e4m3x2_lo_to_f16x2(cb[2 * hf]);
+                            fb[1] = e4m3x2_lo_to_f16x2(cb[2 * hf + 1]);
+                            fb[2] = e4m3x2_hi_to_f16x2(cb[2 * hf]);
+                            fb[3] = e4m3x2_hi_to_f16x2(cb[2 * hf + 1]);
+#pragma unroll
+                            for (int n = 0; n < NT8; ++n) {
+                                mma_f16_16816(aa[n][hf], fa, qf[n][2 * kk + hf][0], qf[n][2 * kk + hf][1]);
+                                mma_f16_16816(ab[n][hf], fb, qf[n][2 * kk + hf][0], qf[n][2 * kk + hf][1]);
+                            }
                         }
                     }
 #pragma unroll
                     for (int n = 0; n < NT8; ++n)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            sa[n][e] = fmaf(al[n][e], 0.0625f, ah[n][e]) * fh[n][e & 1];
-                            sb[n][e] = fmaf(bl[n][e], 0.0625f, bh[n][e]) * fh[n][e & 1];
+                            sa[n][e] = (aa[n][0][e] + aa[n][1][e]) * fh[n][e & 1];
+                            sb[n][e] = (ab[n][0][e] + ab[n][1][e]) * fh[n][e & 1];
                         }
                 }
-                // sa[n][0]: (token a + t_a0, head 2c) [1]: (t_a0, 2c+1) [2]: (t_a1, 2c) [3]: (t_a1, 2c+1); sb: t_b0, t_b1
+                // sa[n][0]: (token a + t_a0, head 2c) [1]: (t_a0, 2c+1) [2]: (t_a1, 2c) [3]: (t_a1, 2c+1); sb: tokens + 16
                 if (ragged) {
                     const bool oa0 = (a + t_a0 >= v_lo) && (a + t_a0 < v_hi), oa1 = (a + t_a1 >= v_lo) && (a + t_a1 < v_hi);
-                    const bool ob0 = (a + t_b0 >= v_lo) && (a + t_b0 < v_hi), ob1 = (a + t_b1 >= v_lo) && (a + t_b1 < v_hi);
+                    const bool ob0 = (a + 16 + t_a0 >= v_lo) && (a + 16 + t_a0 < v_hi);
+                    const bool ob1 = (a + 16 + t_a1 >= v_lo) && (a + 16 + t_a1 < v_hi);
 #pragma unroll
                     for (int n = 0; n < NT8; ++n) {
                         if (!oa0) sa[n][0] = sa[n][1] = -INFINITY;
@@ -798,50 +795,47 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         }
                     }
                 }
-                // ---- weights w = 2^15 * exp2(s - m), each split into four E5M2 terms (three significant
-                //      bits apiece: the first three by truncation, the last by rounding, so a weight is
-                //      carried to 2^-12 of itself down to 2^-31 of the largest), packed and transposed
-                //      into the B operand of O^T += V^T P^T (k = 32 tokens)
-                uint32_t pb[4][NT8][2];
+                // ---- weights w = 2^15 * exp2(s - m) as f16 high and low parts (together ~22 bits of each
+                //      weight; the factor 2^15 keeps weights down to 2^-39 of the largest representable),
+                //      transposed into the B operand of O^T += V^T P^T.  ph[n][q]: block q = rows 0-7 / 8-15
+                //      of tile A, then of tile B.
+                uint32_t ph[NT8][4], pl[NT8][4];
 #pragma unroll
                 for (int n = 0; n < NT8; ++n) {
-                    float wa[4], wb[4];
+                    float w[8];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        wa[e] = fast_exp2(sa[n][e] - m_run[n][e & 1] + P8_SHIFT);
-                        wb[e] = fast_exp2(sb[n][e] - m_run[n][e & 1] + P8_SHIFT);
+                        w[e] = fast_exp2(sa[n][e] - m_run[n][e & 1] + P8_SHIFT);
+                        w[4 + e] = fast_exp2(sb[n][e] - m_run[n][e & 1] + P8_SHIFT);
                     }
-                    l_run[n][0] += (wa[0] + wa[2]) + (wb[0] + wb[2]);
-                    l_run[n][1] += (wa[1] + wa[3]) + (wb[1] + wb[3]);
+                    l_run[n][0] += (w[0] + w[2]) + (w[4] + w[6]);
+                    l_run[n][1] += (w[1] + w[3]) + (w[5] + w[7]);
 #pragma unroll
-                    for (int term = 0; term < 4; ++term) {
-                        float ta[4], tb[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            if (term < 3) {
-                                ta[e] = __uint_as_float(__float_as_uint(wa[e]) & 0xFFE00000u);
-                                tb[e] = __uint_as_float(__float_as_uint(wb[e]) & 0xFFE00000u);
-                                wa[e] -= ta[e];
-                                wb[e] -= tb[e];
-                            } else {
-                                ta[e] = wa[e];
-                                tb[e] = wb[e];
-                            }
-                        }
-                        // 16-bit element (row, head) = {code of tile A, code of tile B}
-                        pb[term][n][0] = movmatrix_trans(pack_e5m2x4(ta[0], tb[0], ta[1], tb[1]));   // rows r
-                        pb[term][n][1] = movmatrix_trans(pack_e5m2x4(ta[2], tb[2], ta[3], tb[3]));   // rows r + 8
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t hi = pack_f16(w[2 * q], w[2 * q + 1]);
+                        const float2 hv = unpack_f16(hi);
+                        const uint32_t lo = pack_f16(w[2 * q] - hv.x, w[2 * q + 1] - hv.y);
+                        ph[n][q] = movmatrix_trans(hi);
+                        pl[n][q] = movmatrix_trans(lo);
                     }
                 }
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    uint32_t vf[4];
-                    ldmatrix_b8_x2_trans(vf, v_base + v8_off + ((((uint32_t)j) ^ v8_sw) << 4));
+                    uint32_t cv[4];
+                    ldmatrix_b8_x2_trans(cv, v_base + v8_off + ((((uint32_t)j) ^ v8_sw) << 4));
 #pragma unroll
-                    for (int n = 0; n < NT8; ++n)
+                    for (int hf = 0; hf < 2; ++hf) {   // tile A's 16 tokens, then tile B's
+                        uint32_t vf[4];
+                        vf[0] = e4m3x2_lo_to_f16x2(cv[2 * hf]);
+                        vf[1] = e4m3x2_lo_to_f16x2(cv[2 * hf + 1]);
+                        vf[2] = e4m3x2_hi_to_f16x2(cv[2 * hf]);
+                        vf[3] = e4m3x2_hi_to_f16x2(cv[2 * hf + 1]);
 #pragma unroll
-                        for (int term = 0; term < 4; ++term)
-                            mma_e4m3_e5m2_16832(o[n][j], vf, pb[term][n][0], pb[term][n][1]);
+                        for (int n = 0; n < NT8; ++n) {
+                            mma_f16_16816(o[n][j], vf, ph[n][2 * hf], ph[n][2 * hf + 1]);
+                            mma_f16_16816(o[n][j], vf, pl[n][2 * hf], pl[n][2 * hf + 1]);
+                        }
+                    }
                 }
                 if (ragged)
                     fence_proxy_async_smem();   // the zeroed rows will be overwritten by a later TMA load

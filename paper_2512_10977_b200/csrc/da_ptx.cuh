@@ -158,12 +158,11 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// ---------------------------------------------------------------- 8-bit (E4M3 / E5M2) fragments
+// ---------------------------------------------------------------- 8-bit (E4M3) cache fragments
 // Two 16x16 matrices of bytes, each read TRANSPOSED: lane i < 16 gives the address of the 16-byte
 // shared-memory row that becomes COLUMN i of matrix 0, lane i >= 16 that of column i - 16 of matrix 1.
 // Lane (r = lane / 4, c = lane % 4) receives, for matrix 0, r[0] = bytes r of rows 4c .. 4c+3 and
-// r[1] = bytes r + 8 of the same rows; r[2], r[3] likewise from matrix 1 -- which is the A fragment
-// (16 x 32 bytes) of mma m16n8k32 when the shared-memory rows are the k index.
+// r[1] = bytes r + 8 of the same rows; r[2], r[3] likewise from matrix 1.
 __device__ __forceinline__ void ldmatrix_b8_x2_trans(uint32_t (&r)[4], uint32_t addr)
 {
     asm volatile("ldmatrix.sync.aligned.m16n16.x2.trans.shared.b8 {%0,%1,%2,%3}, [%4];"
@@ -171,59 +170,45 @@ __device__ __forceinline__ void ldmatrix_b8_x2_trans(uint32_t (&r)[4], uint32_t 
                  : "r"(addr)
                  : "memory");
 }
-// D(16x8, f32) += A(16x32, e4m3, row) * B(32x8, e4m3, col)
-__device__ __forceinline__ void mma_e4m3_e4m3_16832(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-// D(16x8, f32) += A(16x32, e4m3, row) * B(32x8, e5m2, col)
-__device__ __forceinline__ void mma_e4m3_e5m2_16832(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e5m2.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-// Four floats -> four E4M3 (or E5M2) codes in one register, x0 in the lowest byte; round to nearest
-// even, saturating at the largest finite magnitude.
-__device__ __forceinline__ uint32_t pack_e4m3x4(float x0, float x1, float x2, float x3)
+// The two E4M3 codes in the low (high) half of a register, widened exactly to an f16 pair
+// (lower byte -> lower half).  Every E4M3 value is an f16 value.
+__device__ __forceinline__ uint32_t e4m3x2_lo_to_f16x2(uint32_t codes)
 {
     uint32_t d;
     asm("{\n\t.reg .b16 lo, hi;\n\t"
-        "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
-        "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
-        "mov.b32 %0, {lo, hi};\n\t}"
+        "mov.b32 {lo, hi}, %1;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, lo;\n\t}"
         : "=r"(d)
-        : "f"(x0), "f"(x1), "f"(x2), "f"(x3));
-    return d;
-}
-__device__ __forceinline__ uint32_t pack_e5m2x4(float x0, float x1, float x2, float x3)
-{
-    uint32_t d;
-    asm("{\n\t.reg .b16 lo, hi;\n\t"
-        "cvt.rn.satfinite.e5m2x2.f32 lo, %2, %1;\n\t"
-        "cvt.rn.satfinite.e5m2x2.f32 hi, %4, %3;\n\t"
-        "mov.b32 %0, {lo, hi};\n\t}"
-        : "=r"(d)
-        : "f"(x0), "f"(x1), "f"(x2), "f"(x3));
-    return d;
-}
-// The values of the four E4M3 codes of a register (lowest byte first).
-__device__ __forceinline__ void unpack_e4m3x4(uint32_t codes, float (&v)[4])
-{
-    uint32_t h01, h23;
-    asm("{\n\t.reg .b16 lo, hi;\n\t"
-        "mov.b32 {lo, hi}, %2;\n\t"
-        "cvt.rn.f16x2.e4m3x2 %0, lo;\n\t"
-        "cvt.rn.f16x2.e4m3x2 %1, hi;\n\t}"
-        : "=r"(h01), "=r"(h23)
         : "r"(codes));
-    const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&h01));
-    const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&h23));
-    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+    return d;
+}
+__device__ __forceinline__ uint32_t e4m3x2_hi_to_f16x2(uint32_t codes)
+{
+    uint32_t d;
+    asm("{\n\t.reg .b16 lo, hi;\n\t"
+        "mov.b32 {lo, hi}, %1;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, hi;\n\t}"
+        : "=r"(d)
+        : "r"(codes));
+    return d;
+}
+// D(16x8, f32) += A(16x16, f16, row) * B(16x8, f16, col)
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// {lo, hi} -> one register of two f16, `lo` in the low half, both rounded to nearest even.
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi)
+{
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ float2 unpack_f16(uint32_t packed)
+{
+    return __half22float2(*reinterpret_cast<const __half2 *>(&packed));
 }
 
 // ---------------------------------------------------------------- programmatic dependent launch
