@@ -119,15 +119,15 @@ int decode_attn(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
  *   k_pages, v_pages  DA_FP8_E4M3 [num_pages, Hkv, P, 128]; last dim contiguous, base and every
  *                     stride a multiple of 16 bytes; P in {16, 32, 64, 128}
  *   k_scale, v_scale  DEVICE float[Hkv]; NULL means all factors are 1
- *   q                 bf16, finite (a head's query is rescaled by a power of two and split exactly
- *                     into two E4M3 terms; elements below 2^-13 of the head's largest magnitude
- *                     are carried to within 2^-21 of that largest)
+ *   q                 bf16, finite
  *   other arguments, workspace, status and error conventions: as decode_attn().
  *
- * Arithmetic: both products run on the FP8 tensor-core path (mma m16n8k32, fp32 accumulation) with
- * no conversion of the cache: softmax in fp32 as in decode_attn(); every softmax weight enters the
- * PV product as four E5M2 terms, i.e. to 2^-12 of itself down to 2^-31 of the row's largest weight.
- * Output error is therefore about 2^-12 * max|V| in the worst case (observed: ~1e-5 on N(0,1) data).
+ * Arithmetic: the codes are widened to f16 in registers (exact: every E4M3 value is an f16
+ * value) and both products run as f16 tensor-core mma with fp32 accumulation.  A head's query is
+ * scaled by a power of two so that its largest magnitude lies in [2^14, 2^15) and rounded to f16,
+ * which is exact for every element within 2^-28 of the head's largest; the softmax runs in fp32 as in
+ * decode_attn(); every weight enters the PV product as an f16 high part plus an f16 low part
+ * (about 22 bits).  Observed error against the fp64 oracle: ~1e-6 on N(0,1)-like data.
  */
 int decode_attn_fp8kv(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
                       const float *k_scale, const float *v_scale, const da_tensor *block_table,
@@ -172,6 +172,21 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
  */
 int decode_attn_append(const da_tensor *k_new, const da_tensor *v_new, da_tensor *k_pages, da_tensor *v_pages,
                        const da_tensor *block_table, const da_tensor *seq_lens, void *stream);
+
+/*
+ * decode_attn_append_fp8kv -- decode_attn_append() for the 8-bit cache of decode_attn_fp8kv(): the
+ * new token's bf16 K and V rows are quantised and their E4M3 codes written to position L-1:
+ *     code = nearest_e4m3( x / k_scale[g] )      (v_scale[g] for V)
+ * with the quotient taken in fp32 (one correctly rounded division), ties to the even mantissa,
+ * magnitudes beyond 448 saturating to +-448 and NaN giving the code 0x7F.
+ *   k_new, v_new      bf16 [B, Hkv, 128] as in decode_attn_append()
+ *   k_pages, v_pages  DA_FP8_E4M3 pools as in decode_attn_fp8kv(); WRITTEN
+ *   k_scale, v_scale  DEVICE float[Hkv], or NULL for 1
+ * Status, errors and workspace as decode_attn_append().
+ */
+int decode_attn_append_fp8kv(const da_tensor *k_new, const da_tensor *v_new, da_tensor *k_pages,
+                             da_tensor *v_pages, const float *k_scale, const float *v_scale,
+                             const da_tensor *block_table, const da_tensor *seq_lens, void *stream);
 
 /*
  * decode_attn_extend -- attention for Lq NEW tokens per sequence at once, causal among them, over

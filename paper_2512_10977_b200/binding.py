@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
             L.decode_attn.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_fp8kv.restype = ctypes.c_int
             L.decode_attn_fp8kv.argtypes = [T, T, T, vp, vp, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_append_fp8kv.restype = ctypes.c_int
+            L.decode_attn_append_fp8kv.argtypes = [T, T, T, T, vp, vp, T, T, vp]
             L.decode_attn_cascade.restype = ctypes.c_int
             L.decode_attn_cascade.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_append.restype = ctypes.c_int
@@ -233,6 +235,20 @@ def decode_attn_append(k_new, v_new, k_pages, v_pages, block_table, seq_lens,
                          block_table.shape[1], k_pages.device)
         tv = [_view(t) for t in (k_new, v_new, k_pages, v_pages, block_table, seq_lens)]
         _check(lib().decode_attn_append(*[_ref(t) for t in tv], _stream_ptr(stream)))
+
+
+def decode_attn_append_fp8kv(k_new, v_new, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens,
+                             stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Quantise the new token's bf16 K/V rows [B, Hkv, 128] per KV head (code = nearest E4M3 of
+    x / scale[g]) and write the codes into position seq_lens[b]-1 of the 8-bit cache, in place."""
+    with torch.cuda.device(k_pages.device):
+        ensure_workspace(k_new.shape[0], k_new.shape[1], k_pages.shape[1], 128, k_pages.shape[2],
+                         block_table.shape[1], k_pages.device)
+        tv = [_view(t) for t in (k_new, v_new, k_pages, v_pages, block_table, seq_lens)]
+        _check(lib().decode_attn_append_fp8kv(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]),
+                                              k_scale.data_ptr() if k_scale is not None else None,
+                                              v_scale.data_ptr() if v_scale is not None else None,
+                                              _ref(tv[4]), _ref(tv[5]), _stream_ptr(stream)))
 
 
 def decode_attn_extend(q, k_pages, v_pages, block_table, seq_lens, scale: float,

@@ -1299,4 +1299,64 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p)
     }
 }
 
+// The same step for the 8-bit cache: each bf16 element is divided by its KV head's factor in fp32
+// (one correctly rounded division) and rounded to the nearest E4M3 code (ties to even, saturating at
+// +-448, NaN -> 0x7F) by the hardware conversion.  Thread -> (K or V, kv head, 8 elements).
+struct Append8Params {
+    const __nv_bfloat16 *k_new, *v_new;   // [B, Hkv, 128]
+    int64_t kn_sb, kn_sh, vn_sb, vn_sh;
+    uint8_t *k_pages, *v_pages;           // strides in bytes: page, head, token
+    int64_t k_sp, k_sh, k_st, v_sp, v_sh, v_st;
+    const float *k_scale, *v_scale;       // [Hkv] or NULL (1)
+    const int32_t *block_table;
+    int64_t bt_sb;
+    const int32_t *seq_lens;
+    int64_t sl_stride;
+    int32_t *status;
+    int32_t B, Hkv, P, num_pages;
+    int64_t max_pages;
+};
+
+__global__ void __launch_bounds__(256) append8_kernel(const Append8Params p)
+{
+    const int b = blockIdx.x;
+    const int L = p.seq_lens[(int64_t)b * p.sl_stride];
+    if (L <= 0) {
+        if (L < 0 && threadIdx.x == 0)
+            report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
+        return;
+    }
+    const int t = L - 1;
+    if ((int64_t)(t / p.P) >= p.max_pages) {
+        if (threadIdx.x == 0)
+            report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
+        return;
+    }
+    const int page = __ldg(p.block_table + (int64_t)b * p.bt_sb + t / p.P);
+    if ((uint32_t)page >= (uint32_t)p.num_pages) {
+        if (threadIdx.x == 0)
+            report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, b, t / p.P, page);
+        return;
+    }
+    const int row = t % p.P;
+    for (int e = threadIdx.x; e < 2 * p.Hkv * 16; e += blockDim.x) {
+        const int c = e & 15, g = (e >> 4) % p.Hkv, is_v = e / (16 * p.Hkv);
+        const __nv_bfloat16 *src = is_v ? p.v_new + (int64_t)b * p.vn_sb + (int64_t)g * p.vn_sh
+                                        : p.k_new + (int64_t)b * p.kn_sb + (int64_t)g * p.kn_sh;
+        uint8_t *dst = is_v ? p.v_pages + (int64_t)page * p.v_sp + (int64_t)g * p.v_sh + (int64_t)row * p.v_st
+                            : p.k_pages + (int64_t)page * p.k_sp + (int64_t)g * p.k_sh + (int64_t)row * p.k_st;
+        const float *sc = is_v ? p.v_scale : p.k_scale;
+        const float factor = sc ? __ldg(sc + g) : 1.f;
+        const uint4 in = *reinterpret_cast<const uint4 *>(src + c * 8);
+        const uint32_t w[4] = {in.x, in.y, in.z, in.w};
+        uint32_t codes[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+            codes[h] = pack_e4m3x4(__fdiv_rn(bf16_lo_to_float(w[2 * h]), factor), __fdiv_rn(bf16_hi_to_float(w[2 * h]), factor),
+                                   __fdiv_rn(bf16_lo_to_float(w[2 * h + 1]), factor),
+                                   __fdiv_rn(bf16_hi_to_float(w[2 * h + 1]), factor));
+        *reinterpret_cast<uint2 *>(dst + c * 8) = make_uint2(codes[0], codes[1]);
+    }
+}
+
 }  // namespace da

@@ -192,6 +192,19 @@ __device__ __forceinline__ uint32_t e4m3x2_hi_to_f16x2(uint32_t codes)
         : "r"(codes));
     return d;
 }
+// Four floats -> four E4M3 codes in one register, x0 in the lowest byte: round to nearest even,
+// saturating at the largest finite magnitude (448), NaN -> 0x7F.
+__device__ __forceinline__ uint32_t pack_e4m3x4(float x0, float x1, float x2, float x3)
+{
+    uint32_t d;
+    asm("{\n\t.reg .b16 lo, hi;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+        "mov.b32 %0, {lo, hi};\n\t}"
+        : "=r"(d)
+        : "f"(x0), "f"(x1), "f"(x2), "f"(x3));
+    return d;
+}
 // D(16x8, f32) += A(16x16, f16, row) * B(16x8, f16, col)
 __device__ __forceinline__ void mma_f16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {

@@ -685,6 +685,76 @@ int decode_attn_append(const da_tensor *k_new, const da_tensor *v_new, da_tensor
     return DA_OK;
 }
 
+int decode_attn_append_fp8kv(const da_tensor *k_new, const da_tensor *v_new, da_tensor *k_pages, da_tensor *v_pages,
+                             const float *k_scale, const float *v_scale, const da_tensor *block_table,
+                             const da_tensor *seq_lens, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!k_new || !v_new || !k_pages || !v_pages || !block_table || !seq_lens) return DA_ERR_NULL;
+    if (!k_new->data || !v_new->data || !block_table->data || !seq_lens->data) return DA_ERR_NULL;
+    int rc = check_pool(k_pages, DA_FP8_E4M3);
+    if (rc != DA_OK) return rc;
+    rc = check_pool(v_pages, DA_FP8_E4M3);
+    if (rc != DA_OK) return rc;
+    for (int i = 0; i < 4; ++i)
+        if (k_pages->shape[i] != v_pages->shape[i]) return DA_ERR_SHAPE;
+    if (k_new->dtype != DA_BF16 || v_new->dtype != DA_BF16 || block_table->dtype != DA_I32 || seq_lens->dtype != DA_I32)
+        return DA_ERR_DTYPE;
+    if (k_new->ndim != 3 || v_new->ndim != 3 || block_table->ndim != 2 || seq_lens->ndim != 1) return DA_ERR_SHAPE;
+    const int64_t B = k_new->shape[0], Hkv = k_pages->shape[1], P = k_pages->shape[2];
+    if (k_new->shape[1] != Hkv || k_new->shape[2] != HEAD_DIM) return DA_ERR_SHAPE;
+    for (int i = 0; i < 3; ++i)
+        if (v_new->shape[i] != k_new->shape[i]) return DA_ERR_SHAPE;
+    if (block_table->shape[0] != B || seq_lens->shape[0] != B || block_table->shape[1] <= 0) return DA_ERR_SHAPE;
+    if (B < 0 || B > (1 << 24) || k_pages->shape[0] > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+    if (P != 16 && P != 32 && P != 64 && P != 128) return DA_ERR_UNSUPPORTED;
+    const da_tensor *nw[2] = {k_new, v_new};
+    for (const da_tensor *t : nw) {
+        if (t->stride[2] != 1 || !aligned16(t->data) || (t->stride[0] * 2) % 16 != 0 || (t->stride[1] * 2) % 16 != 0)
+            return DA_ERR_STRIDE_ALIGN;
+    }
+    if (block_table->stride[1] != 1) return DA_ERR_STRIDE_ALIGN;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev;
+    DeviceState *st;
+    rc = current_device(&dev, &st);
+    if (rc != DA_OK) return rc;
+    if (!st->ws || st->ws_bytes < 256) return DA_ERR_WORKSPACE;   // the status record lives there
+    if (B == 0) return DA_OK;
+    Append8Params ap;
+    ap.k_new = static_cast<const __nv_bfloat16 *>(k_new->data);
+    ap.v_new = static_cast<const __nv_bfloat16 *>(v_new->data);
+    ap.kn_sb = k_new->stride[0];
+    ap.kn_sh = k_new->stride[1];
+    ap.vn_sb = v_new->stride[0];
+    ap.vn_sh = v_new->stride[1];
+    ap.k_pages = static_cast<uint8_t *>(k_pages->data);
+    ap.v_pages = static_cast<uint8_t *>(v_pages->data);
+    ap.k_sp = k_pages->stride[0];
+    ap.k_sh = k_pages->stride[1];
+    ap.k_st = k_pages->stride[2];
+    ap.v_sp = v_pages->stride[0];
+    ap.v_sh = v_pages->stride[1];
+    ap.v_st = v_pages->stride[2];
+    ap.k_scale = k_scale;
+    ap.v_scale = v_scale;
+    ap.block_table = static_cast<const int32_t *>(block_table->data);
+    ap.bt_sb = block_table->stride[0];
+    ap.seq_lens = static_cast<const int32_t *>(seq_lens->data);
+    ap.sl_stride = seq_lens->stride[0];
+    ap.status = reinterpret_cast<int32_t *>(st->ws);
+    ap.B = (int32_t)B;
+    ap.Hkv = (int32_t)Hkv;
+    ap.P = (int32_t)P;
+    ap.num_pages = (int32_t)k_pages->shape[0];
+    ap.max_pages = block_table->shape[1];
+    append8_kernel<<<(unsigned)B, 256, 0, stream>>>(ap);
+    g_launches.fetch_add(1);
+    DA_CUDA(cudaGetLastError());
+    return DA_OK;
+}
+
 int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
                        const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse, void *stream_)
 {

@@ -317,3 +317,70 @@ def test_c5b_window_sampled(da):
     da.set_option("grid_blocks", 0)
     case = workloads.c5("cuda", 8192, kv_dtype="fp8")
     _sampled_full_size(da, case, [0, int(np.argmax(case.lens))], "c5b fp8")
+
+
+# ------------------------------------------------------------------ quantising append, bit-exact
+
+@pytest.mark.parametrize("P", [16, 64])
+@pytest.mark.parametrize("layout", ["head_major", "token_major"])
+def test_append_quantises_bit_exactly(da, P, layout):
+    lens = [1, 16, 17, 0, 64, 65, 300, 128, 129]
+    case = fp8_case("app8", lens, P, 5 + P, layout=layout, poison=False)
+    gen = torch.Generator().manual_seed(P)
+    # values spread over the whole E4M3 range after division by the factors: ties, subnormals, saturation
+    k_new = (torch.randn((len(lens), 8, 128), generator=gen) * torch.exp2(torch.randint(-12, 6, (len(lens), 8, 128), generator=gen).float()))
+    v_new = torch.randn((len(lens), 8, 128), generator=gen)
+    k_new[0, 0, :4] = torch.tensor([float("nan"), float("inf"), -float("inf"), 0.0])
+    k_new, v_new = k_new.to(torch.bfloat16), v_new.to(torch.bfloat16)
+    dev = workloads.to_device(case, "cuda")
+    da.decode_attn_append_fp8kv(k_new.cuda(), v_new.cuda(), dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale,
+                                dev.block_table, dev.seq_lens)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    oracle.kv_append_fp8_oracle(k_new, v_new, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
+                                case.block_table, case.seq_lens)
+    assert torch.equal(dev.k_pages.cpu(), case.k_pages) and torch.equal(dev.v_pages.cpu(), case.v_pages)
+
+
+def test_every_bf16_value_quantises_as_the_oracle_says(da):
+    """All 65536 bf16 bit patterns through the kernel's quantiser, for a factor that is not a power of two."""
+    allbits = torch.arange(65536, dtype=torch.int32).to(torch.int16).view(torch.bfloat16)     # [65536]
+    B = 65536 // (8 * 128)
+    k_new = allbits.view(B, 8, 128)
+    case = fp8_case("allbf16", [1] * B, 16, 3, poison=False, shuffle=False)
+    dev = workloads.to_device(case, "cuda")
+    da.decode_attn_append_fp8kv(k_new.cuda(), k_new.cuda(), dev.k_pages, dev.v_pages, dev.k_scale, None,
+                                dev.block_table, dev.seq_lens)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    got_k = dev.k_pages.cpu()[case.block_table[:, 0].long(), :, 0]     # [B, 8, 128]
+    got_v = dev.v_pages.cpu()[case.block_table[:, 0].long(), :, 0]
+    for g in range(8):
+        want = oracle.e4m3_quantize(k_new[:, g].contiguous(), float(case.k_scale[g]))
+        assert np.array_equal(got_k[:, g].numpy(), want), g
+    want = oracle.e4m3_quantize(k_new.contiguous(), 1.0)
+    assert np.array_equal(got_v.numpy(), want)
+
+
+def test_decode_loop_append_then_attend(da):
+    lens = np.array([15, 63, 200, 1])
+    case = fp8_case("loop8", lens + 4, 16, 81, poison=False)
+    case.seq_lens[:] = torch.from_numpy(lens.astype(np.int32))
+    dev = workloads.to_device(case, "cuda")
+    gen = torch.Generator().manual_seed(9)
+    for step in range(4):
+        k_new = torch.randn((4, 8, 128), generator=gen).to(torch.bfloat16)
+        v_new = torch.randn((4, 8, 128), generator=gen).to(torch.bfloat16)
+        q = torch.randn((4, 48, 128), generator=gen).to(torch.bfloat16)
+        case.seq_lens += 1
+        dev.seq_lens += 1
+        da.decode_attn_append_fp8kv(k_new.cuda(), v_new.cuda(), dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale,
+                                    dev.block_table, dev.seq_lens)
+        out, lse = da.decode_attn_fp8kv(q.cuda(), dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, dev.block_table,
+                                        dev.seq_lens, 0, case.scale)
+        oracle.kv_append_fp8_oracle(k_new, v_new, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
+                                    case.block_table, case.seq_lens)
+        ref, ref_lse = oracle.decode_attn_fp8kv_oracle(q, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
+                                                       case.block_table, case.seq_lens, 0, case.scale)
+        assert_close(out.cpu().numpy(), ref, f"loop step {step} out")
+        assert_close(lse.cpu().numpy(), ref_lse, f"loop step {step} lse")
+    assert da.read_device_status() == (0, 0, 0, 0)
+    assert torch.equal(dev.k_pages.cpu(), case.k_pages) and torch.equal(dev.v_pages.cpu(), case.v_pages)
