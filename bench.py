@@ -36,8 +36,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the partition kernel, from the ncu
 # capture summarised in profiles/partition_kernel_<workload>.md; valid for that library version only.
-NCU_TRAFFIC = {("c2", 101): 2223268000 + 8050000,
-               ("c2", 102): 2223268000 + 8050000}   # 102 changed the cascade path only, not this kernel
+NCU_TRAFFIC = {("c2", 103): 2223345000 + 7984000}
 WORKLOAD_TEXT = {
     "c1": "c1: 1 seq x 512 tok, page 16, contiguous, seed 0, 3 keys x20",
     "c2": "c2: 64 seqs, len U[1024,16384], 48q/8kv heads, d128, page 16, permuted pool, seed 1",
