@@ -6,7 +6,7 @@
 //
 // prefix_kernel: one block = 128 query rows (row = b * G + head-in-group) of one KV head and one
 // range of 128-token KV tiles.  Per tile:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in TMEM)
-// -> the eight softmax warps read their rows of S (two threads per row, 64 columns each), keep running
+// -> the sixteen softmax warps read their rows of S (four threads per row, 32 columns each), keep running
 // max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts into tensor memory
 // -> O += P_hi V + P_lo V (tcgen05.mma with the A operand in TMEM, accumulating in another TMEM region) -> the softmax
 // threads rescale a row of O in TMEM only when its maximum has grown by more than 2^8 (rare).  A ninth warp
@@ -21,9 +21,11 @@ constexpr int PF_ROWS = 128;                 // query rows per block (UMMA M)
 constexpr int PF_TOK = 128;                  // tokens per KV tile (UMMA N for S, K for PV)
 constexpr int PF_PLANE = PF_TOK * 128;       // one 64-column half of a 128-row tile: 128-byte rows
 constexpr int PF_TILE = 2 * PF_PLANE;        // 32 KB: Q, a K tile, a V tile
-constexpr int PF_DRV = 8;                    // warps 0..7: softmax (two threads per row); warp 8: issues the
-constexpr int PF_LOADER = 9;                 // MMAs (and owns the TMEM allocation); warp 9: issues the TMA loads
-constexpr int PF_THREADS = (PF_LOADER + 1) * 32;
+constexpr int PF_TPR = 4;                    // softmax threads per row (each owns 128 / PF_TPR columns of a tile)
+constexpr int PF_COLS = 128 / PF_TPR;
+constexpr int PF_DRV = 4 * PF_TPR;           // warps 0..15: softmax; warp 16: issues the MMAs (and owns the TMEM
+constexpr int PF_LOADER = PF_DRV + 1;        // allocation); warp 17: issues the TMA loads of K, warp 18 those of V
+constexpr int PF_THREADS = (PF_LOADER + 2) * 32;   // (one tensor copy costs its issuing warp ~90 cycles)
 constexpr int PF_OFF_Q = 0;
 constexpr float PF_RESCALE_LOG2 = 8.f;       // a row's reference maximum moves only when the maximum grew by more
 constexpr uint32_t PF_WAIT_SLEEP_NS = 64;     // softmax warps yield while they wait: the driver warp shares their schedulers
@@ -33,10 +35,14 @@ constexpr int PF_OFF_V = (1 + PF_NB) * PF_TILE;
 constexpr int PF_OFF_BARS = (1 + 2 * PF_NB) * PF_TILE;   // kfull[3], vfull[3], kfree[3], o[3], s[2], p, x
 constexpr int PF_OFF_MISC = PF_OFF_BARS + 128;  // TMEM base address, abort flag
 constexpr int PF_OFF_XCHG = PF_OFF_MISC + 16;   // row maxima / sums swapped between a row's two threads
-constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + 2 * 2 * 128 * 4;
-constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O_tile in [256,384),
-constexpr int PF_TMEM_PH = 384;              // P high parts in [384,448), low parts in [448,512): 128 tokens as
-constexpr int PF_TMEM_PL = 448;              // 64 columns of bf16 pairs, the A operand of the PV product
+constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + PF_TPR * 128 * 4;   // 2 buffers of bf16 maxima, or one of fp32 sums
+static_assert(PF_SMEM_BYTES <= 232448, "one block must fit the 227 KB of shared memory an SM offers");
+constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O_tile in [256,384).
+constexpr int PF_TMEM_PH = 0;                // P(j) overwrites S(j) in place once both threads of a row have read
+constexpr int PF_TMEM_PL = 64;               // their scores: high parts in the buffer's columns [0,64), low parts in
+                                             // [64,128) -- 128 tokens as 64 columns of bf16 pairs, the A operand of
+                                             // the PV product.  So P is double-buffered like S, and the softmax of
+                                             // tile j+1 does not wait for the PV product of tile j.
 
 // The kernel serves two callers.
 //  * cascade (ext = 0): rows = all sequences' heads of one KV group, row = b * G + head; keys = the
@@ -155,6 +161,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+// 16 consecutive 32-bit columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // D += A * B with the A operand in tensor memory (row i in lane i, two bf16 of K per column).
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate)
@@ -227,7 +242,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
         mbar_init(bar_s, 1);
         mbar_init(bar_s + 8, 1);
-        mbar_init(bar_p, 2 * PF_ROWS);
+        mbar_init(bar_p, PF_DRV);
         mbar_init(bar_x, PF_DRV);
         mbar_fence_init();
         tma_prefetch_desc(&tm_k);
@@ -261,18 +276,23 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const uint32_t tmem = tmem_base_s;
     const uint32_t tmem_s = tmem, tmem_o = tmem + 256;   // S(j) lives at tmem_s + 128 * (j & 1)
 
-    if (warp == PF_LOADER) {
-        // ------------------------------------------------------------------ loader warp: TMA
-        // Lane l < 2 * boxes issues one load per call: box l >> 1 (box_rows tokens of one page), plane
+    if (warp == PF_LOADER || warp == PF_LOADER + 1) {
+        // ------------------------------------------------------------------ loader warps: TMA
+        // Warp PF_LOADER loads the K tiles, warp PF_LOADER + 1 the V tiles (issuing a tile's 16 tensor
+        // copies takes a warp ~1500 cycles: one warp for both was the slowest stage of the block).
+        // Lane l < 2 * boxes issues one load per tile: box l >> 1 (box_rows tokens of one page), plane
         // l & 1.  Tiles 0..2 fill the three buffers; after that K(t) follows the completion of the
-        // scores of tile t-3 (bar_kfree) and V(t) the completion of the PV product of tile t-3
-        // (bar_o).  The tensor core finishes S(t-2) before PV(t-3), so the order is K(t), V(t-1).
+        // scores of tile t-3 (bar_kfree) and V(t) the completion of the PV product of tile t-3 (bar_o).
         if (ntiles > 0) {
+            const bool is_v = warp == PF_LOADER + 1;
             const int boxes = PF_TOK / p.box_rows;
             const int box = lane >> 1, pl = lane & 1;
             const bool active = lane < 2 * boxes;
+            const uint32_t bar_full = is_v ? bar_vfull : bar_kfull;
+            const uint32_t bar_free = is_v ? bar_o : bar_kfree;
+            const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
             bool ok = true;
-            int issued_k = 0, issued_v = 0;
+            int issued = 0;
             auto read_page = [&](int j) {   // page id of this lane's box of tile j (0 for idle lanes)
                 if (!active || j >= ntiles)
                     return 0;
@@ -281,9 +301,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     return 0;   // past the sequence's last page: the block table has no entry
                 return __ldg(bt_row + t / p.P);
             };
-            auto load_kv = [&](int j, int page, bool is_v) {   // K or V of tile j into buffer j % 3
+            auto load_tile = [&](int j, int page) {   // tile j into buffer j % 3
                 const int buf = j % PF_NB;
-                const uint32_t bar = (is_v ? bar_vfull : bar_kfull) + 8 * buf;
+                const uint32_t bar = bar_full + 8 * buf;
                 // extend: boxes wholly past the sequence's end are not loaded (their rows are masked)
                 const int t_tile = (t_begin + j) * PF_TOK;
                 const int nbox = p.ext ? min(boxes, (L - t_tile + p.box_rows - 1) / p.box_rows) : boxes;
@@ -298,39 +318,20 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                         page = p.num_pages;   // out of range: TMA fills zeros and still counts the bytes
                     }
                     const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + box * p.box_rows * 128);
-                    tma_load_4d(sb + (is_v ? PF_OFF_V : PF_OFF_K) + off, is_v ? &tm_v : &tm_k, pl * 64, t % p.P, g, page, bar);
+                    tma_load_4d(sb + (is_v ? PF_OFF_V : PF_OFF_K) + off, tm, pl * 64, t % p.P, g, page, bar);
                 }
-                if (is_v)
-                    issued_v = j + 1;
-                else
-                    issued_k = j + 1;
+                issued = j + 1;
             };
-            int pg_k = read_page(0);
-            for (int j = 0; j < PF_NB && j < ntiles; ++j) {
-                const int pg = pg_k;
-                pg_k = read_page(j + 1);
-                load_kv(j, pg, false);
-                load_kv(j, pg, true);
-            }
-            int pg_v = pg_k;   // page ids of tile 3, fetched ahead
-            for (int t = PF_NB; ok && t <= ntiles; ++t) {
-                if (t < ntiles) {
-                    ok = mbar_wait_bounded(bar_kfree + 8 * (t % PF_NB), (uint32_t)(((t - PF_NB) / PF_NB) & 1), abort_flag);
+            int pg = read_page(0);
+            for (int t = 0; ok && t < ntiles; ++t) {
+                if (t >= PF_NB) {
+                    ok = mbar_wait_bounded(bar_free + 8 * (t % PF_NB), (uint32_t)(((t - PF_NB) / PF_NB) & 1), abort_flag);
                     if (!ok)
                         break;
-                    const int pg = pg_k;
-                    pg_k = read_page(t + 1);
-                    load_kv(t, pg, false);
                 }
-                const int tv = t - 1;   // V of the tile before
-                if (tv >= PF_NB) {
-                    ok = mbar_wait_bounded(bar_o + 8 * (tv % PF_NB), (uint32_t)(((tv - PF_NB) / PF_NB) & 1), abort_flag);
-                    if (!ok)
-                        break;
-                    const int pg = pg_v;
-                    pg_v = read_page(tv + 1);
-                    load_kv(tv, pg, true);
-                }
+                const int pg_now = pg;
+                pg = read_page(t + 1);   // fetched one tile ahead
+                load_tile(t, pg_now);
             }
             if (!ok && lane == 0) {
                 if (*abort_flag == 0) {
@@ -342,10 +343,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 // do not leave while copies may still land in shared memory: bounded wait for the
                 // latest fill of each buffer
                 for (int k = 0; k < PF_NB; ++k) {
-                    const int jk = issued_k - 1 - k, jv = issued_v - 1 - k;
+                    const int jk = issued - 1 - k;
                     const uint64_t t0 = globaltimer_ns();
-                    while ((jk >= 0 && !mbar_try_wait(bar_kfull + 8 * (jk % PF_NB), (uint32_t)((jk / PF_NB) & 1))) ||
-                           (jv >= 0 && !mbar_try_wait(bar_vfull + 8 * (jv % PF_NB), (uint32_t)((jv / PF_NB) & 1)))) {
+                    while (jk >= 0 && !mbar_try_wait(bar_full + 8 * (jk % PF_NB), (uint32_t)((jk / PF_NB) & 1))) {
                         if (globaltimer_ns() - t0 > 1000000000ull)
                             break;
                     }
@@ -359,30 +359,37 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         // just released -- so the scores of tile j+1 are ready before the softmax of j ends.
         if (ntiles > 0) {
             bool ok = true;
+            // The issuing thread is the narrowest part of the kernel (one tcgen05.mma takes ~70 cycles
+            // to execute), so nothing is computed per instruction that can be computed once: the matrix
+            // descriptors of Q and of the first K and V buffers are built here, and a step or a buffer
+            // only adds a constant to the descriptor's address field (bits 0-13, in 16-byte units).
+            const uint64_t q_desc = umma_desc(sb + PF_OFF_Q, 16, 1024);
+            const uint64_t k_desc = umma_desc(sb + PF_OFF_K, 16, 1024);
+            const uint64_t v_desc = umma_desc(sb + PF_OFF_V, PF_PLANE, 1024);
+            const uint32_t idesc_s = umma_idesc(PF_ROWS, PF_TOK, false);
+            const uint32_t idesc_o = umma_idesc(PF_ROWS, HEAD_DIM, true);
+            static_assert(PF_OFF_V + PF_NB * PF_TILE <= (1 << 18), "descriptor addresses must stay inside 256 KB");
             auto mma_s = [&](int j) {   // S = Q K^T for tile j
-                const uint32_t kb = sb + PF_OFF_K + (j % PF_NB) * PF_TILE;
-                const uint32_t idesc = umma_idesc(PF_ROWS, PF_TOK, false);
+                const uint64_t kd = k_desc + (uint64_t)(((j % PF_NB) * PF_TILE) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * PF_PLANE + (kk & 3) * 32;
-                    umma_bf16(tmem_s + 128 * (j & 1), umma_desc(sb + PF_OFF_Q + off, 16, 1024), umma_desc(kb + off, 16, 1024),
-                              idesc, kk > 0);
+                    const uint64_t off = (uint64_t)(((kk >> 2) * PF_PLANE + (kk & 3) * 32) >> 4);
+                    umma_bf16(tmem_s + 128 * (j & 1), q_desc + off, kd + off, idesc_s, kk > 0);
                 }
                 umma_commit(bar_s + 8 * (j & 1));
                 umma_commit(bar_kfree + 8 * (j % PF_NB));
             };
             auto mma_o = [&](int j) {   // O_tile = P_hi V + P_lo V for tile j
-                const uint32_t vb = sb + PF_OFF_V + (j % PF_NB) * PF_TILE;
-                const uint32_t idesc = umma_idesc(PF_ROWS, HEAD_DIM, true);
+                const uint64_t vd = v_desc + (uint64_t)(((j % PF_NB) * PF_TILE) >> 4);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    const uint32_t pa = tmem + (half ? PF_TMEM_PL : PF_TMEM_PH);
+                    const uint32_t pa = tmem_s + 128 * (j & 1) + (half ? PF_TMEM_PL : PF_TMEM_PH);
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         // A = P from tensor memory (16 tokens = 8 columns per step); B = V stored
                         // [token][d]: MN-major, planes are the two halves of d (leading offset = plane),
                         // 8-token groups 1024 B apart
-                        umma_bf16_ts(tmem_o, pa + kk * 8, umma_desc(vb + kk * 2048, PF_PLANE, 1024), idesc, j > 0 || half > 0 || kk > 0);
+                        umma_bf16_ts(tmem_o, pa + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || half > 0 || kk > 0);
                     }
                 }
                 umma_commit(bar_o + 8 * (j % PF_NB));
@@ -425,18 +432,29 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------------------------ softmax warps
-        // Two threads per row: warp w and warp w + 4 read the same TMEM lanes (32 * (w % 4) ...), the
-        // first the tile's columns 0..63, the second 64..127 -- of S (tokens) and of O_tile (head_dim).
+        // PF_TPR threads per row: warps w, w + 4, w + 8, ... read the same TMEM lanes (32 * (w % 4) ...),
+        // each its own PF_COLS columns -- of S (tokens) and of O_tile (head_dim).
+        static_assert(PF_COLS == 32, "the TMEM access shapes below are written for 32 columns a thread");
         const int r = 32 * (warp & 3) + lane;            // row of the tile = TMEM lane
-        const int half = warp >> 2;
-        const uint32_t lane_base = ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(half * 64);
-        float *xchg = reinterpret_cast<float *>(smem + PF_OFF_XCHG);   // [2 buffers][2 halves][128 rows]
+        const int part = warp >> 2;                      // which columns
+        const uint32_t lane_sel = (uint32_t)(32 * (warp & 3)) << 16;
+        const uint32_t lane_base = lane_sel + (uint32_t)(part * PF_COLS);
+        // row maxima are swapped as bf16 rounded UP, [2 buffers][PF_TPR parts][128 rows]: every thread of a
+        // row reads the same four values, so they agree on one reference that is >= every score (the
+        // result does not depend on which reference is used, only on its being common); the final sums
+        // of weights go through the same bytes as fp32 [PF_TPR][128]
+        __nv_bfloat16 *xchg = reinterpret_cast<__nv_bfloat16 *>(smem + PF_OFF_XCHG);
         // O accumulates in tensor memory across tiles, relative to a reference maximum m_run that is
         // moved only when a row's maximum has grown by more than PF_RESCALE_LOG2 (weights then stay
         // below 2^PF_RESCALE_LOG2, well inside what the bf16 high + low pair carries); moving it
         // means scaling that row of O, which after the first few tiles is rare.
         float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;
+        // The scale enters inside the exponent (one fma per score).  A masked raw score must come out as
+        // -inf after scaling whatever the scale's sign; a scale of exactly 0 would turn it into NaN
+        // (inf * 0), so 0 is replaced by 1e-30, which changes no weight by more than 1e-24.
+        const float sc = p.scale_log2 == 0.f ? 1e-30f : p.scale_log2;
+        const float neg_inf_raw = sc > 0.f ? -INFINITY : INFINITY;
         // extend: this row's query attends tokens below `limit` (0 for padding rows: nothing)
         const int rr = rt * PF_ROWS + r;
         const int limit = (p.ext && rr < R && L > 0) ? L - p.Lq + rr / p.G + 1 : 0;
@@ -446,32 +464,38 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 break;
             }
             tc_fence_after();
-            // this thread's 64 scores, scaled into the log2 domain, and their maximum
-            float sv[64];
+            // this thread's raw scores (q.k) and the largest scaled one
+            float sv[PF_COLS];
             {
-                uint32_t v[2][32];
-                tmem_ld32_issue(tmem_s + 128 * (j & 1) + lane_base, v[0]);
-                tmem_ld32_issue(tmem_s + 128 * (j & 1) + lane_base + 32, v[1]);
+                uint32_t v[PF_COLS];
+                tmem_ld32_issue(tmem_s + 128 * (j & 1) + lane_base, v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 64; ++i)
-                    sv[i] = __uint_as_float(v[i >> 5][i & 31]) * p.scale_log2;
+                for (int i = 0; i < PF_COLS; ++i)
+                    sv[i] = __uint_as_float(v[i]);
             }
             const int t_tile = (t_begin + j) * PF_TOK;
             if (t_tile + PF_TOK > mask_from) {   // extend, near the end: causal mask by select (K rows past
-                const int t_mine = t_tile + half * 64;   // the sequence's end may hold anything)
+                const int t_mine = t_tile + part * PF_COLS;   // the sequence's end may hold anything)
 #pragma unroll
-                for (int i = 0; i < 64; ++i)
+                for (int i = 0; i < PF_COLS; ++i)
                     if (t_mine + i >= limit)
-                        sv[i] = -INFINITY;
+                        sv[i] = neg_inf_raw;
             }
             float mx = sv[0];
+            if (sc > 0.f) {
 #pragma unroll
-            for (int i = 1; i < 64; ++i)
-                mx = fmaxf(mx, sv[i]);
-            // the row's two halves must use one maximum: swap through shared memory
-            float *xb = xchg + (j & 1) * 256;
-            xb[half * 128 + r] = mx;
+                for (int i = 1; i < PF_COLS; ++i)
+                    mx = fmaxf(mx, sv[i]);
+            } else {
+#pragma unroll
+                for (int i = 1; i < PF_COLS; ++i)
+                    mx = fminf(mx, sv[i]);
+            }
+            mx = (mx == neg_inf_raw) ? -INFINITY : mx * sc;
+            // the row's threads must use one maximum: swap through shared memory
+            __nv_bfloat16 *xb = xchg + (j & 1) * (PF_TPR * 128);
+            xb[part * 128 + r] = __float2bfloat16_ru(mx);
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_x);
@@ -479,41 +503,40 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 ok = false;
                 break;
             }
-            mx = fmaxf(mx, xb[(half ^ 1) * 128 + r]);
+            mx = __bfloat162float(xb[r]);
+#pragma unroll
+            for (int q = 1; q < PF_TPR; ++q)
+                mx = fmaxf(mx, __bfloat162float(xb[q * 128 + r]));
             const bool moved = (m_run == -INFINITY) || (mx > m_run + PF_RESCALE_LOG2);
             const float m_new = moved ? mx : m_run;
             const float alpha = !moved ? 1.f : (m_run == -INFINITY ? 0.f : fast_exp2(m_run - m_new));
             // weights, their sum, and P as bf16 high + low parts (kept in registers for now)
             float lsum = 0.f;
-            uint32_t phi[32], plo[32];
+            uint32_t phi[PF_COLS / 2], plo[PF_COLS / 2];
             const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // a row with nothing to attend yet
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-                const float p0 = fast_exp2(sv[2 * e] - m_use);
-                const float p1 = fast_exp2(sv[2 * e + 1] - m_use);
+            for (int e = 0; e < PF_COLS / 2; ++e) {
+                const float p0 = fast_exp2(fmaf(sv[2 * e], sc, -m_use));
+                const float p1 = fast_exp2(fmaf(sv[2 * e + 1], sc, -m_use));
                 lsum += p0 + p1;
                 phi[e] = pack_bf16(p0, p1);
                 plo[e] = pack_bf16(p0 - bf16_lo_to_float(phi[e]), p1 - bf16_hi_to_float(phi[e]));
             }
-            // the previous tile's PV product must be complete before its P buffer is overwritten, and
-            // before a row of O is rescaled
-            if (j > 0) {
+            // a row of O may be rescaled only once the previous tile's PV product is complete
+            // (tcgen05.ld / .st are warp-wide: all lanes go)
+            if (j > 0 && __any_sync(0xffffffffu, moved)) {
                 if (!mbar_wait_bounded(bar_o + 8 * ((j - 1) % PF_NB), (uint32_t)(((j - 1) / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, moved)) {   // tcgen05.ld / .st are warp-wide: all lanes go
-                    uint32_t v[2][32];
-                    tmem_ld32_issue(tmem_o + lane_base, v[0]);
-                    tmem_ld32_issue(tmem_o + lane_base + 32, v[1]);
-                    tmem_ld_wait();
+                uint32_t v[PF_COLS];
+                tmem_ld32_issue(tmem_o + lane_base, v);
+                tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 64; ++i)
-                        v[i >> 5][i & 31] = __float_as_uint(__uint_as_float(v[i >> 5][i & 31]) * alpha);
-                    tmem_st32(tmem_o + lane_base, v[0]);
-                    tmem_st32(tmem_o + lane_base + 32, v[1]);
-                }
+                for (int i = 0; i < PF_COLS; ++i)
+                    v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                tmem_st32(tmem_o + lane_base, v);
             }
             if (p.ext && t_tile + PF_TOK > L) {
                 // The tile reaches past the sequence's end: those V rows were not loaded, or are a page's
@@ -525,44 +548,50 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 }
                 const int first_bad = max(L - t_tile, 0);
                 uint8_t *vb = smem + PF_OFF_V + (j % PF_NB) * PF_TILE;
-                for (int e = tid; e < (PF_TOK - first_bad) * 16; e += 2 * PF_ROWS) {
+                for (int e = tid; e < (PF_TOK - first_bad) * 16; e += PF_TPR * PF_ROWS) {
                     const int row = first_bad + (e >> 4), ch = e & 15;
                     *reinterpret_cast<uint4 *>(vb + (ch >> 3) * PF_PLANE + row * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
                 }
                 fence_proxy_async_smem();
             }
-            // P into tensor memory: this thread's 64 tokens are 32 columns of bf16 pairs
-            tmem_st32(tmem + PF_TMEM_PH + ((uint32_t)(32 * (warp & 3)) << 16) + half * 32, phi);
-            tmem_st32(tmem + PF_TMEM_PL + ((uint32_t)(32 * (warp & 3)) << 16) + half * 32, plo);
+            // P into tensor memory, over this tile's scores (every thread of the row has read its own: the
+            // maximum exchange above came after the loads): this thread's 32 tokens are 16 columns of bf16 pairs
+            tmem_st16(tmem_s + 128 * (j & 1) + PF_TMEM_PH + lane_sel + part * (PF_COLS / 2), phi);
+            tmem_st16(tmem_s + 128 * (j & 1) + PF_TMEM_PL + lane_sel + part * (PF_COLS / 2), plo);
             tmem_st_wait();
             l_run = l_run * alpha + lsum;
             m_run = m_new;
             tc_fence_before();          // this thread's TMEM reads and writes precede the MMAs that follow
-            mbar_arrive(bar_p);
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(bar_p);     // one arrival per warp: 512 arrivals on one barrier cost hundreds of cycles
         }
-        uint32_t o_raw[2][32];
+        uint32_t o_raw[PF_COLS];
         if (ok && ntiles > 0) {
             if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) % PF_NB), (uint32_t)(((ntiles - 1) / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
                 tc_fence_after();
-                tmem_ld32_issue(tmem_o + lane_base, o_raw[0]);
-                tmem_ld32_issue(tmem_o + lane_base + 32, o_raw[1]);
+                tmem_ld32_issue(tmem_o + lane_base, o_raw);
                 tmem_ld_wait();
             } else {
                 ok = false;
             }
         }
-        // the row's sum of weights is the sum of its two halves' sums (both relative to m_run)
-        float l_row = l_run;
+        // the row's sum of weights is the sum of its threads' sums (all relative to m_run)
+        float l_row = 0.f;
         if (ok && ntiles > 0) {
-            float *xb = xchg + (ntiles & 1) * 256;
-            xb[half * 128 + r] = l_run;
+            // (every thread has read the last maxima before the last PV product could complete)
+            float *xb = reinterpret_cast<float *>(smem + PF_OFF_XCHG);
+            xb[part * 128 + r] = l_run;
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_x);
-            if (mbar_wait_bounded(bar_x, (uint32_t)(ntiles & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS))
-                l_row += xb[(half ^ 1) * 128 + r];
-            else
+            if (mbar_wait_bounded(bar_x, (uint32_t)(ntiles & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
+#pragma unroll
+                for (int q = 0; q < PF_TPR; ++q)
+                    l_row += xb[q * 128 + r];
+            } else {
                 ok = false;
+            }
         }
         if (!ok) {
             if (*abort_flag == 0) {
@@ -575,36 +604,36 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 const bool any = ntiles > 0 && l_row > 0.f;
                 const float inv = any ? 1.f / l_row : 0.f;
                 const float lse_val = any ? (m_run + fast_log2(l_row)) * LN2 : -INFINITY;
-                float vals[64];
+                float vals[PF_COLS];
 #pragma unroll
-                for (int i = 0; i < 64; ++i)
-                    vals[i] = any ? __uint_as_float(o_raw[i >> 5][i & 31]) * inv : 0.f;
+                for (int i = 0; i < PF_COLS; ++i)
+                    vals[i] = any ? __uint_as_float(o_raw[i]) * inv : 0.f;
                 const int h = g * p.G + hd;
                 if (p.ext && p.splits == 1) {
-                    const int64_t at = (int64_t)bseq * p.o_sb + (int64_t)outer * p.o_sq + (int64_t)h * p.o_sh + half * 64;
+                    const int64_t at = (int64_t)bseq * p.o_sb + (int64_t)outer * p.o_sq + (int64_t)h * p.o_sh + part * PF_COLS;
                     if (p.out_bf16) {
                         __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
 #pragma unroll
-                        for (int i = 0; i < 64; ++i)
+                        for (int i = 0; i < PF_COLS; ++i)
                             dst[i] = __float2bfloat16_rn(vals[i]);
                     } else {
                         float *dst = reinterpret_cast<float *>(p.out) + at;
 #pragma unroll
-                        for (int i = 0; i < 64; ++i)
+                        for (int i = 0; i < PF_COLS; ++i)
                             dst[i] = vals[i];
                     }
-                    if (half == 0 && p.lse)
+                    if (part == 0 && p.lse)
                         p.lse[(int64_t)bseq * p.l_sb + (int64_t)outer * p.l_sq + (int64_t)h * p.l_sh] = lse_val;
                 } else {
                     const int Hq = p.Hkv * p.G;
                     const int64_t n_rows = (int64_t)p.B * (p.ext ? p.Lq : 1) * Hq;
                     const int64_t idx = p.ext ? ((int64_t)bseq * p.Lq + outer) * Hq + h : (int64_t)outer * Hq + h;
                     const int64_t at = (int64_t)split * n_rows + idx;
-                    float *dst = p.pre_o + at * HEAD_DIM + half * 64;
+                    float *dst = p.pre_o + at * HEAD_DIM + part * PF_COLS;
 #pragma unroll
-                    for (int i = 0; i < 64; i += 4)
+                    for (int i = 0; i < PF_COLS; i += 4)
                         *reinterpret_cast<float4 *>(dst + i) = make_float4(vals[i], vals[i + 1], vals[i + 2], vals[i + 3]);
-                    if (half == 0)
+                    if (part == 0)
                         p.pre_lse[at] = lse_val;
                 }
             }
