@@ -351,7 +351,12 @@ def run_ours(args):
                 "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                 "kernel_ms": kms, "traffic": None if kv8 else NCU_TRAFFIC.get((args.workload, da.version()))}
-    if Lq:
+    G_ = case.q.shape[1] // case.k_pages.shape[1]
+    ext_stream = bool(Lq) and Lq * G_ <= da.get_option("extend_stream_rows")
+    if ext_stream:
+        # a few new tokens ride through the streaming kernels as a wider group: still bound by HBM
+        roofline["kernel"] = f"partition_kernel ({Lq} query tokens x {G_} heads per KV head)"
+    elif Lq:
         # one kernel, a dense causal contraction: algorithmic flops = QK^T and PV over each query's keys
         Hq, Dh = case.q.shape[1], case.q.shape[2]
         keys = sum(float(L - Lq) * Lq + Lq * (Lq + 1) / 2.0 for L in case.lens)
@@ -387,7 +392,8 @@ def run_ours(args):
                    "l2": "inputs exceed L2 (no flush)" if nbytes > 4 * 126e6 else "inputs fit L2; not flushed",
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "grid_blocks": da.get_option("grid_blocks"),
-                   "path": f"decode_attn_extend, {Lq} new tokens per sequence (causal, tcgen05)" if Lq else
+                   "path": (f"decode_attn_extend, {Lq} new tokens per sequence (causal, " +
+                            ("streaming kernels)" if ext_stream else "tcgen05)")) if Lq else
                            ("cascade (shared prefix on tcgen05)" if prefix else
                             ("decode_attn_fp8kv" if kv8 else "decode_attn"))},
         "frac_of_8TBs": gbs / world / NOMINAL_HBM_GBS, "seq_per_s": seqs,

@@ -197,8 +197,12 @@ int decode_attn_append_fp8kv(const da_tensor *k_new, const da_tensor *v_new, da_
  *
  *     out[b,qi,h,:] = sum_{t <= L_b-Lq+qi} softmax(scale * <q[b,qi,h], K[.., t]>)_t V[.., t]
  *
- * which for Lq = 1 is decode_attn() without a window.  Runs on the tcgen05 tensor cores (the same
- * kernel as the cascade's prefix pass: 128 (query, head) rows of one KV group per thread block).
+ * which for Lq = 1 is decode_attn() without a window.  Two schedules, same result: with at most 16
+ * query rows per KV head (Lq * Hq / Hkv <= 16: a few speculated tokens) the rows ride through the
+ * plan / partition / merge kernels of decode_attn() as one wider head group, each column with its own
+ * causal limit, at the HBM rate; longer query blocks run on the tcgen05 tensor cores (the same kernel
+ * as the cascade's prefix pass: 128 (query, head) rows of one KV group per thread block).  Option
+ * "extend_stream_rows" (0 .. 16, default 16) moves the switch; 0 always takes the tensor-core kernel.
  *
  *   q      bf16 [B, Lq, Hq, 128], last dim contiguous
  *   out    f32 or bf16 [B, Lq, Hq, 128], last dim contiguous
@@ -303,6 +307,8 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
  *   "tail_units"   work units per thread block that are handed out by ticket after the static
  *                  ranges (0 .. 64, default 4; 0 = static ranges only)
  *   "static_frac"  share of the work, in 1/256, covered by the static ranges (default 224)
+ *   "extend_stream_rows"  decode_attn_extend(): most query rows per KV head that go through the
+ *                  streaming kernels instead of the tensor-core kernel (0 .. 16, default 16)
  * Returns DA_ERR_UNSUPPORTED for an unknown name or a value out of range.
  */
 int decode_attn_set_option(const char *name, int64_t value);

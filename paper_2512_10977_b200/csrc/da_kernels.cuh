@@ -89,6 +89,11 @@ struct PartParams {
     int32_t B, Hkv, G, P, box_rows, num_pages, out_bf16;
     float scale_log2;         // scale * log2(e)
     const float *k_scale, *v_scale;   // 8-bit cache: per-KV-head factors (NULL: 1)
+    // Several new tokens per sequence (Lq > 1, causal among them): query token qi of KV group g's head hd
+    // is "virtual head" qi * G + hd of that group; Gv = Lq * G <= 16 of them share one pass over K and V.
+    // Query qi sits at position L - Lq + qi and attends tokens below L - Lq + qi + 1.
+    int32_t Lq, Gv;
+    int64_t q_sq, o_sq, l_sq;         // strides of the query-token dimension (0 when Lq == 1)
 };
 
 struct PlanParams {
@@ -105,6 +110,7 @@ struct PlanParams {
     int32_t *status;
     int32_t B, Hkv, P, window;
     int32_t tile_t;           // tokens per tile (TILE_T or TILE_T8)
+    int32_t min_len;          // a non-empty sequence shorter than this is an error (the new tokens of an extend call)
     int32_t first_token;      // tokens before this one are not attended (the cascade's suffix pass)
     int32_t n_static, n_tail_max, static_frac_q8;   // large units; most ticketed units; share of the
                                                     // line given to the large units, in 1/256
@@ -125,6 +131,8 @@ struct MergeParams {
     float *lse;
     int64_t l_sb, l_sh;
     int32_t B, Hkv, G, heads_pad, out_bf16;
+    int32_t Lq, Gv;           // as in PartParams
+    int64_t o_sq, l_sq;
 };
 
 __device__ __forceinline__ void report_status(int32_t *status, int code, int a, int b, int c)
@@ -210,9 +218,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
                     report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
                 L = 0;
             }
-            if (L > 0 && L < p.first_token) {
+            if (L > 0 && (L < p.first_token || L < p.min_len)) {
                 if (writer)
-                    report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 1, L);
+                    report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, L < p.min_len ? 2 : 1, L);
                 L = 0;
             }
             lo = (p.window > 0 && p.window < L) ? L - p.window : 0;
@@ -605,12 +613,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
             const int head = n * 8 + r;
+            const int hv = head < p.Gv ? head : 0;
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
-                p.q + (int64_t)b * p.q_sb + (int64_t)(g * p.G + (head < p.G ? head : 0)) * p.q_sh);
+                p.q + (int64_t)b * p.q_sb + (int64_t)(hv / p.G) * p.q_sq + (int64_t)(g * p.G + hv % p.G) * p.q_sh);
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
-                qf[n][kk][0] = head < p.G ? __ldg(qrow + 8 * kk + c) : 0u;
-                qf[n][kk][1] = head < p.G ? __ldg(qrow + 8 * kk + 4 + c) : 0u;
+                qf[n][kk][0] = head < p.Gv ? __ldg(qrow + 8 * kk + c) : 0u;
+                qf[n][kk][1] = head < p.Gv ? __ldg(qrow + 8 * kk + 4 + c) : 0u;
             }
         }
     };
@@ -626,15 +635,16 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
             const int head = n * 8 + r;
+            const int hv = head < p.Gv ? head : 0;
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
-                p.q + (int64_t)b * p.q_sb + (int64_t)(g * p.G + (head < p.G ? head : 0)) * p.q_sh);
+                p.q + (int64_t)b * p.q_sb + (int64_t)(hv / p.G) * p.q_sq + (int64_t)(g * p.G + hv % p.G) * p.q_sh);
             uint32_t w[8][2];
             float amax = 0.f;
 #pragma unroll
             for (int i = 0; i < 8; ++i)
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
-                    w[i][hf] = head < p.G ? __ldg(qrow + 8 * i + 2 * c + hf) : 0u;
+                    w[i][hf] = head < p.Gv ? __ldg(qrow + 8 * i + 2 * c + hf) : 0u;
                     amax = fmaxf(amax, fmaxf(fabsf(bf16_lo_to_float(w[i][hf])), fabsf(bf16_hi_to_float(w[i][hf]))));
                 }
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
@@ -894,6 +904,18 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         if (!ok1) s[n][2] = s[n][3] = -INFINITY;
                     }
                 }
+                if (p.Lq > 1 && a + 16 > L - p.Lq + 1) {
+                    // several new tokens: the query of column (virtual head) v attends tokens below
+                    // L - Lq + v / G + 1 only
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int lim = L - p.Lq + (n * 8 + 2 * c + e) / p.G + 1;
+                            if (a + r >= lim) s[n][e] = -INFINITY;
+                            if (a + r + 8 >= lim) s[n][2 + e] = -INFINITY;
+                        }
+                }
                 // ---- online softmax in the log2 domain: column (head) maxima over the 16 tokens
                 float mx[NT8][2];
                 bool grew = false;
@@ -934,10 +956,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
                 for (int n = 0; n < NT8; ++n) {
                     float pv[4];
-                    pv[0] = fast_exp2(s[n][0] - m_run[n][0]);
-                    pv[1] = fast_exp2(s[n][1] - m_run[n][1]);
-                    pv[2] = fast_exp2(s[n][2] - m_run[n][0]);
-                    pv[3] = fast_exp2(s[n][3] - m_run[n][1]);
+                    // (a column that has seen no token yet keeps m = -inf: exp2(-inf - 0) = 0, not NaN)
+                    const float m0u = m_run[n][0] == -INFINITY ? 0.f : m_run[n][0];
+                    const float m1u = m_run[n][1] == -INFINITY ? 0.f : m_run[n][1];
+                    pv[0] = fast_exp2(s[n][0] - m0u);
+                    pv[1] = fast_exp2(s[n][1] - m1u);
+                    pv[2] = fast_exp2(s[n][2] - m0u);
+                    pv[3] = fast_exp2(s[n][3] - m1u);
                     l_run[n][0] += pv[0] + pv[2];
                     l_run[n][1] += pv[1] + pv[3];
                     const uint32_t h01 = pack_bf16(pv[0], pv[1]);
@@ -1025,7 +1050,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         {
             const int d = tid;   // 0..127
             const float vmul = (KV8 && p.v_scale) ? __ldg(p.v_scale + g) : 1.f;
-            for (int head = 0; head < p.G; ++head) {
+            for (int head = 0; head < p.Gv; ++head) {
                 float M = st_m[head];
 #pragma unroll
                 for (int w = 1; w < NCW; ++w)
@@ -1038,17 +1063,18 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     den += st_l[w * HEADS + head] * f;
                     num += xbuf[(w * HEADS + head) * HEAD_DIM + dx] * f;
                 }
-                const float val = KV8 ? (num / den) * vmul : num / den;
-                const float lse_nat = (M + fast_log2(den)) * LN2;
+                // (den = 0: a piece in which this column's query attends nothing -- several new tokens only)
+                const float val = den > 0.f ? (KV8 ? (num / den) * vmul : num / den) : 0.f;
+                const float lse_nat = den > 0.f ? (M + fast_log2(den)) * LN2 : -INFINITY;
                 if (whole) {
-                    const int h = g * p.G + head;
+                    const int qi = head / p.G, h = g * p.G + head % p.G;
+                    const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h * p.o_sh + d;
                     if (p.out_bf16)
-                        reinterpret_cast<__nv_bfloat16 *>(p.out)[(int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d] =
-                            __float2bfloat16_rn(val);
+                        reinterpret_cast<__nv_bfloat16 *>(p.out)[at] = __float2bfloat16_rn(val);
                     else
-                        reinterpret_cast<float *>(p.out)[(int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d] = val;
+                        reinterpret_cast<float *>(p.out)[at] = val;
                     if (d == 0 && p.lse)
-                        p.lse[(int64_t)b * p.l_sb + (int64_t)h * p.l_sh] = lse_nat;
+                        p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h * p.l_sh] = lse_nat;
                 } else {
                     p.part_o[((int64_t)slot * HEADS + head) * HEAD_DIM + d] = val;
                     if (d == 0)
@@ -1142,8 +1168,8 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
             }
         return list[(size_t)k * p.merge_seg + i];
     };
-    auto store = [&](int b, int h, float4 v, float lse_val) {
-        const int64_t at = (int64_t)b * p.o_sb + (int64_t)h * p.o_sh + d;
+    auto store = [&](int b, int qi, int h, float4 v, float lse_val) {
+        const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h * p.o_sh + d;
         if (p.out_bf16) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
             __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
@@ -1162,7 +1188,7 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
             }
         }
         if (ln == 0 && p.lse)
-            p.lse[(int64_t)b * p.l_sb + (int64_t)h * p.l_sh] = lse_val;
+            p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h * p.l_sh] = lse_val;
     };
     // splits [k0, k0 + 32) of entry e (pair id, first slot, first unit, splits), one head
     auto warp_merge = [&](const int4 &e, int head, int k0) {
@@ -1212,15 +1238,16 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
     };
     auto finish = [&](const int4 &e, int head, const MergeAcc &a) {
         const float inv = 1.f / a.den;
-        store(e.x / p.Hkv, (e.x % p.Hkv) * p.G + head,
+        // head = virtual head: query token head / G, head head % G of the pair's KV group
+        store(e.x / p.Hkv, head / p.G, (e.x % p.Hkv) * p.G + head % p.G,
               make_float4(a.acc.x * inv, a.acc.y * inv, a.acc.z * inv, a.acc.w * inv), a.M + __logf(a.den));
     };
 
     // ---- pairs with many splits: one (pair, head) per block at a time, handed out from the last
     //      block down so that they rarely meet the warp-sized items below in the same block
-    for (int item = (int)(gridDim.x - 1 - blockIdx.x); item < n_big * p.G; item += gridDim.x) {
-        const int4 e = entry(p.merge_big, cnt.n_big, item / p.G);
-        const int head = item % p.G;
+    for (int item = (int)(gridDim.x - 1 - blockIdx.x); item < n_big * p.Gv; item += gridDim.x) {
+        const int4 e = entry(p.merge_big, cnt.n_big, item / p.Gv);
+        const int head = item % p.Gv;
         MergeAcc a = {-INFINITY, 0.f, make_float4(0.f, 0.f, 0.f, 0.f)};
         for (int k0 = warp * 32; k0 < e.w; k0 += MERGE_WARPS * 32)
             merge_fold(a, warp_merge(e, head, k0));
@@ -1235,17 +1262,17 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
         __syncthreads();
     }
     // ---- pairs with at most 32 splits: one (pair, head) per warp
-    for (int item = blockIdx.x * MERGE_WARPS + warp; item < n_small * p.G; item += gridDim.x * MERGE_WARPS) {
-        const int4 e = entry(p.merge_small, cnt.n_small, item / p.G);
-        const int head = item % p.G;
+    for (int item = blockIdx.x * MERGE_WARPS + warp; item < n_small * p.Gv; item += gridDim.x * MERGE_WARPS) {
+        const int4 e = entry(p.merge_small, cnt.n_small, item / p.Gv);
+        const int head = item % p.Gv;
         finish(e, head, warp_merge(e, head, 0));
     }
     // ---- empty sequences
     for (int b = blockIdx.x; b < p.B; b += gridDim.x) {
         if (p.seq_info[b].w != 0)
             continue;
-        for (int h = warp; h < p.Hkv * p.G; h += MERGE_WARPS)
-            store(b, h, make_float4(0.f, 0.f, 0.f, 0.f), -INFINITY);
+        for (int h = warp; h < p.Lq * p.Hkv * p.G; h += MERGE_WARPS)
+            store(b, h / (p.Hkv * p.G), h % (p.Hkv * p.G), make_float4(0.f, 0.f, 0.f, 0.f), -INFINITY);
     }
 }
 

@@ -16,7 +16,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 103;
+constexpr int kVersion = 104;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -29,6 +29,8 @@ std::atomic<int64_t> g_launches{0};
 int64_t g_opt_grid_blocks = 0;   // 0 = two blocks per SM
 int64_t g_opt_tail_units = 4;    // ticketed units per thread block (0: one static range per block only)
 int64_t g_opt_static_frac = 224; // share of the work given to the static ranges, in 1/256
+int64_t g_opt_extend_stream_rows = 16;   // decode_attn_extend: Lq * (Hq / Hkv) up to this many rows go through the
+                                         // streaming (partition) kernel, more through the tcgen05 kernel; 0: never
 cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
 
 struct DeviceState {
@@ -303,7 +305,7 @@ int set_kernel_attrs()
 }
 
 int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const Dims &d, uint8_t *ws,
-                const WsLayout &lay, int nblocks, int n_tail, cudaStream_t stream, int tile_t = TILE_T)
+                const WsLayout &lay, int nblocks, int n_tail, cudaStream_t stream, int tile_t = TILE_T, int min_len = 0)
 {
     PlanParams pp;
     pp.seq_lens = static_cast<const int32_t *>(sl->data);
@@ -322,6 +324,7 @@ int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const 
     pp.P = (int32_t)d.P;
     pp.window = window;
     pp.tile_t = tile_t;
+    pp.min_len = min_len;
     pp.first_token = first_token;
     pp.n_static = nblocks;
     pp.n_tail_max = n_tail;
@@ -339,7 +342,8 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
                 const da_tensor *q,
                 const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl, int32_t window,
                 float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, int32_t first_token = 0,
-                bool kv8 = false, const float *k_scale = nullptr, const float *v_scale = nullptr)
+                bool kv8 = false, const float *k_scale = nullptr, const float *v_scale = nullptr, int Lq = 1,
+                int64_t q_sq = 0, int64_t o_sq = 0, int64_t l_sq = 0)
 {
     int rc;
     if (!st->attrs_set) {
@@ -358,7 +362,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     rc = get_tmap(v, box_rows, kv8 ? 0 : 2, &tm_v);
     if (rc != DA_OK) return rc;
 
-    rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream, tile_t);
+    rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream, tile_t, Lq > 1 ? Lq : 0);
     if (rc != DA_OK) return rc;
 
     PartParams pa;
@@ -389,7 +393,12 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pa.scale_log2 = scale * LOG2E;
     pa.k_scale = k_scale;
     pa.v_scale = v_scale;
-    const int nt8 = d.G <= 8 ? 1 : 2;
+    pa.Lq = Lq;
+    pa.Gv = (int32_t)(Lq * d.G);
+    pa.q_sq = q_sq;
+    pa.o_sq = o_sq;
+    pa.l_sq = l_sq;
+    const int nt8 = pa.Gv <= 8 ? 1 : 2;
     const bool timed = g_ev_before && g_ev_after;
     if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
     // Both dependent kernels are launched with programmatic stream serialization: their blocks may
@@ -438,6 +447,10 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     mp.G = pa.G;
     mp.heads_pad = nt8 * 8;
     mp.out_bf16 = pa.out_bf16;
+    mp.Lq = pa.Lq;
+    mp.Gv = pa.Gv;
+    mp.o_sq = o_sq;
+    mp.l_sq = l_sq;
     cfg.gridDim = dim3((unsigned)(4 * st->sm_count));
     cfg.blockDim = dim3((unsigned)MERGE_THREADS);
     cfg.dynamicSmemBytes = 0;
@@ -804,6 +817,24 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
         DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
         st->attrs_set = true;
     }
+    if (Lq * G <= g_opt_extend_stream_rows && Lq * G <= kMaxGroup) {
+        // A few new tokens (speculated tokens, short appends): their Lq * G query rows per KV head ride
+        // through the streaming kernels as one wider group, at the HBM rate of decode_attn(); the
+        // tensor-core kernel below would fill only Lq * G of its 128 rows.
+        Dims d;
+        d.B = B; d.Hq = Hq; d.Hkv = Hkv; d.G = G; d.P = P; d.num_pages = k_pages->shape[0]; d.max_pages = max_pages;
+        da_tensor q3 = *q, o3 = *out, l3;
+        q3.ndim = 3; q3.shape[1] = Hq; q3.shape[2] = HEAD_DIM; q3.stride[1] = q->stride[2]; q3.stride[2] = 1;
+        o3.ndim = 3; o3.shape[1] = Hq; o3.shape[2] = HEAD_DIM; o3.stride[1] = out->stride[2]; o3.stride[2] = 1;
+        if (lse) {
+            l3 = *lse;
+            l3.ndim = 2; l3.shape[1] = Hq; l3.stride[1] = lse->stride[2];
+        }
+        const int n_tail = tail_units_for(nblocks);
+        return launch_path(st, d, ws, lay, nblocks, n_tail, &q3, k_pages, v_pages, block_table, seq_lens, 0, scale, &o3,
+                           lse ? &l3 : nullptr, stream, 0, false, nullptr, nullptr, (int)Lq, q->stride[1], out->stride[1],
+                           lse ? lse->stride[1] : 0);
+    }
     const int box_rows = P < PF_TOK ? (int)P : PF_TOK;
     CUtensorMap tm_k, tm_v;
     rc = get_tmap(k_pages, box_rows, 1, &tm_k);
@@ -1088,6 +1119,11 @@ int decode_attn_set_option(const char *name, int64_t value)
         g_opt_static_frac = value;
         return DA_OK;
     }
+    if (std::strcmp(name, "extend_stream_rows") == 0) {
+        if (value < 0 || value > kMaxGroup) return DA_ERR_UNSUPPORTED;
+        g_opt_extend_stream_rows = value;
+        return DA_OK;
+    }
     return DA_ERR_UNSUPPORTED;
 }
 
@@ -1098,6 +1134,7 @@ int64_t decode_attn_get_option(const char *name)
     if (std::strcmp(name, "grid_blocks") == 0) return g_opt_grid_blocks;
     if (std::strcmp(name, "tail_units") == 0) return g_opt_tail_units;
     if (std::strcmp(name, "static_frac") == 0) return g_opt_static_frac;
+    if (std::strcmp(name, "extend_stream_rows") == 0) return g_opt_extend_stream_rows;
     return -1;
 }
 

@@ -93,3 +93,57 @@ def test_extend_errors(da):
     out, lse = da.decode_attn_extend(q, case.k_pages, case.v_pages, case.block_table, sl, 1.0)
     assert da.read_device_status()[0] == 2
     assert (out[0] == 0).all()
+
+
+# ------------------------------------------------------------------ a few new tokens: the streaming path
+
+@pytest.mark.parametrize("Hq,Hkv,Lq", [(48, 8, 2), (8, 8, 16), (16, 8, 8), (32, 8, 4), (32, 8, 3), (24, 8, 5), (48, 8, 1)])
+@pytest.mark.parametrize("P", [16, 64])
+def test_few_new_tokens_stream_and_tensor_core_paths_agree_with_the_oracle(da, Hq, Hkv, Lq, P):
+    """Lq * (Hq / Hkv) <= 16 query rows per KV head go through the plan / partition / merge kernels as one
+    wider group (per-column causal limits); option extend_stream_rows = 0 forces the tcgen05 kernel."""
+    lens = [Lq, Lq + 1, 15 + Lq, 16 + Lq, 63 + Lq, 64 + Lq, 65 + Lq, 1000, 0, 2500]
+    lens = [L if L == 0 else max(L, Lq) for L in lens]
+    try:
+        for rows, grid in ((16, 0), (16, 1), (16, 7), (0, 0)):
+            da.set_option("extend_stream_rows", rows)
+            da.set_option("grid_blocks", grid)
+            got, got_lse, ref, ref_lse = run_case(da, lens, Lq, P, 5 * Lq + P + Hq, Hq=Hq, Hkv=Hkv, poison=True,
+                                                  pool_pages=400 if P == 16 else 120, pad_table_to=170 if P == 16 else 50)
+            assert np.isfinite(got[[i for i, L in enumerate(lens) if L]]).all()
+            assert_close(got, ref, f"few tokens rows={rows} grid={grid} out")
+            assert_close(got_lse, ref_lse, f"few tokens rows={rows} grid={grid} lse")
+            assert (got[8] == 0).all() and np.isneginf(got_lse[8]).all()
+    finally:
+        da.set_option("extend_stream_rows", 16)
+        da.set_option("grid_blocks", 0)
+
+
+def test_few_new_tokens_bf16_out_strided_views_and_errors(da):
+    lens, Lq = [300, 70, 2, 1030], 2
+    case = workloads.build_case("extv", lens, 16, 91, "cpu")
+    q = torch.randn((4, Lq, 48, 128), generator=torch.Generator().manual_seed(2)).to(torch.bfloat16)
+    ref, ref_lse = oracle.extend_attn_oracle(q, case.k_pages, case.v_pages, case.block_table, case.seq_lens, case.scale)
+    dev = workloads.to_device(case, "cuda")
+    q_big = torch.zeros((4, Lq + 1, 50, 256), dtype=torch.bfloat16, device="cuda")
+    q_view = q_big[:, 1:, 1:49, :128]
+    q_view.copy_(q)
+    out_big = torch.full((4, Lq, 48, 384), 7.0, device="cuda")
+    out_view = out_big[..., 128:256]
+    lse_big = torch.full((Lq, 4, 48), 7.0, device="cuda")
+    lse_view = lse_big.permute(1, 0, 2)
+    da.decode_attn_extend(q_view, dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, dev.scale, out=out_view, lse=lse_view)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    assert_close(out_view.cpu().numpy(), ref, "strided out")
+    assert_close(lse_view.cpu().numpy(), ref_lse, "strided lse")
+    assert (out_big[..., :128] == 7).all() and (out_big[..., 256:] == 7).all()
+    out16, _ = da.decode_attn_extend(q.cuda(), dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, dev.scale,
+                                     out_dtype=torch.bfloat16)
+    assert_bf16_close(out16.float().cpu().numpy().astype(np.float64), ref, "bf16 out")
+    sl = dev.seq_lens.clone()
+    sl[1] = 1                                # fewer tokens than the query block
+    out, lse = da.decode_attn_extend(q.cuda(), dev.k_pages, dev.v_pages, dev.block_table, sl, dev.scale)
+    st = da.read_device_status()
+    assert st[0] == 2 and st[1] == 1
+    assert (out[1] == 0).all() and torch.isneginf(lse[1]).all()
+    assert_close(out[0].cpu().numpy(), ref[0], "other sequences are unaffected")
