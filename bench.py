@@ -36,7 +36,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the partition kernel, from the ncu
 # capture summarised in profiles/partition_kernel_<workload>.md; valid for that library version only.
-NCU_TRAFFIC = {("c2", 103): 2223345000 + 7984000}
+NCU_TRAFFIC = {("c2", 104): 2223380000 + 7997000}
+NCU_TRAFFIC_FP8 = {("c2", 104): 1112405000 + 6407000}   # profiles/partition_kernel_fp8_c2.md
 WORKLOAD_TEXT = {
     "c1": "c1: 1 seq x 512 tok, page 16, contiguous, seed 0, 3 keys x20",
     "c2": "c2: 64 seqs, len U[1024,16384], 48q/8kv heads, d128, page 16, permuted pool, seed 1",
@@ -350,7 +351,8 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "partition_kernel (8-bit cache)" if kv8 else "partition_kernel",
                 "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                "kernel_ms": kms, "traffic": None if kv8 else NCU_TRAFFIC.get((args.workload, da.version()))}
+                "kernel_ms": kms, "traffic": NCU_TRAFFIC_FP8.get((args.workload, da.version())) if kv8 else
+                NCU_TRAFFIC.get((args.workload, da.version()))}
     G_ = case.q.shape[1] // case.k_pages.shape[1]
     ext_stream = bool(Lq) and Lq * G_ <= da.get_option("extend_stream_rows")
     if ext_stream:
