@@ -272,8 +272,17 @@ def run_ours(args):
     launches0 = da.launch_count()
     t_all0 = torch.cuda.Event(enable_timing=True)
     t_all1 = torch.cuda.Event(enable_timing=True)
+    # --flush-l2: a 512 MB write between steps evicts the 126 MB L2 (for workloads whose inputs fit it or
+    # are partly re-read from it); the flush itself is outside every step's events
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=device) if args.flush_l2 else None
+
+    def flush():
+        if flush_buf is not None:
+            flush_buf.zero_()
+
     t_all0.record(stream)
     for i in range(K):
+        flush()
         starts[i].record(stream)
         step()
         stops[i].record(stream)
@@ -282,7 +291,7 @@ def run_ours(args):
     launches = da.launch_count() - launches0
     ms_total = t_all0.elapsed_time(t_all1)
     per_step = [a.elapsed_time(b) for a, b in zip(starts, stops)]
-    ms_per_step = ms_total / K
+    ms_per_step = sum(per_step) / K if args.flush_l2 else ms_total / K
 
     # ---- the partition kernel alone (the dominant kernel), bracketed inside the library
     kernel_ms = None
@@ -291,6 +300,7 @@ def run_ours(args):
         lib.decode_attn_set_profile_events.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
         durs = []
         for i in range(K):
+            flush()
             lib.decode_attn_set_profile_events(kev0[i].cuda_event, kev1[i].cuda_event)
             step()
         lib.decode_attn_set_profile_events(None, None)
@@ -331,13 +341,24 @@ def run_ours(args):
     for _ in range(3):
         e2e_step()
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(K):
-        e2e_step()
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1) / K
+    if args.flush_l2:
+        ee0 = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+        ee1 = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+        for i in range(K):
+            flush()
+            ee0[i].record(stream)
+            e2e_step()
+            ee1[i].record(stream)
+        barrier()
+        e2e_ms = sum(a.elapsed_time(b) for a, b in zip(ee0, ee1)) / K
+    else:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(K):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / K
     assert torch.equal(out_h, out.cpu()), "host-io result differs from the device-resident call"
 
     gbs, seqs, ms = aggregate_replicas(nbytes, case.B, ms_per_step, device)
@@ -391,7 +412,8 @@ def run_ours(args):
         "dtype": "fp8 e4m3 (f32 accumulate)" if kv8 else "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD_TEXT[args.workload] + kv_text(args), "sequences": case.B,
                    "attended_tokens": int(case.attended_tokens().sum()), "algorithmic_bytes": nbytes,
-                   "l2": "inputs exceed L2 (no flush)" if nbytes > 4 * 126e6 else "inputs fit L2; not flushed",
+                   "l2": ("flushed between steps (512 MB write, outside the timed events)" if args.flush_l2 else
+                          ("inputs exceed L2 (no flush)" if nbytes > 4 * 126e6 else "inputs fit L2; not flushed")),
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "grid_blocks": da.get_option("grid_blocks"),
                    "path": (f"decode_attn_extend, {Lq} new tokens per sequence (causal, " +
@@ -428,6 +450,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extend", type=int, default=0, metavar="LQ",
                     help="time decode_attn_extend with LQ new (causal) query tokens per sequence instead of decode_attn")
+    ap.add_argument("--flush-l2", action="store_true",
+                    help="write 512 MB between steps so that every step starts with a cold L2 (c1, c5a, c5b)")
     ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
                     help="cache element type: bf16 (decode_attn, the headline) or fp8 (decode_attn_fp8kv)")
     ap.add_argument("--cascade", action="store_true",
