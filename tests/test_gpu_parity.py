@@ -142,6 +142,20 @@ def test_all_sequences_empty(da):
     assert (got == 0).all() and np.isneginf(got_lse).all()
 
 
+@pytest.mark.parametrize("B", [1025, 1500, 4096, 4097, 6000])
+def test_many_sequences(da, B):
+    """Batches beyond one pass of the plan kernel's scan (1024 sequences) and beyond what its shared
+    memory holds (4096: the work units are then cut from the global copy of the prefix)."""
+    rng = np.random.default_rng(B)
+    lens = rng.integers(0, 150, size=B)
+    lens[rng.integers(0, B, size=5)] = 700
+    case = workloads.build_case("many", lens, 16, B, "cpu")
+    for grid in (0, 3):
+        got, got_lse = check(da, case, f"B={B} grid={grid}", grid)
+    for b in np.nonzero(lens == 0)[0][:20]:
+        assert (got[b] == 0).all() and np.isneginf(got_lse[b]).all()
+
+
 def test_token_major_layout(da):
     case = workloads.build_case("tm", [513, 40, 1300], 16, 21, "cpu", layout="token_major")
     assert case.k_pages.stride(1) < case.k_pages.stride(2)
