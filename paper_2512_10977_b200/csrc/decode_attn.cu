@@ -481,6 +481,17 @@ int run(const da_tensor *q, const da_tensor *k, const da_tensor *v, const da_ten
                        out, lse, stream, 0, kv8, k_scale, v_scale);
 }
 
+// The device-side address of a pinned, mapped host buffer (NULL for pageable or unknown memory).
+void *mapped_device_pointer(const void *host_ptr)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host_ptr) != cudaSuccess) {
+        cudaGetLastError();   // not an error of the call being made
+        return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 bool contiguous(const da_tensor *t)
 {
     int64_t expect = 1;
@@ -950,16 +961,24 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
     qd.data = ws + lay.stg_q;
     btd.data = ws + lay.stg_bt;
     sld.data = ws + lay.stg_sl;
-    od.data = ws + lay.stg_out;
+    // Results: when the host buffers are pinned and mapped into the device's address space the kernels
+    // write them directly (the stores travel while the rest of the batch is still streaming, and no
+    // copy is queued after the kernels); otherwise they go to staging and are copied back.
+    void *out_dev = mapped_device_pointer(out_host->data);
+    void *lse_dev = lse_host ? mapped_device_pointer(lse_host->data) : nullptr;
+    const bool direct = out_dev && (!lse_host || lse_dev);
+    od.data = direct ? out_dev : ws + lay.stg_out;
     if (lse_host) {
         ld = *lse_host;
-        ld.data = ws + lay.stg_lse;
+        ld.data = direct ? lse_dev : ws + lay.stg_lse;
     }
     rc = run(&qd, k_pages, v_pages, &btd, &sld, window, scale, &od, lse_host ? &ld : nullptr, stream);
     if (rc != DA_OK) return rc;
-    DA_CUDA(cudaMemcpyAsync(out_host->data, ws + lay.stg_out, (size_t)d.B * d.Hq * HEAD_DIM * out_item, cudaMemcpyDeviceToHost, stream));
-    if (lse_host)
-        DA_CUDA(cudaMemcpyAsync(lse_host->data, ws + lay.stg_lse, (size_t)d.B * d.Hq * 4, cudaMemcpyDeviceToHost, stream));
+    if (!direct) {
+        DA_CUDA(cudaMemcpyAsync(out_host->data, ws + lay.stg_out, (size_t)d.B * d.Hq * HEAD_DIM * out_item, cudaMemcpyDeviceToHost, stream));
+        if (lse_host)
+            DA_CUDA(cudaMemcpyAsync(lse_host->data, ws + lay.stg_lse, (size_t)d.B * d.Hq * 4, cudaMemcpyDeviceToHost, stream));
+    }
     return DA_OK;
 }
 

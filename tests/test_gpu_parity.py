@@ -218,6 +218,33 @@ def test_host_io_matches_device_call(da):
         assert torch.equal(out_h, want.cpu()) and torch.equal(lse_h, want_lse.cpu())
 
 
+def test_host_io_with_pageable_buffers_takes_the_staged_path(da):
+    case = workloads.build_case("hostio2", [700, 33, 2100, 1, 0], 16, 38, "cpu")
+    dev = workloads.to_device(case, "cuda")
+    want, want_lse = da.decode_attn(dev.q, dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, 0, dev.scale)
+    out_h = torch.full(case.q.shape, 5.0, dtype=torch.float32)            # pageable
+    lse_h = torch.full(case.q.shape[:2], 5.0, dtype=torch.float32)
+    da.decode_attn_host_io(case.q, dev.k_pages, dev.v_pages, case.block_table, case.seq_lens, 0, dev.scale, out_h, lse_h)
+    torch.cuda.synchronize()
+    assert torch.equal(out_h, want.cpu()) and torch.equal(lse_h, want_lse.cpu())
+    # pinned out, pageable lse: still staged (both must be mapped for direct writes)
+    out_p = torch.full(case.q.shape, 5.0, dtype=torch.float32).pin_memory()
+    lse_h.fill_(5)
+    da.decode_attn_host_io(case.q, dev.k_pages, dev.v_pages, case.block_table, case.seq_lens, 0, dev.scale, out_p, lse_h)
+    torch.cuda.synchronize()
+    assert torch.equal(out_p, want.cpu()) and torch.equal(lse_h, want_lse.cpu())
+    # bf16 results written directly into pinned memory
+    out_b = torch.zeros(case.q.shape, dtype=torch.bfloat16).pin_memory()
+    lse_p = torch.zeros(case.q.shape[:2], dtype=torch.float32).pin_memory()
+    da.decode_attn_host_io(case.q.pin_memory(), dev.k_pages, dev.v_pages, case.block_table.pin_memory(),
+                           case.seq_lens.pin_memory(), 0, dev.scale, out_b, lse_p)
+    torch.cuda.synchronize()
+    want_b, _ = da.decode_attn(dev.q, dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, 0, dev.scale,
+                               out_dtype=torch.bfloat16)
+    assert torch.equal(out_b, want_b.cpu()) and torch.equal(lse_p, want_lse.cpu())
+    assert da.read_device_status() == (0, 0, 0, 0)
+
+
 # ------------------------------------------------------------------ indexing, bit-exact
 
 def _probe_case(P, lens, window, seed):
