@@ -221,7 +221,8 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
  * asynchronous; they must stay valid until the stream reaches the end of the call); k_pages and
  * v_pages stay DEVICE views (the cache is resident state).  The inputs are staged into the
  * registered workspace with cudaMemcpyAsync, decode_attn() runs on the staged copies, and out/lse
- * are copied back, all on `stream`, without synchronising.  Host views must be contiguous.  If out
+ * are copied back, all on `stream`, without synchronising.  Host views must be contiguous.  Pinned,
+ * mapped input buffers are gathered into the staging area by one kernel instead of three copies.  If out
  * and lse are pinned memory that is mapped into the device's address space (cudaHostAlloc /
  * cudaHostRegister under unified addressing, which is what torch's pin_memory() gives), the kernels
  * write them directly instead of going through staging and a copy; the results are complete when

@@ -1386,4 +1386,34 @@ __global__ void __launch_bounds__(256) append8_kernel(const Append8Params p)
     }
 }
 
+// =====================================================================================  host-input staging
+// decode_attn_host_io: the three per-step inputs (q, block table, lengths) are read straight out of the
+// caller's pinned, mapped host buffers by all SMs at once and written to the staging area -- one launch
+// instead of three DMA copies, each of which costs several microseconds before its first byte moves.
+struct StageParams {
+    const uint8_t *src[3];
+    uint8_t *dst[3];
+    unsigned long long bytes[3];   // multiples of 4
+};
+
+__global__ void __launch_bounds__(256) stage_inputs_kernel(const StageParams p)
+{
+    const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, nthr = (size_t)gridDim.x * blockDim.x;
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        const uint8_t *s = p.src[r];
+        uint8_t *d = p.dst[r];
+        const size_t n = p.bytes[r];
+        size_t done = 0;
+        if (((reinterpret_cast<uintptr_t>(s) | reinterpret_cast<uintptr_t>(d)) & 15u) == 0) {
+            const size_t n16 = n / 16;
+            for (size_t i = tid; i < n16; i += nthr)
+                reinterpret_cast<uint4 *>(d)[i] = reinterpret_cast<const uint4 *>(s)[i];
+            done = n16 * 16;
+        }
+        for (size_t i = done / 4 + tid; i < n / 4; i += nthr)
+            reinterpret_cast<uint32_t *>(d)[i] = reinterpret_cast<const uint32_t *>(s)[i];
+    }
+}
+
 }  // namespace da

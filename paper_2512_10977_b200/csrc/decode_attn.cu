@@ -954,9 +954,32 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
     }
     if (d.B == 0) return DA_OK;
     const size_t out_item = out_host->dtype == DA_BF16 ? 2 : 4;
-    DA_CUDA(cudaMemcpyAsync(ws + lay.stg_q, q_host->data, (size_t)d.B * d.Hq * HEAD_DIM * 2, cudaMemcpyHostToDevice, stream));
-    DA_CUDA(cudaMemcpyAsync(ws + lay.stg_bt, block_table_host->data, (size_t)d.B * d.max_pages * 4, cudaMemcpyHostToDevice, stream));
-    DA_CUDA(cudaMemcpyAsync(ws + lay.stg_sl, seq_lens_host->data, (size_t)d.B * 4, cudaMemcpyHostToDevice, stream));
+    // Inputs: from pinned, mapped host buffers one kernel gathers all three into the staging area;
+    // from other memory, three copies.
+    {
+        const size_t nb[3] = {(size_t)d.B * d.Hq * HEAD_DIM * 2, (size_t)d.B * d.max_pages * 4, (size_t)d.B * 4};
+        const void *hp[3] = {q_host->data, block_table_host->data, seq_lens_host->data};
+        const size_t at[3] = {lay.stg_q, lay.stg_bt, lay.stg_sl};
+        StageParams sp;
+        bool all_mapped = true;
+        for (int r = 0; r < 3; ++r) {
+            sp.src[r] = static_cast<const uint8_t *>(mapped_device_pointer(hp[r]));
+            sp.dst[r] = ws + at[r];
+            sp.bytes[r] = nb[r];
+            all_mapped = all_mapped && sp.src[r] != nullptr && (reinterpret_cast<uintptr_t>(sp.src[r]) & 3u) == 0;
+        }
+        if (all_mapped) {
+            int dev = 0, sms = 148;
+            DA_CUDA(cudaGetDevice(&dev));
+            if (dev >= 0 && dev < kMaxDevices && g_dev[dev].sm_count > 0) sms = g_dev[dev].sm_count;
+            stage_inputs_kernel<<<(unsigned)(2 * sms), 256, 0, stream>>>(sp);
+            g_launches.fetch_add(1);
+            DA_CUDA(cudaGetLastError());
+        } else {
+            for (int r = 0; r < 3; ++r)
+                DA_CUDA(cudaMemcpyAsync(ws + at[r], hp[r], nb[r], cudaMemcpyHostToDevice, stream));
+        }
+    }
     da_tensor qd = *q_host, btd = *block_table_host, sld = *seq_lens_host, od = *out_host, ld;
     qd.data = ws + lay.stg_q;
     btd.data = ws + lay.stg_bt;
