@@ -7,11 +7,13 @@
 // prefix_kernel: one block = 128 query rows (row = b * G + head-in-group) of one KV head and one
 // range of 128-token KV tiles.  Per tile:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in TMEM)
 // -> the sixteen softmax warps read their rows of S (four threads per row, 32 columns each), keep running
-// max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts into tensor memory
-// -> O += P_hi V + P_lo V (tcgen05.mma with the A operand in TMEM, accumulating in another TMEM region) -> the softmax
-// threads rescale a row of O in TMEM only when its maximum has grown by more than 2^8 (rare).  A ninth warp
-// issues the MMAs and a tenth the TMA loads (one warp doing both spent most of a tile's time issuing).  Result: a normalised partial (O / l, lse) per (split, b, h),
-// combined with the per-sequence suffix attention by cascade_merge_kernel.
+// max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts over their scores in tensor
+// memory -> O += P_hi V + P_lo V (tcgen05.mma with the A operand in TMEM, accumulating in another TMEM
+// region) -> the softmax threads rescale a row of O in TMEM only when its maximum has grown by more than
+// 2^8 (rare).  One more warp issues the MMAs and two more the TMA loads, one for K and one for V (issuing a
+// tile's tensor copies is slow enough that one warp doing it all set the pace of the block).  Result: a
+// normalised partial (O / l, lse) per (split, b, h), combined with the per-sequence suffix attention by
+// cascade_merge_kernel.
 #pragma once
 #include "da_kernels.cuh"
 
