@@ -147,3 +147,26 @@ def test_few_new_tokens_bf16_out_strided_views_and_errors(da):
     assert st[0] == 2 and st[1] == 1
     assert (out[1] == 0).all() and torch.isneginf(lse[1]).all()
     assert_close(out[0].cpu().numpy(), ref[0], "other sequences are unaffected")
+
+
+# ------------------------------------------------------------------ the benchmark's configurations at full size
+
+@pytest.mark.parametrize("Lq", [2, 512])
+def test_c2_full_size_extend_sampled(da, Lq):
+    """c2's cache with Lq new tokens per sequence, as `bench.py --extend` times it; sampled sequences and
+    query tokens against the single-token oracle on a cache cut at each query's position."""
+    da.set_option("grid_blocks", 0)
+    case = workloads.c2("cuda")
+    B = case.B
+    q = torch.randn((B, Lq, 48, 128), device="cuda", generator=torch.Generator(device="cuda").manual_seed(7)).to(torch.bfloat16)
+    out, lse = da.decode_attn_extend(q, case.k_pages, case.v_pages, case.block_table, case.seq_lens, case.scale)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    assert torch.isfinite(out).all() and torch.isfinite(lse).all()
+    ids = sorted({int(np.argmin(case.lens)), int(np.argmax(case.lens)), 17})
+    sub = workloads.host_subcase(case, ids)
+    for qi in sorted({0, Lq // 2, Lq - 1}):
+        cut = (sub.lens - Lq + qi + 1).astype(np.int32)
+        ref, ref_lse = oracle.decode_attn_oracle(q[ids, qi].cpu().contiguous(), sub.k_pages, sub.v_pages, sub.block_table,
+                                                 cut, 0, sub.scale)
+        assert_close(out[ids, qi].cpu().numpy(), ref, f"c2 extend Lq={Lq} qi={qi} out")
+        assert_close(lse[ids, qi].cpu().numpy(), ref_lse, f"c2 extend Lq={Lq} qi={qi} lse")
