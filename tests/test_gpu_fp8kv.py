@@ -384,3 +384,10 @@ def test_decode_loop_append_then_attend(da):
         assert_close(lse.cpu().numpy(), ref_lse, f"loop step {step} lse")
     assert da.read_device_status() == (0, 0, 0, 0)
     assert torch.equal(dev.k_pages.cpu(), case.k_pages) and torch.equal(dev.v_pages.cpu(), case.v_pages)
+
+
+def test_c3_scattered_in_large_pool_sampled(da):
+    da.set_option("grid_blocks", 0)
+    case = workloads.c3("cuda", kv_dtype="fp8")
+    ids = sorted({int(np.argmin(case.lens)), int(np.argmax(case.lens)), 5, 128, 255})
+    _sampled_full_size(da, case, ids, "c3 fp8")
