@@ -329,11 +329,9 @@ def run_ours(args):
             da.decode_attn_cascade(q_d, case.k_pages, case.v_pages, bt_d, sl_d, prefix, case.scale,
                                    out=out, lse=lse, stream=stream)
             out_h.copy_(out, non_blocking=True); lse_h.copy_(lse, non_blocking=True)
-        elif kv8:   # no host-io entry point for the 8-bit cache: same copies, made here on the same stream
-            q_d.copy_(q_h, non_blocking=True); bt_d.copy_(bt_h, non_blocking=True); sl_d.copy_(sl_h, non_blocking=True)
-            da.decode_attn_fp8kv(q_d, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt_d, sl_d,
-                                 case.window, case.scale, out=out, lse=lse, stream=stream)
-            out_h.copy_(out, non_blocking=True); lse_h.copy_(lse, non_blocking=True)
+        elif kv8:
+            da.decode_attn_fp8kv_host_io(q_h, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt_h, sl_h,
+                                         case.window, case.scale, out_h, lse_h, stream=stream)
         else:
             da.decode_attn_host_io(q_h, case.k_pages, case.v_pages, bt_h, sl_h, case.window, case.scale,
                                    out_h, lse_h, stream=stream)

@@ -233,6 +233,12 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
                         int32_t window, float scale, da_tensor *out_host, da_tensor *lse_host,
                         void *stream);
 
+/* The same for the 8-bit cache of decode_attn_fp8kv(): k_pages / v_pages and the factors stay on the DEVICE. */
+int decode_attn_fp8kv_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tensor *v_pages,
+                              const float *k_scale, const float *v_scale, const da_tensor *block_table_host,
+                              const da_tensor *seq_lens_host, int32_t window, float scale,
+                              da_tensor *out_host, da_tensor *lse_host, void *stream);
+
 /*
  * decode_attn_static_scratch -- decode_attn() for callers that cannot allocate device memory.
  * (The paper has no counterpart; this is a packaging variant of the same kernels.)

@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
             L.decode_attn_extend.argtypes = [T, T, T, T, T, ctypes.c_float, T, T, vp]
             L.decode_attn_host_io.restype = ctypes.c_int
             L.decode_attn_host_io.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_fp8kv_host_io.restype = ctypes.c_int
+            L.decode_attn_fp8kv_host_io.argtypes = [T, T, T, vp, vp, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_static_scratch.restype = ctypes.c_int
             L.decode_attn_static_scratch.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp, vp]
             L.decode_attn_workspace_bytes.restype = ctypes.c_size_t
@@ -279,6 +281,20 @@ def decode_attn_host_io(q_host, k_pages, v_pages, block_table_host, seq_lens_hos
         _check(lib().decode_attn_host_io(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
                                          int(window), float(scale), _ref(tv[5]), _ref(tv[6]),
                                          _stream_ptr(stream)))
+    return out_host, lse_host
+
+
+def decode_attn_fp8kv_host_io(q_host, k_pages, v_pages, k_scale, v_scale, block_table_host, seq_lens_host, window: int,
+                              scale: float, out_host, lse_host=None, stream: Optional[torch.cuda.Stream] = None):
+    """``decode_attn_host_io`` for the 8-bit cache (pools and factors on the device, per-step tensors on the host)."""
+    with torch.cuda.device(k_pages.device):
+        _auto_workspace(q_host, k_pages, block_table_host)
+        tv = [_view(t) for t in (q_host, k_pages, v_pages, block_table_host, seq_lens_host, out_host, lse_host)]
+        _check(lib().decode_attn_fp8kv_host_io(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]),
+                                               k_scale.data_ptr() if k_scale is not None else None,
+                                               v_scale.data_ptr() if v_scale is not None else None,
+                                               _ref(tv[3]), _ref(tv[4]), int(window), float(scale), _ref(tv[5]), _ref(tv[6]),
+                                               _stream_ptr(stream)))
     return out_host, lse_host
 
 

@@ -927,13 +927,18 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
     return DA_OK;
 }
 
-int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tensor *v_pages,
-                        const da_tensor *block_table_host, const da_tensor *seq_lens_host, int32_t window, float scale,
-                        da_tensor *out_host, da_tensor *lse_host, void *stream_)
+}  // extern "C"
+
+namespace {
+// decode_attn_host_io / decode_attn_fp8kv_host_io
+int run_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tensor *v_pages,
+                const da_tensor *block_table_host, const da_tensor *seq_lens_host, int32_t window, float scale,
+                da_tensor *out_host, da_tensor *lse_host, cudaStream_t stream, bool kv8, const float *k_scale,
+                const float *v_scale)
 {
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     Dims d;
-    int rc = validate(q_host, k_pages, v_pages, block_table_host, seq_lens_host, out_host, lse_host, &d);
+    int rc = validate(q_host, k_pages, v_pages, block_table_host, seq_lens_host, out_host, lse_host, &d,
+                      kv8 ? DA_FP8_E4M3 : DA_BF16);
     if (rc != DA_OK) return rc;
     if (!contiguous(q_host) || !contiguous(block_table_host) || !contiguous(seq_lens_host) || !contiguous(out_host) ||
         (lse_host && !contiguous(lse_host)))
@@ -994,7 +999,7 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
         ld = *lse_host;
         ld.data = direct ? lse_dev : ws + lay.stg_lse;
     }
-    rc = run(&qd, k_pages, v_pages, &btd, &sld, window, scale, &od, lse_host ? &ld : nullptr, stream);
+    rc = run(&qd, k_pages, v_pages, &btd, &sld, window, scale, &od, lse_host ? &ld : nullptr, stream, kv8, k_scale, v_scale);
     if (rc != DA_OK) return rc;
     if (!direct) {
         DA_CUDA(cudaMemcpyAsync(out_host->data, ws + lay.stg_out, (size_t)d.B * d.Hq * HEAD_DIM * out_item, cudaMemcpyDeviceToHost, stream));
@@ -1002,6 +1007,26 @@ int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const
             DA_CUDA(cudaMemcpyAsync(lse_host->data, ws + lay.stg_lse, (size_t)d.B * d.Hq * 4, cudaMemcpyDeviceToHost, stream));
     }
     return DA_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int decode_attn_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tensor *v_pages,
+                        const da_tensor *block_table_host, const da_tensor *seq_lens_host, int32_t window, float scale,
+                        da_tensor *out_host, da_tensor *lse_host, void *stream)
+{
+    return run_host_io(q_host, k_pages, v_pages, block_table_host, seq_lens_host, window, scale, out_host, lse_host,
+                       static_cast<cudaStream_t>(stream), false, nullptr, nullptr);
+}
+
+int decode_attn_fp8kv_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tensor *v_pages,
+                              const float *k_scale, const float *v_scale, const da_tensor *block_table_host,
+                              const da_tensor *seq_lens_host, int32_t window, float scale, da_tensor *out_host,
+                              da_tensor *lse_host, void *stream)
+{
+    return run_host_io(q_host, k_pages, v_pages, block_table_host, seq_lens_host, window, scale, out_host, lse_host,
+                       static_cast<cudaStream_t>(stream), true, k_scale, v_scale);
 }
 
 int decode_attn_static_scratch(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,

@@ -391,3 +391,24 @@ def test_c3_scattered_in_large_pool_sampled(da):
     case = workloads.c3("cuda", kv_dtype="fp8")
     ids = sorted({int(np.argmin(case.lens)), int(np.argmax(case.lens)), 5, 128, 255})
     _sampled_full_size(da, case, ids, "c3 fp8")
+
+
+def test_host_io_matches_device_call(da):
+    case = fp8_case("hostio8", [700, 33, 2100, 1, 0], 16, 37)
+    dev = workloads.to_device(case, "cuda")
+    want, want_lse = da.decode_attn_fp8kv(dev.q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, dev.block_table,
+                                          dev.seq_lens, 9, dev.scale)
+    q_h, bt_h, sl_h = (t.pin_memory() for t in (case.q, case.block_table, case.seq_lens))
+    out_h = torch.empty(case.q.shape, dtype=torch.float32).pin_memory()
+    lse_h = torch.empty(case.q.shape[:2], dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        out_h.fill_(5)
+        da.decode_attn_fp8kv_host_io(q_h, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, bt_h, sl_h, 9, dev.scale,
+                                     out_h, lse_h)
+        torch.cuda.synchronize()
+        assert torch.equal(out_h, want.cpu()) and torch.equal(lse_h, want_lse.cpu())
+    out_p = torch.full(case.q.shape, 5.0, dtype=torch.float32)     # pageable: the staged path
+    da.decode_attn_fp8kv_host_io(case.q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, case.block_table,
+                                 case.seq_lens, 9, dev.scale, out_p, None)
+    torch.cuda.synchronize()
+    assert torch.equal(out_p, want.cpu())
