@@ -106,10 +106,9 @@ def _view(t: Optional[torch.Tensor]) -> Optional[DaTensor]:
     d = DaTensor()
     d.data = t.data_ptr()
     d.dtype = _DTYPES[t.dtype]
-    d.ndim = t.dim()
-    for i in range(t.dim()):
-        d.shape[i] = t.shape[i]
-        d.stride[i] = t.stride(i)
+    n = d.ndim = t.dim()
+    d.shape[0:n] = tuple(t.shape)
+    d.stride[0:n] = t.stride()
     return d
 
 
@@ -117,8 +116,14 @@ def _ref(d: Optional[DaTensor]):
     return ctypes.byref(d) if d is not None else None
 
 
+_have_cuda = None
+
+
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
-    if not torch.cuda.is_available():
+    global _have_cuda
+    if _have_cuda is None:
+        _have_cuda = torch.cuda.is_available()
+    if not _have_cuda:
         raise RuntimeError("decode_attn needs a CUDA device; there is no CPU path")
     s = stream if stream is not None else torch.cuda.current_stream()
     return s.cuda_stream
@@ -132,8 +137,12 @@ def launch_count() -> int:
     return int(lib().decode_attn_launch_count())
 
 
+_ws_seen = {}   # (device, extents) -> bytes needed, for the current launch options
+
+
 def set_option(name: str, value: int) -> None:
     _check(lib().decode_attn_set_option(name.encode(), int(value)))
+    _ws_seen.clear()   # the workspace size depends on the launch options
 
 
 def get_option(name: str) -> int:
@@ -149,8 +158,14 @@ def ensure_workspace(B: int, Hq: int, Hkv: int, D: int, P: int, max_pages: int,
     """Make sure the current device has a registered workspace large enough for these extents.
     The buffer is a torch allocation owned here; the library only borrows the pointer."""
     dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    key = (dev.index, B, Hq, Hkv, D, P, max_pages)
+    need = _ws_seen.get(key)
+    cur = _workspaces.get(dev.index)
+    if need is not None and cur is not None and cur.numel() >= need:
+        return cur    # seen before with these options, and the registered buffer is large enough
     with torch.cuda.device(dev):
         need = workspace_bytes(B, Hq, Hkv, D, P, max_pages)
+        _ws_seen[key] = need
         cur = _workspaces.get(dev.index)
         if cur is None or cur.numel() < need:
             torch.cuda.synchronize()
