@@ -87,6 +87,7 @@ struct PartParams {
     float *part_lse;          // [2 * units][HEADS]
     int32_t *status;
     int32_t B, Hkv, G, P, box_rows, num_pages, out_bf16;
+    int32_t log2_P;           // P = 1 << log2_P
     float scale_log2;         // scale * log2(e)
     const float *k_scale, *v_scale;   // 8-bit cache: per-KV-head factors (NULL: 1)
     // Several new tokens per sequence (Lq > 1, causal among them): query token qi of KV group g's head hd
@@ -432,6 +433,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         int b = 0, g = 0, rel = 0, remaining = 0, cnt = 0, i = 0;
         int4 si = make_int4(0, 0, 0, 0);
         bool first_item = true;
+        const int box_tok = box * p.box_rows;   // this lane's first token within a tile
+        const int32_t *bt_row = p.block_table;  // block-table row of the cursor's sequence (set in open_pair)
         auto take_ticket = [&]() {
             int t = 0;
             if (lane == 0)
@@ -458,6 +461,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     if (si.w > 0) {
                         cnt = min(si.w - rel, remaining);
                         i = 0;
+                        bt_row = p.block_table + (int64_t)b * p.bt_sb;
                         return true;
                     }
                     ++b;   // an empty sequence (only reachable with g == 0)
@@ -470,12 +474,12 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         struct Tile { int page, row, t0, g, b, lo, L, flags, slot; bool need; };
         auto fetch = [&](Tile &t) {   // describe the cursor's tile and start its block-table read
             t.t0 = (si.z + rel + i) * TT;
-            const int tok0 = t.t0 + box * p.box_rows;
+            const int tok0 = t.t0 + box_tok;
             t.need = active && tok0 < si.y && tok0 + p.box_rows > si.x;
             t.page = 0;
-            t.row = tok0 % p.P;
+            t.row = tok0 & (p.P - 1);           // P is a power of two: no divisions in this loop
             if (t.need)
-                t.page = __ldg(p.block_table + (int64_t)b * p.bt_sb + tok0 / p.P);
+                t.page = __ldg(bt_row + (tok0 >> p.log2_P));
             t.g = g; t.b = b; t.lo = si.x; t.L = si.y;
             t.flags = (i == cnt - 1 ? TILE_ITEM_END : 0) | (cnt == si.w ? TILE_WHOLE : 0);
             t.slot = 2 * u + (first_item ? 0 : 1);

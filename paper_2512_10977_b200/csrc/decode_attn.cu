@@ -387,6 +387,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pa.Hkv = (int32_t)d.Hkv;
     pa.G = (int32_t)d.G;
     pa.P = (int32_t)d.P;
+    pa.log2_P = d.P == 16 ? 4 : (d.P == 32 ? 5 : (d.P == 64 ? 6 : 7));
     pa.box_rows = box_rows;
     pa.num_pages = (int32_t)d.num_pages;
     pa.out_bf16 = out->dtype == DA_BF16;
