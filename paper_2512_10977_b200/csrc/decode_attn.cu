@@ -16,7 +16,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 104;
+constexpr int kVersion = 105;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
