@@ -471,7 +471,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     return false;
             }
         };
-        struct Tile { int page, row, t0, g, b, lo, L, flags, slot; bool need; };
+        struct Tile { int page, row, t0, g, b, lo, L, flags, slot; bool need, valid; };
         auto fetch = [&](Tile &t) {   // describe the cursor's tile and start its block-table read
             t.t0 = (si.z + rel + i) * TT;
             const int tok0 = t.t0 + box_tok;
@@ -498,16 +498,18 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             return true;
         };
 
-        Tile cur, nxt;
-        bool have = open_unit() && open_pair();
-        if (have)
-            fetch(cur);
-        while (have) {
-            // issue the next tile's block-table read before waiting for a free stage
-            const bool n_have = advance();
-            if (n_have)
-                fetch(nxt);
-
+        // Three tile records in rotation: a tile is described (and its block-table entry requested) two
+        // tiles before its copies are issued, so that the entry has two tile periods to arrive, and no
+        // record is ever copied (copying a register with a load in flight would wait for the load).
+        bool cursor_ok = open_unit() && open_pair();
+        auto fill = [&](Tile &t) {   // describe the cursor's tile, then move the cursor on
+            t.valid = cursor_ok;
+            if (cursor_ok) {
+                fetch(t);
+                cursor_ok = advance();
+            }
+        };
+        auto issue = [&](Tile &cur) {   // the tile's descriptor and copies into the next free stage
             const int stage = it % NSTAGES;
             const uint32_t phase = (it / NSTAGES) & 1u;
             if (cur.need && (uint32_t)cur.page >= (uint32_t)p.num_pages) {
@@ -515,10 +517,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 cur.need = false;   // skip the load; the rows keep whatever the stage held
             }
             const uint32_t mask = __ballot_sync(0xffffffffu, cur.need);
-            if (!mbar_wait_bounded(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) {
-                aborted = true;
-                break;
-            }
+            if (!mbar_wait_bounded(bar_empty + 8 * stage, phase ^ 1u, abort_flag))
+                return false;
             if (lane == 0) {
                 meta[2 * stage] = make_int4(cur.b, cur.g, cur.t0, cur.flags);
                 meta[2 * stage + 1] = make_int4(cur.lo, cur.L, cur.slot, 0);
@@ -533,8 +533,21 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     tma_load_5d(dst, tm, 0, cur.row, 0, cur.g, cur.page, bar_full + 8 * stage);
             }
             ++it;
-            have = n_have;
-            cur = nxt;
+            return true;
+        };
+        Tile t0, t1, t2;
+        fill(t0);
+        fill(t1);
+        for (;;) {
+            fill(t2);
+            if (!t0.valid) break;
+            if (!issue(t0)) { aborted = true; break; }
+            fill(t0);
+            if (!t1.valid) break;
+            if (!issue(t1)) { aborted = true; break; }
+            fill(t1);
+            if (!t2.valid) break;
+            if (!issue(t2)) { aborted = true; break; }
         }
         if (!aborted) {
             // tell the consumers that nothing follows
