@@ -36,8 +36,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the partition kernel, from the ncu
 # capture summarised under profiles/ (one file per kernel and workload); valid for that library version only.
-NCU_TRAFFIC = {("c2", 106): 2223297000 + 8080000}
-NCU_TRAFFIC_FP8 = {("c2", 106): 1112420000 + 6245000}   # the 8-bit-cache kernel's capture
+NCU_TRAFFIC = {("c2", 107): 2223315000 + 7977000}
+NCU_TRAFFIC_FP8 = {("c2", 107): 1112425000 + 7460000}   # the 8-bit-cache kernel's capture
 WORKLOAD_TEXT = {
     "c1": "c1: 1 seq x 512 tok, page 16, contiguous, seed 0, 3 keys x20",
     "c2": "c2: 64 seqs, len U[1024,16384], 48q/8kv heads, d128, page 16, permuted pool, seed 1",

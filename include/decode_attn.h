@@ -216,6 +216,18 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
                        da_tensor *lse, void *stream);
 
 /*
+ * decode_attn_fp8kv_extend -- decode_attn_extend() over the 8-bit cache of decode_attn_fp8kv(), for a
+ * few new tokens per sequence (speculated tokens): Lq * Hq / Hkv must not exceed 16 (else
+ * DA_ERR_UNSUPPORTED: longer query blocks need the tensor-core kernel, which reads a bf16 cache).
+ * Runs on the streaming kernels with per-column causal limits.  Arguments as decode_attn_extend()
+ * and decode_attn_fp8kv().
+ */
+int decode_attn_fp8kv_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                             const float *k_scale, const float *v_scale, const da_tensor *block_table,
+                             const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse,
+                             void *stream);
+
+/*
  * decode_attn_host_io -- the same call for a caller whose per-step tensors are in HOST memory.
  * q, block_table, seq_lens, out and lse are HOST views (pinned memory makes the copies
  * asynchronous; they must stay valid until the stream reaches the end of the call); k_pages and

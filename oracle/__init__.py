@@ -280,3 +280,19 @@ def kv_append_fp8_oracle(k_new, v_new, k_pages, v_pages, k_scale, v_scale, block
                                   bt.ctypes.data, bt.shape[1], sl.ctypes.data)
     if rc != 0:
         raise RuntimeError(f"kv_append_fp8_oracle failed with code {rc}")
+
+
+def extend_attn_fp8kv_oracle(q, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens, scale: float,
+                             num_threads: int = 0):
+    """``extend_attn_oracle`` over the 8-bit cache: query qi of sequence b is single-token attention over a
+    cache cut to L_b - Lq + qi + 1 tokens.  q: bf16 [B, Lq, Hq, D]."""
+    B, Lq, Hq, D = q.shape
+    sl = np.asarray(seq_lens, dtype=np.int64)
+    out = np.zeros((B, Lq, Hq, D))
+    lse = np.full((B, Lq, Hq), -np.inf)
+    for qi in range(Lq):
+        cut = np.where(sl > 0, sl - Lq + qi + 1, 0).astype(np.int32)
+        o, l = decode_attn_fp8kv_oracle(q[:, qi].contiguous(), k_pages, v_pages, k_scale, v_scale, block_table, cut,
+                                        0, scale, num_threads)
+        out[:, qi], lse[:, qi] = o, l
+    return out, lse

@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
             L.decode_attn_append.argtypes = [T, T, T, T, T, T, vp]
             L.decode_attn_extend.restype = ctypes.c_int
             L.decode_attn_extend.argtypes = [T, T, T, T, T, ctypes.c_float, T, T, vp]
+            L.decode_attn_fp8kv_extend.restype = ctypes.c_int
+            L.decode_attn_fp8kv_extend.argtypes = [T, T, T, vp, vp, T, T, ctypes.c_float, T, T, vp]
             L.decode_attn_host_io.restype = ctypes.c_int
             L.decode_attn_host_io.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_fp8kv_host_io.restype = ctypes.c_int
@@ -283,6 +285,26 @@ def decode_attn_extend(q, k_pages, v_pages, block_table, seq_lens, scale: float,
         tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
         _check(lib().decode_attn_extend(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
                                         float(scale), _ref(tv[5]), _ref(tv[6]), _stream_ptr(stream)))
+    return out, lse
+
+
+def decode_attn_fp8kv_extend(q, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens, scale: float,
+                             out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                             stream: Optional[torch.cuda.Stream] = None, out_dtype=torch.float32):
+    """``decode_attn_extend`` over the 8-bit cache, for a few new tokens (Lq * Hq / Hkv <= 16)."""
+    if out is None:
+        out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    with torch.cuda.device(k_pages.device):
+        ensure_workspace(q.shape[0], q.shape[2], k_pages.shape[1], q.shape[3], k_pages.shape[2],
+                         block_table.shape[1], k_pages.device)
+        tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
+        _check(lib().decode_attn_fp8kv_extend(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]),
+                                              k_scale.data_ptr() if k_scale is not None else None,
+                                              v_scale.data_ptr() if v_scale is not None else None,
+                                              _ref(tv[3]), _ref(tv[4]), float(scale), _ref(tv[5]), _ref(tv[6]),
+                                              _stream_ptr(stream)))
     return out, lse
 
 

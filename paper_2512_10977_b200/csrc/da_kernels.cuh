@@ -788,6 +788,20 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         if (!ob1) sb[n][2] = sb[n][3] = -INFINITY;
                     }
                 }
+                if (p.Lq > 1 && a + 32 > L - p.Lq + 1) {
+                    // several new tokens: the query of column (virtual head) v attends tokens below
+                    // L - Lq + v / G + 1 only
+#pragma unroll
+                    for (int n = 0; n < NT8; ++n)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int lim = L - p.Lq + (n * 8 + 2 * c + e) / p.G + 1;
+                            if (a + t_a0 >= lim) sa[n][e] = -INFINITY;
+                            if (a + t_a1 >= lim) sa[n][2 + e] = -INFINITY;
+                            if (a + 16 + t_a0 >= lim) sb[n][e] = -INFINITY;
+                            if (a + 16 + t_a1 >= lim) sb[n][2 + e] = -INFINITY;
+                        }
+                }
                 // ---- online softmax in the log2 domain: column (head) maxima over the 32 tokens
                 float mx[NT8][2];
                 bool grew = false;
@@ -830,10 +844,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
                 for (int n = 0; n < NT8; ++n) {
                     float w[8];
+                    // (a column that has seen no token yet keeps m = -inf: exp2(-inf) = 0, not NaN)
+                    const float mu[2] = {m_run[n][0] == -INFINITY ? 0.f : m_run[n][0] - P8_SHIFT,
+                                         m_run[n][1] == -INFINITY ? 0.f : m_run[n][1] - P8_SHIFT};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        w[e] = fast_exp2(sa[n][e] - m_run[n][e & 1] + P8_SHIFT);
-                        w[4 + e] = fast_exp2(sb[n][e] - m_run[n][e & 1] + P8_SHIFT);
+                        w[e] = fast_exp2(sa[n][e] - mu[e & 1]);
+                        w[4 + e] = fast_exp2(sb[n][e] - mu[e & 1]);
                     }
                     l_run[n][0] += (w[0] + w[2]) + (w[4] + w[6]);
                     l_run[n][1] += (w[1] + w[3]) + (w[5] + w[7]);

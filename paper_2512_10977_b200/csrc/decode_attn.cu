@@ -16,7 +16,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 106;
+constexpr int kVersion = 107;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -779,10 +779,14 @@ int decode_attn_append_fp8kv(const da_tensor *k_new, const da_tensor *v_new, da_
     return DA_OK;
 }
 
-int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
-                       const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse, void *stream_)
+}  // extern "C"
+
+namespace {
+// decode_attn_extend / decode_attn_fp8kv_extend
+int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
+               const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, bool kv8,
+               const float *k_scale, const float *v_scale)
 {
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return DA_ERR_NULL;
     if (!q->data || !block_table->data || !seq_lens->data || !out->data || (lse && !lse->data)) return DA_ERR_NULL;
     if (q->dtype != DA_BF16 || block_table->dtype != DA_I32 || seq_lens->dtype != DA_I32) return DA_ERR_DTYPE;
@@ -790,9 +794,9 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
     if (lse && lse->dtype != DA_F32) return DA_ERR_DTYPE;
     if (q->ndim != 4 || out->ndim != 4 || block_table->ndim != 2 || seq_lens->ndim != 1 || (lse && lse->ndim != 3))
         return DA_ERR_SHAPE;
-    int rc = check_pool(k_pages);
+    int rc = check_pool(k_pages, kv8 ? DA_FP8_E4M3 : DA_BF16);
     if (rc != DA_OK) return rc;
-    rc = check_pool(v_pages);
+    rc = check_pool(v_pages, kv8 ? DA_FP8_E4M3 : DA_BF16);
     if (rc != DA_OK) return rc;
     for (int i = 0; i < 4; ++i)
         if (k_pages->shape[i] != v_pages->shape[i]) return DA_ERR_SHAPE;
@@ -828,7 +832,7 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
         DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
         st->attrs_set = true;
     }
-    if (Lq * G <= g_opt_extend_stream_rows && Lq * G <= kMaxGroup) {
+    if ((Lq * G <= g_opt_extend_stream_rows || kv8) && Lq * G <= kMaxGroup) {
         // A few new tokens (speculated tokens, short appends): their Lq * G query rows per KV head ride
         // through the streaming kernels as one wider group, at the HBM rate of decode_attn(); the
         // tensor-core kernel below would fill only Lq * G of its 128 rows.
@@ -843,9 +847,11 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
         }
         const int n_tail = tail_units_for(nblocks);
         return launch_path(st, d, ws, lay, nblocks, n_tail, &q3, k_pages, v_pages, block_table, seq_lens, 0, scale, &o3,
-                           lse ? &l3 : nullptr, stream, 0, false, nullptr, nullptr, (int)Lq, q->stride[1], out->stride[1],
+                           lse ? &l3 : nullptr, stream, 0, kv8, k_scale, v_scale, (int)Lq, q->stride[1], out->stride[1],
                            lse ? lse->stride[1] : 0);
     }
+    if (kv8)
+        return DA_ERR_UNSUPPORTED;   // the tensor-core kernel reads a bf16 cache only
     const int box_rows = P < PF_TOK ? (int)P : PF_TOK;
     CUtensorMap tm_k, tm_v;
     rc = get_tmap(k_pages, box_rows, 1, &tm_k);
@@ -926,6 +932,24 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
         DA_CUDA(cudaGetLastError());
     }
     return DA_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
+                       const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse, void *stream)
+{
+    return run_extend(q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, static_cast<cudaStream_t>(stream), false,
+                      nullptr, nullptr);
+}
+
+int decode_attn_fp8kv_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const float *k_scale,
+                             const float *v_scale, const da_tensor *block_table, const da_tensor *seq_lens, float scale,
+                             da_tensor *out, da_tensor *lse, void *stream)
+{
+    return run_extend(q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, static_cast<cudaStream_t>(stream), true,
+                      k_scale, v_scale);
 }
 
 }  // extern "C"

@@ -412,3 +412,32 @@ def test_host_io_matches_device_call(da):
                                  case.seq_lens, 9, dev.scale, out_p, None)
     torch.cuda.synchronize()
     assert torch.equal(out_p, want.cpu())
+
+
+# ------------------------------------------------------------------ a few new tokens over the 8-bit cache
+
+@pytest.mark.parametrize("Hq,Hkv,Lq", [(48, 8, 2), (8, 8, 16), (16, 8, 8), (32, 8, 3), (24, 8, 5), (48, 8, 1)])
+@pytest.mark.parametrize("P", [16, 64])
+def test_few_new_tokens_over_the_fp8_cache(da, Hq, Hkv, Lq, P):
+    lens = [Lq, Lq + 1, 31 + Lq, 32 + Lq, 127 + Lq, 128 + Lq, 129 + Lq, 1000, 0, 2500]
+    lens = [L if L == 0 else max(L, Lq) for L in lens]
+    case = fp8_case("ext8", lens, P, 7 * Lq + P + Hq, Hq=Hq, Hkv=Hkv, poison=True,
+                    pool_pages=400 if P == 16 else 120, pad_table_to=170 if P == 16 else 50)
+    q = torch.randn((len(lens), Lq, Hq, 128), generator=torch.Generator().manual_seed(Lq)).to(torch.bfloat16)
+    ref, ref_lse = oracle.extend_attn_fp8kv_oracle(q, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
+                                                   case.block_table, case.seq_lens, case.scale)
+    dev = workloads.to_device(case, "cuda")
+    try:
+        for grid in (0, 1, 7):
+            da.set_option("grid_blocks", grid)
+            out, lse = da.decode_attn_fp8kv_extend(q.cuda(), dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale,
+                                                   dev.block_table, dev.seq_lens, dev.scale)
+            assert da.read_device_status() == (0, 0, 0, 0)
+            assert_close(out.cpu().numpy(), ref, f"fp8 extend grid={grid} out")
+            assert_close(lse.cpu().numpy(), ref_lse, f"fp8 extend grid={grid} lse")
+    finally:
+        da.set_option("grid_blocks", 0)
+    with pytest.raises(da.DecodeAttnError) as e:     # more than 16 query rows per KV head
+        big = torch.zeros((len(lens), 17, Hq, 128), dtype=torch.bfloat16, device="cuda")
+        da.decode_attn_fp8kv_extend(big, dev.k_pages, dev.v_pages, None, None, dev.block_table, dev.seq_lens, 1.0)
+    assert e.value.status == 5

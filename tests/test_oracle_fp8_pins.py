@@ -221,3 +221,17 @@ def test_planted_slips_are_seen():
     # bias 8 instead of 7 would halve every K: emulate by halving k_scale
     half = run8(case, k_scale=case.k_scale * 0.5)
     assert np.abs(half[1] - base_lse).max() > 1e-2
+
+
+def test_extend_over_codes_reproduces_the_bf16_extend_oracle():
+    """Unit factors and a cache widened exactly to bf16: the causal multi-token oracle over codes must equal the
+    (separately pinned) bf16 one bit for bit."""
+    case = tiny8([13, 4, 0, 22], P=4, seed=71, poison=False)
+    q = torch.randn((4, 3, 6, 8), generator=torch.Generator().manual_seed(3)).to(torch.bfloat16)
+    lens = np.where(case.seq_lens.numpy() > 0, np.maximum(case.seq_lens.numpy(), 3), 0)
+    assert (lens == case.seq_lens.numpy()).all()
+    k, v = widened(case)
+    want = oracle.extend_attn_oracle(q, k, v, case.block_table, case.seq_lens, case.scale)
+    got = oracle.extend_attn_fp8kv_oracle(q, case.k_pages, case.v_pages, None, None, case.block_table, case.seq_lens,
+                                          case.scale)
+    assert np.array_equal(want[0], got[0]) and np.array_equal(want[1], got[1])
