@@ -332,6 +332,12 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
  *   "static_frac"  share of the work, in 1/256, covered by the static ranges (default 224)
  *   "extend_stream_rows"  decode_attn_extend(): most query rows per KV head that go through the
  *                  streaming kernels instead of the tensor-core kernel (0 .. 16, default 16)
+ *   "kv_evict_first"  L2 priority of the K and V page loads: 1 = "evict first" (pages that are read
+ *                  once do not push the query rows, block table, plan and partial results out of L2),
+ *                  0 = normal (better when sequences share pages, which are then re-read from L2),
+ *                  2 = chosen per call on the device (default): normal when at least a quarter of the
+ *                  non-empty sequences start on the same physical page as the first sequence or as
+ *                  their predecessor in the batch, else evict first.  Results do not depend on it.
  * Returns DA_ERR_UNSUPPORTED for an unknown name or a value out of range.
  */
 int decode_attn_set_option(const char *name, int64_t value);

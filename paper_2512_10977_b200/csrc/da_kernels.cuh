@@ -29,7 +29,8 @@ constexpr int PLAN_THREADS = 1024;
 constexpr int PLAN_SMEM_SEQS = 4096;
 constexpr int MIN_TAIL_UNIT_TILES = 4;      // a ticketed unit is never cut smaller than this
 constexpr int PLAN_BLOCKS = 8;              // the plan kernel's grid: each block cuts a slice of the units
-constexpr int MERGE_WARP_SPLITS = 32;       // pairs cut into more splits are merged by a whole block
+constexpr int MERGE_WARP_SPLITS = 8;        // pairs cut into more splits are merged by a whole block
+                                            // (a warp keeps eight partial rows in flight: one pass)
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
@@ -63,7 +64,8 @@ struct PlanHeader {
     int n_static;         // = thread blocks of the partition kernel
     int n_tail;           // ticketed units (0: none)
     int ticket;           // next ticketed unit to hand out (reset by the plan kernel)
-    int pad[3];
+    int kv_evict_first;   // K and V loads carry the L2 "evict first" policy (no pages seem to be shared)
+    int pad[2];
 };
 // Split pairs found by plan block k: how many with <= MERGE_WARP_SPLITS splits, how many with more.
 struct MergeCounts {
@@ -88,6 +90,7 @@ struct PartParams {
     int32_t *status;
     int32_t B, Hkv, G, P, box_rows, num_pages, out_bf16;
     int32_t log2_P;           // P = 1 << log2_P
+
     float scale_log2;         // scale * log2(e)
     const float *k_scale, *v_scale;   // 8-bit cache: per-KV-head factors (NULL: 1)
     // Several new tokens per sequence (Lq > 1, causal among them): query token qi of KV group g's head hd
@@ -113,6 +116,11 @@ struct PlanParams {
     int32_t tile_t;           // tokens per tile (TILE_T or TILE_T8)
     int32_t min_len;          // a non-empty sequence shorter than this is an error (the new tokens of an extend call)
     int32_t first_token;      // tokens before this one are not attended (the cascade's suffix pass)
+    // L2 policy of the K/V loads: 0 normal, 1 evict first, 2 decide here -- evict first unless many
+    // sequences start on the same physical page (a shared prefix is re-read from L2 by every sharer).
+    int32_t kv_policy;
+    const int32_t *block_table;   // only read for kv_policy 2 (may be NULL otherwise)
+    int64_t bt_sb;
     int32_t n_static, n_tail_max, static_frac_q8;   // large units; most ticketed units; share of the
                                                     // line given to the large units, in 1/256
     int64_t max_pages;
@@ -199,13 +207,20 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     __shared__ int running_s;
     __shared__ int prefix_s[PLAN_SMEM_SEQS + 1];   // copy of the prefix for the searches below
     __shared__ PlanHeader hdr_s;
+    __shared__ int nonempty_s, same_start_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     grid_launch_dependents();   // the partition kernel may set up its blocks while the plan is made
+    // The plan kernel is itself launched with programmatic serialization, so that its blocks can be
+    // placed while the kernel before it in the stream drains: nothing is read or written before that
+    // kernel is complete.
+    grid_dependency_wait();
     const bool writer = blockIdx.x == 0;
     if (tid == 0) {
         running_s = 0;
         n_small_s = 0;
         n_big_s = 0;
+        nonempty_s = 0;
+        same_start_s = 0;
     }
     __syncthreads();
 
@@ -223,6 +238,16 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
                 if (writer)
                     report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, L < p.min_len ? 2 : 1, L);
                 L = 0;
+            }
+            if (writer && p.kv_policy == 2 && L > p.first_token) {
+                // Does this sequence start (after the tokens a cascade call skips) on the same page as the
+                // first sequence, or as the one before it?  Entries are compared, never used as page ids;
+                // the other rows' entries exist (L <= max_pages * P was checked) but may be unspecified.
+                const int64_t j = p.first_token / p.P;
+                const int pg = __ldg(p.block_table + (int64_t)b * p.bt_sb + j);
+                atomicAdd(&nonempty_s, 1);
+                if (b > 0 && (pg == __ldg(p.block_table + j) || pg == __ldg(p.block_table + (int64_t)(b - 1) * p.bt_sb + j)))
+                    atomicAdd(&same_start_s, 1);
             }
             lo = (p.window > 0 && p.window < L) ? L - p.window : 0;
             lo = max(lo, min(p.first_token, L));
@@ -295,7 +320,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         h.q_tail = n_tail ? tail_w / n_tail : 0;
         h.r_tail = n_tail ? (int)(tail_w % n_tail) : 0;
         h.ticket = 0;
-        h.pad[0] = h.pad[1] = h.pad[2] = 0;
+        h.kv_evict_first = p.kv_policy == 2 ? (4 * same_start_s < nonempty_s || nonempty_s < 2) : p.kv_policy;
+        h.pad[0] = h.pad[1] = 0;
         hdr_s = h;
         if (writer)
             *p.hdr = h;
@@ -427,6 +453,9 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         const int n_static = p.hdr->n_static, n_units = n_static + p.hdr->n_tail;
         uint32_t it = 0;
         bool aborted = false;
+        // K and V pass through L2 once (unless sequences share pages: then the caller may ask for the
+        // normal priority, under which re-read pages stay in L2 longer)
+        const uint64_t kv_policy = p.hdr->kv_evict_first ? l2_policy_evict_first() : l2_policy_evict_normal();
 
         // cursor over this block's tiles: unit u, pair (b, g), tile i of cnt
         int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
@@ -528,9 +557,9 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             if (cur.need) {
                 const uint32_t dst = smem_base + stage * STAGE_BYTES + is_v * KV_BYTES + box * box_bytes;
                 if constexpr (KV8)
-                    tma_load_4d(dst, tm, 0, cur.row, cur.g, cur.page, bar_full + 8 * stage);
+                    tma_load_4d_hint(dst, tm, 0, cur.row, cur.g, cur.page, bar_full + 8 * stage, kv_policy);
                 else
-                    tma_load_5d(dst, tm, 0, cur.row, 0, cur.g, cur.page, bar_full + 8 * stage);
+                    tma_load_5d_hint(dst, tm, 0, cur.row, 0, cur.g, cur.page, bar_full + 8 * stage, kv_policy);
             }
             ++it;
             return true;
@@ -647,23 +676,32 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     // within 2^-28 of the head's largest (smaller ones are off by at most 2^-25 of the scaled value).
     // qf[n][i] is the fragment of k step i (16 dims): lane (r, c) holds head r, dims 16i + 4c .. + 3.
     // fh[n][e]: what turns the raw products of head 2c + e into log2-domain scores.
-    auto load_q8 = [&](uint32_t (&qf)[NT8][8][2], float (&fh)[NT8][2], int b, int g) {
-        const float ks = p.k_scale ? __ldg(p.k_scale + g) : 1.f;
+    // Two steps, so that the loads of the next item's vectors can fly while this item is combined:
+    // load_q8_raw only issues the loads (bf16 pairs), q8_fragments turns them into the fragments.
+    auto load_q8_raw = [&](uint32_t (&w)[NT8][8][2], float &ks, int b, int g) {
+        ks = p.k_scale ? __ldg(p.k_scale + g) : 1.f;
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
             const int head = n * 8 + r;
             const int hv = head < p.Gv ? head : 0;
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
                 p.q + (int64_t)b * p.q_sb + (int64_t)(hv / p.G) * p.q_sq + (int64_t)(g * p.G + hv % p.G) * p.q_sh);
-            uint32_t w[8][2];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf)
+                    w[n][i][hf] = head < p.Gv ? __ldg(qrow + 8 * i + 2 * c + hf) : 0u;
+        }
+    };
+    auto q8_fragments = [&](uint32_t (&qf)[NT8][8][2], float (&fh)[NT8][2], const uint32_t (&w)[NT8][8][2], float ks) {
+#pragma unroll
+        for (int n = 0; n < NT8; ++n) {
             float amax = 0.f;
 #pragma unroll
             for (int i = 0; i < 8; ++i)
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    w[i][hf] = head < p.Gv ? __ldg(qrow + 8 * i + 2 * c + hf) : 0u;
-                    amax = fmaxf(amax, fmaxf(fabsf(bf16_lo_to_float(w[i][hf])), fabsf(bf16_hi_to_float(w[i][hf]))));
-                }
+                for (int hf = 0; hf < 2; ++hf)
+                    amax = fmaxf(amax, fmaxf(fabsf(bf16_lo_to_float(w[n][i][hf])), fabsf(bf16_hi_to_float(w[n][i][hf]))));
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
             // f = 2^(14 - exponent of amax), kept inside the normal fp32 range
@@ -674,7 +712,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             for (int i = 0; i < 8; ++i)
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf)
-                    qf[n][i][hf] = pack_f16(bf16_lo_to_float(w[i][hf]) * f, bf16_hi_to_float(w[i][hf]) * f);
+                    qf[n][i][hf] = pack_f16(bf16_lo_to_float(w[n][i][hf]) * f, bf16_hi_to_float(w[n][i][hf]) * f);
             const float fin = (1.f / f) * ks * p.scale_log2;   // the same in all four lanes of head r
             fh[n][0] = __shfl_sync(0xffffffffu, fin, 8 * c);
             fh[n][1] = __shfl_sync(0xffffffffu, fin, 8 * c + 4);
@@ -691,7 +729,10 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     uint32_t qf[NT8][8][2];
     float fh[NT8][2];
     if constexpr (KV8) {
-        load_q8(qf, fh, m0.x, m0.y);
+        uint32_t w[NT8][8][2];
+        float ks;
+        load_q8_raw(w, ks, m0.x, m0.y);
+        q8_fragments(qf, fh, w, ks);
     } else {
         load_q(qf, m0.x, m0.y);
 #pragma unroll
@@ -1042,10 +1083,12 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         //      (m, l, O) and write the pair's result or partial.
         const bool stop = (m0.w & TILE_STOP) != 0;
         uint32_t qn[NT8][8][2];
-        float fn[NT8][2];
+        float ks_next = 1.f;
+        // 8-bit cache: this item's V factor (asked for here, used after the barrier below)
+        const float vmul = (KV8 && p.v_scale) ? __ldg(p.v_scale + g) : 1.f;
         if (!stop) {
             if constexpr (KV8)
-                load_q8(qn, fn, m0.x, m0.y);
+                load_q8_raw(qn, ks_next, m0.x, m0.y);
             else
                 load_q(qn, m0.x, m0.y);
         }
@@ -1082,37 +1125,74 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             return;
         }
         {
-            const int d = tid;   // 0..127
-            const float vmul = (KV8 && p.v_scale) ? __ldg(p.v_scale + g) : 1.f;
-            for (int head = 0; head < p.Gv; ++head) {
-                float M = st_m[head];
-#pragma unroll
-                for (int w = 1; w < NCW; ++w)
-                    M = fmaxf(M, st_m[w * HEADS + head]);
-                float den = 0.f, num = 0.f;
-                const int dx = d ^ (8 * ((head >> 1) & 3));
+            // Warp w folds heads w, w + 4, ...: lane -> output dims 4 lane .. 4 lane + 3.  A short loop
+            // on purpose: this code runs once per item, so its instructions are fetched cold each time,
+            // and a compact body costs far less than a long unrolled one.
+            const uint64_t part_policy = l2_policy_evict_last();   // partial results wait in L2 for the merge kernel
+#pragma unroll 1
+            for (int head = warp; head < p.Gv; head += NCW) {
+                float mw[NCW], lw[NCW], f[NCW];
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {
-                    const float f = fast_exp2(st_m[w * HEADS + head] - M);   // 0 for a warp that saw no token
-                    den += st_l[w * HEADS + head] * f;
-                    num += xbuf[(w * HEADS + head) * HEAD_DIM + dx] * f;
+                    mw[w] = st_m[w * HEADS + head];
+                    lw[w] = st_l[w * HEADS + head];
                 }
-                // (den = 0: a piece in which this column's query attends nothing -- several new tokens only)
-                const float val = den > 0.f ? (KV8 ? (num / den) * vmul : num / den) : 0.f;
-                const float lse_nat = den > 0.f ? (M + fast_log2(den)) * LN2 : -INFINITY;
+                const float *xrow = xbuf + head * HEAD_DIM + ((4 * lane) ^ (8 * ((head >> 1) & 3)));
+                float4 x[NCW];
+#pragma unroll
+                for (int w = 0; w < NCW; ++w)
+                    x[w] = *reinterpret_cast<const float4 *>(xrow + w * HEADS * HEAD_DIM);
+                float M = mw[0];
+#pragma unroll
+                for (int w = 1; w < NCW; ++w)
+                    M = fmaxf(M, mw[w]);
+                float den = 0.f;
+                float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int w = 0; w < NCW; ++w) {
+                    f[w] = fast_exp2(mw[w] - M);   // 0 for a warp that saw no token
+                    den += lw[w] * f[w];
+                    num.x += x[w].x * f[w];
+                    num.y += x[w].y * f[w];
+                    num.z += x[w].z * f[w];
+                    num.w += x[w].w * f[w];
+                }
+                // (den = 0, or NaN when no warp saw a token: a piece in which this column's query attends
+                //  nothing -- several new tokens only)
+                const bool some = den > 0.f;
+                const float inv = some ? (KV8 ? vmul / den : 1.f / den) : 0.f;
+                const float lse_nat = some ? (M + fast_log2(den)) * LN2 : -INFINITY;
+                const float4 val = some ? make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv)
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
                 if (whole) {
-                    const int qi = head / p.G, h = g * p.G + head % p.G;
-                    const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h * p.o_sh + d;
-                    if (p.out_bf16)
-                        reinterpret_cast<__nv_bfloat16 *>(p.out)[at] = __float2bfloat16_rn(val);
-                    else
-                        reinterpret_cast<float *>(p.out)[at] = val;
-                    if (d == 0 && p.lse)
-                        p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h * p.l_sh] = lse_nat;
+                    const int qi = p.Lq > 1 ? head / p.G : 0;
+                    const int h_out = g * p.G + (head - qi * p.G);
+                    const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h_out * p.o_sh + 4 * lane;
+                    if (p.out_bf16) {
+                        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
+                        const uint32_t lo = pack_bf16(val.x, val.y), hi = pack_bf16(val.z, val.w);
+                        if ((reinterpret_cast<uintptr_t>(o) & 7u) == 0) {
+                            *reinterpret_cast<uint2 *>(o) = make_uint2(lo, hi);
+                        } else {
+                            reinterpret_cast<uint16_t *>(o)[0] = (uint16_t)lo;
+                            reinterpret_cast<uint16_t *>(o)[1] = (uint16_t)(lo >> 16);
+                            reinterpret_cast<uint16_t *>(o)[2] = (uint16_t)hi;
+                            reinterpret_cast<uint16_t *>(o)[3] = (uint16_t)(hi >> 16);
+                        }
+                    } else {
+                        float *o = reinterpret_cast<float *>(p.out) + at;
+                        if ((reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+                            *reinterpret_cast<float4 *>(o) = val;
+                        } else {
+                            o[0] = val.x; o[1] = val.y; o[2] = val.z; o[3] = val.w;
+                        }
+                    }
+                    if (lane == 0 && p.lse)
+                        p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h_out * p.l_sh] = lse_nat;
                 } else {
-                    p.part_o[((int64_t)slot * HEADS + head) * HEAD_DIM + d] = val;
-                    if (d == 0)
-                        p.part_lse[(int64_t)slot * HEADS + head] = lse_nat;
+                    st_global_v4_hint(p.part_o + ((int64_t)slot * HEADS + head) * HEAD_DIM + 4 * lane, val, part_policy);
+                    if (lane == 0)
+                        st_global_f32_hint(p.part_lse + (int64_t)slot * HEADS + head, lse_nat, part_policy);
                 }
             }
         }
@@ -1126,19 +1206,16 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         ++items;
         if (stop)
             return;
-#pragma unroll
-        for (int n = 0; n < NT8; ++n)
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                qf[n][kk][0] = qn[n][kk][0];
-                qf[n][kk][1] = qn[n][kk][1];
-            }
         if constexpr (KV8) {
+            q8_fragments(qf, fh, qn, ks_next);
+        } else {
 #pragma unroll
-            for (int n = 0; n < NT8; ++n) {
-                fh[n][0] = fn[n][0];
-                fh[n][1] = fn[n][1];
-            }
+            for (int n = 0; n < NT8; ++n)
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    qf[n][kk][0] = qn[n][kk][0];
+                    qf[n][kk][1] = qn[n][kk][1];
+                }
         }
     }
 }
@@ -1180,6 +1257,7 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
 {
     __shared__ MergeAcc s_part[MERGE_WARPS][MERGE_LANES];
     const int warp = threadIdx.x / MERGE_LANES, ln = threadIdx.x % MERGE_LANES, d = ln * 4;
+    grid_launch_dependents();   // a following kernel launched the same way may place its blocks now
     grid_dependency_wait();     // partials and the plan are complete and visible
     const PlanHeader hdr = *p.hdr;
     const MergeCounts cnt = *p.merge_counts;
@@ -1224,14 +1302,26 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
         if (ln == 0 && p.lse)
             p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h * p.l_sh] = lse_val;
     };
-    // splits [k0, k0 + 32) of entry e (pair id, first slot, first unit, splits), one head
-    auto warp_merge = [&](const int4 &e, int head, int k0) {
+    // splits [k0, min(k_end, k0 + 32)) of entry e (pair id, first slot, first unit, splits), one head
+    auto warp_merge = [&](const int4 &e, int head, int k0, int k_end) {
         const int k = k0 + ln;
-        const bool valid = k < e.w;
+        const bool valid = k < k_end;
         int uu = e.z + k;
         if (e.z < n_full && uu >= n_full)
             uu += gap;   // skip the static units that hold no tiles
         const int slot = (k == 0) ? e.y : 2 * uu;
+        const int n = min(k_end - k0, 32);
+        auto row = [&](int sl) {
+            return *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)sl * p.heads_pad + head) * HEAD_DIM + d);
+        };
+        // the first eight partial rows are asked for together with the lse values (their addresses do
+        // not depend on them): one round trip to memory less
+        float4 o0[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int sl = __shfl_sync(0xffffffffu, slot, j);
+            o0[j] = j < n ? row(sl) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         const float l = valid ? p.part_lse[(int64_t)slot * p.heads_pad + head] : -INFINITY;
         MergeAcc a;
         a.M = l;
@@ -1244,9 +1334,16 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
         for (int o = 16; o > 0; o >>= 1)
             a.den += __shfl_xor_sync(0xffffffffu, a.den, o);
         a.acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        const int n = min(e.w - k0, 32);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float wj = __shfl_sync(0xffffffffu, w, j);   // 0 past the last split
+            a.acc.x += wj * o0[j].x;
+            a.acc.y += wj * o0[j].y;
+            a.acc.z += wj * o0[j].z;
+            a.acc.w += wj * o0[j].w;
+        }
         // 8 independent loads in flight per lane and pass
-        for (int s0 = 0; s0 < n; s0 += 8) {
+        for (int s0 = 8; s0 < n; s0 += 8) {
             float4 o[8];
             float ws[8];
 #pragma unroll
@@ -1256,7 +1353,7 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
                 const int sl = __shfl_sync(0xffffffffu, slot, s2 & 31);
                 o[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (s2 < n)
-                    o[j] = *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)sl * p.heads_pad + head) * HEAD_DIM + d);
+                    o[j] = row(sl);
                 else
                     ws[j] = 0.f;
             }
@@ -1283,8 +1380,12 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
         const int4 e = entry(p.merge_big, cnt.n_big, item / p.Gv);
         const int head = item % p.Gv;
         MergeAcc a = {-INFINITY, 0.f, make_float4(0.f, 0.f, 0.f, 0.f)};
-        for (int k0 = warp * 32; k0 < e.w; k0 += MERGE_WARPS * 32)
-            merge_fold(a, warp_merge(e, head, k0));
+        // the splits are dealt to the eight warps in equal chunks (of at least eight, the number of
+        // rows a warp asks for at once), so that up to 64 splits cost one round trip to memory
+        const int chunk = max(8, (e.w + MERGE_WARPS - 1) / MERGE_WARPS);
+        const int k_end = min(e.w, (warp + 1) * chunk);
+        for (int k0 = warp * chunk; k0 < k_end; k0 += 32)
+            merge_fold(a, warp_merge(e, head, k0, k_end));
         s_part[warp][ln] = a;
         __syncthreads();
         if (warp == 0) {
@@ -1299,7 +1400,7 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
     for (int item = blockIdx.x * MERGE_WARPS + warp; item < n_small * p.Gv; item += gridDim.x * MERGE_WARPS) {
         const int4 e = entry(p.merge_small, cnt.n_small, item / p.Gv);
         const int head = item % p.Gv;
-        finish(e, head, warp_merge(e, head, 0));
+        finish(e, head, warp_merge(e, head, 0, e.w));
     }
     // ---- empty sequences
     for (int b = blockIdx.x; b < p.B; b += gridDim.x) {

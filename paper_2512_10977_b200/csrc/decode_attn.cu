@@ -16,7 +16,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 107;
+constexpr int kVersion = 108;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -29,6 +29,7 @@ std::atomic<int64_t> g_launches{0};
 int64_t g_opt_grid_blocks = 0;   // 0 = two blocks per SM
 int64_t g_opt_tail_units = 4;    // ticketed units per thread block (0: one static range per block only)
 int64_t g_opt_static_frac = 224; // share of the work given to the static ranges, in 1/256
+int64_t g_opt_kv_evict_first = 2; // L2 policy of the K and V loads: 0 normal, 1 evict first, 2 chosen by the plan kernel
 int64_t g_opt_extend_stream_rows = 16;   // decode_attn_extend: Lq * (Hq / Hkv) up to this many rows go through the
                                          // streaming (partition) kernel, more through the tcgen05 kernel; 0: never
 cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
@@ -305,7 +306,8 @@ int set_kernel_attrs()
 }
 
 int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const Dims &d, uint8_t *ws,
-                const WsLayout &lay, int nblocks, int n_tail, cudaStream_t stream, int tile_t = TILE_T, int min_len = 0)
+                const WsLayout &lay, int nblocks, int n_tail, cudaStream_t stream, int tile_t = TILE_T, int min_len = 0,
+                const da_tensor *bt = nullptr)
 {
     PlanParams pp;
     pp.seq_lens = static_cast<const int32_t *>(sl->data);
@@ -326,13 +328,27 @@ int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const 
     pp.tile_t = tile_t;
     pp.min_len = min_len;
     pp.first_token = first_token;
+    pp.block_table = (bt && d.max_pages > 0) ? static_cast<const int32_t *>(bt->data) : nullptr;
+    pp.bt_sb = bt ? bt->stride[0] : 0;
+    pp.kv_policy = (int32_t)g_opt_kv_evict_first;
+    if (pp.kv_policy == 2 && !pp.block_table) pp.kv_policy = 1;
     pp.n_static = nblocks;
     pp.n_tail_max = n_tail;
     pp.static_frac_q8 = (int32_t)g_opt_static_frac;
     pp.max_pages = d.max_pages;
-    plan_kernel<<<PLAN_BLOCKS, PLAN_THREADS, 0, stream>>>(pp);
+    // Programmatic stream serialization: the blocks may be placed while the kernel before this one in
+    // the stream finishes; the kernel waits on the device before it reads or writes anything.
+    cudaLaunchAttribute pdl;
+    pdl.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)PLAN_BLOCKS);
+    cfg.blockDim = dim3((unsigned)PLAN_THREADS);
+    cfg.stream = stream;
+    cfg.attrs = &pdl;
+    cfg.numAttrs = 1;
+    DA_CUDA(cudaLaunchKernelEx(&cfg, plan_kernel, pp));
     g_launches.fetch_add(1);
-    DA_CUDA(cudaGetLastError());
     return DA_OK;
 }
 
@@ -362,7 +378,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     rc = get_tmap(v, box_rows, kv8 ? 0 : 2, &tm_v);
     if (rc != DA_OK) return rc;
 
-    rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream, tile_t, Lq > 1 ? Lq : 0);
+    rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream, tile_t, Lq > 1 ? Lq : 0, bt);
     if (rc != DA_OK) return rc;
 
     PartParams pa;
@@ -1210,6 +1226,11 @@ int decode_attn_set_option(const char *name, int64_t value)
         g_opt_static_frac = value;
         return DA_OK;
     }
+    if (std::strcmp(name, "kv_evict_first") == 0) {
+        if (value < 0 || value > 2) return DA_ERR_UNSUPPORTED;
+        g_opt_kv_evict_first = value;
+        return DA_OK;
+    }
     if (std::strcmp(name, "extend_stream_rows") == 0) {
         if (value < 0 || value > kMaxGroup) return DA_ERR_UNSUPPORTED;
         g_opt_extend_stream_rows = value;
@@ -1225,6 +1246,7 @@ int64_t decode_attn_get_option(const char *name)
     if (std::strcmp(name, "grid_blocks") == 0) return g_opt_grid_blocks;
     if (std::strcmp(name, "tail_units") == 0) return g_opt_tail_units;
     if (std::strcmp(name, "static_frac") == 0) return g_opt_static_frac;
+    if (std::strcmp(name, "kv_evict_first") == 0) return g_opt_kv_evict_first;
     if (std::strcmp(name, "extend_stream_rows") == 0) return g_opt_extend_stream_rows;
     return -1;
 }

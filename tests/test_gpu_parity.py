@@ -125,6 +125,23 @@ def test_any_mix_of_static_and_ticketed_units_gives_the_same_answer(da, tail, fr
         da.set_option("static_frac", 224)
 
 
+@pytest.mark.parametrize("policy", [0, 1, 2])
+def test_l2_priority_of_the_page_loads_does_not_change_the_answer(da, policy):
+    """The K/V loads' L2 policy (normal, evict first, chosen on the device from how many sequences
+    start on the same page) is a cache hint only: same result with and without a shared prefix."""
+    unique = workloads.build_case("pol_u", [2500, 3, 900, 0, 64, 4097], 16, 31, "cpu")
+    shared = workloads.build_case("pol_s", [2500, 640, 900, 1300, 4097], 16, 32, "cpu", shared_prefix_tokens=640)
+    try:
+        da.set_option("kv_evict_first", policy)
+        assert da.get_option("kv_evict_first") == policy
+        for case, what in ((unique, "unique pages"), (shared, "shared prefix")):
+            check(da, case, f"{what}, policy {policy}")
+    finally:
+        da.set_option("kv_evict_first", 2)
+    with pytest.raises(Exception):
+        da.set_option("kv_evict_first", 3)
+
+
 @pytest.mark.parametrize("B", [1, 2, 3, 7])
 @pytest.mark.parametrize("P", [16, 64])
 def test_batches_with_empty_sequences(da, B, P):
