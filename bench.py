@@ -36,8 +36,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the partition kernel, from the ncu
 # capture summarised under profiles/ (one file per kernel and workload); valid for that library version only.
-NCU_TRAFFIC = {("c2", 107): 2223315000 + 7977000}
-NCU_TRAFFIC_FP8 = {("c2", 107): 1112425000 + 7460000}   # the 8-bit-cache kernel's capture
+NCU_TRAFFIC = {("c2", 108): 2222443000 + 3706000}
+NCU_TRAFFIC_FP8 = {("c2", 108): 1111734000 + 6661000}   # the 8-bit-cache kernel's capture
 WORKLOAD_TEXT = {
     "c1": "c1: 1 seq x 512 tok, page 16, contiguous, seed 0, 3 keys x20",
     "c2": "c2: 64 seqs, len U[1024,16384], 48q/8kv heads, d128, page 16, permuted pool, seed 1",
@@ -205,8 +205,8 @@ def run_ours(args):
 
     case = make_case(args, device)
     kv8 = args.kv == "fp8"
-    if kv8 and (args.cascade or args.extend):
-        raise SystemExit("--kv fp8 applies to decode_attn only")
+    if kv8 and args.cascade:
+        raise SystemExit("--kv fp8 applies to decode_attn and to --extend with a few new tokens")
     out = torch.empty(case.q.shape, dtype=torch.float32, device=device)
     lse = torch.empty(case.q.shape[:2], dtype=torch.float32, device=device)
     nbytes = case.algorithmic_bytes(4)
@@ -233,7 +233,10 @@ def run_ours(args):
         nbytes += case.B * (Lq - 1) * (Hq_ * Dh_ * 2 + Hq_ * Dh_ * 4 + Hq_ * 4)   # the extra queries' q, out, lse
 
     def step():
-        if Lq:
+        if Lq and kv8:
+            da.decode_attn_fp8kv_extend(q_ext, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
+                                        case.block_table, case.seq_lens, case.scale, out=out, lse=lse, stream=stream)
+        elif Lq:
             da.decode_attn_extend(q_ext, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
                                   case.scale, out=out, lse=lse, stream=stream)
         elif prefix:
@@ -322,7 +325,12 @@ def run_ours(args):
     def e2e_step():
         if Lq:
             q_d.copy_(q_h, non_blocking=True); bt_d.copy_(bt_h, non_blocking=True); sl_d.copy_(sl_h, non_blocking=True)
-            da.decode_attn_extend(q_d, case.k_pages, case.v_pages, bt_d, sl_d, case.scale, out=out, lse=lse, stream=stream)
+            if kv8:
+                da.decode_attn_fp8kv_extend(q_d, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt_d, sl_d,
+                                            case.scale, out=out, lse=lse, stream=stream)
+            else:
+                da.decode_attn_extend(q_d, case.k_pages, case.v_pages, bt_d, sl_d, case.scale, out=out, lse=lse,
+                                      stream=stream)
             out_h.copy_(out, non_blocking=True); lse_h.copy_(lse, non_blocking=True)
         elif prefix:   # the cascade has no host-io entry point: same copies, made here on the same stream
             q_d.copy_(q_h, non_blocking=True); bt_d.copy_(bt_h, non_blocking=True); sl_d.copy_(sl_h, non_blocking=True)
@@ -373,10 +381,11 @@ def run_ours(args):
                 "kernel_ms": kms, "traffic": NCU_TRAFFIC_FP8.get((args.workload, da.version())) if kv8 else
                 NCU_TRAFFIC.get((args.workload, da.version()))}
     G_ = case.q.shape[1] // case.k_pages.shape[1]
-    ext_stream = bool(Lq) and Lq * G_ <= da.get_option("extend_stream_rows")
+    ext_stream = bool(Lq) and (kv8 or Lq * G_ <= da.get_option("extend_stream_rows"))
     if ext_stream:
         # a few new tokens ride through the streaming kernels as a wider group: still bound by HBM
         roofline["kernel"] = f"partition_kernel ({Lq} query tokens x {G_} heads per KV head)"
+        roofline["traffic"] = None   # the ncu capture is of the single-token call
     elif Lq:
         # one kernel, a dense causal contraction: algorithmic flops = QK^T and PV over each query's keys
         Hq, Dh = case.q.shape[1], case.q.shape[2]
@@ -414,7 +423,7 @@ def run_ours(args):
                           ("inputs exceed L2 (no flush)" if nbytes > 4 * 126e6 else "inputs fit L2; not flushed")),
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "grid_blocks": da.get_option("grid_blocks"),
-                   "path": (f"decode_attn_extend, {Lq} new tokens per sequence (causal, " +
+                   "path": (f"decode_attn{'_fp8kv' if kv8 else ''}_extend, {Lq} new tokens per sequence (causal, " +
                             ("streaming kernels)" if ext_stream else "tcgen05)")) if Lq else
                            ("cascade (shared prefix on tcgen05)" if prefix else
                             ("decode_attn_fp8kv" if kv8 else "decode_attn"))},
