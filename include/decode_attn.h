@@ -352,6 +352,24 @@ int64_t decode_attn_get_option(const char *name);
  */
 int decode_attn_set_profile_events(void *before, void *after);
 
+/*
+ * decode_attn_timeline -- diagnostic of the timeline build only (the same sources compiled with
+ * -DDA_TIMELINE into a second library; the normal library returns DA_ERR_UNSUPPORTED and keeps no
+ * stamps).  In that build the plan, partition and merge kernels leave global-timer stamps (ns) of
+ * their most recent launch in a device table; this call waits for the device, copies the table to
+ * `host_out` and, if `clear` is non-zero, zeroes it.
+ *   host_out   HOST, DECODE_ATTN_TIMELINE_ROWS x DECODE_ATTN_TIMELINE_COLS values, row-major:
+ *              rows 0..1023 = thread blocks of the partition kernel (columns: 0 entry, 1 past the wait
+ *              for the plan, 2 first tile ready, 3 last tile consumed, 4 exit, 5 tiles consumed,
+ *              6 (sequence, KV head) items finished); rows 1024..1031 = the merge kernel's first eight
+ *              blocks (0 resident, 1 released, 2 exit); row 1032 column 2 = the last merge block's
+ *              exit; rows 1036..1043 = the plan kernel's blocks (0 entry, 1 exit)
+ *   capacity   values `host_out` can hold; DA_ERR_SHAPE if fewer than rows x cols
+ */
+#define DECODE_ATTN_TIMELINE_ROWS 1048
+#define DECODE_ATTN_TIMELINE_COLS 8
+int decode_attn_timeline(unsigned long long *host_out, int64_t capacity, int32_t clear);
+
 const char *decode_attn_strerror(int status);
 int decode_attn_last_cuda_error(void); /* cudaError_t of the last failing CUDA call, else 0 */
 int decode_attn_version(void);

@@ -14,7 +14,8 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libdecode_attn.so")
+# DECODE_ATTN_LIBRARY names another build of the same library (the timeline build); default: the in-tree one
+_LIB_PATH = os.environ.get("DECODE_ATTN_LIBRARY") or os.path.join(_HERE, "libdecode_attn.so")
 _lock = threading.Lock()
 _lib = None
 _workspaces = {}   # device index -> torch uint8 tensor kept alive while registered
@@ -34,6 +35,16 @@ class DecodeAttnError(RuntimeError):
 class DaTensor(ctypes.Structure):
     _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("ndim", ctypes.c_int32),
                 ("shape", ctypes.c_int64 * 4), ("stride", ctypes.c_int64 * 4)]
+
+
+def use_library(path: str) -> None:
+    """Load another build of the library (the timeline build) instead of the in-tree default.  Must be
+    called before the first library call of the process."""
+    global _LIB_PATH
+    with _lock:
+        if _lib is not None:
+            raise RuntimeError("the library is already loaded")
+        _LIB_PATH = os.path.abspath(path)
 
 
 def lib() -> ctypes.CDLL:
@@ -85,6 +96,8 @@ def lib() -> ctypes.CDLL:
             L.decode_attn_last_cuda_error.restype = ctypes.c_int
             L.decode_attn_version.restype = ctypes.c_int
             L.decode_attn_launch_count.restype = i64
+            L.decode_attn_timeline.restype = ctypes.c_int
+            L.decode_attn_timeline.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), i64, i32]
             _lib = L
     return _lib
 
@@ -129,6 +142,18 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
         raise RuntimeError("decode_attn needs a CUDA device; there is no CPU path")
     s = stream if stream is not None else torch.cuda.current_stream()
     return s.cuda_stream
+
+
+TIMELINE_ROWS, TIMELINE_COLS = 1048, 8
+
+
+def timeline(clear: bool = True):
+    """The kernels' global-timer stamps of their last launch as a [TIMELINE_ROWS, TIMELINE_COLS] int64
+    array (timeline build of the library only; see include/decode_attn.h for the rows)."""
+    import numpy as np
+    buf = (ctypes.c_ulonglong * (TIMELINE_ROWS * TIMELINE_COLS))()
+    _check(lib().decode_attn_timeline(buf, TIMELINE_ROWS * TIMELINE_COLS, 1 if clear else 0))
+    return np.frombuffer(buf, dtype=np.uint64).astype(np.int64).reshape(TIMELINE_ROWS, TIMELINE_COLS)
 
 
 def version() -> int:

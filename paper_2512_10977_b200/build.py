@@ -33,5 +33,24 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+TIMELINE_LIB = os.path.join(_HERE, "libdecode_attn_timeline.so")
+
+
+def build_timeline(force: bool = False) -> str:
+    """The diagnostic variant of the library (-DDA_TIMELINE: the kernels keep global-timer stamps of
+    their phases).  Built on demand by ``timeline.py``; the normal library carries none of it."""
+    if not force and os.path.exists(TIMELINE_LIB):
+        t = os.path.getmtime(TIMELINE_LIB)
+        if not any(os.path.getmtime(os.path.join(CSRC, f)) > t for f in SOURCES + HEADERS):
+            return TIMELINE_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = TIMELINE_LIB + f".tmp{os.getpid()}"
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-DDA_TIMELINE",
+           "-shared", "-Xcompiler", "-fPIC", "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, TIMELINE_LIB)
+    return TIMELINE_LIB
+
+
 if __name__ == "__main__":
     print(build(force=True, verbose=True))

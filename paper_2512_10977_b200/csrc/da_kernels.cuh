@@ -34,6 +34,25 @@ constexpr int MERGE_WARP_SPLITS = 8;        // pairs cut into more splits are me
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 
+// Timeline build (-DDA_TIMELINE, a diagnostic library beside the normal one): the kernels leave
+// %globaltimer stamps in g_timeline, which decode_attn_timeline() copies out.  Rows 0 .. 1023: thread
+// blocks of the partition kernel -- column 0 entry, 1 past the wait for the plan, 2 first tile ready,
+// 3 last tile consumed, 4 exit, 5 tiles consumed, 6 (b, kv head) items finished.  Rows TL_MERGE .. + 7:
+// the merge kernel's first eight blocks -- 0 resident, 1 released by the partition kernel, 2 exit;
+// row TL_MERGE + 8, column 2: the latest exit of any merge block.  Rows TL_PLAN .. + 7: the plan
+// kernel's blocks -- 0 entry, 1 exit.  In the normal build DA_TL() is empty and nothing is kept.
+constexpr int TL_ROWS = 1048, TL_COLS = 8, TL_MERGE = 1024, TL_PLAN = 1036;
+#ifdef DA_TIMELINE
+__device__ unsigned long long g_timeline[TL_ROWS][TL_COLS];
+#define DA_TL(row, col) (g_timeline[(row)][(col)] = globaltimer_ns())
+#define DA_TL_SET(row, col, value) (g_timeline[(row)][(col)] = (unsigned long long)(value))
+#define DA_TL_MAX(row, col) atomicMax(&g_timeline[(row)][(col)], (unsigned long long)globaltimer_ns())
+#else
+#define DA_TL(row, col) ((void)0)
+#define DA_TL_SET(row, col, value) ((void)0)
+#define DA_TL_MAX(row, col) ((void)0)
+#endif
+
 // flags of a tile's descriptor (written by the producer warp, read by the consumer warps)
 constexpr int TILE_ITEM_END = 1;   // last tile this unit holds of its (b, kv head) pair
 constexpr int TILE_WHOLE = 2;      // the unit holds every tile of the pair: write `out` directly
@@ -209,6 +228,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     __shared__ PlanHeader hdr_s;
     __shared__ int nonempty_s, same_start_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0)
+        DA_TL(TL_PLAN + blockIdx.x, 0);
     grid_launch_dependents();   // the partition kernel may set up its blocks while the plan is made
     // The plan kernel is itself launched with programmatic serialization, so that its blocks can be
     // placed while the kernel before it in the stream drains: nothing is read or written before that
@@ -384,6 +405,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     if (tid == 0) {
         p.merge_counts->n_small[blockIdx.x] = n_small_s;
         p.merge_counts->n_big[blockIdx.x] = n_big_s;
+        DA_TL(TL_PLAN + blockIdx.x, 1);
     }
 }
 
@@ -420,6 +442,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const uint32_t bar_epi = bar_empty + NSTAGES * 8;   // two barriers for the consumers' epilogue
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0 && blockIdx.x < TL_MERGE)
+        DA_TL(blockIdx.x, 0);
 
     if ((smem_base & 1023u) != 0) {   // the swizzle pattern is a function of the address bits
         if (tid == 0)
@@ -441,6 +465,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     grid_launch_dependents();   // lets the merge kernel's blocks become resident early
     __syncthreads();
     grid_dependency_wait();     // the plan (and everything before it in the stream) is complete
+    if (tid == 0 && blockIdx.x < TL_MERGE)
+        DA_TL(blockIdx.x, 1);
 
     if (warp == NCW) {
         // ------------------------------------------------------------------ producer warp
@@ -724,6 +750,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         return;
     }
     int4 m0 = meta[0], m1 = meta[1];
+    if (tid == 0 && blockIdx.x < TL_MERGE)
+        DA_TL(blockIdx.x, 2);
     if (m0.w & TILE_STOP)
         return;
     uint32_t qf[NT8][8][2];
@@ -1067,6 +1095,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             if (lane == 0)
                 mbar_arrive(bar_empty + 8 * stage);
             ++it;
+            if (tid == 0 && blockIdx.x < TL_MERGE)
+                DA_TL(blockIdx.x, 3);
             // the next tile (of this item, or the first of the next one, or the stop mark)
             const int nstage = it % NSTAGES;
             if (!mbar_wait_bounded(bar_full + 8 * nstage, (it / NSTAGES) & 1u, abort_flag)) {
@@ -1204,8 +1234,14 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             return;
         }
         ++items;
-        if (stop)
+        if (stop) {
+            if (tid == 0 && blockIdx.x < TL_MERGE) {
+                DA_TL(blockIdx.x, 4);
+                DA_TL_SET(blockIdx.x, 5, it);
+                DA_TL_SET(blockIdx.x, 6, items);
+            }
             return;
+        }
         if constexpr (KV8) {
             q8_fragments(qf, fh, qn, ks_next);
         } else {
@@ -1258,7 +1294,11 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
     __shared__ MergeAcc s_part[MERGE_WARPS][MERGE_LANES];
     const int warp = threadIdx.x / MERGE_LANES, ln = threadIdx.x % MERGE_LANES, d = ln * 4;
     grid_launch_dependents();   // a following kernel launched the same way may place its blocks now
+    if (threadIdx.x == 0 && blockIdx.x < 8)
+        DA_TL(TL_MERGE + blockIdx.x, 0);
     grid_dependency_wait();     // partials and the plan are complete and visible
+    if (threadIdx.x == 0 && blockIdx.x < 8)
+        DA_TL(TL_MERGE + blockIdx.x, 1);
     const PlanHeader hdr = *p.hdr;
     const MergeCounts cnt = *p.merge_counts;
     const int n_full = static_units_in_use(hdr);
@@ -1408,6 +1448,11 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
             continue;
         for (int h = warp; h < p.Lq * p.Hkv * p.G; h += MERGE_WARPS)
             store(b, h / (p.Hkv * p.G), h % (p.Hkv * p.G), make_float4(0.f, 0.f, 0.f, 0.f), -INFINITY);
+    }
+    if (threadIdx.x == 0) {
+        if (blockIdx.x < 8)
+            DA_TL(TL_MERGE + blockIdx.x, 2);
+        DA_TL_MAX(TL_MERGE + 8, 2);
     }
 }
 

@@ -1274,6 +1274,26 @@ const char *decode_attn_strerror(int status)
     }
 }
 
+int decode_attn_timeline(unsigned long long *host_out, int64_t capacity, int32_t clear)
+{
+#ifdef DA_TIMELINE
+    constexpr int64_t n = (int64_t)da::TL_ROWS * da::TL_COLS;
+    if (!host_out) return DA_ERR_NULL;
+    if (capacity < n) return DA_ERR_SHAPE;
+    std::lock_guard<std::mutex> lock(g_mu);
+    DA_CUDA(cudaMemcpyFromSymbol(host_out, da::g_timeline, (size_t)n * 8));   // waits for the device's work
+    if (clear) {
+        void *sym = nullptr;
+        DA_CUDA(cudaGetSymbolAddress(&sym, da::g_timeline));
+        DA_CUDA(cudaMemset(sym, 0, (size_t)n * 8));
+    }
+    return DA_OK;
+#else
+    (void)host_out; (void)capacity; (void)clear;
+    return DA_ERR_UNSUPPORTED;
+#endif
+}
+
 int decode_attn_last_cuda_error(void) { return g_last_cuda_error.load(); }
 int decode_attn_version(void) { return kVersion; }
 int64_t decode_attn_launch_count(void) { return g_launches.load(); }

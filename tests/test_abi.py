@@ -45,6 +45,14 @@ def test_status_strings_and_version(pkg):
     assert L.decode_attn_strerror(99).decode() == "unknown status"
 
 
+def test_the_normal_build_keeps_no_timeline(pkg):
+    # the stamps exist only in the -DDA_TIMELINE build; the normal library says so without touching CUDA
+    buf = (ctypes.c_ulonglong * 16)()
+    assert pkg.lib().decode_attn_timeline(buf, 16, 0) == 5   # DA_ERR_UNSUPPORTED
+    with pytest.raises(pkg.DecodeAttnError):
+        pkg.timeline()
+
+
 def test_options(pkg):
     assert pkg.get_option("grid_blocks") == 0
     pkg.set_option("grid_blocks", 7)
