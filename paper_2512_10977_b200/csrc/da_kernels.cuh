@@ -40,7 +40,7 @@ constexpr float LN2 = 0.6931471805599453f;
 // 3 last tile consumed, 4 exit, 5 tiles consumed, 6 (b, kv head) items finished.  Rows TL_MERGE .. + 7:
 // the merge kernel's first eight blocks -- 0 resident, 1 released by the partition kernel, 2 exit;
 // row TL_MERGE + 8, column 2: the latest exit of any merge block.  Rows TL_PLAN .. + 7: the plan
-// kernel's blocks -- 0 entry, 1 exit.  In the normal build DA_TL() is empty and nothing is kept.
+// kernel's blocks -- 0 entry, 1 exit, 2 past the wait for the kernel before it in the stream.  In the normal build DA_TL() is empty and nothing is kept.
 constexpr int TL_ROWS = 1048, TL_COLS = 8, TL_MERGE = 1024, TL_PLAN = 1036;
 #ifdef DA_TIMELINE
 __device__ unsigned long long g_timeline[TL_ROWS][TL_COLS];
@@ -235,6 +235,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     // placed while the kernel before it in the stream drains: nothing is read or written before that
     // kernel is complete.
     grid_dependency_wait();
+    if (tid == 0)
+        DA_TL(TL_PLAN + blockIdx.x, 2);
     const bool writer = blockIdx.x == 0;
     if (tid == 0) {
         running_s = 0;

@@ -64,7 +64,8 @@ def main() -> None:
     q = lambda col, f: rel(f(part[:, col]))
     print(f"workload {args.workload}, cache {args.kv}: {used.sum()} partition blocks, {int(part[:, 5].sum())} tiles, "
           f"{int(part[:, 6].sum())} (sequence, KV head) items; back-to-back calls every {period_ns:.0f} ns")
-    print(f"plan kernel        : start 0, last block done {rel(tl[PLAN:PLAN + 8, 1].max())}")
+    print(f"plan kernel        : first block enters 0, last passes the wait for the kernel before it "
+          f"{rel(tl[PLAN:PLAN + 8, 2].max())}, last block done {rel(tl[PLAN:PLAN + 8, 1].max())}")
     print(f"partition kernel   : first block enters {q(0, np.min)}, last passes the wait for the plan {q(1, np.max)}")
     print(f"  first tile ready : min {q(2, np.min)}  median {q(2, np.median)}  max {q(2, np.max)}")
     print(f"  last tile done   : min {q(3, np.min)}  median {q(3, np.median)}  max {q(3, np.max)}")
