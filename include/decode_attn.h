@@ -364,7 +364,7 @@ int decode_attn_set_profile_events(void *before, void *after);
  *              6 (sequence, KV head) items finished); rows 1024..1031 = the merge kernel's first eight
  *              blocks (0 resident, 1 released, 2 exit); row 1032 column 2 = the last merge block's
  *              exit; rows 1036..1043 = the plan kernel's blocks (0 entry, 1 exit, 2 past the wait for the
- *              kernel before it in the stream)
+ *              kernel before it in the stream, 3 lengths scanned, 4 cut made, 5 units written)
  *   capacity   values `host_out` can hold; DA_ERR_SHAPE if fewer than rows x cols
  */
 #define DECODE_ATTN_TIMELINE_ROWS 1048

@@ -25,10 +25,12 @@ static_assert(TILE_T8 * 128 == KV_BYTES, "both cache types fill a stage");
 constexpr float P8_SHIFT = 15.f;            // 8-bit cache: softmax weights are carried as 2^15 * p (f16 high + low)
 constexpr int STAGE_BYTES = 2 * KV_BYTES;   // K tile followed by V tile
 constexpr int NTHREADS = (NCW + 1) * 32;    // + one producer warp
-constexpr int PLAN_THREADS = 1024;
+constexpr int PLAN_THREADS = 512;
 constexpr int PLAN_SMEM_SEQS = 4096;
 constexpr int MIN_TAIL_UNIT_TILES = 4;      // a ticketed unit is never cut smaller than this
-constexpr int PLAN_BLOCKS = 8;              // the plan kernel's grid: each block cuts a slice of the units
+constexpr int PLAN_BLOCKS = 16;             // the plan kernel's grid: each block cuts a slice of the units
+                                            // (16 x 512 threads: with 8 x 1024 the 32 warps of an SM spent 1.5 us
+                                            // issuing the ~300 instructions that cut one unit per thread)
 constexpr int MERGE_WARP_SPLITS = 8;        // pairs cut into more splits are merged by a whole block
                                             // (a warp keeps eight partial rows in flight: one pass)
 constexpr float LOG2E = 1.4426950408889634f;
@@ -40,7 +42,8 @@ constexpr float LN2 = 0.6931471805599453f;
 // 3 last tile consumed, 4 exit, 5 tiles consumed, 6 (b, kv head) items finished.  Rows TL_MERGE .. + 7:
 // the merge kernel's first eight blocks -- 0 resident, 1 released by the partition kernel, 2 exit;
 // row TL_MERGE + 8, column 2: the latest exit of any merge block.  Rows TL_PLAN .. + 7: the plan
-// kernel's blocks -- 0 entry, 1 exit, 2 past the wait for the kernel before it in the stream.  In the normal build DA_TL() is empty and nothing is kept.
+// kernel's blocks -- 0 entry, 1 exit, 2 past the wait for the kernel before it in the stream, 3 lengths scanned, 4 cut made,
+// 5 units written.  In the normal build DA_TL() is empty and nothing is kept.
 constexpr int TL_ROWS = 1048, TL_COLS = 8, TL_MERGE = 1024, TL_PLAN = 1036;
 #ifdef DA_TIMELINE
 __device__ unsigned long long g_timeline[TL_ROWS][TL_COLS];
@@ -251,6 +254,18 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
         const int b = base + tid;
         int lo = 0, L = 0, first = 0, nt = 0;
         if (b < p.B) {
+            // Does this sequence start (after the tokens a cascade call skips) on the same page as the first
+            // sequence, or as the one before it?  The three entries are asked for together with the length
+            // (entry first_token / P exists in every row: the host checked it against max_pages); they are
+            // compared, never used as page ids, and may be unspecified for sequences that end before them.
+            const bool probe = writer && p.kv_policy == 2;
+            int pg = 0, pg_first = 0, pg_prev = 0;
+            if (probe) {
+                const int64_t j = p.first_token / p.P;
+                pg = __ldg(p.block_table + (int64_t)b * p.bt_sb + j);
+                pg_first = __ldg(p.block_table + j);
+                pg_prev = __ldg(p.block_table + (int64_t)(b > 0 ? b - 1 : 0) * p.bt_sb + j);
+            }
             L = p.seq_lens[(int64_t)b * p.sl_stride];
             if (L < 0 || (int64_t)L > p.max_pages * (int64_t)p.P) {
                 if (writer)
@@ -262,14 +277,9 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
                     report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, L < p.min_len ? 2 : 1, L);
                 L = 0;
             }
-            if (writer && p.kv_policy == 2 && L > p.first_token) {
-                // Does this sequence start (after the tokens a cascade call skips) on the same page as the
-                // first sequence, or as the one before it?  Entries are compared, never used as page ids;
-                // the other rows' entries exist (L <= max_pages * P was checked) but may be unspecified.
-                const int64_t j = p.first_token / p.P;
-                const int pg = __ldg(p.block_table + (int64_t)b * p.bt_sb + j);
+            if (probe && L > p.first_token) {
                 atomicAdd(&nonempty_s, 1);
-                if (b > 0 && (pg == __ldg(p.block_table + j) || pg == __ldg(p.block_table + (int64_t)(b - 1) * p.bt_sb + j)))
+                if (b > 0 && (pg == pg_first || pg == pg_prev))
                     atomicAdd(&same_start_s, 1);
             }
             lo = (p.window > 0 && p.window < L) ? L - p.window : 0;
@@ -291,14 +301,15 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
             warp_tot[warp] = incl;
         __syncthreads();
         if (warp == 0) {
-            int w = warp_tot[lane];
+            int w = lane < PLAN_THREADS / 32 ? warp_tot[lane] : 0;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const int y = __shfl_up_sync(0xffffffffu, w, o);
                 if (lane >= o)
                     w += y;
             }
-            warp_tot[lane] = w;   // inclusive over warps
+            if (lane < PLAN_THREADS / 32)
+                warp_tot[lane] = w;   // inclusive over warps
         }
         __syncthreads();
         const int run = running_s;
@@ -318,6 +329,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     }
     const int tiles_per_head = running_s;
     const bool in_smem = p.B <= PLAN_SMEM_SEQS;
+    if (tid == 0)
+        DA_TL(TL_PLAN + blockIdx.x, 3);
     if (tid == 0) {
         if (writer)
             p.prefix[p.B] = tiles_per_head;
@@ -350,6 +363,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
             *p.hdr = h;
     }
     __syncthreads();   // this block's global writes are visible to itself after the barrier
+    if (tid == 0)
+        DA_TL(TL_PLAN + blockIdx.x, 4);
     // With more sequences than fit in shared memory the searches read block 0's global copy.
     // (Blocks cannot wait for one another, so in that case block 0 alone cuts all the units.)
     const int *prefix = in_smem ? prefix_s : p.prefix;
@@ -405,6 +420,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     }
     __syncthreads();
     if (tid == 0) {
+        DA_TL(TL_PLAN + blockIdx.x, 5);
         p.merge_counts->n_small[blockIdx.x] = n_small_s;
         p.merge_counts->n_big[blockIdx.x] = n_big_s;
         DA_TL(TL_PLAN + blockIdx.x, 1);

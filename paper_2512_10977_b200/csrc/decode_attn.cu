@@ -331,7 +331,8 @@ int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const 
     pp.block_table = (bt && d.max_pages > 0) ? static_cast<const int32_t *>(bt->data) : nullptr;
     pp.bt_sb = bt ? bt->stride[0] : 0;
     pp.kv_policy = (int32_t)g_opt_kv_evict_first;
-    if (pp.kv_policy == 2 && !pp.block_table) pp.kv_policy = 1;
+    // the plan kernel compares entry first_token / P of the rows: it must exist
+    if (pp.kv_policy == 2 && (!pp.block_table || (int64_t)first_token / d.P >= d.max_pages)) pp.kv_policy = 1;
     pp.n_static = nblocks;
     pp.n_tail_max = n_tail;
     pp.static_frac_q8 = (int32_t)g_opt_static_frac;

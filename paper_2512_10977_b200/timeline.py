@@ -66,6 +66,8 @@ def main() -> None:
           f"{int(part[:, 6].sum())} (sequence, KV head) items; back-to-back calls every {period_ns:.0f} ns")
     print(f"plan kernel        : first block enters 0, last passes the wait for the kernel before it "
           f"{rel(tl[PLAN:PLAN + 8, 2].max())}, last block done {rel(tl[PLAN:PLAN + 8, 1].max())}")
+    pl = tl[PLAN:PLAN + 8]
+    print(f"  plan block 0     : lengths scanned {rel(pl[0, 3])}, cut made {rel(pl[0, 4])}, units written {rel(pl[0, 5])}, exit {rel(pl[0, 1])}")
     print(f"partition kernel   : first block enters {q(0, np.min)}, last passes the wait for the plan {q(1, np.max)}")
     print(f"  first tile ready : min {q(2, np.min)}  median {q(2, np.median)}  max {q(2, np.max)}")
     print(f"  last tile done   : min {q(3, np.min)}  median {q(3, np.median)}  max {q(3, np.max)}")
