@@ -29,8 +29,6 @@ constexpr int PLAN_THREADS = 512;
 constexpr int PLAN_SMEM_SEQS = 4096;
 constexpr int MIN_TAIL_UNIT_TILES = 4;      // a ticketed unit is never cut smaller than this
 constexpr int PLAN_BLOCKS = 16;             // the plan kernel's grid: each block cuts a slice of the units
-                                            // (16 x 512 threads: with 8 x 1024 the 32 warps of an SM spent 1.5 us
-                                            // issuing the ~300 instructions that cut one unit per thread)
 constexpr int MERGE_WARP_SPLITS = 8;        // pairs cut into more splits are merged by a whole block
                                             // (a warp keeps eight partial rows in flight: one pass)
 constexpr float LOG2E = 1.4426950408889634f;
