@@ -159,9 +159,9 @@ def test_all_sequences_empty(da):
     assert (got == 0).all() and np.isneginf(got_lse).all()
 
 
-@pytest.mark.parametrize("B", [1025, 1500, 4096, 4097, 6000])
+@pytest.mark.parametrize("B", [512, 513, 1025, 1500, 4096, 4097, 6000])
 def test_many_sequences(da, B):
-    """Batches beyond one pass of the plan kernel's scan (1024 sequences) and beyond what its shared
+    """Batches beyond one pass of the plan kernel's scan (512 sequences) and beyond what its shared
     memory holds (4096: the work units are then cut from the global copy of the prefix)."""
     rng = np.random.default_rng(B)
     lens = rng.integers(0, 150, size=B)
