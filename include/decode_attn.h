@@ -28,15 +28,24 @@
  *
  * Conventions.  Every function returns a da_status (0 = ok) and never throws,
  * aborts or synchronises unless it says so.  Pointers inside da_tensor are
- * DEVICE pointers unless a function says HOST.  The library owns no memory:
- * scratch comes from the caller through decode_attn_set_workspace().  Work is
+ * DEVICE pointers unless a function says HOST.  The library allocates no
+ * memory: scratch comes from the caller through decode_attn_set_workspace()
+ * (one entry point, decode_attn_static_scratch(), uses a fixed array inside the
+ * library image instead).  Work is
  * enqueued on the given CUDA stream and the call returns at once.  Arguments a
  * host can check (NULL, dtype, shape, stride, alignment, workspace size) are
- * rejected before anything is launched.  Errors that depend on device data (a
- * page id outside the pool, a sequence longer than its block-table row) are
- * found on the device: the offending access is skipped or clamped (never a
- * trap, never an unbounded wait), a status word is set, and
- * decode_attn_read_device_status() returns it.
+ * rejected before anything is launched.  Errors that depend on device data are
+ * found on the device (never a trap, never an unbounded wait); a status record
+ * is set, decode_attn_read_device_status() returns it, and the affected rows
+ * are marked in the result:
+ *   - a block-table entry outside [0, num_pages): that page is not read, and
+ *     out and lse of every (sequence, query head) whose KV head needed it are
+ *     NaN (in decode_attn_cascade(), a bad entry inside the shared prefix makes
+ *     every row NaN, since every row attends it);
+ *   - a length below 0, beyond its block-table row, or below what the call
+ *     requires (the shared prefix, the new tokens of an extend call): the
+ *     sequence is treated as empty, out = 0 and lse = -inf.
+ * Other sequences of the batch are not affected.
  */
 #ifndef DECODE_ATTN_H_
 #define DECODE_ATTN_H_
@@ -66,7 +75,9 @@ typedef enum {
     DA_DEV_OK = 0,
     DA_DEV_BAD_PAGE = 1,   /* block-table entry outside [0, num_pages); that load was skipped */
     DA_DEV_BAD_SEQLEN = 2, /* seq_len < 0 or > max_pages * P; the sequence was treated as empty */
-    DA_DEV_TIMEOUT = 3     /* a bounded wait inside a kernel ran out; results are invalid  */
+    DA_DEV_TIMEOUT = 3,    /* a bounded wait inside a kernel ran out; results are invalid  */
+    DA_DEV_BOUNDS = 4      /* diagnostic build only: a kernel formed an index outside one of its own
+                              arrays; record = {4, site, index, extent}; that access was skipped    */
 } da_dev_status;
 
 /* A strided view.  `stride` is in ELEMENTS.  Nothing is owned. */
@@ -147,7 +158,8 @@ int decode_attn_fp8kv(const da_tensor *q, const da_tensor *k_pages, const da_ten
  *
  *   shared_prefix_tokens  a multiple of 128, at most max_pages * P; <= 0 means no shared prefix
  *                         (plain decode_attn).  Every seq_lens[b] must be >= shared_prefix_tokens
- *                         (a shorter one sets DA_DEV_BAD_SEQLEN in the device status).
+ *                         (a shorter one sets DA_DEV_BAD_SEQLEN in the device status and is treated
+ *                         as empty: out = 0, lse = -inf).
  *   The page ids of the prefix are read from row 0 of the block table; that the other rows agree
  *   is the caller's promise and is not checked.
  * Other arguments, results, workspace and error conventions: as decode_attn().
@@ -273,7 +285,12 @@ int decode_attn_fp8kv_host_io(const da_tensor *q_host, const da_tensor *k_pages,
  * array, the work is cut into one static range per thread block only (as with "tail_units" 0).
  *
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
- * that device current); make that first call outside any stream capture.  All calls on a device
+ * that device current); make that first call outside any stream capture.  When the 6 MiB are
+ * reserved: when the CUDA runtime loads this library's device code on that device -- with lazy
+ * module loading that is the first library call on it that launches a kernel or looks up a
+ * symbol, not process start.  A server that sizes its KV pool from "all the memory that is free" should therefore
+ * make one library call on each device (this one with B = 0 will do) BEFORE it measures free memory,
+ * or that first call can itself fail with an out-of-memory error.  All calls on a device
  * share the one array, which still holds the previous call's contents when the next one starts
  * (the call clears the only part that must start at zero, its status record): two calls that
  * overlap on the GPU race on it, so keep them on one stream or order them yourself.
@@ -338,6 +355,17 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
  *                  2 = chosen per call on the device (default): normal when at least a quarter of the
  *                  non-empty sequences start on the same physical page as the first sequence or as
  *                  their predecessor in the batch, else evict first.  Results do not depend on it.
+ * The diagnostic build of the library (the same sources compiled with -DDA_TIMELINE -DDA_DIAG
+ * -DDA_BOUNDS_CHECK into a second shared object; the normal library knows none of these names) adds
+ *   "diag_wait_limit_us"  how long a bounded wait inside a kernel lasts before it gives up with
+ *                  DA_DEV_TIMEOUT (default 2,000,000 = the normal build's fixed 2 s)
+ *   "diag_withhold_partition_tile", "diag_withhold_prefix_tile"   tile number (counted per thread
+ *                  block, from 0) whose copies AND barrier arrival the loader of thread block 0 leaves
+ *                  out in the partition / prefix kernel; -1 (default) = none.  Nothing is issued for that
+ *                  tile, so the warps waiting for it run into the limit above and the kernel leaves
+ *                  through its give-up path: a way to test that path without faulting or hanging the
+ *                  device.  The results of such a call are invalid; the next call is unaffected.
+ * and checks every index its kernels form into their own arrays (DA_DEV_BOUNDS).
  * Returns DA_ERR_UNSUPPORTED for an unknown name or a value out of range.
  */
 int decode_attn_set_option(const char *name, int64_t value);
@@ -353,9 +381,9 @@ int64_t decode_attn_get_option(const char *name);
 int decode_attn_set_profile_events(void *before, void *after);
 
 /*
- * decode_attn_timeline -- diagnostic of the timeline build only (the same sources compiled with
- * -DDA_TIMELINE into a second library; the normal library returns DA_ERR_UNSUPPORTED and keeps no
- * stamps).  In that build the plan, partition and merge kernels leave global-timer stamps (ns) of
+ * decode_attn_timeline -- diagnostic build only (the same sources compiled with -DDA_TIMELINE,
+ * -DDA_DIAG and -DDA_BOUNDS_CHECK into a second library; the normal library returns
+ * DA_ERR_UNSUPPORTED and keeps no stamps).  In that build the plan, partition and merge kernels leave global-timer stamps (ns) of
  * their most recent launch in a device table; this call waits for the device, copies the table to
  * `host_out` and, if `clear` is non-zero, zeroes it.
  *   host_out   HOST, DECODE_ATTN_TIMELINE_ROWS x DECODE_ATTN_TIMELINE_COLS values, row-major:

@@ -33,23 +33,27 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
-TIMELINE_LIB = os.path.join(_HERE, "libdecode_attn_timeline.so")
+DIAG_LIB = os.path.join(_HERE, "libdecode_attn_diag.so")
+DIAG_FLAGS = ["-DDA_TIMELINE", "-DDA_DIAG", "-DDA_BOUNDS_CHECK"]
 
 
-def build_timeline(force: bool = False) -> str:
-    """The diagnostic variant of the library (-DDA_TIMELINE: the kernels keep global-timer stamps of
-    their phases).  Built on demand by ``timeline.py``; the normal library carries none of it."""
-    if not force and os.path.exists(TIMELINE_LIB):
-        t = os.path.getmtime(TIMELINE_LIB)
+def build_diag(force: bool = False) -> str:
+    """The diagnostic variant of the library, from the same sources: -DDA_TIMELINE (the kernels keep
+    global-timer stamps of their phases), -DDA_DIAG (the limit of the kernels' bounded waits becomes
+    an option, and one tile's copies can be withheld so that a wait runs out) and -DDA_BOUNDS_CHECK
+    (every index into the kernels' own arrays is checked into the status record).  Used by
+    ``timeline.py`` and the diagnostic tests; the normal library carries none of it."""
+    if not force and os.path.exists(DIAG_LIB):
+        t = os.path.getmtime(DIAG_LIB)
         if not any(os.path.getmtime(os.path.join(CSRC, f)) > t for f in SOURCES + HEADERS):
-            return TIMELINE_LIB
+            return DIAG_LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = TIMELINE_LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-DDA_TIMELINE",
+    tmp = DIAG_LIB + f".tmp{os.getpid()}"
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17"] + DIAG_FLAGS + [
            "-shared", "-Xcompiler", "-fPIC", "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.run(cmd, check=True)
-    os.replace(tmp, TIMELINE_LIB)
-    return TIMELINE_LIB
+    os.replace(tmp, DIAG_LIB)
+    return DIAG_LIB
 
 
 if __name__ == "__main__":

@@ -118,6 +118,8 @@ struct PartParams {
     // Query qi sits at position L - Lq + qi and attends tokens below L - Lq + qi + 1.
     int32_t Lq, Gv;
     int64_t q_sq, o_sq, l_sq;         // strides of the query-token dimension (0 when Lq == 1)
+    int32_t unit_cap;                 // rows of unit_work; the partial arrays hold 2 * unit_cap slots
+    int64_t max_pages;                // entries in a block-table row
 };
 
 struct PlanParams {
@@ -162,6 +164,8 @@ struct MergeParams {
     int32_t B, Hkv, G, heads_pad, out_bf16;
     int32_t Lq, Gv;           // as in PartParams
     int64_t o_sq, l_sq;
+    int32_t unit_cap;         // as in PartParams
+    int32_t *status;
 };
 
 __device__ __forceinline__ void report_status(int32_t *status, int code, int a, int b, int c)
@@ -172,6 +176,24 @@ __device__ __forceinline__ void report_status(int32_t *status, int code, int a, 
         status[3] = c;
     }
 }
+
+// Bounds-check build (-DDA_BOUNDS_CHECK, part of the diagnostic library; compute-sanitizer's stand-in
+// where that tool is not available): every index the kernels form into the plan arrays, the merge
+// lists, the partial slots, the block table and the result tensors is compared with its extent first.
+// An index outside it is recorded in the status record as {DA_DEV_BOUNDS, site, index, extent} and the
+// access is skipped.  In the normal build DA_IN_RANGE() is `true` and costs nothing.
+#ifdef DA_BOUNDS_CHECK
+__device__ __forceinline__ bool in_range(int32_t *status, long long idx, long long extent, int site)
+{
+    if (idx >= 0 && idx < extent)
+        return true;
+    report_status(status, 4 /* DA_DEV_BOUNDS */, site, (int)idx, (int)extent);
+    return false;
+}
+#define DA_IN_RANGE(status, idx, extent, site) ::da::in_range((status), (long long)(idx), (long long)(extent), (site))
+#else
+#define DA_IN_RANGE(status, idx, extent, site) true
+#endif
 
 // Start of range c of a cut with quotient q and remainder r.
 __host__ __device__ __forceinline__ long long cut_start(long long q, int r, int c)
@@ -406,15 +428,21 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
                         const int ns = pair_splits(h, w0, nt, &uf);
                         // the pair is the first item of unit `prev` only if that unit starts at it
                         const int4 e = make_int4(b * p.Hkv + g, 2 * prev + (prev_start == w0 ? 0 : 1), prev, ns);
-                        if (ns > MERGE_WARP_SPLITS)
-                            my_big[atomicAdd(&n_big_s, 1)] = e;
-                        else
-                            my_small[atomicAdd(&n_small_s, 1)] = e;
+                        if (ns > MERGE_WARP_SPLITS) {
+                            const int at = atomicAdd(&n_big_s, 1);
+                            if (DA_IN_RANGE(p.status, at, p.merge_seg, 1))
+                                my_big[at] = e;
+                        } else {
+                            const int at = atomicAdd(&n_small_s, 1);
+                            if (DA_IN_RANGE(p.status, at, p.merge_seg, 2))
+                                my_small[at] = e;
+                        }
                     }
                 }
             }
         }
-        p.unit_work[u] = uw;
+        if (DA_IN_RANGE(p.status, u, units_max, 3))
+            p.unit_work[u] = uw;
     }
     __syncthreads();
     if (tid == 0) {
@@ -515,6 +543,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         };
         auto open_unit = [&]() {   // make u a unit that has tiles, taking tickets past empty ones
             while (u >= 0) {
+                if (!DA_IN_RANGE(p.status, u, p.unit_cap, 4))
+                    return false;
                 const int4 uw = p.unit_work[u];
                 if (uw.w > 0) {
                     b = uw.x; g = uw.y; rel = uw.z; remaining = uw.w;
@@ -528,6 +558,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         auto open_pair = [&]() {   // position on the next (b, g) pair that has tiles; false at the end
             for (;;) {
                 while (remaining > 0) {
+                    if (!DA_IN_RANGE(p.status, b, p.B, 5))
+                        return false;
                     si = p.seq_info[b];
                     if (si.w > 0) {
                         cnt = min(si.w - rel, remaining);
@@ -549,6 +581,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             t.need = active && tok0 < si.y && tok0 + p.box_rows > si.x;
             t.page = 0;
             t.row = tok0 & (p.P - 1);           // P is a power of two: no divisions in this loop
+            if (t.need && !DA_IN_RANGE(p.status, tok0 >> p.log2_P, p.max_pages, 6))
+                t.need = false;
             if (t.need)
                 t.page = __ldg(bt_row + (tok0 >> p.log2_P));
             t.g = g; t.b = b; t.lo = si.x; t.L = si.y;
@@ -583,20 +617,28 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         auto issue = [&](Tile &cur) {   // the tile's descriptor and copies into the next free stage
             const int stage = it % NSTAGES;
             const uint32_t phase = (it / NSTAGES) & 1u;
-            if (cur.need && (uint32_t)cur.page >= (uint32_t)p.num_pages) {
+            // A page id outside the pool: the load is skipped (the rows keep whatever the stage held) and
+            // the tile is marked, so that the consumers write NaN for this (sequence, KV head) pair
+            // instead of a finite result computed from stale rows.
+            const bool bad_page = cur.need && (uint32_t)cur.page >= (uint32_t)p.num_pages;
+            if (bad_page) {
                 report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, cur.b, (cur.t0 + box * p.box_rows) / p.P, cur.page);
-                cur.need = false;   // skip the load; the rows keep whatever the stage held
+                cur.need = false;
             }
+            const uint32_t poisoned = __ballot_sync(0xffffffffu, bad_page);
             const uint32_t mask = __ballot_sync(0xffffffffu, cur.need);
             if (!mbar_wait_bounded(bar_empty + 8 * stage, phase ^ 1u, abort_flag))
                 return false;
-            if (lane == 0) {
+            // (diagnostic build only: one tile of block 0 can be left out altogether -- no arrival, no
+            //  copies -- so that the consumers' bounded wait for it runs out)
+            const bool withheld = DA_WITHHOLD(0, blockIdx.x, it);
+            if (lane == 0 && !withheld) {
                 meta[2 * stage] = make_int4(cur.b, cur.g, cur.t0, cur.flags);
-                meta[2 * stage + 1] = make_int4(cur.lo, cur.L, cur.slot, 0);
+                meta[2 * stage + 1] = make_int4(cur.lo, cur.L, cur.slot, poisoned != 0u);
                 mbar_arrive_expect_tx(bar_full + 8 * stage, (uint32_t)__popc(mask) * box_bytes);
             }
             __syncwarp();
-            if (cur.need) {
+            if (cur.need && !withheld) {
                 const uint32_t dst = smem_base + stage * STAGE_BYTES + is_v * KV_BYTES + box * box_bytes;
                 if constexpr (KV8)
                     tma_load_4d_hint(dst, tm, 0, cur.row, cur.g, cur.page, bar_full + 8 * stage, kv_policy);
@@ -643,7 +685,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     const uint32_t j = it - 1 - k;
                     const uint64_t t_begin = globaltimer_ns();
                     while (!mbar_try_wait(bar_full + 8 * (j % NSTAGES), (j / NSTAGES) & 1u)) {
-                        if (globaltimer_ns() - t_begin > 1000000000ull)
+                        if (globaltimer_ns() - t_begin > DA_WAIT_LIMIT_NS / 2)
                             break;
                     }
                 }
@@ -787,6 +829,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     for (;;) {   // one (b, kv head) item per iteration
         const int b = m0.x, g = m0.y, lo = m1.x, L = m1.y, slot = m1.z;
         const bool whole = (m0.w & TILE_WHOLE) != 0;
+        bool poisoned = false;   // a tile of this item lost rows to a bad page id: the result is NaN
         float m_run[NT8][2], l_run[NT8][2], o[NT8][8][4];
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
@@ -803,6 +846,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             const int a = m0.z + WT * warp;     // first token of this warp's rows
             const int v_lo = max(a, lo), v_hi = min(a + WT, L);
             const bool item_end = (m0.w & TILE_ITEM_END) != 0;
+            poisoned |= m1.w != 0;
             if constexpr (KV8) {
               if (v_lo < v_hi) {
                 const uint32_t k_base = smem_base + stage * STAGE_BYTES;
@@ -1207,13 +1251,20 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 //  nothing -- several new tokens only)
                 const bool some = den > 0.f;
                 const float inv = some ? (KV8 ? vmul / den : 1.f / den) : 0.f;
-                const float lse_nat = some ? (M + fast_log2(den)) * LN2 : -INFINITY;
-                const float4 val = some ? make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv)
-                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                float lse_nat = some ? (M + fast_log2(den)) * LN2 : -INFINITY;
+                float4 val = some ? make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv)
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (poisoned) {   // (a NaN partial makes the merged result NaN as well)
+                    lse_nat = __int_as_float(0x7fc00000);
+                    val = make_float4(lse_nat, lse_nat, lse_nat, lse_nat);
+                }
                 if (whole) {
                     const int qi = p.Lq > 1 ? head / p.G : 0;
                     const int h_out = g * p.G + (head - qi * p.G);
                     const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h_out * p.o_sh + 4 * lane;
+                    if (!DA_IN_RANGE(p.status, b, p.B, 7) || !DA_IN_RANGE(p.status, h_out, p.Hkv * p.G, 8) ||
+                        !DA_IN_RANGE(p.status, qi, p.Lq, 9))
+                        continue;
                     if (p.out_bf16) {
                         __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
                         const uint32_t lo = pack_bf16(val.x, val.y), hi = pack_bf16(val.z, val.w);
@@ -1236,6 +1287,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     if (lane == 0 && p.lse)
                         p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h_out * p.l_sh] = lse_nat;
                 } else {
+                    if (!DA_IN_RANGE(p.status, slot, 2 * p.unit_cap, 10))
+                        continue;
                     st_global_v4_hint(p.part_o + ((int64_t)slot * HEADS + head) * HEAD_DIM + 4 * lane, val, part_policy);
                     if (lane == 0)
                         st_global_f32_hint(p.part_lse + (int64_t)slot * HEADS + head, lse_nat, part_policy);
@@ -1334,9 +1387,14 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
                 i -= per_block[j];
                 ++k;
             }
+        if (!DA_IN_RANGE(p.status, i, p.merge_seg, 11))
+            return make_int4(0, 0, 0, 0);   // (no splits: the entry is skipped below)
         return list[(size_t)k * p.merge_seg + i];
     };
     auto store = [&](int b, int qi, int h, float4 v, float lse_val) {
+        if (!DA_IN_RANGE(p.status, b, p.B, 12) || !DA_IN_RANGE(p.status, h, p.Hkv * p.G, 13) ||
+            !DA_IN_RANGE(p.status, qi, p.Lq, 14))
+            return;
         const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h * p.o_sh + d;
         if (p.out_bf16) {
             __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
@@ -1365,7 +1423,9 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
         int uu = e.z + k;
         if (e.z < n_full && uu >= n_full)
             uu += gap;   // skip the static units that hold no tiles
-        const int slot = (k == 0) ? e.y : 2 * uu;
+        int slot = (k == 0) ? e.y : 2 * uu;
+        if (valid && !DA_IN_RANGE(p.status, slot, 2 * p.unit_cap, 15))
+            slot = 0;
         const int n = min(k_end - k0, 32);
         auto row = [&](int sl) {
             return *reinterpret_cast<const float4 *>(p.part_o + ((int64_t)sl * p.heads_pad + head) * HEAD_DIM + d);
@@ -1435,6 +1495,10 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
     for (int item = (int)(gridDim.x - 1 - blockIdx.x); item < n_big * p.Gv; item += gridDim.x) {
         const int4 e = entry(p.merge_big, cnt.n_big, item / p.Gv);
         const int head = item % p.Gv;
+#ifdef DA_BOUNDS_CHECK
+        if (e.w == 0)
+            continue;   // an entry the check above refused
+#endif
         MergeAcc a = {-INFINITY, 0.f, make_float4(0.f, 0.f, 0.f, 0.f)};
         // the splits are dealt to the eight warps in equal chunks (of at least eight, the number of
         // rows a warp asks for at once), so that up to 64 splits cost one round trip to memory
@@ -1456,6 +1520,10 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
     for (int item = blockIdx.x * MERGE_WARPS + warp; item < n_small * p.Gv; item += gridDim.x * MERGE_WARPS) {
         const int4 e = entry(p.merge_small, cnt.n_small, item / p.Gv);
         const int head = item % p.Gv;
+#ifdef DA_BOUNDS_CHECK
+        if (e.w == 0)
+            continue;
+#endif
         finish(e, head, warp_merge(e, head, 0, e.w));
     }
     // ---- empty sequences

@@ -35,7 +35,7 @@ constexpr int PF_NB = 3;                     // K and V buffers (tiles in flight
 constexpr int PF_OFF_K = PF_TILE;
 constexpr int PF_OFF_V = (1 + PF_NB) * PF_TILE;
 constexpr int PF_OFF_BARS = (1 + 2 * PF_NB) * PF_TILE;   // kfull[3], vfull[3], kfree[3], o[3], s[2], p, x
-constexpr int PF_OFF_MISC = PF_OFF_BARS + 128;  // TMEM base address, abort flag
+constexpr int PF_OFF_MISC = PF_OFF_BARS + 128;  // TMEM base address, abort flag, "a page id was bad" flag
 constexpr int PF_OFF_XCHG = PF_OFF_MISC + 16;   // row maxima / sums swapped between a row's two threads
 constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + PF_TPR * 128 * 4;   // 2 buffers of bf16 maxima, or one of fp32 sums
 static_assert(PF_SMEM_BYTES <= 232448, "one block must fit the 227 KB of shared memory an SM offers");
@@ -193,6 +193,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     extern __shared__ __align__(1024) uint8_t smem[];   // no static shared memory: keeps the base 1024-B aligned
     uint32_t &tmem_base_s = *reinterpret_cast<uint32_t *>(smem + PF_OFF_MISC);
     int &abort_s = *reinterpret_cast<int *>(smem + PF_OFF_MISC + 4);
+    volatile int *poison_s = reinterpret_cast<volatile int *>(smem + PF_OFF_MISC + 8);
     const uint32_t sb = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // per K/V buffer (tile t uses buffer t % 3): K loaded, V loaded, K no longer needed (scores complete),
@@ -236,6 +237,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     }
     if (tid == 0) {
         abort_s = 0;
+        *poison_s = 0;
         for (int i = 0; i < PF_NB; ++i) {
             mbar_init(bar_kfull + 8 * i, 1);
             mbar_init(bar_vfull + 8 * i, 1);
@@ -309,16 +311,24 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 // extend: boxes wholly past the sequence's end are not loaded (their rows are masked)
                 const int t_tile = (t_begin + j) * PF_TOK;
                 const int nbox = p.ext ? min(boxes, (L - t_tile + p.box_rows - 1) / p.box_rows) : boxes;
-                if (lane == 0)
+                const bool mine = active && box < nbox;
+                const int t = t_tile + box * p.box_rows;
+                if (mine && (uint32_t)page >= (uint32_t)p.num_pages) {
+                    // A page id outside the pool.  The copy is made from just past the pool instead (the
+                    // tensor map fills zeros there and still counts the bytes), and the block is marked:
+                    // its rows are written as NaN, not as a finite result over zeroed keys.
+                    if (!is_v && pl == 0)
+                        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, bseq, t / p.P, page);
+                    *poison_s = 1;
+                    page = p.num_pages;
+                }
+                // (diagnostic build only: the K loader of block 0 can leave one tile out altogether)
+                const bool withheld = !is_v && DA_WITHHOLD(1, blockIdx.x, j);
+                __syncwarp();   // the mark above precedes lane 0's arrival, which the later stages build on
+                if (lane == 0 && !withheld)
                     mbar_arrive_expect_tx(bar, (uint32_t)(nbox * p.box_rows * 256));
                 __syncwarp();
-                if (active && box < nbox) {
-                    const int t = t_tile + box * p.box_rows;
-                    if ((uint32_t)page >= (uint32_t)p.num_pages) {
-                        if (!is_v && pl == 0)
-                            report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, bseq, t / p.P, page);
-                        page = p.num_pages;   // out of range: TMA fills zeros and still counts the bytes
-                    }
+                if (mine && !withheld) {
                     const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + box * p.box_rows * 128);
                     tma_load_4d(sb + (is_v ? PF_OFF_V : PF_OFF_K) + off, tm, pl * 64, t % p.P, g, page, bar);
                 }
@@ -348,7 +358,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     const int jk = issued - 1 - k;
                     const uint64_t t0 = globaltimer_ns();
                     while (jk >= 0 && !mbar_try_wait(bar_full + 8 * (jk % PF_NB), (uint32_t)((jk / PF_NB) & 1))) {
-                        if (globaltimer_ns() - t0 > 1000000000ull)
+                        if (globaltimer_ns() - t0 > DA_WAIT_LIMIT_NS / 2)
                             break;
                     }
                 }
@@ -461,7 +471,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         const int rr = rt * PF_ROWS + r;
         const int limit = (p.ext && rr < R && L > 0) ? L - p.Lq + rr / p.G + 1 : 0;
         for (int j = 0; j < ntiles; ++j) {
-            if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
+            if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                 ok = false;
                 break;
             }
@@ -501,7 +511,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_x);
-            if (!mbar_wait_bounded(bar_x, (uint32_t)(j & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
+            if (!mbar_wait_bounded(bar_x, (uint32_t)(j & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                 ok = false;
                 break;
             }
@@ -527,7 +537,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             // a row of O may be rescaled only once the previous tile's PV product is complete
             // (tcgen05.ld / .st are warp-wide: all lanes go)
             if (j > 0 && __any_sync(0xffffffffu, moved)) {
-                if (!mbar_wait_bounded(bar_o + 8 * ((j - 1) % PF_NB), (uint32_t)(((j - 1) / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
+                if (!mbar_wait_bounded(bar_o + 8 * ((j - 1) % PF_NB), (uint32_t)(((j - 1) / PF_NB) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                     ok = false;
                     break;
                 }
@@ -544,7 +554,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 // The tile reaches past the sequence's end: those V rows were not loaded, or are a page's
                 // unused tail, and may hold NaN, which a zero weight would not hide.  Clear them (both
                 // planes, 128 bytes a row) once V has landed, before the PV product reads them.
-                if (!mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
+                if (!mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                     ok = false;
                     break;
                 }
@@ -570,7 +580,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
         uint32_t o_raw[PF_COLS];
         if (ok && ntiles > 0) {
-            if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) % PF_NB), (uint32_t)(((ntiles - 1) / PF_NB) & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
+            if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) % PF_NB), (uint32_t)(((ntiles - 1) / PF_NB) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                 tc_fence_after();
                 tmem_ld32_issue(tmem_o + lane_base, o_raw);
                 tmem_ld_wait();
@@ -587,7 +597,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_x);
-            if (mbar_wait_bounded(bar_x, (uint32_t)(ntiles & 1), abort_flag, 2000000000ull, PF_WAIT_SLEEP_NS)) {
+            if (mbar_wait_bounded(bar_x, (uint32_t)(ntiles & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
 #pragma unroll
                 for (int q = 0; q < PF_TPR; ++q)
                     l_row += xb[q * 128 + r];
@@ -604,12 +614,14 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             if (rr < R) {
                 const int outer = rr / p.G, hd = rr % p.G;   // sequence (cascade) or query token (extend)
                 const bool any = ntiles > 0 && l_row > 0.f;
+                const bool poisoned = *poison_s != 0;   // (every copy of this block was issued long before)
+                const float nan = __int_as_float(0x7fc00000);
                 const float inv = any ? 1.f / l_row : 0.f;
-                const float lse_val = any ? (m_run + fast_log2(l_row)) * LN2 : -INFINITY;
+                const float lse_val = poisoned ? nan : (any ? (m_run + fast_log2(l_row)) * LN2 : -INFINITY);
                 float vals[PF_COLS];
 #pragma unroll
                 for (int i = 0; i < PF_COLS; ++i)
-                    vals[i] = any ? __uint_as_float(o_raw[i]) * inv : 0.f;
+                    vals[i] = poisoned ? nan : (any ? __uint_as_float(o_raw[i]) * inv : 0.f);
                 const int h = g * p.G + hd;
                 if (p.ext && p.splits == 1) {
                     const int64_t at = (int64_t)bseq * p.o_sb + (int64_t)outer * p.o_sq + (int64_t)h * p.o_sh + part * PF_COLS;
@@ -654,6 +666,8 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 struct CascadeMergeParams {
     const float *pre_o, *pre_lse;   // [splits][n][128], [splits][n]   with n = B * Lq * Hq
     const float *suf_o, *suf_lse;   // [n][128], [n]; may be NULL (extend: no separate suffix pass)
+    const int4 *seq_info;           // the suffix pass's plan {lo, L, ..}: L == 0 marks a sequence that is empty or
+                                    // was refused (shorter than the prefix) -> 0 / -inf; may be NULL
     void *out;
     int64_t o_sb, o_sq, o_sh;
     float *lse;
@@ -688,14 +702,21 @@ __global__ void __launch_bounds__(256) cascade_merge_kernel(const CascadeMergePa
         fold(p.suf_lse[idx], p.suf_o + idx * HEAD_DIM);
     for (int s = 0; s < p.splits; ++s)
         fold(p.pre_lse[(int64_t)s * n + idx], p.pre_o + ((int64_t)s * n + idx) * HEAD_DIM);
+    const int h = (int)(idx % p.Hq), qi = (int)((idx / p.Hq) % p.Lq), b = (int)(idx / ((int64_t)p.Hq * p.Lq));
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     float lse_val = -INFINITY;
-    if (den > 0.f) {
+    const bool empty = p.seq_info && p.seq_info[b].y == 0;
+    if (empty) {
+        // nothing to attend
+    } else if (den > 0.f) {
         const float inv = 1.f / den;
         v = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
         lse_val = M + __logf(den);
+    } else if (den != den) {
+        // a NaN partial (rows lost to a bad page id) makes the result NaN
+        v = make_float4(den, den, den, den);
+        lse_val = den;
     }
-    const int h = (int)(idx % p.Hq), qi = (int)((idx / p.Hq) % p.Lq), b = (int)(idx / ((int64_t)p.Hq * p.Lq));
     const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h * p.o_sh + d;
     if (p.out_bf16) {
         __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;

@@ -64,13 +64,29 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// How long a bounded wait may last.  The diagnostic build (-DDA_DIAG) reads the limit from a device
+// variable that a test can shorten, so that the give-up paths can be exercised in milliseconds by a
+// wait that nothing satisfies; the normal build has the constant.
+#ifdef DA_DIAG
+__device__ unsigned long long g_diag_wait_limit_ns = 2000000000ull;
+// The loader of thread block 0 leaves out the copies AND the barrier arrival of its tile number
+// g_diag_withhold[0] (partition kernel) / [1] (prefix kernel); -1: never.  Nothing is issued for that
+// tile, so nothing can land late; the warps that wait for it run into the limit above.
+__device__ int g_diag_withhold[2] = {-1, -1};
+#define DA_WAIT_LIMIT_NS (::da::g_diag_wait_limit_ns)
+#define DA_WITHHOLD(which, block, tile) ((block) == 0 && (int)(tile) == ::da::g_diag_withhold[(which)])
+#else
+#define DA_WAIT_LIMIT_NS 2000000000ull
+#define DA_WITHHOLD(which, block, tile) false
+#endif
+
 // Waits until the phase with the given parity has completed.  Every wait is bounded: after
 // `limit_ns` without completion, or as soon as another thread of the block has raised the
 // abort flag, it gives up and returns false, so a pipeline bug cannot hang the device.
 // `sleep_ns` > 0 makes a waiting warp yield its issue slots between probes (for waits whose
 // outcome depends on another warp of the same scheduler getting to run).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                                  uint64_t limit_ns = 2000000000ull, uint32_t sleep_ns = 0)
+                                                  uint64_t limit_ns, uint32_t sleep_ns = 0)
 {
     if (mbar_try_wait(bar, parity))
         return true;
@@ -90,6 +106,10 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
                 return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    return mbar_wait_bounded(bar, parity, abort_flag, DA_WAIT_LIMIT_NS, 0);
 }
 
 // Orders this thread's earlier generic-proxy shared-memory writes before later async-proxy

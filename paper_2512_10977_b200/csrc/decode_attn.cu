@@ -16,7 +16,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 108;
+constexpr int kVersion = 109;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -33,6 +33,9 @@ int64_t g_opt_kv_evict_first = 2; // L2 policy of the K and V loads: 0 normal, 1
 int64_t g_opt_extend_stream_rows = 16;   // decode_attn_extend: Lq * (Hq / Hkv) up to this many rows go through the
                                          // streaming (partition) kernel, more through the tcgen05 kernel; 0: never
 cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
+#ifdef DA_DIAG
+int64_t g_host_wait_limit_us = 2000000, g_host_withhold[2] = {-1, -1};   // host copies of the device variables
+#endif
 
 struct DeviceState {
     void *ws = nullptr;
@@ -247,6 +250,7 @@ int check_pool(const da_tensor *t, int32_t dtype = DA_BF16)
     if (!t->data) return DA_ERR_NULL;
     if (t->dtype != dtype) return DA_ERR_DTYPE;
     if (t->ndim != 4) return DA_ERR_SHAPE;
+    if (t->shape[0] <= 0 || t->shape[1] <= 0 || t->shape[2] <= 0) return DA_ERR_SHAPE;
     if (t->shape[3] != HEAD_DIM) return DA_ERR_UNSUPPORTED;
     if (t->stride[3] != 1 || !aligned16(t->data)) return DA_ERR_STRIDE_ALIGN;
     const int64_t item = dtype == DA_FP8_E4M3 ? 1 : 2;
@@ -416,6 +420,8 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pa.q_sq = q_sq;
     pa.o_sq = o_sq;
     pa.l_sq = l_sq;
+    pa.unit_cap = nblocks + n_tail;
+    pa.max_pages = d.max_pages;
     const int nt8 = pa.Gv <= 8 ? 1 : 2;
     const bool timed = g_ev_before && g_ev_after;
     if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
@@ -468,6 +474,8 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     mp.Gv = pa.Gv;
     mp.o_sq = o_sq;
     mp.l_sq = l_sq;
+    mp.unit_cap = pa.unit_cap;
+    mp.status = pa.status;
     cfg.gridDim = dim3((unsigned)(4 * st->sm_count));
     cfg.blockDim = dim3((unsigned)MERGE_THREADS);
     cfg.dynamicSmemBytes = 0;
@@ -640,6 +648,7 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     cm.pre_lse = pf.pre_lse;
     cm.suf_o = reinterpret_cast<const float *>(ws + lay.suf_o);
     cm.suf_lse = reinterpret_cast<const float *>(ws + lay.suf_lse);
+    cm.seq_info = reinterpret_cast<const int4 *>(ws + lay.seq_info);
     cm.out = out->data;
     cm.o_sb = out->stride[0];
     cm.o_sq = 0;
@@ -820,6 +829,7 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
     const int64_t B = q->shape[0], Lq = q->shape[1], Hq = q->shape[2];
     const int64_t Hkv = k_pages->shape[1], P = k_pages->shape[2], max_pages = block_table->shape[1];
     if (q->shape[3] != HEAD_DIM) return DA_ERR_UNSUPPORTED;
+    if (Hkv <= 0 || k_pages->shape[0] <= 0) return DA_ERR_SHAPE;   // (before Hkv divides anything)
     if (B < 0 || Lq <= 0 || Hq <= 0 || max_pages <= 0 || Hq % Hkv != 0) return DA_ERR_SHAPE;
     if (P != 16 && P != 32 && P != 64 && P != 128) return DA_ERR_UNSUPPORTED;
     if (B > (1 << 20) || Lq > (1 << 20) || k_pages->shape[0] > 0x7fffffffll || max_pages * P > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
@@ -931,6 +941,7 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
         cm.pre_lse = pf.pre_lse;
         cm.suf_o = nullptr;
         cm.suf_lse = nullptr;
+        cm.seq_info = nullptr;
         cm.out = out->data;
         cm.o_sb = pf.o_sb;
         cm.o_sq = pf.o_sq;
@@ -1237,6 +1248,24 @@ int decode_attn_set_option(const char *name, int64_t value)
         g_opt_extend_stream_rows = value;
         return DA_OK;
     }
+#ifdef DA_DIAG
+    // Diagnostic build only; each writes a device variable of the current device (synchronously).
+    if (std::strcmp(name, "diag_wait_limit_us") == 0) {
+        if (value < 1 || value > 2000000) return DA_ERR_UNSUPPORTED;
+        const unsigned long long ns = (unsigned long long)value * 1000ull;
+        DA_CUDA(cudaMemcpyToSymbol(da::g_diag_wait_limit_ns, &ns, sizeof ns));
+        g_host_wait_limit_us = value;
+        return DA_OK;
+    }
+    if (std::strcmp(name, "diag_withhold_partition_tile") == 0 || std::strcmp(name, "diag_withhold_prefix_tile") == 0) {
+        if (value < -1 || value > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+        const int which = std::strcmp(name, "diag_withhold_prefix_tile") == 0;
+        const int v = (int)value;
+        DA_CUDA(cudaMemcpyToSymbol(da::g_diag_withhold, &v, sizeof v, (size_t)which * sizeof(int)));
+        g_host_withhold[which] = value;
+        return DA_OK;
+    }
+#endif
     return DA_ERR_UNSUPPORTED;
 }
 
@@ -1249,6 +1278,11 @@ int64_t decode_attn_get_option(const char *name)
     if (std::strcmp(name, "static_frac") == 0) return g_opt_static_frac;
     if (std::strcmp(name, "kv_evict_first") == 0) return g_opt_kv_evict_first;
     if (std::strcmp(name, "extend_stream_rows") == 0) return g_opt_extend_stream_rows;
+#ifdef DA_DIAG
+    if (std::strcmp(name, "diag_wait_limit_us") == 0) return g_host_wait_limit_us;
+    if (std::strcmp(name, "diag_withhold_partition_tile") == 0) return g_host_withhold[0];
+    if (std::strcmp(name, "diag_withhold_prefix_tile") == 0) return g_host_withhold[1];
+#endif
     return -1;
 }
 

@@ -24,7 +24,7 @@ def main() -> None:
     args = ap.parse_args()
 
     from . import binding, build
-    binding.use_library(build.build_timeline())
+    binding.use_library(build.build_diag())
     import torch
     sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
     import workloads

@@ -53,6 +53,13 @@ def test_the_normal_build_keeps_no_timeline(pkg):
         pkg.timeline()
 
 
+def test_the_normal_build_knows_no_diagnostic_option(pkg):
+    # shortening the kernels' wait limit or withholding a tile exists only in the diagnostic build
+    for name in ("diag_wait_limit_us", "diag_withhold_partition_tile", "diag_withhold_prefix_tile"):
+        assert pkg.lib().decode_attn_set_option(name.encode(), 1) == 5   # DA_ERR_UNSUPPORTED
+        assert pkg.get_option(name) == -1
+
+
 def test_options(pkg):
     assert pkg.get_option("grid_blocks") == 0
     pkg.set_option("grid_blocks", 7)

@@ -92,16 +92,39 @@ def test_cascade_argument_and_device_errors(da):
     assert e.value.status == 2                                   # longer than a block-table row
     sl = case.seq_lens.clone()
     sl[1] = 100                                                  # shorter than the prefix
-    da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, sl, 256, case.scale)
+    out, lse = da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, sl, 256, case.scale)
     assert da.read_device_status()[0] == 2
+    # ... and that sequence is treated as empty, the others are unaffected
+    assert (out[1] == 0).all() and torch.isneginf(lse[1]).all()
+    want, want_lse = da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens, 256, case.scale)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    keep = [b for b in range(case.q.shape[0]) if b != 1]
+    assert torch.allclose(out[keep], want[keep], atol=2e-5, rtol=1e-4) and torch.allclose(lse[keep], want_lse[keep], atol=2e-5, rtol=1e-4)
+    # a page id outside the pool inside the shared prefix: every row attends it, so every row is NaN
+    bt = case.block_table.clone()
+    bt[:, 3] = 10 ** 6
+    out, lse = da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, bt, case.seq_lens, 256, case.scale)
+    st = da.read_device_status()
+    assert st[0] == 1 and st[3] == 10 ** 6
+    assert torch.isnan(out).all() and torch.isnan(lse).all()
+    # ... and one in a single sequence's own tokens marks that sequence only
+    bt = case.block_table.clone()
+    own = 256 // case.k_pages.shape[2]                           # first page after the prefix
+    b_long = int(torch.argmax(case.seq_lens))
+    bt[b_long, own] = -7
+    out, lse = da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, bt, case.seq_lens, 256, case.scale)
+    assert da.read_device_status()[0] == 1
+    assert torch.isnan(out[b_long]).all() and torch.isnan(lse[b_long]).all()
+    keep = [b for b in range(case.q.shape[0]) if b != b_long]
+    assert torch.allclose(out[keep], want[keep], atol=2e-5, rtol=1e-4) and torch.allclose(lse[keep], want_lse[keep], atol=2e-5, rtol=1e-4)
 
 
-def test_c5a_full_size_cascade_sampled(da):
+def test_c5a_full_size_cascade_every_fourth_sequence(da):
     case = workloads.c5("cuda", 0)
     out, lse = da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
                                       16384, case.scale)
     assert da.read_device_status() == (0, 0, 0, 0)
-    ids = [0, int(np.argmin(case.lens)), int(np.argmax(case.lens)), 77]
+    ids = sorted(set(range(0, case.B, 4)) | {int(np.argmin(case.lens)), int(np.argmax(case.lens)), 77})
     sub = workloads.host_subcase(case, ids)
     ref, ref_lse = oracle.decode_attn_oracle(sub.q, sub.k_pages, sub.v_pages, sub.block_table, sub.seq_lens, 0, sub.scale)
     assert_close(out[ids].cpu().numpy(), ref, "c5a cascade out")

@@ -290,7 +290,7 @@ def test_device_side_errors_set_the_status_word_without_faulting(da):
 
 # ------------------------------------------------------------------ the workloads at full size
 
-def _sampled_full_size(da, case, ids, what):
+def _full_size(da, case, ids, what):
     out, lse = da.decode_attn_fp8kv(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table,
                                     case.seq_lens, case.window, case.scale)
     assert da.read_device_status() == (0, 0, 0, 0)
@@ -301,22 +301,22 @@ def _sampled_full_size(da, case, ids, what):
     assert_close(lse[ids].cpu().numpy(), ref_lse, what + " lse")
 
 
-def test_c2_full_size_sampled(da):
+def test_c2_full_size_every_sequence(da):
     da.set_option("grid_blocks", 0)
     case = workloads.c2("cuda", kv_dtype="fp8")
-    ids = sorted({int(np.argmin(case.lens)), int(np.argmax(case.lens)), 0, 31, 63})
-    _sampled_full_size(da, case, ids, "c2 fp8")
+    _full_size(da, case, list(range(case.B)), "c2 fp8")
 
 
-def test_c4_long_context_page64_sampled(da):
+def test_c4_long_context_page64_every_sequence(da):
     da.set_option("grid_blocks", 0)
-    _sampled_full_size(da, workloads.c4("cuda", kv_dtype="fp8"), [0, 7], "c4 fp8")
+    case = workloads.c4("cuda", kv_dtype="fp8")
+    _full_size(da, case, list(range(case.B)), "c4 fp8")
 
 
-def test_c5b_window_sampled(da):
+def test_c5b_window_every_eighth_sequence(da):
     da.set_option("grid_blocks", 0)
     case = workloads.c5("cuda", 8192, kv_dtype="fp8")
-    _sampled_full_size(da, case, [0, int(np.argmax(case.lens))], "c5b fp8")
+    _full_size(da, case, sorted(set(range(0, case.B, 8)) | {int(np.argmax(case.lens))}), "c5b fp8")
 
 
 # ------------------------------------------------------------------ quantising append, bit-exact
@@ -386,11 +386,11 @@ def test_decode_loop_append_then_attend(da):
     assert torch.equal(dev.k_pages.cpu(), case.k_pages) and torch.equal(dev.v_pages.cpu(), case.v_pages)
 
 
-def test_c3_scattered_in_large_pool_sampled(da):
+def test_c3_scattered_in_large_pool_every_fourth_sequence(da):
     da.set_option("grid_blocks", 0)
     case = workloads.c3("cuda", kv_dtype="fp8")
-    ids = sorted({int(np.argmin(case.lens)), int(np.argmax(case.lens)), 5, 128, 255})
-    _sampled_full_size(da, case, ids, "c3 fp8")
+    ids = sorted(set(range(0, case.B, 4)) | {int(np.argmin(case.lens)), int(np.argmax(case.lens))})
+    _full_size(da, case, ids, "c3 fp8")
 
 
 def test_host_io_matches_device_call(da):

@@ -14,7 +14,7 @@ import sys
 sys.path.insert(0, %r)
 import numpy as np, torch
 from paper_2512_10977_b200 import binding, build
-binding.use_library(build.build_timeline())
+binding.use_library(build.build_diag())
 import oracle, workloads
 case = workloads.build_case("tl", [2500, 3, 900, 0, 64, 4097, 130, 9000], 16, 5, "cpu")
 ref, ref_lse = oracle.decode_attn_oracle(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens, 0, case.scale)

@@ -2,7 +2,8 @@
 (a server whose KV-cache pool owns all of HBM, or a step that cannot take cudaMalloc's
 device-wide synchronisation).  Its scratch is a fixed array inside the library, shared by every
 call, so the check runs it twice in a row on different batches and compares each result with
-what decode_attn() gives for the same inputs through its caller-provided workspace.
+what decode_attn() gives for the same inputs through its caller-provided workspace -- and with the
+fp64 CPU oracle, so that a slip the two entry points share would not pass either.
 
 Collected last on purpose: a run that stops at the first failure has then already run every
 other test."""
@@ -10,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import workloads
 
 pytestmark = pytest.mark.gpu
@@ -33,14 +35,19 @@ def test_static_scratch_matches_decode_attn_on_two_calls_in_a_row():
         da.decode_attn_static_scratch(c.q, c.k_pages, c.v_pages, c.block_table, c.seq_lens, c.window, c.scale,
                                       o, l, s)
     torch.cuda.synchronize()
-    for (w_out, w_lse), o, l, s in zip(want, outs, lses, status):
+    for c, (w_out, w_lse), o, l, s in zip(cases, want, outs, lses, status):
         assert s.tolist() == [0, 0, 0, 0]
-        got, ref = o.cpu().numpy().astype(np.float64), w_out.cpu().numpy().astype(np.float64)
-        assert (np.abs(got - ref) <= 1e-3 + 1e-3 * np.abs(ref)).all()
-        gl, rl = l.cpu().numpy().astype(np.float64), w_lse.cpu().numpy().astype(np.float64)
-        both_ninf = np.isneginf(gl) & np.isneginf(rl)      # empty sequences: -inf on both sides
-        gl, rl = np.where(both_ninf, 0.0, gl), np.where(both_ninf, 0.0, rl)
-        assert (np.abs(gl - rl) <= 1e-3 + 1e-3 * np.abs(rl)).all()
+        host = workloads.to_device(c, "cpu")
+        o_ref, l_ref = oracle.decode_attn_oracle(host.q, host.k_pages, host.v_pages, host.block_table,
+                                                 host.seq_lens, host.window, host.scale)
+        for ref, rl in ((w_out.cpu().numpy().astype(np.float64), w_lse.cpu().numpy().astype(np.float64)),
+                        (np.asarray(o_ref, dtype=np.float64), np.asarray(l_ref, dtype=np.float64))):
+            got = o.cpu().numpy().astype(np.float64)
+            assert (np.abs(got - ref) <= 1e-3 + 1e-3 * np.abs(ref)).all()
+            gl = l.cpu().numpy().astype(np.float64)
+            both_ninf = np.isneginf(gl) & np.isneginf(rl)      # empty sequences: -inf on both sides
+            gl, rl = np.where(both_ninf, 0.0, gl), np.where(both_ninf, 0.0, rl)
+            assert (np.abs(gl - rl) <= 1e-3 + 1e-3 * np.abs(rl)).all()
 
 
 def test_static_scratch_reports_device_errors_and_refuses_oversize_batches():
