@@ -398,6 +398,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     const int u_end = ((int)blockIdx.x < nblk) ? min(u_begin + slice, units_max) : u_begin;
     int4 *my_small = p.merge_small + (size_t)blockIdx.x * p.merge_seg;
     int4 *my_big = p.merge_big + (size_t)blockIdx.x * p.merge_seg;
+    // room in this block's segment of the lists; a block that cuts all the units alone (nblk == 1) fills
+    // the segments one after another, which the merge kernel's walk over the per-block counts reads back
+    // as one contiguous list
+    [[maybe_unused]] const int list_room = nblk == 1 ? p.merge_seg * PLAN_BLOCKS : p.merge_seg;
     for (int u = u_begin + tid; u < u_end; u += PLAN_THREADS) {
         int4 uw = make_int4(0, 0, 0, 0);
         if (u < n_units) {
@@ -430,11 +434,11 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
                         const int4 e = make_int4(b * p.Hkv + g, 2 * prev + (prev_start == w0 ? 0 : 1), prev, ns);
                         if (ns > MERGE_WARP_SPLITS) {
                             const int at = atomicAdd(&n_big_s, 1);
-                            if (DA_IN_RANGE(p.status, at, p.merge_seg, 1))
+                            if (DA_IN_RANGE(p.status, at, list_room, 1))
                                 my_big[at] = e;
                         } else {
                             const int at = atomicAdd(&n_small_s, 1);
-                            if (DA_IN_RANGE(p.status, at, p.merge_seg, 2))
+                            if (DA_IN_RANGE(p.status, at, list_room, 2))
                                 my_small[at] = e;
                         }
                     }
@@ -965,11 +969,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         }
                     }
                 }
-                // ---- weights w = 2^15 * exp2(s - m) as f16 high and low parts (together ~22 bits of each
-                //      weight; the factor 2^15 keeps weights down to 2^-39 of the largest representable),
-                //      transposed into the B operand of O^T += V^T P^T.  ph[n][q]: block q = rows 0-7 / 8-15
-                //      of tile A, then of tile B.
-                uint32_t ph[NT8][4], pl[NT8][4];
+                // ---- weights w = 2^15 * exp2(s - m) rounded to f16 (11 significant bits: each weight is off
+                //      by at most 2^-11 of itself, so a row of the result by at most 2^-11 * sum_t p_t |v_t|,
+                //      half the 1e-3 bar for values of unit size; the sum of weights keeps the unrounded
+                //      values.  The factor 2^15 keeps weights down to 2^-29 of the largest in f16's normal
+                //      range), transposed into the B operand of O^T += V^T P^T.  ph[n][q]: block q = rows
+                //      0-7 / 8-15 of tile A, then of tile B.
+                uint32_t ph[NT8][4];
 #pragma unroll
                 for (int n = 0; n < NT8; ++n) {
                     float w[8];
@@ -984,13 +990,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     l_run[n][0] += (w[0] + w[2]) + (w[4] + w[6]);
                     l_run[n][1] += (w[1] + w[3]) + (w[5] + w[7]);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint32_t hi = pack_f16(w[2 * q], w[2 * q + 1]);
-                        const float2 hv = unpack_f16(hi);
-                        const uint32_t lo = pack_f16(w[2 * q] - hv.x, w[2 * q + 1] - hv.y);
-                        ph[n][q] = movmatrix_trans(hi);
-                        pl[n][q] = movmatrix_trans(lo);
-                    }
+                    for (int q = 0; q < 4; ++q)
+                        ph[n][q] = movmatrix_trans(pack_f16(w[2 * q], w[2 * q + 1]));
                 }
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -1004,10 +1005,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         vf[2] = e4m3x2_hi_to_f16x2(cv[2 * hf]);
                         vf[3] = e4m3x2_hi_to_f16x2(cv[2 * hf + 1]);
 #pragma unroll
-                        for (int n = 0; n < NT8; ++n) {
+                        for (int n = 0; n < NT8; ++n)
                             mma_f16_16816(o[n][j], vf, ph[n][2 * hf], ph[n][2 * hf + 1]);
-                            mma_f16_16816(o[n][j], vf, pl[n][2 * hf], pl[n][2 * hf + 1]);
-                        }
                     }
                 }
                 if (ragged)
@@ -1387,7 +1386,7 @@ __global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergePara
                 i -= per_block[j];
                 ++k;
             }
-        if (!DA_IN_RANGE(p.status, i, p.merge_seg, 11))
+        if (!DA_IN_RANGE(p.status, (long long)k * p.merge_seg + i, (long long)p.merge_seg * PLAN_BLOCKS, 11))
             return make_int4(0, 0, 0, 0);   // (no splits: the entry is skipped below)
         return list[(size_t)k * p.merge_seg + i];
     };

@@ -118,3 +118,15 @@ def test_null_and_malformed_arguments_are_rejected_before_any_cuda_call(pkg):
     assert call(q, k, v, bt, sl, view(3, (B, Hq, D)), lse) == 3                   # out dtype
     null_q = view(1, (B, Hq, D), data=0)
     assert call(null_q, k, v, bt, sl, out, lse) == 1
+    # pools without KV heads or without pages: a status, never a division fault on the host -- from the
+    # single-token call and from the multi-token one (whose group size is Hq / Hkv)
+    def pool(shape):
+        t = view(1, shape)
+        t.stride[0], t.stride[1], t.stride[2] = P * D * 8, P * D, D      # (zero extents must not make zero strides)
+        return t
+    q4, out4, lse3 = view(1, (B, 1, Hq, D)), view(2, (B, 1, Hq, D)), view(2, (B, 1, Hq))
+    ext = lambda kk, vv: L.decode_attn_extend(ctypes.byref(q4), ctypes.byref(kk), ctypes.byref(vv), ctypes.byref(bt),
+                                              ctypes.byref(sl), 1.0, ctypes.byref(out4), ctypes.byref(lse3), None)
+    for shape in ((10, 0, P, D), (0, Hkv, P, D)):
+        assert call(q, pool(shape), pool(shape), bt, sl, out, lse) == 2
+        assert ext(pool(shape), pool(shape)) == 2

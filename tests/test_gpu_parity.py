@@ -449,15 +449,15 @@ def test_host_side_argument_errors(da):
     with pytest.raises(TypeError):
         call(**args(bt=case.block_table.long()))
     # pools without KV heads or without pages: refused with a status (never a division fault on the host),
-    # by the single-token call and by the multi-token one
+    # by the single-token call and by the multi-token one (torch hands an empty tensor over as a NULL pointer)
     q4 = case.q[:, None].contiguous()
     for k, v in ((case.k_pages[:, :0], case.v_pages[:, :0]), (case.k_pages[:0], case.v_pages[:0])):
         with pytest.raises(da.DecodeAttnError) as e:
             call(**args(k=k, v=v))
-        assert e.value.status == 2
+        assert e.value.status in (1, 2)
         with pytest.raises(da.DecodeAttnError) as e:
             da.decode_attn_extend(q4, k, v, case.block_table, case.seq_lens, 1.0)
-        assert e.value.status == 2
+        assert e.value.status in (1, 2)
     assert da.read_device_status() == (0, 0, 0, 0)
 
 
