@@ -41,17 +41,30 @@ constexpr float LN2 = 0.6931471805599453f;
 // the merge kernel's first eight blocks -- 0 resident, 1 released by the partition kernel, 2 exit;
 // row TL_MERGE + 8, column 2: the latest exit of any merge block.  Rows TL_PLAN .. + 7: the plan
 // kernel's blocks -- 0 entry, 1 exit, 2 past the wait for the kernel before it in the stream, 3 lengths scanned, 4 cut made,
-// 5 units written.  In the normal build DA_TL() is empty and nothing is kept.
-constexpr int TL_ROWS = 1048, TL_COLS = 8, TL_MERGE = 1024, TL_PLAN = 1036;
+// 5 units written.  Rows TL_PREFIX .. + 5: thread block 0 of the prefix kernel, cycles (clock64) that one
+// warp of each role spent in its phases, summed over the block's tiles -- softmax warp 0: 0 waiting for the
+// scores, 1 loading them and agreeing on the row maximum, 2 weights (exp2, high/low parts, a rescale of O),
+// 3 storing P and arriving, 4 after the last tile, 5 tiles, 6 cycles from entry to the end, 7 the same span
+// in ns; score MMA warp: 0 waiting for the PV products, 1 for K, 2 issuing; the two PV MMA warps: 0 waiting for
+// P, 1 for V, 2 issuing; the K and V loader warps: 0 waiting for a free buffer, 1 issuing the copies.
+// In the normal build DA_TL() is empty and nothing is kept.
+constexpr int TL_ROWS = 1056, TL_COLS = 8, TL_MERGE = 1024, TL_PLAN = 1036, TL_PREFIX = 1044;
 #ifdef DA_TIMELINE
 __device__ unsigned long long g_timeline[TL_ROWS][TL_COLS];
 #define DA_TL(row, col) (g_timeline[(row)][(col)] = globaltimer_ns())
 #define DA_TL_SET(row, col, value) (g_timeline[(row)][(col)] = (unsigned long long)(value))
 #define DA_TL_MAX(row, col) atomicMax(&g_timeline[(row)][(col)], (unsigned long long)globaltimer_ns())
+// phase counters: `acc` is a per-thread array, DA_PH(acc, slot, t) adds the cycles since t and restarts t
+#define DA_PH_DECL(acc, t) long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long t = clock64()
+#define DA_PH(acc, slot, t) do { const long long now_ = clock64(); acc[(slot)] += now_ - (t); (t) = now_; } while (0)
+#define DA_PH_STORE(row, acc) do { for (int i_ = 0; i_ < 8; ++i_) g_timeline[(row)][i_] = (unsigned long long)acc[i_]; } while (0)
 #else
 #define DA_TL(row, col) ((void)0)
 #define DA_TL_SET(row, col, value) ((void)0)
 #define DA_TL_MAX(row, col) ((void)0)
+#define DA_PH_DECL(acc, t) ((void)0)
+#define DA_PH(acc, slot, t) ((void)0)
+#define DA_PH_STORE(row, acc) ((void)0)
 #endif
 
 // flags of a tile's descriptor (written by the producer warp, read by the consumer warps)
@@ -969,13 +982,11 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         }
                     }
                 }
-                // ---- weights w = 2^15 * exp2(s - m) rounded to f16 (11 significant bits: each weight is off
-                //      by at most 2^-11 of itself, so a row of the result by at most 2^-11 * sum_t p_t |v_t|,
-                //      half the 1e-3 bar for values of unit size; the sum of weights keeps the unrounded
-                //      values.  The factor 2^15 keeps weights down to 2^-29 of the largest in f16's normal
-                //      range), transposed into the B operand of O^T += V^T P^T.  ph[n][q]: block q = rows
-                //      0-7 / 8-15 of tile A, then of tile B.
-                uint32_t ph[NT8][4];
+                // ---- weights w = 2^15 * exp2(s - m) as f16 high and low parts (together ~22 bits of each
+                //      weight; the factor 2^15 keeps weights down to 2^-39 of the largest representable),
+                //      transposed into the B operand of O^T += V^T P^T.  ph[n][q]: block q = rows 0-7 / 8-15
+                //      of tile A, then of tile B.
+                uint32_t ph[NT8][4], pl[NT8][4];
 #pragma unroll
                 for (int n = 0; n < NT8; ++n) {
                     float w[8];
@@ -990,8 +1001,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     l_run[n][0] += (w[0] + w[2]) + (w[4] + w[6]);
                     l_run[n][1] += (w[1] + w[3]) + (w[5] + w[7]);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        ph[n][q] = movmatrix_trans(pack_f16(w[2 * q], w[2 * q + 1]));
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t hi = pack_f16(w[2 * q], w[2 * q + 1]);
+                        const float2 hv = unpack_f16(hi);
+                        const uint32_t lo = pack_f16(w[2 * q] - hv.x, w[2 * q + 1] - hv.y);
+                        ph[n][q] = movmatrix_trans(hi);
+                        pl[n][q] = movmatrix_trans(lo);
+                    }
                 }
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -1005,8 +1021,10 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         vf[2] = e4m3x2_hi_to_f16x2(cv[2 * hf]);
                         vf[3] = e4m3x2_hi_to_f16x2(cv[2 * hf + 1]);
 #pragma unroll
-                        for (int n = 0; n < NT8; ++n)
+                        for (int n = 0; n < NT8; ++n) {
                             mma_f16_16816(o[n][j], vf, ph[n][2 * hf], ph[n][2 * hf + 1]);
+                            mma_f16_16816(o[n][j], vf, pl[n][2 * hf], pl[n][2 * hf + 1]);
+                        }
                     }
                 }
                 if (ragged)

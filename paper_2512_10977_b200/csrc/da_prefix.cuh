@@ -10,10 +10,13 @@
 // max / sum in the log2 domain, write P = exp2(S - m) as bf16 high and low parts over their scores in tensor
 // memory -> O += P_hi V + P_lo V (tcgen05.mma with the A operand in TMEM, accumulating in another TMEM
 // region) -> the softmax threads rescale a row of O in TMEM only when its maximum has grown by more than
-// 2^8 (rare).  One more warp issues the MMAs and two more the TMA loads, one for K and one for V (issuing a
-// tile's tensor copies is slow enough that one warp doing it all set the pace of the block).  Result: a
-// normalised partial (O / l, lse) per (split, b, h), combined with the per-sequence suffix attention by
-// cascade_merge_kernel.
+// 2^8 (rare).  Three more warps issue the MMAs -- one the score products, one the P_hi V products, one the
+// P_lo V products into an accumulator of its own: a thread that issues a tcgen05.mma is held for about
+// 70 ns, longer than the tensor core needs for a 128 x 128 x 16 product, so a single issuing thread keeps
+// the pipe less than half busy; issued from several warps the same instructions run back to back -- and two
+// more the TMA loads, one for K and one for V (issuing a tile's tensor copies is slow enough that one warp
+// doing it all set the pace of the block).  Result: a normalised partial (O / l, lse) per (split, b, h),
+// combined with the per-sequence suffix attention by cascade_merge_kernel.
 #pragma once
 #include "da_kernels.cuh"
 
@@ -25,8 +28,9 @@ constexpr int PF_PLANE = PF_TOK * 128;       // one 64-column half of a 128-row 
 constexpr int PF_TILE = 2 * PF_PLANE;        // 32 KB: Q, a K tile, a V tile
 constexpr int PF_TPR = 4;                    // softmax threads per row (each owns 128 / PF_TPR columns of a tile)
 constexpr int PF_COLS = 128 / PF_TPR;
-constexpr int PF_DRV = 4 * PF_TPR;           // warps 0..15: softmax; warp 16: issues the MMAs (and owns the TMEM
-constexpr int PF_LOADER = PF_DRV + 1;        // allocation); warp 17: issues the TMA loads of K, warp 18 those of V
+constexpr int PF_DRV = 4 * PF_TPR;           // warps 0..15: softmax; warp 16: issues the score MMAs (and owns the TMEM
+constexpr int PF_PV = PF_DRV + 1;            // allocation); warps 17, 18: issue the P_hi V and the P_lo V MMAs;
+constexpr int PF_LOADER = PF_DRV + 3;        // warp 19: issues the TMA loads of K, warp 20 those of V
 constexpr int PF_THREADS = (PF_LOADER + 2) * 32;   // (one tensor copy costs its issuing warp ~90 cycles)
 constexpr int PF_OFF_Q = 0;
 constexpr float PF_RESCALE_LOG2 = 8.f;       // a row's reference maximum moves only when the maximum grew by more
@@ -39,7 +43,8 @@ constexpr int PF_OFF_MISC = PF_OFF_BARS + 128;  // TMEM base address, abort flag
 constexpr int PF_OFF_XCHG = PF_OFF_MISC + 16;   // row maxima / sums swapped between a row's two threads
 constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + PF_TPR * 128 * 4;   // 2 buffers of bf16 maxima, or one of fp32 sums
 static_assert(PF_SMEM_BYTES <= 232448, "one block must fit the 227 KB of shared memory an SM offers");
-constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O_tile in [256,384).
+constexpr int PF_TMEM_COLS = 512;            // S buffers in columns [0,128) and [128,256), O in [256,384) (the P_hi V
+                                             // products) and [384,512) (the P_lo V products; added at the end).
 constexpr int PF_TMEM_PH = 0;                // P(j) overwrites S(j) in place once both threads of a row have read
 constexpr int PF_TMEM_PL = 64;               // their scores: high parts in the buffer's columns [0,64), low parts in
                                              // [64,128) -- 128 tokens as 64 columns of bf16 pairs, the A operand of
@@ -242,7 +247,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             mbar_init(bar_kfull + 8 * i, 1);
             mbar_init(bar_vfull + 8 * i, 1);
             mbar_init(bar_kfree + 8 * i, 1);
-            mbar_init(bar_o + 8 * i, 1);
+            mbar_init(bar_o + 8 * i, 2);   // the two PV products of a tile, committed by their issuing warps
         }
         mbar_init(bar_s, 1);
         mbar_init(bar_s + 8, 1);
@@ -278,7 +283,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
-    const uint32_t tmem_s = tmem, tmem_o = tmem + 256;   // S(j) lives at tmem_s + 128 * (j & 1)
+    const uint32_t tmem_s = tmem, tmem_o = tmem + 256, tmem_o2 = tmem + 384;   // S(j) lives at tmem_s + 128 * (j & 1)
 
     if (warp == PF_LOADER || warp == PF_LOADER + 1) {
         // ------------------------------------------------------------------ loader warps: TMA
@@ -335,16 +340,21 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 issued = j + 1;
             };
             int pg = read_page(0);
+            DA_PH_DECL(ph, ph_t);
             for (int t = 0; ok && t < ntiles; ++t) {
                 if (t >= PF_NB) {
                     ok = mbar_wait_bounded(bar_free + 8 * (t % PF_NB), (uint32_t)(((t - PF_NB) / PF_NB) & 1), abort_flag);
                     if (!ok)
                         break;
                 }
+                DA_PH(ph, 0, ph_t);
                 const int pg_now = pg;
                 pg = read_page(t + 1);   // fetched one tile ahead
                 load_tile(t, pg_now);
+                DA_PH(ph, 1, ph_t);
             }
+            if (blockIdx.x == 0 && lane == 0)
+                DA_PH_STORE(TL_PREFIX + 4 + (int)is_v, ph);
             if (!ok && lane == 0) {
                 if (*abort_flag == 0) {
                     *abort_flag = 1;
@@ -365,21 +375,17 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         }
     } else if (warp == PF_DRV) {
-        // ------------------------------------------------------------------ MMA warp
-        // All lanes wait together; lane 0 issues.  Order on the tensor core: S(0), S(1), then for every
-        // tile j: PV(j) as soon as P(j) is written, and S(j+2) into the S buffer the softmax of j has
-        // just released -- so the scores of tile j+1 are ready before the softmax of j ends.
+        // ------------------------------------------------------------------ score MMA warp
+        // All lanes wait together; lane 0 issues.  S(0), S(1), then S(j+2) into the S buffer of tile j as
+        // soon as both PV products of tile j are complete (they read P(j) from that buffer) -- so the scores
+        // of tile j+1 are ready before the softmax of j ends.  Nothing is computed per instruction that can
+        // be computed once: the matrix descriptors of Q and of the first K buffer are built here, and a step
+        // or a buffer only adds a constant to the descriptor's address field (bits 0-13, in 16-byte units).
         if (ntiles > 0) {
             bool ok = true;
-            // The issuing thread is the narrowest part of the kernel (one tcgen05.mma takes ~70 cycles
-            // to execute), so nothing is computed per instruction that can be computed once: the matrix
-            // descriptors of Q and of the first K and V buffers are built here, and a step or a buffer
-            // only adds a constant to the descriptor's address field (bits 0-13, in 16-byte units).
             const uint64_t q_desc = umma_desc(sb + PF_OFF_Q, 16, 1024);
             const uint64_t k_desc = umma_desc(sb + PF_OFF_K, 16, 1024);
-            const uint64_t v_desc = umma_desc(sb + PF_OFF_V, PF_PLANE, 1024);
             const uint32_t idesc_s = umma_idesc(PF_ROWS, PF_TOK, false);
-            const uint32_t idesc_o = umma_idesc(PF_ROWS, HEAD_DIM, true);
             static_assert(PF_OFF_V + PF_NB * PF_TILE <= (1 << 18), "descriptor addresses must stay inside 256 KB");
             auto mma_s = [&](int j) {   // S = Q K^T for tile j
                 const uint64_t kd = k_desc + (uint64_t)(((j % PF_NB) * PF_TILE) >> 4);
@@ -390,21 +396,6 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 }
                 umma_commit(bar_s + 8 * (j & 1));
                 umma_commit(bar_kfree + 8 * (j % PF_NB));
-            };
-            auto mma_o = [&](int j) {   // O_tile = P_hi V + P_lo V for tile j
-                const uint64_t vd = v_desc + (uint64_t)(((j % PF_NB) * PF_TILE) >> 4);
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const uint32_t pa = tmem_s + 128 * (j & 1) + (half ? PF_TMEM_PL : PF_TMEM_PH);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        // A = P from tensor memory (16 tokens = 8 columns per step); B = V stored
-                        // [token][d]: MN-major, planes are the two halves of d (leading offset = plane),
-                        // 8-token groups 1024 B apart
-                        umma_bf16_ts(tmem_o, pa + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || half > 0 || kk > 0);
-                    }
-                }
-                umma_commit(bar_o + 8 * (j % PF_NB));
             };
             auto kfull = [&](int j) {
                 return mbar_wait_bounded(bar_kfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag);
@@ -418,28 +409,64 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     __syncwarp();
                 }
             }
-            for (int j = 0; ok && j < ntiles; ++j) {
-                ok = mbar_wait_bounded(bar_p, (uint32_t)(j & 1), abort_flag) &&
-                     mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag);
+            DA_PH_DECL(ph, ph_t);
+            for (int j = 0; ok && j + 2 < ntiles; ++j) {
+                ok = mbar_wait_bounded(bar_o + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag);
+                DA_PH(ph, 0, ph_t);
+                ok = ok && kfull(j + 2);
+                DA_PH(ph, 1, ph_t);
                 if (!ok)
                     break;
                 tc_fence_after();
                 if (lane == 0)
-                    mma_o(j);
+                    mma_s(j + 2);
                 __syncwarp();
-                if (j + 2 < ntiles) {
-                    ok = kfull(j + 2);
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-                    if (lane == 0)
-                        mma_s(j + 2);
-                    __syncwarp();
-                }
+                DA_PH(ph, 2, ph_t);
             }
+            if (blockIdx.x == 0 && lane == 0)
+                DA_PH_STORE(TL_PREFIX + 1, ph);
             if (!ok && lane == 0 && *abort_flag == 0) {
                 *abort_flag = 1;
                 report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -7, (int)blockIdx.x, 0);
+            }
+        }
+    } else if (warp == PF_PV || warp == PF_PV + 1) {
+        // ------------------------------------------------------------------ PV MMA warps
+        // Warp PF_PV accumulates P_hi V in tmem_o, warp PF_PV + 1 P_lo V in tmem_o2: for every tile, as soon
+        // as P is written and V has landed.  A = P from tensor memory (16 tokens = 8 columns per step);
+        // B = V stored [token][d]: MN-major, planes are the two halves of d (leading offset = plane),
+        // 8-token groups 1024 B apart.
+        if (ntiles > 0) {
+            bool ok = true;
+            const bool low = warp == PF_PV + 1;
+            const uint64_t v_desc = umma_desc(sb + PF_OFF_V, PF_PLANE, 1024);
+            const uint32_t idesc_o = umma_idesc(PF_ROWS, HEAD_DIM, true);
+            const uint32_t acc = low ? tmem_o2 : tmem_o;
+            DA_PH_DECL(ph, ph_t);
+            for (int j = 0; ok && j < ntiles; ++j) {
+                ok = mbar_wait_bounded(bar_p, (uint32_t)(j & 1), abort_flag);
+                DA_PH(ph, 0, ph_t);
+                ok = ok && mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag);
+                DA_PH(ph, 1, ph_t);
+                if (!ok)
+                    break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint64_t vd = v_desc + (uint64_t)(((j % PF_NB) * PF_TILE) >> 4);
+                    const uint32_t pa = tmem_s + 128 * (j & 1) + (low ? PF_TMEM_PL : PF_TMEM_PH);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        umma_bf16_ts(acc, pa + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || kk > 0);
+                    umma_commit(bar_o + 8 * (j % PF_NB));
+                }
+                __syncwarp();
+                DA_PH(ph, 2, ph_t);
+            }
+            if (blockIdx.x == 0 && lane == 0)
+                DA_PH_STORE(TL_PREFIX + 2 + (int)low, ph);
+            if (!ok && lane == 0 && *abort_flag == 0) {
+                *abort_flag = 1;
+                report_status(p.status, 3 /* DA_DEV_TIMEOUT */, -7, (int)blockIdx.x, 1 + (int)low);
             }
         }
     } else {
@@ -470,11 +497,17 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         // extend: this row's query attends tokens below `limit` (0 for padding rows: nothing)
         const int rr = rt * PF_ROWS + r;
         const int limit = (p.ext && rr < R && L > 0) ? L - p.Lq + rr / p.G + 1 : 0;
+        DA_PH_DECL(ph, ph_t);
+#ifdef DA_TIMELINE
+        const long long ph_begin = ph_t;
+        const unsigned long long ph_ns = globaltimer_ns();
+#endif
         for (int j = 0; j < ntiles; ++j) {
             if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                 ok = false;
                 break;
             }
+            DA_PH(ph, 0, ph_t);
             tc_fence_after();
             // this thread's raw scores (q.k) and the largest scaled one
             float sv[PF_COLS];
@@ -519,6 +552,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 #pragma unroll
             for (int q = 1; q < PF_TPR; ++q)
                 mx = fmaxf(mx, __bfloat162float(xb[q * 128 + r]));
+            DA_PH(ph, 1, ph_t);
             const bool moved = (m_run == -INFINITY) || (mx > m_run + PF_RESCALE_LOG2);
             const float m_new = moved ? mx : m_run;
             const float alpha = !moved ? 1.f : (m_run == -INFINITY ? 0.f : fast_exp2(m_run - m_new));
@@ -542,13 +576,17 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     break;
                 }
                 tc_fence_after();
-                uint32_t v[PF_COLS];
-                tmem_ld32_issue(tmem_o + lane_base, v);
-                tmem_ld_wait();
+#pragma unroll 1
+                for (int a = 0; a < 2; ++a) {
+                    const uint32_t at = (a ? tmem_o2 : tmem_o) + lane_base;
+                    uint32_t v[PF_COLS];
+                    tmem_ld32_issue(at, v);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < PF_COLS; ++i)
-                    v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                tmem_st32(tmem_o + lane_base, v);
+                    for (int i = 0; i < PF_COLS; ++i)
+                        v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                    tmem_st32(at, v);
+                }
             }
             if (p.ext && t_tile + PF_TOK > L) {
                 // The tile reaches past the sequence's end: those V rows were not loaded, or are a page's
@@ -566,6 +604,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 }
                 fence_proxy_async_smem();
             }
+            DA_PH(ph, 2, ph_t);
             // P into tensor memory, over this tile's scores (every thread of the row has read its own: the
             // maximum exchange above came after the loads): this thread's 32 tokens are 16 columns of bf16 pairs
             tmem_st16(tmem_s + 128 * (j & 1) + PF_TMEM_PH + lane_sel + part * (PF_COLS / 2), phi);
@@ -577,13 +616,19 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_p);     // one arrival per warp: 512 arrivals on one barrier cost hundreds of cycles
+            DA_PH(ph, 3, ph_t);
         }
         uint32_t o_raw[PF_COLS];
         if (ok && ntiles > 0) {
             if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) % PF_NB), (uint32_t)(((ntiles - 1) / PF_NB) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                 tc_fence_after();
+                uint32_t o_low[PF_COLS];
                 tmem_ld32_issue(tmem_o + lane_base, o_raw);
+                tmem_ld32_issue(tmem_o2 + lane_base, o_low);
                 tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < PF_COLS; ++i)   // the two products' sums: O = P_hi V + P_lo V
+                    o_raw[i] = __float_as_uint(__uint_as_float(o_raw[i]) + __uint_as_float(o_low[i]));
             } else {
                 ok = false;
             }
@@ -652,6 +697,15 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 }
             }
         }
+#ifdef DA_TIMELINE
+        DA_PH(ph, 4, ph_t);
+        if (blockIdx.x == 0 && tid == 0) {
+            ph[5] = ntiles;
+            ph[6] = ph_t - ph_begin;
+            ph[7] = (long long)(globaltimer_ns() - ph_ns);
+            DA_PH_STORE(TL_PREFIX, ph);
+        }
+#endif
     }
     tc_fence_before();
     __syncthreads();
