@@ -187,10 +187,11 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
         "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
         : "memory");
 }
-// The K/V pools are read here through a 4-D tiled map {d, token, head, page} with box {64, box_rows, 1, 1}:
+// The K pool is read here through a 4-D tiled map {d, token, head, page} with box {64, box_rows, 1, 1}:
 // one box is one 64-column plane of box_rows token rows, so a plane of a tile is contiguous and
-// its 8-row groups are 1024 bytes apart, which is what the matrix descriptors above assume.
-// (tma_load_4d itself is in da_ptx.cuh.)
+// its 8-row groups are 1024 bytes apart, which is what the matrix descriptors above assume; the V pool
+// through the 5-D map of the partition kernel (both planes of box_rows rows per box).
+// (The loads themselves are in da_ptx.cuh.)
 
 __global__ void __launch_bounds__(PF_THREADS, 1)
 prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const PrefixParams p)
@@ -289,14 +290,21 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         // ------------------------------------------------------------------ loader warps: TMA
         // Warp PF_LOADER loads the K tiles, warp PF_LOADER + 1 the V tiles (issuing a tile's 16 tensor
         // copies takes a warp ~1500 cycles: one warp for both was the slowest stage of the block).
-        // Lane l < 2 * boxes issues one load per tile: box l >> 1 (box_rows tokens of one page), plane
-        // l & 1.  Tiles 0..2 fill the three buffers; after that K(t) follows the completion of the
-        // scores of tile t-3 (bar_kfree) and V(t) the completion of the PV product of tile t-3 (bar_o).
+        // K: lane l < 2 * boxes issues one load per tile: box l >> 1 (box_rows tokens of one page), plane
+        // l & 1 -- the score product reads a K tile as 128 rows of one 64-column plane after the other, so
+        // a copy cannot span both planes.  V: lane l < boxes issues one load per tile, box l with both of
+        // its planes (the pool seen as {64 columns, token, half, head, page}: half as many copies, and the
+        // TMA unit's ~85 cycles per copy are what the loaders spend their time on); the tile is then its
+        // boxes one after the other, each box_rows rows of the first 64 columns followed by box_rows rows
+        // of the other 64, which suits the PV product: each of its steps reads 16 token rows, and the
+        // distance between the planes is just its descriptor's leading offset.  Tiles 0..2 fill the three
+        // buffers; after that K(t) follows the completion of the scores of tile t-3 (bar_kfree) and V(t)
+        // the completion of the PV products of tile t-3 (bar_o).
         if (ntiles > 0) {
             const bool is_v = warp == PF_LOADER + 1;
             const int boxes = PF_TOK / p.box_rows;
-            const int box = lane >> 1, pl = lane & 1;
-            const bool active = lane < 2 * boxes;
+            const int box = is_v ? lane : lane >> 1, pl = is_v ? 0 : lane & 1;
+            const bool active = lane < (is_v ? boxes : 2 * boxes);
             const uint32_t bar_full = is_v ? bar_vfull : bar_kfull;
             const uint32_t bar_free = is_v ? bar_o : bar_kfree;
             const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
@@ -334,8 +342,11 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     mbar_arrive_expect_tx(bar, (uint32_t)(nbox * p.box_rows * 256));
                 __syncwarp();
                 if (mine && !withheld) {
-                    const uint32_t off = (uint32_t)(buf * PF_TILE + pl * PF_PLANE + box * p.box_rows * 128);
-                    tma_load_4d(sb + (is_v ? PF_OFF_V : PF_OFF_K) + off, tm, pl * 64, t % p.P, g, page, bar);
+                    if (is_v)
+                        tma_load_5d(sb + PF_OFF_V + (uint32_t)(buf * PF_TILE + box * p.box_rows * 256), tm, 0, t % p.P, 0, g, page, bar);
+                    else
+                        tma_load_4d(sb + PF_OFF_K + (uint32_t)(buf * PF_TILE + pl * PF_PLANE + box * p.box_rows * 128), tm,
+                                    pl * 64, t % p.P, g, page, bar);
                 }
                 issued = j + 1;
             };
@@ -439,8 +450,10 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         if (ntiles > 0) {
             bool ok = true;
             const bool low = warp == PF_PV + 1;
-            const uint64_t v_desc = umma_desc(sb + PF_OFF_V, PF_PLANE, 1024);
+            // a V tile is its boxes one after the other, each box its two 64-column planes of box_rows rows
+            const uint64_t v_desc = umma_desc(sb + PF_OFF_V, (uint32_t)p.box_rows * 128u, 1024);
             const uint32_t idesc_o = umma_idesc(PF_ROWS, HEAD_DIM, true);
+            const int log2_br = 31 - __clz(p.box_rows);
             const uint32_t acc = low ? tmem_o2 : tmem_o;
             DA_PH_DECL(ph, ph_t);
             for (int j = 0; ok && j < ntiles; ++j) {
@@ -455,8 +468,12 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     const uint64_t vd = v_desc + (uint64_t)(((j % PF_NB) * PF_TILE) >> 4);
                     const uint32_t pa = tmem_s + 128 * (j & 1) + (low ? PF_TMEM_PL : PF_TMEM_PH);
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        umma_bf16_ts(acc, pa + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), idesc_o, j > 0 || kk > 0);
+                    for (int kk = 0; kk < 8; ++kk) {
+                        // tokens 16 kk .. 16 kk + 15: box (16 kk) / box_rows, row (16 kk) % box_rows of it
+                        const uint32_t t16 = 16u * kk;
+                        const uint32_t off = ((t16 >> log2_br) << (log2_br + 8)) + (t16 & ((uint32_t)p.box_rows - 1u)) * 128u;
+                        umma_bf16_ts(acc, pa + kk * 8, vd + (uint64_t)(off >> 4), idesc_o, j > 0 || kk > 0);
+                    }
                     umma_commit(bar_o + 8 * (j % PF_NB));
                 }
                 __syncwarp();
@@ -600,7 +617,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 uint8_t *vb = smem + PF_OFF_V + (j % PF_NB) * PF_TILE;
                 for (int e = tid; e < (PF_TOK - first_bad) * 16; e += PF_TPR * PF_ROWS) {
                     const int row = first_bad + (e >> 4), ch = e & 15;
-                    *reinterpret_cast<uint4 *>(vb + (ch >> 3) * PF_PLANE + row * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    const int bx = row / p.box_rows, rr_ = row % p.box_rows;   // box-major tile: see the loader warps
+                    *reinterpret_cast<uint4 *>(vb + bx * p.box_rows * 256 + (ch >> 3) * p.box_rows * 128 + rr_ * 128 + ((ch & 7) << 4)) =
+                        make_uint4(0, 0, 0, 0);
                 }
                 fence_proxy_async_smem();
             }

@@ -178,9 +178,9 @@ int get_encoder()
 // {64, box_rows, 2, 1, 1}, 128-byte swizzle.  Splitting head_dim into two halves keeps the inner box
 // extent at the swizzle span (128 bytes) while one TMA operation still brings all 128 columns of
 // box_rows tokens: in shared memory a box is two planes of box_rows 128-byte rows.
-// planes = 2: the partition kernel's view.  planes = 1: a 4-D view {d, token, kv head, page} with
-// box {64, box_rows, 1, 1} (one 64-column half per box), used by the prefix kernel, whose matrix
-// descriptors want each half of a tile contiguous.
+// planes = 2: the partition kernel's view, and the prefix kernel's view of V.  planes = 1: a 4-D view
+// {d, token, kv head, page} with box {64, box_rows, 1, 1} (one 64-column half per box), the prefix
+// kernel's view of K, whose score product wants each half of a tile contiguous.
 int get_tmap(const da_tensor *t, int box_rows, int planes, CUtensorMap *out)
 {
     TmapKey key;
@@ -596,7 +596,7 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     CUtensorMap tm_k, tm_v;
     rc = get_tmap(k_pages, box_rows, 1, &tm_k);
     if (rc != DA_OK) return rc;
-    rc = get_tmap(v_pages, box_rows, 1, &tm_v);
+    rc = get_tmap(v_pages, box_rows, 2, &tm_v);   // (K: one plane per box; V: both)
     if (rc != DA_OK) return rc;
     PrefixParams pf;
     pf.q = static_cast<const __nv_bfloat16 *>(q->data);
@@ -883,7 +883,7 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
     CUtensorMap tm_k, tm_v;
     rc = get_tmap(k_pages, box_rows, 1, &tm_k);
     if (rc != DA_OK) return rc;
-    rc = get_tmap(v_pages, box_rows, 1, &tm_v);
+    rc = get_tmap(v_pages, box_rows, 2, &tm_v);   // (K: one plane per box; V: both)
     if (rc != DA_OK) return rc;
 
     PrefixParams pf;
