@@ -24,7 +24,7 @@ constexpr int KV_BYTES = TILE_T * 256;      // a K (or V) tile: TILE_T rows of 1
 static_assert(TILE_T8 * 128 == KV_BYTES, "both cache types fill a stage");
 constexpr float P8_SHIFT = 15.f;            // 8-bit cache: softmax weights are carried as 2^15 * p (f16 high + low)
 constexpr int STAGE_BYTES = 2 * KV_BYTES;   // K tile followed by V tile
-constexpr int NTHREADS = (NCW + 1) * 32;    // + one producer warp
+constexpr int NTHREADS = (NCW + 1) * 32;    // + one producer warp (with two column sets: 2 * NCW + 1 warps)
 constexpr int PLAN_THREADS = 512;
 constexpr int PLAN_SMEM_SEQS = 4096;
 constexpr int MIN_TAIL_UNIT_TILES = 4;      // a ticketed unit is never cut smaller than this
@@ -72,18 +72,27 @@ constexpr int TILE_ITEM_END = 1;   // last tile this unit holds of its (b, kv he
 constexpr int TILE_WHOLE = 2;      // the unit holds every tile of the pair: write `out` directly
 constexpr int TILE_STOP = 4;       // no more work for this block (carries no data)
 
-template <int NT8>
+// A thread block's consumer warps form CSETS column sets of NCW warps.  Warp (set cs, token group tw) owns
+// tokens WT * tw .. of every tile and the NT8 column tiles (8 query heads each) cs * NT8 .. of the KV
+// group's (virtual) heads: one set of 1 or 2 column tiles serves up to 16 heads with two blocks per SM;
+// two sets of 2 or 3 serve up to 32 or 48 (several new tokens per sequence) with one block per SM -- both
+// sets read the same K and V tiles from shared memory, so K and V still cross HBM once.
+template <int NT8, int CSETS>
 struct PartCfg {
-    static constexpr int NSTAGES = (NT8 == 1) ? 3 : 2;
-    static constexpr int HEADS = NT8 * 8;                                // padded heads per KV group
+    static constexpr int NSTAGES = CSETS == 1 ? ((NT8 == 1) ? 3 : 2) : ((NT8 == 2) ? 4 : 3);
+    static constexpr int HEADS_SET = NT8 * 8;                            // padded heads of one column set
+    static constexpr int HEADS = CSETS * HEADS_SET;                      // padded heads per KV group
+    static constexpr int THREADS = (NCW * CSETS + 1) * 32;               // consumer warps + one producer warp
+    static constexpr int MIN_BLOCKS = CSETS == 1 ? 2 : 1;
     static constexpr int XBUF_BYTES = NCW * HEADS * HEAD_DIM * 4;        // cross-warp combine buffer
     static constexpr int STATS_BYTES = 2 * NCW * HEADS * 4;              // (m, l) per warp and head
     static constexpr int OFF_XBUF = NSTAGES * STAGE_BYTES;
     static constexpr int OFF_STATS = OFF_XBUF + XBUF_BYTES;
     static constexpr int OFF_META = OFF_STATS + STATS_BYTES;             // two int4 per stage
-    static constexpr int OFF_BARS = OFF_META + NSTAGES * 32;             // full[NSTAGES], empty[NSTAGES], epi[2]
-    static constexpr int OFF_FLAGS = OFF_BARS + (2 * NSTAGES + 2) * 8;   // abort flag
+    static constexpr int OFF_BARS = OFF_META + NSTAGES * 32;             // full[NSTAGES], empty[NSTAGES], epi[2 * CSETS]
+    static constexpr int OFF_FLAGS = OFF_BARS + (2 * NSTAGES + 2 * CSETS) * 8;   // abort flag
     static constexpr int SMEM_BYTES = OFF_FLAGS + 16;
+    static_assert(SMEM_BYTES <= 232448, "a block must fit the 227 KB of shared memory an SM offers");
 };
 
 // What the plan kernel decides, read by the other two kernels.  Units 0 .. n_static-1 cut
@@ -481,12 +490,13 @@ __device__ __forceinline__ uint32_t row_offset(int row, int box_rows)
     return (uint32_t)((row / box_rows) * (box_rows * 256) + (row % box_rows) * 128);
 }
 
-template <int NT8, bool KV8>
-__global__ void __launch_bounds__(NTHREADS, 2)
+template <int NT8, bool KV8, int CSETS>
+__global__ void __launch_bounds__((PartCfg<NT8, CSETS>::THREADS), (PartCfg<NT8, CSETS>::MIN_BLOCKS))
 partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const PartParams p)
 {
-    using C = PartCfg<NT8>;
+    using C = PartCfg<NT8, CSETS>;
+    constexpr int HS = C::HEADS_SET;                   // padded heads of one column set
     constexpr int TT = KV8 ? TILE_T8 : TILE_T;        // tokens per tile
     constexpr uint32_t ROW_BYTES = KV8 ? 128u : 256u;  // one token row of one KV head
     constexpr int NSTAGES = C::NSTAGES;
@@ -500,7 +510,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAGS);
     const uint32_t bar_full = smem_base + C::OFF_BARS;
     const uint32_t bar_empty = bar_full + NSTAGES * 8;
-    const uint32_t bar_epi = bar_empty + NSTAGES * 8;   // two barriers for the consumers' epilogue
+    const uint32_t bar_epi0 = bar_empty + NSTAGES * 8;  // two barriers per column set for the consumers' epilogue
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0 && blockIdx.x < TL_MERGE)
@@ -515,10 +525,10 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         *abort_flag = 0;
         for (int s = 0; s < NSTAGES; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, NCW);
+            mbar_init(bar_empty + 8 * s, NCW * CSETS);
         }
-        mbar_init(bar_epi, NCW);
-        mbar_init(bar_epi + 8, NCW);
+        for (int s = 0; s < 2 * CSETS; ++s)
+            mbar_init(bar_epi0 + 8 * s, NCW);
         mbar_fence_init();
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
@@ -529,7 +539,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     if (tid == 0 && blockIdx.x < TL_MERGE)
         DA_TL(blockIdx.x, 1);
 
-    if (warp == NCW) {
+    if (warp == NCW * CSETS) {
         // ------------------------------------------------------------------ producer warp
         // Lane -> (box, K|V).  A box is box_rows token rows (all 128 columns) of one page.
         const int nboxes = TT / p.box_rows;
@@ -715,11 +725,15 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     // They follow the tile descriptors the producer leaves with each stage.  A failed (timed-out)
     // wait raises the abort flag and leaves at once; every other wait then gives up quickly too.
     const int r = lane >> 2, c = lane & 3;
+    const int tw = CSETS == 1 ? warp : warp % NCW;      // token group: this warp's rows of every tile
+    const int cs = CSETS == 1 ? 0 : warp / NCW;         // column set
+    const int col0 = cs * HS;                           // first (virtual) head of this warp's column tiles
+    const uint32_t bar_epi = bar_epi0 + 16 * cs;
     uint32_t it = 0, items = 0;
     // per-lane offsets used by the ldmatrix address patterns
-    const int k_row = 16 * warp + (lane & 7) + ((lane >> 3) & 1) * 8;   // K: matrices 1,3 are rows +8
+    const int k_row = 16 * tw + (lane & 7) + ((lane >> 3) & 1) * 8;     // K: matrices 1,3 are rows +8
     const int k_chunk = lane >> 4;                                      //    matrices 2,3 are chunk +1
-    const int v_row = 16 * warp + (lane & 7) + (lane >> 4) * 8;         // V: matrices 2,3 are rows +8
+    const int v_row = 16 * tw + (lane & 7) + (lane >> 4) * 8;           // V: matrices 2,3 are rows +8
     const int v_chunk = (lane >> 3) & 1;                                //    matrices 1,3 are chunk +1
     const uint32_t plane_bytes = (uint32_t)p.box_rows * 128u;
     const uint32_t k_off = row_offset(k_row, p.box_rows), v_off = row_offset(v_row, p.box_rows);
@@ -741,11 +755,11 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     auto tok8 = [](int x) { return x < 8 ? x : 8 + ((x + 4) & 7); };
     const int x8 = (lane & 7) + ((lane >> 3) & 1) * 8;          // QK ldmatrix: row of the 16-row tile
     const int k8_chunk = lane >> 4;                             //              16-byte half of the 32-dim step
-    const int row_a8 = 32 * warp + tok8(x8), row_b8 = row_a8 + 16;
+    const int row_a8 = 32 * tw + tok8(x8), row_b8 = row_a8 + 16;
     const uint32_t ka8_off = (uint32_t)row_a8 * 128u, kb8_off = (uint32_t)row_b8 * 128u;
     const uint32_t ka8_sw = (uint32_t)(row_a8 & 7), kb8_sw = (uint32_t)(row_b8 & 7);
     const int slot_row = 8 * ((lane >> 1) & 1) + 2 * ((lane & 15) >> 2) + (lane & 1);   // PV: tile row of k slot `lane`
-    const int row_v8 = 32 * warp + tok8(slot_row) + 16 * (lane >> 4);
+    const int row_v8 = 32 * tw + tok8(slot_row) + 16 * (lane >> 4);
     const uint32_t v8_off = (uint32_t)row_v8 * 128u, v8_sw = (uint32_t)(row_v8 & 7);
     const int t_a0 = tok8(r), t_a1 = tok8(r + 8);               // tokens of this lane's scores (tile B: + 16)
 
@@ -759,7 +773,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     auto load_q = [&](uint32_t (&qf)[NT8][8][2], int b, int g) {
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
-            const int head = n * 8 + r;
+            const int head = col0 + n * 8 + r;
             const int hv = head < p.Gv ? head : 0;
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
                 p.q + (int64_t)b * p.q_sb + (int64_t)(hv / p.G) * p.q_sq + (int64_t)(g * p.G + hv % p.G) * p.q_sh);
@@ -783,7 +797,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         ks = p.k_scale ? __ldg(p.k_scale + g) : 1.f;
 #pragma unroll
         for (int n = 0; n < NT8; ++n) {
-            const int head = n * 8 + r;
+            const int head = col0 + n * 8 + r;
             const int hv = head < p.Gv ? head : 0;
             const uint32_t *qrow = reinterpret_cast<const uint32_t *>(
                 p.q + (int64_t)b * p.q_sb + (int64_t)(hv / p.G) * p.q_sq + (int64_t)(g * p.G + hv % p.G) * p.q_sh);
@@ -860,7 +874,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         for (;;) {   // the item's tiles; (m0, m1) describe the tile in stage it % NSTAGES, already full
             const int stage = it % NSTAGES;
             constexpr int WT = KV8 ? 32 : 16;   // tokens of a tile that one warp owns
-            const int a = m0.z + WT * warp;     // first token of this warp's rows
+            const int a = m0.z + WT * tw;       // first token of this warp's rows
             const int v_lo = max(a, lo), v_hi = min(a + WT, L);
             const bool item_end = (m0.w & TILE_ITEM_END) != 0;
             poisoned |= m1.w != 0;
@@ -875,7 +889,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         const int rr = e >> 3, ch = e & 7;
                         const int t = a + rr;
                         if (t < v_lo || t >= v_hi) {
-                            const uint32_t addr = v_base + (uint32_t)(32 * warp + rr) * 128u + (ch << 4);
+                            const uint32_t addr = v_base + (uint32_t)(32 * tw + rr) * 128u + (ch << 4);
                             asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
                         }
                     }
@@ -941,7 +955,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     for (int n = 0; n < NT8; ++n)
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            const int lim = L - p.Lq + (n * 8 + 2 * c + e) / p.G + 1;
+                            const int lim = L - p.Lq + (col0 + n * 8 + 2 * c + e) / p.G + 1;
                             if (a + t_a0 >= lim) sa[n][e] = -INFINITY;
                             if (a + t_a1 >= lim) sa[n][2 + e] = -INFINITY;
                             if (a + 16 + t_a0 >= lim) sb[n][e] = -INFINITY;
@@ -1042,7 +1056,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         const int rr = e >> 4, ch = e & 15;
                         const int t = a + rr;
                         if (t < v_lo || t >= v_hi) {
-                            const uint32_t addr = v_base + row_offset(16 * warp + rr, p.box_rows) +
+                            const uint32_t addr = v_base + row_offset(16 * tw + rr, p.box_rows) +
                                                   (ch >> 3) * plane_bytes + ((ch & 7) << 4);
                             asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
                         }
@@ -1091,7 +1105,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     for (int n = 0; n < NT8; ++n)
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            const int lim = L - p.Lq + (n * 8 + 2 * c + e) / p.G + 1;
+                            const int lim = L - p.Lq + (col0 + n * 8 + 2 * c + e) / p.G + 1;
                             if (a + r >= lim) s[n][e] = -INFINITY;
                             if (a + r + 8 >= lim) s[n][2 + e] = -INFINITY;
                         }
@@ -1209,12 +1223,12 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 l += __shfl_xor_sync(0xffffffffu, l, 16);
                 if (r == 0) {
                     // (8-bit cache: the weights were carried times 2^15, i.e. relative to m - 15)
-                    st_m[warp * HEADS + n * 8 + 2 * c + e] = KV8 ? m_run[n][e] - P8_SHIFT : m_run[n][e];
-                    st_l[warp * HEADS + n * 8 + 2 * c + e] = l;
+                    st_m[tw * HEADS + col0 + n * 8 + 2 * c + e] = KV8 ? m_run[n][e] - P8_SHIFT : m_run[n][e];
+                    st_l[tw * HEADS + col0 + n * 8 + 2 * c + e] = l;
                 }
             }
             // xbuf[warp][head][d ^ 8*((head>>1)&3)] : conflict-free for these stores and the reads below
-            float *xb = xbuf + (warp * HEADS + n * 8 + 2 * c) * HEAD_DIM;
+            float *xb = xbuf + (tw * HEADS + col0 + n * 8 + 2 * c) * HEAD_DIM;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int d0 = (16 * j + r) ^ (8 * c), d1 = (16 * j + r + 8) ^ (8 * c);
@@ -1232,12 +1246,12 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             return;
         }
         {
-            // Warp w folds heads w, w + 4, ...: lane -> output dims 4 lane .. 4 lane + 3.  A short loop
+            // Warp w of a column set folds the set's heads w, w + 4, ...: lane -> output dims 4 lane .. 4 lane + 3.  A short loop
             // on purpose: this code runs once per item, so its instructions are fetched cold each time,
             // and a compact body costs far less than a long unrolled one.
             const uint64_t part_policy = l2_policy_evict_last();   // partial results wait in L2 for the merge kernel
 #pragma unroll 1
-            for (int head = warp; head < p.Gv; head += NCW) {
+            for (int head = col0 + tw; head < min(p.Gv, col0 + HS); head += NCW) {
                 float mw[NCW], lw[NCW], f[NCW];
 #pragma unroll
                 for (int w = 0; w < NCW; ++w) {

@@ -514,12 +514,52 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         // extend: this row's query attends tokens below `limit` (0 for padding rows: nothing)
         const int rr = rt * PF_ROWS + r;
         const int limit = (p.ext && rr < R && L > 0) ? L - p.Lq + rr / p.G + 1 : 0;
+        // extend, a tile that reaches past the sequence's end: those V rows were not loaded, or are a page's
+        // unused tail, and may hold NaN, which a zero weight would not hide.  All softmax threads clear them
+        // (both planes, 128 bytes a row) once V has landed, before the PV product reads them.
+        auto clear_v_tail = [&](int j, int t_tile) {
+            if (!mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS))
+                return false;
+            const int first_bad = max(L - t_tile, 0);
+            uint8_t *vb = smem + PF_OFF_V + (j % PF_NB) * PF_TILE;
+            for (int e = tid; e < (PF_TOK - first_bad) * 16; e += PF_TPR * PF_ROWS) {
+                const int row = first_bad + (e >> 4), ch = e & 15;
+                const int bx = row / p.box_rows, rr_ = row % p.box_rows;   // box-major tile: see the loader warps
+                *reinterpret_cast<uint4 *>(vb + bx * p.box_rows * 256 + (ch >> 3) * p.box_rows * 128 + rr_ * 128 + ((ch & 7) << 4)) =
+                    make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async_smem();
+            return true;
+        };
+        // A warp whose 32 rows all lie past the block's last query row (a few new tokens fill only the first
+        // rows of the tile; the last row tile of a batch) computes nothing: it only keeps pace with the
+        // barriers its fellows use -- the maximum exchange, the tail clearing, the hand-over of P.
+        const bool has_rows = rt * PF_ROWS + 32 * (warp & 3) < R;
         DA_PH_DECL(ph, ph_t);
 #ifdef DA_TIMELINE
         const long long ph_begin = ph_t;
         const unsigned long long ph_ns = globaltimer_ns();
 #endif
-        for (int j = 0; j < ntiles; ++j) {
+        for (int j = 0; !has_rows && ntiles > 0 && j <= ntiles; ++j) {
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(bar_x);   // tiles 0 .. ntiles-1: the maxima; once more: the final sums
+            if (!mbar_wait_bounded(bar_x, (uint32_t)(j & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
+                ok = false;
+                break;
+            }
+            if (j == ntiles)
+                break;
+            const int t_tile = (t_begin + j) * PF_TOK;
+            if (p.ext && t_tile + PF_TOK > L && !clear_v_tail(j, t_tile)) {
+                ok = false;
+                break;
+            }
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(bar_p);
+        }
+        for (int j = 0; has_rows && j < ntiles; ++j) {
             if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                 ok = false;
                 break;
@@ -605,23 +645,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     tmem_st32(at, v);
                 }
             }
-            if (p.ext && t_tile + PF_TOK > L) {
-                // The tile reaches past the sequence's end: those V rows were not loaded, or are a page's
-                // unused tail, and may hold NaN, which a zero weight would not hide.  Clear them (both
-                // planes, 128 bytes a row) once V has landed, before the PV product reads them.
-                if (!mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
-                    ok = false;
-                    break;
-                }
-                const int first_bad = max(L - t_tile, 0);
-                uint8_t *vb = smem + PF_OFF_V + (j % PF_NB) * PF_TILE;
-                for (int e = tid; e < (PF_TOK - first_bad) * 16; e += PF_TPR * PF_ROWS) {
-                    const int row = first_bad + (e >> 4), ch = e & 15;
-                    const int bx = row / p.box_rows, rr_ = row % p.box_rows;   // box-major tile: see the loader warps
-                    *reinterpret_cast<uint4 *>(vb + bx * p.box_rows * 256 + (ch >> 3) * p.box_rows * 128 + rr_ * 128 + ((ch & 7) << 4)) =
-                        make_uint4(0, 0, 0, 0);
-                }
-                fence_proxy_async_smem();
+            if (p.ext && t_tile + PF_TOK > L && !clear_v_tail(j, t_tile)) {
+                ok = false;
+                break;
             }
             DA_PH(ph, 2, ph_t);
             // P into tensor memory, over this tile's scores (every thread of the row has read its own: the
@@ -638,7 +664,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             DA_PH(ph, 3, ph_t);
         }
         uint32_t o_raw[PF_COLS];
-        if (ok && ntiles > 0) {
+        if (ok && ntiles > 0 && has_rows) {
             if (mbar_wait_bounded(bar_o + 8 * ((ntiles - 1) % PF_NB), (uint32_t)(((ntiles - 1) / PF_NB) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                 tc_fence_after();
                 uint32_t o_low[PF_COLS];
@@ -654,7 +680,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
         // the row's sum of weights is the sum of its threads' sums (all relative to m_run)
         float l_row = 0.f;
-        if (ok && ntiles > 0) {
+        if (ok && ntiles > 0 && has_rows) {
             // (every thread has read the last maxima before the last PV product could complete)
             float *xb = reinterpret_cast<float *>(smem + PF_OFF_XCHG);
             xb[part * 128 + r] = l_run;

@@ -21,7 +21,8 @@ constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
 constexpr int kMaxPrefixSplits = 4;
-constexpr int kMaxGroup = 16;
+constexpr int kMaxGroup = 16;        // query heads per KV head
+constexpr int kMaxStreamRows = 48;   // query rows per KV head (new tokens x heads) the streaming kernels take
 
 std::mutex g_mu;
 std::atomic<int> g_last_cuda_error{0};
@@ -127,8 +128,9 @@ struct WsLayout {
     size_t pre_o, pre_lse, suf_o, suf_lse, total;   // cascade scratch
 };
 
-// `units` = thread blocks of the partition kernel x (1 + ticketed units per block)
-WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int units)
+// `units` = thread blocks of the partition kernel x (1 + ticketed units per block); `heads_pad` = most padded
+// (virtual) heads per KV group whose partial results the slots must hold
+WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int units, int heads_pad = kMaxStreamRows)
 {
     WsLayout w;
     size_t off = 0;
@@ -146,8 +148,8 @@ WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int unit
     w.unit_work = take((size_t)units * 16);
     w.merge_small = take((size_t)w.merge_seg * PLAN_BLOCKS * 16);
     w.merge_big = take((size_t)w.merge_seg * PLAN_BLOCKS * 16);
-    w.part_lse = take((size_t)2 * units * kMaxGroup * 4);
-    w.part_o = take((size_t)2 * units * kMaxGroup * HEAD_DIM * 4);
+    w.part_lse = take((size_t)2 * units * heads_pad * 4);
+    w.part_o = take((size_t)2 * units * heads_pad * HEAD_DIM * 4);
     w.stg_q = take((size_t)B * Hq * D * 2);
     w.stg_bt = take((size_t)B * max_pages * 4);
     w.stg_sl = take((size_t)B * 4);
@@ -299,13 +301,42 @@ int validate(const da_tensor *q, const da_tensor *k, const da_tensor *v, const d
     return DA_OK;
 }
 
-template <int NT8>
+template <int NT8, int CSETS>
 int set_kernel_attrs()
 {
-    DA_CUDA(cudaFuncSetAttribute(partition_kernel<NT8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 PartCfg<NT8>::SMEM_BYTES));
-    DA_CUDA(cudaFuncSetAttribute(partition_kernel<NT8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 PartCfg<NT8>::SMEM_BYTES));
+    DA_CUDA(cudaFuncSetAttribute(partition_kernel<NT8, false, CSETS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PartCfg<NT8, CSETS>::SMEM_BYTES));
+    DA_CUDA(cudaFuncSetAttribute(partition_kernel<NT8, true, CSETS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PartCfg<NT8, CSETS>::SMEM_BYTES));
+    return DA_OK;
+}
+
+int set_all_kernel_attrs(DeviceState *st)
+{
+    if (st->attrs_set) return DA_OK;
+    int rc = set_kernel_attrs<1, 1>();
+    if (rc != DA_OK) return rc;
+    rc = set_kernel_attrs<2, 1>();
+    if (rc != DA_OK) return rc;
+    rc = set_kernel_attrs<2, 2>();
+    if (rc != DA_OK) return rc;
+    rc = set_kernel_attrs<3, 2>();
+    if (rc != DA_OK) return rc;
+    DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
+    st->attrs_set = true;
+    return DA_OK;
+}
+
+// One instance of the partition kernel: NT8 column tiles of 8 heads per warp, CSETS column sets.
+template <int NT8, int CSETS>
+int launch_partition(cudaLaunchConfig_t &cfg, bool kv8, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PartParams &pa)
+{
+    cfg.blockDim = dim3((unsigned)PartCfg<NT8, CSETS>::THREADS);
+    cfg.dynamicSmemBytes = PartCfg<NT8, CSETS>::SMEM_BYTES;
+    if (kv8)
+        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<NT8, true, CSETS>, tm_k, tm_v, pa));
+    else
+        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<NT8, false, CSETS>, tm_k, tm_v, pa));
     return DA_OK;
 }
 
@@ -366,14 +397,16 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
                 bool kv8 = false, const float *k_scale = nullptr, const float *v_scale = nullptr, int Lq = 1,
                 int64_t q_sq = 0, int64_t o_sq = 0, int64_t l_sq = 0)
 {
-    int rc;
-    if (!st->attrs_set) {
-        rc = set_kernel_attrs<1>();
-        if (rc != DA_OK) return rc;
-        rc = set_kernel_attrs<2>();
-        if (rc != DA_OK) return rc;
-        DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
-        st->attrs_set = true;
+    int rc = set_all_kernel_attrs(st);
+    if (rc != DA_OK) return rc;
+    // Up to 16 (virtual) heads per KV group: one column set, two blocks per SM.  17 .. 48 (several new tokens
+    // per sequence): two column sets in a block of nine warps, one block per SM.
+    const int gv = (int)(Lq * d.G);
+    const int csets = gv <= 16 ? 1 : 2;
+    const int nt8 = gv <= 8 ? 1 : (gv <= 32 ? 2 : 3);
+    if (csets == 2 && g_opt_grid_blocks <= 0) {
+        nblocks = st->sm_count;
+        n_tail = tail_units_for(nblocks);
     }
     const int tile_t = kv8 ? TILE_T8 : TILE_T;
     const int box_rows = d.P < tile_t ? (int)d.P : tile_t;
@@ -422,7 +455,6 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pa.l_sq = l_sq;
     pa.unit_cap = nblocks + n_tail;
     pa.max_pages = d.max_pages;
-    const int nt8 = pa.Gv <= 8 ? 1 : 2;
     const bool timed = g_ev_before && g_ev_after;
     if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
     // Both dependent kernels are launched with programmatic stream serialization: their blocks may
@@ -433,19 +465,18 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pdl.val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)nblocks);
-    cfg.blockDim = dim3(NTHREADS);
     cfg.stream = stream;
     cfg.attrs = &pdl;
     cfg.numAttrs = 1;
-    cfg.dynamicSmemBytes = nt8 == 1 ? PartCfg<1>::SMEM_BYTES : PartCfg<2>::SMEM_BYTES;
-    if (nt8 == 1 && !kv8)
-        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<1, false>, tm_k, tm_v, pa));
-    else if (nt8 == 1)
-        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<1, true>, tm_k, tm_v, pa));
-    else if (!kv8)
-        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<2, false>, tm_k, tm_v, pa));
+    if (csets == 1 && nt8 == 1)
+        rc = launch_partition<1, 1>(cfg, kv8, tm_k, tm_v, pa);
+    else if (csets == 1)
+        rc = launch_partition<2, 1>(cfg, kv8, tm_k, tm_v, pa);
+    else if (nt8 == 2)
+        rc = launch_partition<2, 2>(cfg, kv8, tm_k, tm_v, pa);
     else
-        DA_CUDA(cudaLaunchKernelEx(&cfg, partition_kernel<2, true>, tm_k, tm_v, pa));
+        rc = launch_partition<3, 2>(cfg, kv8, tm_k, tm_v, pa);
+    if (rc != DA_OK) return rc;
     g_launches.fetch_add(1);
     if (timed) DA_CUDA(cudaEventRecord(g_ev_after, stream));
 
@@ -468,7 +499,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     mp.B = pa.B;
     mp.Hkv = pa.Hkv;
     mp.G = pa.G;
-    mp.heads_pad = nt8 * 8;
+    mp.heads_pad = csets * nt8 * 8;
     mp.out_bf16 = pa.out_bf16;
     mp.Lq = pa.Lq;
     mp.Gv = pa.Gv;
@@ -851,18 +882,12 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
     if (!st->ws || st->ws_bytes < lay.total) return DA_ERR_WORKSPACE;
     if (B == 0) return DA_OK;
     uint8_t *ws = static_cast<uint8_t *>(st->ws);
-    if (!st->attrs_set) {
-        rc = set_kernel_attrs<1>();
-        if (rc != DA_OK) return rc;
-        rc = set_kernel_attrs<2>();
-        if (rc != DA_OK) return rc;
-        DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
-        st->attrs_set = true;
-    }
-    if ((Lq * G <= g_opt_extend_stream_rows || kv8) && Lq * G <= kMaxGroup) {
+    rc = set_all_kernel_attrs(st);
+    if (rc != DA_OK) return rc;
+    if ((Lq * G <= g_opt_extend_stream_rows || kv8) && Lq * G <= kMaxStreamRows) {
         // A few new tokens (speculated tokens, short appends): their Lq * G query rows per KV head ride
-        // through the streaming kernels as one wider group, at the HBM rate of decode_attn(); the
-        // tensor-core kernel below would fill only Lq * G of its 128 rows.
+        // through the streaming kernels as one wider group, K and V crossing HBM once as in decode_attn();
+        // the tensor-core kernel below would fill only Lq * G of its 128 rows.
         Dims d;
         d.B = B; d.Hq = Hq; d.Hkv = Hkv; d.G = G; d.P = P; d.num_pages = k_pages->shape[0]; d.max_pages = max_pages;
         da_tensor q3 = *q, o3 = *out, l3;
@@ -1097,7 +1122,7 @@ int decode_attn_static_scratch(const da_tensor *q, const da_tensor *k_pages, con
     rc = current_device(&dev, &st);
     if (rc != DA_OK) return rc;
     const int nblocks = grid_blocks_for(st);
-    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks);
+    const WsLayout lay = ws_layout(d.B, d.Hq, HEAD_DIM, d.max_pages, nblocks, kMaxGroup);
     // beyond the fixed array: refuse, never spill into an allocation
     if (d.B > kStaticMaxSeqs || nblocks > kStaticMaxBlocks || lay.stg_q > kStaticScratchBytes)
         return DA_ERR_WORKSPACE;
@@ -1244,7 +1269,7 @@ int decode_attn_set_option(const char *name, int64_t value)
         return DA_OK;
     }
     if (std::strcmp(name, "extend_stream_rows") == 0) {
-        if (value < 0 || value > kMaxGroup) return DA_ERR_UNSUPPORTED;
+        if (value < 0 || value > kMaxStreamRows) return DA_ERR_UNSUPPORTED;
         g_opt_extend_stream_rows = value;
         return DA_OK;
     }

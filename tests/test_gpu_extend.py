@@ -97,15 +97,19 @@ def test_extend_errors(da):
 
 # ------------------------------------------------------------------ a few new tokens: the streaming path
 
-@pytest.mark.parametrize("Hq,Hkv,Lq", [(48, 8, 2), (8, 8, 16), (16, 8, 8), (32, 8, 4), (32, 8, 3), (24, 8, 5), (48, 8, 1)])
+@pytest.mark.parametrize("Hq,Hkv,Lq", [(48, 8, 2), (8, 8, 16), (16, 8, 8), (32, 8, 4), (32, 8, 3), (24, 8, 5), (48, 8, 1),
+                                       # 17 .. 48 query rows per KV head: two column sets per thread block
+                                       (48, 8, 3), (48, 8, 4), (48, 8, 5), (48, 8, 8), (8, 8, 17), (8, 8, 33), (64, 8, 6),
+                                       (128, 8, 3), (32, 2, 2)])
 @pytest.mark.parametrize("P", [16, 64])
 def test_few_new_tokens_stream_and_tensor_core_paths_agree_with_the_oracle(da, Hq, Hkv, Lq, P):
-    """Lq * (Hq / Hkv) <= 16 query rows per KV head go through the plan / partition / merge kernels as one
-    wider group (per-column causal limits); option extend_stream_rows = 0 forces the tcgen05 kernel."""
+    """Lq * (Hq / Hkv) <= 48 query rows per KV head go through the plan / partition / merge kernels as one
+    wider group (per-column causal limits; beyond 16 rows as two column sets of warps over the same K and V
+    tiles); option extend_stream_rows = 0 forces the tcgen05 kernel."""
     lens = [Lq, Lq + 1, 15 + Lq, 16 + Lq, 63 + Lq, 64 + Lq, 65 + Lq, 1000, 0, 2500]
     lens = [L if L == 0 else max(L, Lq) for L in lens]
     try:
-        for rows, grid in ((16, 0), (16, 1), (16, 7), (0, 0)):
+        for rows, grid in ((48, 0), (48, 1), (48, 7), (48, 300), (0, 0)):
             da.set_option("extend_stream_rows", rows)
             da.set_option("grid_blocks", grid)
             got, got_lse, ref, ref_lse = run_case(da, lens, Lq, P, 5 * Lq + P + Hq, Hq=Hq, Hkv=Hkv, poison=True,

@@ -416,7 +416,9 @@ def test_host_io_matches_device_call(da):
 
 # ------------------------------------------------------------------ a few new tokens over the 8-bit cache
 
-@pytest.mark.parametrize("Hq,Hkv,Lq", [(48, 8, 2), (8, 8, 16), (16, 8, 8), (32, 8, 3), (24, 8, 5), (48, 8, 1)])
+@pytest.mark.parametrize("Hq,Hkv,Lq", [(48, 8, 2), (8, 8, 16), (16, 8, 8), (32, 8, 3), (24, 8, 5), (48, 8, 1),
+                                       # 17 .. 48 query rows per KV head: two column sets per thread block
+                                       (48, 8, 3), (48, 8, 4), (48, 8, 5), (48, 8, 8), (8, 8, 17), (8, 8, 33)])
 @pytest.mark.parametrize("P", [16, 64])
 def test_few_new_tokens_over_the_fp8_cache(da, Hq, Hkv, Lq, P):
     lens = [Lq, Lq + 1, 31 + Lq, 32 + Lq, 127 + Lq, 128 + Lq, 129 + Lq, 1000, 0, 2500]
@@ -437,7 +439,7 @@ def test_few_new_tokens_over_the_fp8_cache(da, Hq, Hkv, Lq, P):
             assert_close(lse.cpu().numpy(), ref_lse, f"fp8 extend grid={grid} lse")
     finally:
         da.set_option("grid_blocks", 0)
-    with pytest.raises(da.DecodeAttnError) as e:     # more than 16 query rows per KV head
-        big = torch.zeros((len(lens), 17, Hq, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(da.DecodeAttnError) as e:     # more than 48 query rows per KV head
+        big = torch.zeros((len(lens), 49, Hq, 128), dtype=torch.bfloat16, device="cuda")
         da.decode_attn_fp8kv_extend(big, dev.k_pages, dev.v_pages, None, None, dev.block_table, dev.seq_lens, 1.0)
     assert e.value.status == 5
