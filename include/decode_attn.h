@@ -214,7 +214,7 @@ int decode_attn_append_fp8kv(const da_tensor *k_new, const da_tensor *v_new, da_
  * plan / partition / merge kernels of decode_attn() as one wider head group, each column with its own
  * causal limit, at the HBM rate; longer query blocks run on the tcgen05 tensor cores (the same kernel
  * as the cascade's prefix pass: 128 (query, head) rows of one KV group per thread block).  Option
- * "extend_stream_rows" (0 .. 16, default 16) moves the switch; 0 always takes the tensor-core kernel.
+ * "extend_stream_rows" (0 .. 48, default 16) moves the switch; 0 always takes the tensor-core kernel.
  *
  *   q      bf16 [B, Lq, Hq, 128], last dim contiguous
  *   out    f32 or bf16 [B, Lq, Hq, 128], last dim contiguous
@@ -229,7 +229,7 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
 
 /*
  * decode_attn_fp8kv_extend -- decode_attn_extend() over the 8-bit cache of decode_attn_fp8kv(), for a
- * few new tokens per sequence (speculated tokens): Lq * Hq / Hkv must not exceed 16 (else
+ * few new tokens per sequence (speculated tokens): Lq * Hq / Hkv must not exceed 48 (else
  * DA_ERR_UNSUPPORTED: longer query blocks need the tensor-core kernel, which reads a bf16 cache).
  * Runs on the streaming kernels with per-column causal limits.  Arguments as decode_attn_extend()
  * and decode_attn_fp8kv().
@@ -348,7 +348,14 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
  *                  ranges (0 .. 64, default 4; 0 = static ranges only)
  *   "static_frac"  share of the work, in 1/256, covered by the static ranges (default 224)
  *   "extend_stream_rows"  decode_attn_extend(): most query rows per KV head that go through the
- *                  streaming kernels instead of the tensor-core kernel (0 .. 16, default 16)
+ *                  streaming kernels instead of the tensor-core kernel (0 .. 48, default 16; beyond 16 rows
+ *                  the thread blocks carry a second set of consumer warps for the further columns)
+ *   "direct_path"  1 (default): a call small enough that every (sequence, KV head) pair, cut into at most
+ *                  eight pieces of at most eight tiles, fits one wave of thread blocks (judged from B, the
+ *                  block table's width and the window, since the lengths are on the device) runs as ONE
+ *                  kernel: each block derives its piece from seq_lens itself and the block that finishes a
+ *                  pair last folds the pieces.  0: always plan + partition + merge.  Only taken while
+ *                  "grid_blocks" is 0.
  *   "kv_evict_first"  L2 priority of the K and V page loads: 1 = "evict first" (pages that are read
  *                  once do not push the query rows, block table, plan and partial results out of L2),
  *                  0 = normal (better when sequences share pages, which are then re-read from L2),

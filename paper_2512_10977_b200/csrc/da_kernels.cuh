@@ -71,6 +71,8 @@ __device__ unsigned long long g_timeline[TL_ROWS][TL_COLS];
 constexpr int TILE_ITEM_END = 1;   // last tile this unit holds of its (b, kv head) pair
 constexpr int TILE_WHOLE = 2;      // the unit holds every tile of the pair: write `out` directly
 constexpr int TILE_STOP = 4;       // no more work for this block (carries no data)
+constexpr int TILE_SPLITS_SHIFT = 8;   // direct mode: bits 8.. = blocks that share the tile's pair
+constexpr int DIRECT_MAX_PAIRS = 512;  // direct mode: (sequence, KV head) pairs of a call (one counter each)
 
 // A thread block's consumer warps form CSETS column sets of NCW warps.  Warp (set cs, token group tw) owns
 // tokens WT * tw .. of every tile and the NT8 column tiles (8 query heads each) cs * NT8 .. of the KV
@@ -142,6 +144,14 @@ struct PartParams {
     int64_t q_sq, o_sq, l_sq;         // strides of the query-token dimension (0 when Lq == 1)
     int32_t unit_cap;                 // rows of unit_work; the partial arrays hold 2 * unit_cap slots
     int64_t max_pages;                // entries in a block-table row
+    // Direct mode (direct_splits > 0; small calls, one token per sequence): no plan and no merge kernel.
+    // Block x takes piece x % direct_splits of pair x / direct_splits = (b, kv head), works its tiles out
+    // from seq_lens[b] itself and writes a partial to slot x; the block that finishes a pair last (a counter
+    // per pair, left at zero again) folds the pieces and writes the result.
+    int32_t direct_splits, window;
+    const int32_t *seq_lens;
+    int64_t sl_stride;
+    int32_t *pair_counters;           // [DIRECT_MAX_PAIRS], zero between calls
 };
 
 struct PlanParams {
@@ -547,18 +557,20 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         const bool active = lane < nboxes * 2;
         const uint32_t box_bytes = (uint32_t)p.box_rows * ROW_BYTES;
         const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
-        const int n_static = p.hdr->n_static, n_units = n_static + p.hdr->n_tail;
+        const bool direct = p.direct_splits > 0;
+        const int n_static = direct ? 0 : p.hdr->n_static, n_units = direct ? 0 : n_static + p.hdr->n_tail;
         uint32_t it = 0;
         bool aborted = false;
         // K and V pass through L2 once (unless sequences share pages: then the caller may ask for the
         // normal priority, under which re-read pages stay in L2 longer)
-        const uint64_t kv_policy = p.hdr->kv_evict_first ? l2_policy_evict_first() : l2_policy_evict_normal();
+        const uint64_t kv_policy = (!direct && p.hdr->kv_evict_first) ? l2_policy_evict_first() : l2_policy_evict_normal();
 
         // cursor over this block's tiles: unit u, pair (b, g), tile i of cnt
         int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
         int b = 0, g = 0, rel = 0, remaining = 0, cnt = 0, i = 0;
         int4 si = make_int4(0, 0, 0, 0);
         bool first_item = true;
+        int direct_flags = 0;
         const int box_tok = box * p.box_rows;   // this lane's first token within a tile
         const int32_t *bt_row = p.block_table;  // block-table row of the cursor's sequence (set in open_pair)
         auto take_ticket = [&]() {
@@ -613,11 +625,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             if (t.need)
                 t.page = __ldg(bt_row + (tok0 >> p.log2_P));
             t.g = g; t.b = b; t.lo = si.x; t.L = si.y;
-            t.flags = (i == cnt - 1 ? TILE_ITEM_END : 0) | (cnt == si.w ? TILE_WHOLE : 0);
-            t.slot = 2 * u + (first_item ? 0 : 1);
+            t.flags = (i == cnt - 1 ? TILE_ITEM_END : 0) | (cnt == si.w ? TILE_WHOLE : 0) | direct_flags;
+            t.slot = direct ? (int)blockIdx.x : 2 * u + (first_item ? 0 : 1);
         };
         auto advance = [&]() {   // step to the next tile; false when the block has no more work
             if (++i == cnt) {
+                if (direct)
+                    return false;   // one piece of one pair per block
                 remaining -= cnt;
                 rel = 0;
                 first_item = false;
@@ -633,7 +647,48 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         // Three tile records in rotation: a tile is described (and its block-table entry requested) two
         // tiles before its copies are issued, so that the entry has two tile periods to arrive, and no
         // record is ever copied (copying a register with a load in flight would wait for the load).
-        bool cursor_ok = open_unit() && open_pair();
+        bool cursor_ok;
+        if (direct) {
+            // this block's pair and piece; the sequence's attended range and tiles, as the plan kernel would
+            // have worked them out
+            const int pair = (int)blockIdx.x / p.direct_splits, piece = (int)blockIdx.x % p.direct_splits;
+            b = pair / p.Hkv;
+            g = pair % p.Hkv;
+            int L = p.seq_lens[(int64_t)b * p.sl_stride];
+            if (L < 0 || (int64_t)L > p.max_pages * (int64_t)p.P) {
+                if (lane == 0 && g == 0 && piece == 0)
+                    report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, b, 0, L);
+                L = 0;
+            }
+            const int lo = (p.window > 0 && p.window < L) ? L - p.window : 0;
+            const int first = lo / TT, nt = L > lo ? (L - 1) / TT - first + 1 : 0;
+            const int pieces = min(p.direct_splits, nt);   // pieces that hold tiles: the first `pieces`
+            si = make_int4(lo, L, first, nt);
+            bt_row = p.block_table + (int64_t)b * p.bt_sb;
+            cursor_ok = piece < pieces;
+            if (cursor_ok) {
+                rel = (int)((long long)nt * piece / pieces);
+                cnt = (int)((long long)nt * (piece + 1) / pieces) - rel;
+                direct_flags = pieces << TILE_SPLITS_SHIFT;
+            } else if (nt == 0 && piece == 0) {
+                // an empty sequence: out = 0, lse = -inf for the pair's heads (lane -> four output dims)
+                for (int hd = 0; hd < p.G; ++hd) {
+                    const int h_out = g * p.G + hd;
+                    const int64_t at = (int64_t)b * p.o_sb + (int64_t)h_out * p.o_sh + 4 * lane;
+                    if (p.out_bf16) {
+                        uint16_t *o = reinterpret_cast<uint16_t *>(p.out) + at;
+                        o[0] = o[1] = o[2] = o[3] = 0;
+                    } else {
+                        float *o = reinterpret_cast<float *>(p.out) + at;
+                        o[0] = o[1] = o[2] = o[3] = 0.f;
+                    }
+                    if (lane == 0 && p.lse)
+                        p.lse[(int64_t)b * p.l_sb + (int64_t)h_out * p.l_sh] = -INFINITY;
+                }
+            }
+        } else {
+            cursor_ok = open_unit() && open_pair();
+        }
         auto fill = [&](Tile &t) {   // describe the cursor's tile, then move the cursor on
             t.valid = cursor_ok;
             if (cursor_ok) {
@@ -834,6 +889,51 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
     };
 
+    // the result row of (sequence b, virtual head `head` of KV group g): lane -> four output dims
+    auto store_result = [&](int b, int g, int head, const float4 &val, float lse_nat) {
+        const int qi = p.Lq > 1 ? head / p.G : 0;
+        const int h_out = g * p.G + (head - qi * p.G);
+        const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h_out * p.o_sh + 4 * lane;
+        if (!DA_IN_RANGE(p.status, b, p.B, 7) || !DA_IN_RANGE(p.status, h_out, p.Hkv * p.G, 8) ||
+            !DA_IN_RANGE(p.status, qi, p.Lq, 9))
+            return;
+        if (p.out_bf16) {
+            __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
+            const uint32_t lo = pack_bf16(val.x, val.y), hi = pack_bf16(val.z, val.w);
+            if ((reinterpret_cast<uintptr_t>(o) & 7u) == 0) {
+                *reinterpret_cast<uint2 *>(o) = make_uint2(lo, hi);
+            } else {
+                reinterpret_cast<uint16_t *>(o)[0] = (uint16_t)lo;
+                reinterpret_cast<uint16_t *>(o)[1] = (uint16_t)(lo >> 16);
+                reinterpret_cast<uint16_t *>(o)[2] = (uint16_t)hi;
+                reinterpret_cast<uint16_t *>(o)[3] = (uint16_t)(hi >> 16);
+            }
+        } else {
+            float *o = reinterpret_cast<float *>(p.out) + at;
+            if ((reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+                *reinterpret_cast<float4 *>(o) = val;
+            } else {
+                o[0] = val.x; o[1] = val.y; o[2] = val.z; o[3] = val.w;
+            }
+        }
+        if (lane == 0 && p.lse)
+            p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h_out * p.l_sh] = lse_nat;
+    };
+
+    uint32_t qf[NT8][8][2];
+    float fh[NT8][2];
+    // Direct mode: the block's pair follows from its index, so its query rows are asked for before the first
+    // tile's descriptor arrives (the producer's length -> block table -> copy chain runs meanwhile).
+    const bool q_early = p.direct_splits > 0;
+    uint32_t qw[KV8 ? NT8 : 1][8][2];
+    float ks_first = 1.f;
+    if (q_early) {
+        const int pair = (int)blockIdx.x / p.direct_splits;
+        if constexpr (KV8)
+            load_q8_raw(qw, ks_first, pair / p.Hkv, pair % p.Hkv);
+        else
+            load_q(qf, pair / p.Hkv, pair % p.Hkv);
+    }
     if (!mbar_wait_bounded(bar_full, 0u, abort_flag)) {
         give_up(-3);
         return;
@@ -843,15 +943,13 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         DA_TL(blockIdx.x, 2);
     if (m0.w & TILE_STOP)
         return;
-    uint32_t qf[NT8][8][2];
-    float fh[NT8][2];
     if constexpr (KV8) {
-        uint32_t w[NT8][8][2];
-        float ks;
-        load_q8_raw(w, ks, m0.x, m0.y);
-        q8_fragments(qf, fh, w, ks);
+        if (!q_early)
+            load_q8_raw(qw, ks_first, m0.x, m0.y);
+        q8_fragments(qf, fh, qw, ks_first);
     } else {
-        load_q(qf, m0.x, m0.y);
+        if (!q_early)
+            load_q(qf, m0.x, m0.y);
 #pragma unroll
         for (int n = 0; n < NT8; ++n)
             fh[n][0] = fh[n][1] = 0.f;
@@ -860,6 +958,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     for (;;) {   // one (b, kv head) item per iteration
         const int b = m0.x, g = m0.y, lo = m1.x, L = m1.y, slot = m1.z;
         const bool whole = (m0.w & TILE_WHOLE) != 0;
+        const int pieces = m0.w >> TILE_SPLITS_SHIFT;   // direct mode: blocks that share this pair (else 0)
         bool poisoned = false;   // a tile of this item lost rows to a bad page id: the result is NaN
         float m_run[NT8][2], l_run[NT8][2], o[NT8][8][4];
 #pragma unroll
@@ -1290,33 +1389,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     val = make_float4(lse_nat, lse_nat, lse_nat, lse_nat);
                 }
                 if (whole) {
-                    const int qi = p.Lq > 1 ? head / p.G : 0;
-                    const int h_out = g * p.G + (head - qi * p.G);
-                    const int64_t at = (int64_t)b * p.o_sb + (int64_t)qi * p.o_sq + (int64_t)h_out * p.o_sh + 4 * lane;
-                    if (!DA_IN_RANGE(p.status, b, p.B, 7) || !DA_IN_RANGE(p.status, h_out, p.Hkv * p.G, 8) ||
-                        !DA_IN_RANGE(p.status, qi, p.Lq, 9))
-                        continue;
-                    if (p.out_bf16) {
-                        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + at;
-                        const uint32_t lo = pack_bf16(val.x, val.y), hi = pack_bf16(val.z, val.w);
-                        if ((reinterpret_cast<uintptr_t>(o) & 7u) == 0) {
-                            *reinterpret_cast<uint2 *>(o) = make_uint2(lo, hi);
-                        } else {
-                            reinterpret_cast<uint16_t *>(o)[0] = (uint16_t)lo;
-                            reinterpret_cast<uint16_t *>(o)[1] = (uint16_t)(lo >> 16);
-                            reinterpret_cast<uint16_t *>(o)[2] = (uint16_t)hi;
-                            reinterpret_cast<uint16_t *>(o)[3] = (uint16_t)(hi >> 16);
-                        }
-                    } else {
-                        float *o = reinterpret_cast<float *>(p.out) + at;
-                        if ((reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
-                            *reinterpret_cast<float4 *>(o) = val;
-                        } else {
-                            o[0] = val.x; o[1] = val.y; o[2] = val.z; o[3] = val.w;
-                        }
-                    }
-                    if (lane == 0 && p.lse)
-                        p.lse[(int64_t)b * p.l_sb + (int64_t)qi * p.l_sq + (int64_t)h_out * p.l_sh] = lse_nat;
+                    store_result(b, g, head, val, lse_nat);
                 } else {
                     if (!DA_IN_RANGE(p.status, slot, 2 * p.unit_cap, 10))
                         continue;
@@ -1326,12 +1399,66 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 }
             }
         }
+        if (pieces > 1)
+            __threadfence();   // direct mode: this thread's partial stores are visible device-wide before the count below
         __syncwarp();
         if (lane == 0)
             mbar_arrive(bar_epi + 8);
         if (!mbar_wait_bounded(bar_epi + 8, items & 1u, abort_flag)) {
             give_up(-5);
             return;
+        }
+        if (pieces > 1) {
+            // Direct mode, a pair cut into pieces: the block that counts last folds them (the merge kernel's
+            // rule: M = max lse_k; w_k = exp(lse_k - M); out = sum w_k O_k / sum w_k; lse = M + ln sum w_k) and
+            // leaves the counter at zero for the next call.  A block has one item in this mode, so the first
+            // epilogue barrier is free for one more rendezvous (its second phase).
+            volatile int *fold_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAGS + 4);
+            const int pair = (int)blockIdx.x / p.direct_splits;
+            if (tid == 0) {
+                const int last = DA_IN_RANGE(p.status, pair, DIRECT_MAX_PAIRS, 16) && atomicAdd(p.pair_counters + pair, 1) == pieces - 1;
+                if (last)
+                    p.pair_counters[pair] = 0;
+                *fold_flag = last;
+            }
+            __syncwarp();
+            if (lane == 0)
+                mbar_arrive(bar_epi);
+            if (!mbar_wait_bounded(bar_epi, (items & 1u) ^ 1u, abort_flag)) {
+                give_up(-6);
+                return;
+            }
+            if (*fold_flag) {
+                __threadfence();   // the other blocks' partials were published before their counts
+                const int slot0 = pair * p.direct_splits;
+                for (int head = tw; head < p.Gv; head += NCW) {
+                    float lk[8], M = -INFINITY;
+                    float4 ok_[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const bool on = k < pieces;
+                        lk[k] = on ? __ldcg(p.part_lse + (int64_t)(slot0 + k) * HEADS + head) : -INFINITY;
+                        ok_[k] = on ? __ldcg(reinterpret_cast<const float4 *>(p.part_o + ((int64_t)(slot0 + k) * HEADS + head) * HEAD_DIM) + lane)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+                        M = fmaxf(M, lk[k]);
+                    }
+                    float den = 0.f;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        // (a piece that saw no token has lse = -inf and weighs nothing; a NaN piece -- rows lost
+                        //  to a bad page id -- makes the result NaN)
+                        const float w = (k < pieces && lk[k] != -INFINITY) ? __expf(lk[k] - M) : 0.f;
+                        den += w;
+                        acc.x += w * ok_[k].x;
+                        acc.y += w * ok_[k].y;
+                        acc.z += w * ok_[k].z;
+                        acc.w += w * ok_[k].w;
+                    }
+                    const float inv = 1.f / den;
+                    store_result(b, g, head, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv), M + __logf(den));
+                }
+            }
         }
         ++items;
         if (stop) {

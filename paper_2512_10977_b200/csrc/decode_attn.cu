@@ -5,6 +5,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstring>
@@ -31,6 +32,7 @@ int64_t g_opt_grid_blocks = 0;   // 0 = two blocks per SM
 int64_t g_opt_tail_units = 4;    // ticketed units per thread block (0: one static range per block only)
 int64_t g_opt_static_frac = 224; // share of the work given to the static ranges, in 1/256
 int64_t g_opt_kv_evict_first = 2; // L2 policy of the K and V loads: 0 normal, 1 evict first, 2 chosen by the plan kernel
+int64_t g_opt_direct_path = 1;    // small calls (every pair fits one wave of blocks) skip the plan and merge kernels
 int64_t g_opt_extend_stream_rows = 16;   // decode_attn_extend: Lq * (Hq / Hkv) up to this many rows go through the
                                          // streaming (partition) kernel, more through the tcgen05 kernel; 0: never
 cudaEvent_t g_ev_before = nullptr, g_ev_after = nullptr;
@@ -121,8 +123,10 @@ int tail_units_for(int nblocks)
     return t > 0 ? (int)t : 0;
 }
 
+constexpr size_t kWsHeadBytes = 4096;   // status record and the direct path's pair counters: zero between calls
+
 struct WsLayout {
-    size_t status, hdr, merge_counts, seq_info, prefix, unit_work, merge_small, merge_big, part_lse, part_o;
+    size_t status, counters, hdr, merge_counts, seq_info, prefix, unit_work, merge_small, merge_big, part_lse, part_o;
     int merge_seg;
     size_t stg_q, stg_bt, stg_sl, stg_out, stg_lse;
     size_t pre_o, pre_lse, suf_o, suf_lse, total;   // cascade scratch
@@ -140,6 +144,8 @@ WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int unit
         return at;
     };
     w.status = take(16);
+    w.counters = take((size_t)DIRECT_MAX_PAIRS * 4);   // (256 + 2048 bytes: inside the head that set_workspace clears)
+    static_assert(256 + DIRECT_MAX_PAIRS * 4 <= kWsHeadBytes, "the cleared head holds the status record and the counters");
     w.hdr = take(sizeof(PlanHeader));
     w.merge_counts = take(sizeof(MergeCounts));
     w.merge_seg = (units + PLAN_BLOCKS - 1) / PLAN_BLOCKS;   // a plan block lists at most one pair per unit it cuts
@@ -416,8 +422,28 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     rc = get_tmap(v, box_rows, kv8 ? 0 : 2, &tm_v);
     if (rc != DA_OK) return rc;
 
-    rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream, tile_t, Lq > 1 ? Lq : 0, bt);
-    if (rc != DA_OK) return rc;
+    // Direct path: a call whose (sequence, KV head) pairs, each cut into a few pieces, fit one wave of thread
+    // blocks is launched as ONE kernel -- every block works out its own piece from seq_lens, and the block that
+    // finishes a pair last folds the pieces -- instead of plan + partition + merge, whose fixed costs (two
+    // more launches, the plan's round trips) exceed the work of such a call.  The host cannot see the lengths:
+    // it bounds a pair's tiles by the block-table row (and the window).
+    int direct_splits = 0;
+    if (g_opt_direct_path && g_opt_grid_blocks <= 0 && Lq == 1 && first_token == 0 && d.B * d.Hkv <= DIRECT_MAX_PAIRS) {
+        int64_t tiles_max = (d.max_pages * d.P + tile_t - 1) / tile_t;
+        if (window > 0) tiles_max = std::min<int64_t>(tiles_max, (int64_t)window / tile_t + 2);
+        const int64_t pairs = d.B * d.Hkv, wave = 2 * (int64_t)st->sm_count;
+        int64_t s = std::min<int64_t>(8, std::max<int64_t>(1, tiles_max));       // one tile a piece where the wave has room
+        s = std::min<int64_t>(s, wave / std::max<int64_t>(pairs, 1));
+        if (s >= 1 && tiles_max <= 8 * s)   // at most eight tiles a piece: beyond that the planned split balances better
+            direct_splits = (int)s;
+    }
+    if (direct_splits) {
+        nblocks = (int)(d.B * d.Hkv) * direct_splits;   // <= two per SM <= the slots the workspace was sized for
+        n_tail = 0;
+    } else {
+        rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream, tile_t, Lq > 1 ? Lq : 0, bt);
+        if (rc != DA_OK) return rc;
+    }
 
     PartParams pa;
     pa.q = static_cast<const __nv_bfloat16 *>(q->data);
@@ -455,6 +481,11 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pa.l_sq = l_sq;
     pa.unit_cap = nblocks + n_tail;
     pa.max_pages = d.max_pages;
+    pa.direct_splits = direct_splits;
+    pa.window = window;
+    pa.seq_lens = static_cast<const int32_t *>(sl->data);
+    pa.sl_stride = sl->stride[0];
+    pa.pair_counters = reinterpret_cast<int32_t *>(ws + lay.counters);
     const bool timed = g_ev_before && g_ev_after;
     if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
     // Both dependent kernels are launched with programmatic stream serialization: their blocks may
@@ -479,6 +510,8 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     if (rc != DA_OK) return rc;
     g_launches.fetch_add(1);
     if (timed) DA_CUDA(cudaEventRecord(g_ev_after, stream));
+    if (direct_splits)
+        return DA_OK;   // the partition kernel wrote the results itself
 
     MergeParams mp;
     mp.seq_info = pa.seq_info;
@@ -1175,7 +1208,7 @@ int decode_attn_set_workspace(void *dev_ptr, size_t bytes)
     }
     if (reinterpret_cast<uintptr_t>(dev_ptr) & 255u) return DA_ERR_STRIDE_ALIGN;
     if (bytes < 256) return DA_ERR_WORKSPACE;
-    DA_CUDA(cudaMemsetAsync(dev_ptr, 0, 256, 0));
+    DA_CUDA(cudaMemsetAsync(dev_ptr, 0, bytes < kWsHeadBytes ? bytes : kWsHeadBytes, 0));
     DA_CUDA(cudaStreamSynchronize(0));
     st->ws = dev_ptr;
     st->ws_bytes = bytes;
@@ -1199,6 +1232,16 @@ int decode_attn_read_device_status(void *stream_, int32_t *host_status4)
     DA_CUDA(cudaMemcpyAsync(host_status4, ws, 16, cudaMemcpyDeviceToHost, stream));
     DA_CUDA(cudaMemsetAsync(ws, 0, 16, stream));
     DA_CUDA(cudaStreamSynchronize(stream));
+    if (host_status4[0] == DA_DEV_TIMEOUT) {
+        // a call that gave up may have left the direct path's pair counters part-way: start them at zero again
+        std::lock_guard<std::mutex> lock(g_mu);
+        int dev;
+        DeviceState *st;
+        if (current_device(&dev, &st) == DA_OK && st->ws == ws && st->ws_bytes >= kWsHeadBytes) {
+            DA_CUDA(cudaMemsetAsync(static_cast<uint8_t *>(ws) + 256, 0, kWsHeadBytes - 256, stream));
+            DA_CUDA(cudaStreamSynchronize(stream));
+        }
+    }
     return DA_OK;
 }
 
@@ -1268,6 +1311,11 @@ int decode_attn_set_option(const char *name, int64_t value)
         g_opt_kv_evict_first = value;
         return DA_OK;
     }
+    if (std::strcmp(name, "direct_path") == 0) {
+        if (value < 0 || value > 1) return DA_ERR_UNSUPPORTED;
+        g_opt_direct_path = value;
+        return DA_OK;
+    }
     if (std::strcmp(name, "extend_stream_rows") == 0) {
         if (value < 0 || value > kMaxStreamRows) return DA_ERR_UNSUPPORTED;
         g_opt_extend_stream_rows = value;
@@ -1303,6 +1351,7 @@ int64_t decode_attn_get_option(const char *name)
     if (std::strcmp(name, "static_frac") == 0) return g_opt_static_frac;
     if (std::strcmp(name, "kv_evict_first") == 0) return g_opt_kv_evict_first;
     if (std::strcmp(name, "extend_stream_rows") == 0) return g_opt_extend_stream_rows;
+    if (std::strcmp(name, "direct_path") == 0) return g_opt_direct_path;
 #ifdef DA_DIAG
     if (std::strcmp(name, "diag_wait_limit_us") == 0) return g_host_wait_limit_us;
     if (std::strcmp(name, "diag_withhold_partition_tile") == 0) return g_host_withhold[0];

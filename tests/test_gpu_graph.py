@@ -21,7 +21,17 @@ def da():
     return pkg
 
 
-def test_append_and_decode_replayed_from_a_cuda_graph(da):
+@pytest.mark.parametrize("direct", [1, 0])
+def test_append_and_decode_replayed_from_a_cuda_graph(da, direct):
+    """direct = 1: this small batch runs as one kernel per call; 0: as plan + partition + merge."""
+    da.set_option("direct_path", direct)
+    try:
+        _append_and_decode_replayed(da, 2 if direct else 4)
+    finally:
+        da.set_option("direct_path", 1)
+
+
+def _append_and_decode_replayed(da, launches_per_step):
     lens = np.array([15, 63, 200, 1, 1000])
     steps = 5
     case = workloads.build_case("graph", lens + steps + 1, 16, 91, "cpu", poison=False)
@@ -72,7 +82,8 @@ def test_append_and_decode_replayed_from_a_cuda_graph(da):
         side.synchronize()
         with torch.cuda.graph(graph, stream=side):
             step_on(side)
-    assert da.launch_count() - launches_before == 4      # append, plan, partition, merge: recorded, not run
+    # append + (partition | plan, partition, merge): recorded, not run
+    assert da.launch_count() - launches_before == launches_per_step
     graph.replay()
     torch.cuda.synchronize()
     ref, ref_lse = reference(kn, vn, qn)

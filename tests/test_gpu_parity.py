@@ -416,6 +416,37 @@ def test_plan_covers_every_attended_token_exactly_once(da, window):
         da.set_option("tail_units", 4)
 
 
+# ------------------------------------------------------------------ small calls: one kernel instead of three
+
+@pytest.mark.parametrize("lens,P,window", [([512], 16, 0), ([1, 2, 63, 64, 65, 300], 16, 0), ([700, 0, 33, 129], 64, 0),
+                                           ([900, 250, 3], 16, 100), ([2048] * 4, 128, 0), ([0, 0], 16, 0)])
+def test_direct_and_planned_paths_agree_with_the_oracle(da, lens, P, window):
+    """A call whose pairs fit one wave of thread blocks runs as one kernel (every block finds its piece from
+    seq_lens, the last block of a pair folds the pieces); option direct_path = 0 sends the same call through
+    plan + partition + merge.  Both must match the oracle, twice in a row (the pair counters are left at zero)."""
+    case = workloads.build_case("direct", lens, P, 300 + P + len(lens), "cpu", window=window)
+    ref, ref_lse = oracle_of(case)
+    dev = workloads.to_device(case, "cuda")
+    da.set_option("grid_blocks", 0)
+    try:
+        for direct, launches in ((1, 1), (1, 1), (0, 3)):
+            da.set_option("direct_path", direct)
+            for dtype in (torch.float32, torch.bfloat16):
+                n0 = da.launch_count()
+                out, lse = da.decode_attn(dev.q, dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, dev.window,
+                                          dev.scale, out_dtype=dtype)
+                assert da.launch_count() - n0 == launches
+                assert da.read_device_status() == (0, 0, 0, 0)
+                got = out.float().cpu().numpy().astype(np.float64)
+                if dtype == torch.float32:
+                    assert_close(got, ref, f"direct={direct} out")
+                else:
+                    assert_bf16_close(got, ref, f"direct={direct} out(bf16)")
+                assert_close(lse.cpu().numpy(), ref_lse, f"direct={direct} lse")
+    finally:
+        da.set_option("direct_path", 1)
+
+
 # ------------------------------------------------------------------ errors, on the host and on the device
 
 def test_host_side_argument_errors(da):
