@@ -31,15 +31,15 @@ constexpr int PF_COLS = 128 / PF_TPR;
 constexpr int PF_DRV = 4 * PF_TPR;           // warps 0..15: softmax; warp 16: issues the score MMAs (and owns the TMEM
 constexpr int PF_PV = PF_DRV + 1;            // allocation); warps 17, 18: issue the P_hi V and the P_lo V MMAs;
 constexpr int PF_LOADER = PF_DRV + 3;        // warp 19: issues the TMA loads of K, warp 20 those of V
-constexpr int PF_THREADS = (PF_LOADER + 2) * 32;   // (one tensor copy costs its issuing warp ~90 cycles)
+constexpr int PF_THREADS = (PF_LOADER + 5) * 32;   // + one idle warp: whole warpgroups, for the register hand-over   // (one tensor copy costs its issuing warp ~90 cycles)
 constexpr int PF_OFF_Q = 0;
 constexpr float PF_RESCALE_LOG2 = 8.f;       // a row's reference maximum moves only when the maximum grew by more
 constexpr uint32_t PF_WAIT_SLEEP_NS = 64;     // softmax warps yield while they wait: the driver warp shares their schedulers
 constexpr int PF_NB = 3;                     // K and V buffers (tiles in flight)
 constexpr int PF_OFF_K = PF_TILE;
 constexpr int PF_OFF_V = (1 + PF_NB) * PF_TILE;
-constexpr int PF_OFF_BARS = (1 + 2 * PF_NB) * PF_TILE;   // kfull[3], vfull[3], kfree[3], o[3], s[2], p, x
-constexpr int PF_OFF_MISC = PF_OFF_BARS + 128;  // TMEM base address, abort flag, "a page id was bad" flag
+constexpr int PF_OFF_BARS = (1 + 2 * PF_NB) * PF_TILE;   // kfull[3], vfull[3], kfree[3], o[3], s[2], p, x[4]
+constexpr int PF_OFF_MISC = PF_OFF_BARS + 160;  // TMEM base address, abort flag, "a page id was bad" flag
 constexpr int PF_OFF_XCHG = PF_OFF_MISC + 16;   // row maxima / sums swapped between a row's two threads
 constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + PF_TPR * 128 * 4;   // 2 buffers of bf16 maxima, or one of fp32 sums
 static_assert(PF_SMEM_BYTES <= 232448, "one block must fit the 227 KB of shared memory an SM offers");
@@ -205,7 +205,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     // per K/V buffer (tile t uses buffer t % 3): K loaded, V loaded, K no longer needed (scores complete),
     // PV product complete; per S buffer (t & 1): scores complete; P written; row-maximum exchange
     const uint32_t bar_kfull = sb + PF_OFF_BARS, bar_vfull = bar_kfull + 24, bar_kfree = bar_kfull + 48, bar_o = bar_kfull + 72,
-                   bar_s = bar_kfull + 96, bar_p = bar_kfull + 112, bar_x = bar_kfull + 120;
+                   bar_s = bar_kfull + 96, bar_p = bar_kfull + 112, bar_x0 = bar_kfull + 120;   // x: one per 32 rows
     volatile int *abort_flag = &abort_s;
 
     // block -> (row tile, kv head, [sequence,] split)
@@ -245,15 +245,16 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         abort_s = 0;
         *poison_s = 0;
         for (int i = 0; i < PF_NB; ++i) {
-            mbar_init(bar_kfull + 8 * i, 1);
-            mbar_init(bar_vfull + 8 * i, 1);
+            mbar_init(bar_kfull + 8 * i, 2);   // two loader warps per operand, each arrives with its bytes
+            mbar_init(bar_vfull + 8 * i, 2);
             mbar_init(bar_kfree + 8 * i, 1);
             mbar_init(bar_o + 8 * i, 2);   // the two PV products of a tile, committed by their issuing warps
         }
         mbar_init(bar_s, 1);
         mbar_init(bar_s + 8, 1);
         mbar_init(bar_p, PF_DRV);
-        mbar_init(bar_x, PF_DRV);
+        for (int i = 0; i < 4; ++i)
+            mbar_init(bar_x0 + 8 * i, PF_TPR);   // the row-maximum exchange of one quarter of the rows: its PF_TPR warps
         mbar_fence_init();
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
@@ -286,7 +287,14 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const uint32_t tmem = tmem_base_s;
     const uint32_t tmem_s = tmem, tmem_o = tmem + 256, tmem_o2 = tmem + 384;   // S(j) lives at tmem_s + 128 * (j & 1)
 
-    if (warp == PF_LOADER || warp == PF_LOADER + 1) {
+    // Registers: the block is launched with 80 a thread; the MMA-issuing, loader and idle warps (two whole
+    // warpgroups) give theirs back down to 40 and the sixteen softmax warps take 96 -- 16 x 32 x 96 + 8 x 32 x 40
+    // = 59,392 of the 24 x 32 x 80 = 61,440 the block holds, so the increase cannot wait for registers that
+    // never come.
+    if (warp >= PF_LOADER + 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");   // the idle warp
+    } else if (warp >= PF_LOADER) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // ------------------------------------------------------------------ loader warps: TMA
         // Warp PF_LOADER loads the K tiles, warp PF_LOADER + 1 the V tiles (issuing a tile's 16 tensor
         // copies takes a warp ~1500 cycles: one warp for both was the slowest stage of the block).
@@ -301,10 +309,13 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         // buffers; after that K(t) follows the completion of the scores of tile t-3 (bar_kfree) and V(t)
         // the completion of the PV products of tile t-3 (bar_o).
         if (ntiles > 0) {
-            const bool is_v = warp == PF_LOADER + 1;
+            const bool is_v = warp >= PF_LOADER + 2;
+            const int half = (warp - PF_LOADER) & 1;            // each operand's copies are shared by two warps
             const int boxes = PF_TOK / p.box_rows;
-            const int box = is_v ? lane : lane >> 1, pl = is_v ? 0 : lane & 1;
-            const bool active = lane < (is_v ? boxes : 2 * boxes);
+            const int copies = is_v ? boxes : 2 * boxes, per_warp = max(1, copies / 2);
+            const int ci = lane + half * per_warp;              // this lane's copy of the tile
+            const int box = is_v ? ci : ci >> 1, pl = is_v ? 0 : ci & 1;
+            const bool active = lane < per_warp && ci < copies;
             const uint32_t bar_full = is_v ? bar_vfull : bar_kfull;
             const uint32_t bar_free = is_v ? bar_o : bar_kfree;
             const CUtensorMap *tm = is_v ? &tm_v : &tm_k;
@@ -337,9 +348,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 }
                 // (diagnostic build only: the K loader of block 0 can leave one tile out altogether)
                 const bool withheld = !is_v && DA_WITHHOLD(1, blockIdx.x, j);
-                __syncwarp();   // the mark above precedes lane 0's arrival, which the later stages build on
-                if (lane == 0 && !withheld)
-                    mbar_arrive_expect_tx(bar, (uint32_t)(nbox * p.box_rows * 256));
+                const uint32_t n_mine = (uint32_t)__popc(__ballot_sync(0xffffffffu, mine));   // (also orders the mark above
+                if (lane == 0 && !withheld)                                                    //  before lane 0's arrival)
+                    mbar_arrive_expect_tx(bar, n_mine * (uint32_t)p.box_rows * (is_v ? 256u : 128u));
                 __syncwarp();
                 if (mine && !withheld) {
                     if (is_v)
@@ -364,7 +375,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 load_tile(t, pg_now);
                 DA_PH(ph, 1, ph_t);
             }
-            if (blockIdx.x == 0 && lane == 0)
+            if (blockIdx.x == 0 && lane == 0 && half == 0)
                 DA_PH_STORE(TL_PREFIX + 4 + (int)is_v, ph);
             if (!ok && lane == 0) {
                 if (*abort_flag == 0) {
@@ -386,6 +397,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         }
     } else if (warp == PF_DRV) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // ------------------------------------------------------------------ score MMA warp
         // All lanes wait together; lane 0 issues.  S(0), S(1), then S(j+2) into the S buffer of tile j as
         // soon as both PV products of tile j are complete (they read P(j) from that buffer) -- so the scores
@@ -442,6 +454,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         }
     } else if (warp == PF_PV || warp == PF_PV + 1) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
         // ------------------------------------------------------------------ PV MMA warps
         // Warp PF_PV accumulates P_hi V in tmem_o, warp PF_PV + 1 P_lo V in tmem_o2: for every tile, as soon
         // as P is written and V has landed.  A = P from tensor memory (16 tokens = 8 columns per step);
@@ -487,6 +500,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 96;");
         // ------------------------------------------------------------------ softmax warps
         // PF_TPR threads per row: warps w, w + 4, w + 8, ... read the same TMEM lanes (32 * (w % 4) ...),
         // each its own PF_COLS columns -- of S (tokens) and of O_tile (head_dim).
@@ -533,23 +547,15 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         };
         // A warp whose 32 rows all lie past the block's last query row (a few new tokens fill only the first
         // rows of the tile; the last row tile of a batch) computes nothing: it only keeps pace with the
-        // barriers its fellows use -- the maximum exchange, the tail clearing, the hand-over of P.
+        // barriers its fellows use -- the tail clearing and the hand-over of P.
         const bool has_rows = rt * PF_ROWS + 32 * (warp & 3) < R;
         DA_PH_DECL(ph, ph_t);
 #ifdef DA_TIMELINE
         const long long ph_begin = ph_t;
         const unsigned long long ph_ns = globaltimer_ns();
 #endif
-        for (int j = 0; !has_rows && ntiles > 0 && j <= ntiles; ++j) {
-            __syncwarp();
-            if (lane == 0)
-                mbar_arrive(bar_x);   // tiles 0 .. ntiles-1: the maxima; once more: the final sums
-            if (!mbar_wait_bounded(bar_x, (uint32_t)(j & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
-                ok = false;
-                break;
-            }
-            if (j == ntiles)
-                break;
+        const uint32_t bar_x = bar_x0 + 8 * (warp & 3);   // shared with the other warps that hold these 32 rows
+        for (int j = 0; !has_rows && j < ntiles; ++j) {
             const int t_tile = (t_begin + j) * PF_TOK;
             if (p.ext && t_tile + PF_TOK > L && !clear_v_tail(j, t_tile)) {
                 ok = false;
@@ -558,6 +564,11 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_p);
+            // (no second arrival before every warp has made its first: wait for this tile's hand-over)
+            if (!mbar_wait_bounded(bar_p, (uint32_t)(j & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
+                ok = false;
+                break;
+            }
         }
         for (int j = 0; has_rows && j < ntiles; ++j) {
             if (!mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
