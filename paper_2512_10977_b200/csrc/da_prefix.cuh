@@ -34,7 +34,7 @@ constexpr int PF_LOADER = PF_DRV + 3;        // warp 19: issues the TMA loads of
 constexpr int PF_THREADS = (PF_LOADER + 5) * 32;   // + one idle warp: whole warpgroups, for the register hand-over   // (one tensor copy costs its issuing warp ~90 cycles)
 constexpr int PF_OFF_Q = 0;
 constexpr float PF_RESCALE_LOG2 = 8.f;       // a row's reference maximum moves only when the maximum grew by more
-constexpr uint32_t PF_WAIT_SLEEP_NS = 64;     // softmax warps yield while they wait: the driver warp shares their schedulers
+constexpr uint32_t PF_WAIT_SLEEP_NS = 32;     // softmax warps yield while they wait: the driver warp shares their schedulers
 constexpr int PF_NB = 3;                     // K and V buffers (tiles in flight)
 constexpr int PF_OFF_K = PF_TILE;
 constexpr int PF_OFF_V = (1 + PF_NB) * PF_TILE;
