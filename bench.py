@@ -273,8 +273,6 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
     rank 0's JSON line for it (None on the other ranks)."""
     case = make_case(args, device, workload)
     kv8 = args.kv == "fp8"
-    if kv8 and args.cascade:
-        raise SystemExit("--kv fp8 applies to decode_attn and to --extend with a few new tokens")
     out = torch.empty(case.q.shape, dtype=torch.float32, device=device)
     lse = torch.empty(case.q.shape[:2], dtype=torch.float32, device=device)
     nbytes = case.algorithmic_bytes(4)
@@ -307,6 +305,9 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
         elif Lq:
             da.decode_attn_extend(q_ext, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
                                   case.scale, out=out, lse=lse, stream=stream)
+        elif prefix and kv8:
+            da.decode_attn_fp8kv_cascade(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table,
+                                         case.seq_lens, prefix, case.scale, out=out, lse=lse, stream=stream)
         elif prefix:
             da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
                                    prefix, case.scale, out=out, lse=lse, stream=stream)
@@ -415,8 +416,12 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
             out_h.copy_(out, non_blocking=True); lse_h.copy_(lse, non_blocking=True)
         elif prefix:   # the cascade has no host-io entry point: same copies, made here on the same stream
             q_d.copy_(q_h, non_blocking=True); bt_d.copy_(bt_h, non_blocking=True); sl_d.copy_(sl_h, non_blocking=True)
-            da.decode_attn_cascade(q_d, case.k_pages, case.v_pages, bt_d, sl_d, prefix, case.scale,
-                                   out=out, lse=lse, stream=stream)
+            if kv8:
+                da.decode_attn_fp8kv_cascade(q_d, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt_d, sl_d,
+                                             prefix, case.scale, out=out, lse=lse, stream=stream)
+            else:
+                da.decode_attn_cascade(q_d, case.k_pages, case.v_pages, bt_d, sl_d, prefix, case.scale,
+                                       out=out, lse=lse, stream=stream)
             out_h.copy_(out, non_blocking=True); lse_h.copy_(lse, non_blocking=True)
         elif kv8:
             da.decode_attn_fp8kv_host_io(q_h, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt_h, sl_h,
@@ -508,7 +513,8 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
                    "grid_blocks": da.get_option("grid_blocks"),
                    "path": (f"decode_attn{'_fp8kv' if kv8 else ''}_extend, {Lq} new tokens per sequence (causal, " +
                             ("streaming kernels)" if ext_stream else "tcgen05)")) if Lq else
-                           ("cascade (shared prefix on tcgen05)" if prefix else
+                           (("cascade over the 8-bit cache (shared prefix widened to bf16, then tcgen05)" if kv8 else
+                             "cascade (shared prefix on tcgen05)") if prefix else
                             ("decode_attn_fp8kv" if kv8 else "decode_attn"))},
         "frac_of_8TBs": gbs / world / NOMINAL_HBM_GBS, "seq_per_s": seqs,
         "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),

@@ -170,6 +170,28 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
                         void *stream);
 
 /*
+ * decode_attn_fp8kv_cascade -- decode_attn_cascade() over the 8-bit cache of decode_attn_fp8kv(): the sessions'
+ * shared initial prompt (paper Sec. 3.2 "Generate Kernel", App. B) is the largest block of cache a server
+ * would keep in 8 bits.  Same result as decode_attn_fp8kv() without a window.  The tokens past the prefix go
+ * through the streaming kernels' 8-bit instances; the prefix's E4M3 codes are first widened -- exactly, every
+ * E4M3 value is a bf16 value -- into a bf16 copy in `prefix_scratch`, which the tensor-core kernel then
+ * attends once for the whole batch, with k_scale[g] folded into the score scale and v_scale[g] into the
+ * result, so no rounding is added to the dequantised values.
+ *
+ *   prefix_scratch        DEVICE, caller-owned, 256-byte aligned, at least
+ *                         decode_attn_fp8kv_cascade_scratch_bytes(shared_prefix_tokens, Hkv, P) bytes
+ *                         (= 2 x prefix tokens x Hkv x 128 x 2: K copy, then V copy); rewritten by every call,
+ *                         so calls that share it must not overlap on the GPU.  Too small: DA_ERR_WORKSPACE.
+ * Other arguments, requirements on shared_prefix_tokens, results, workspace and error conventions: as
+ * decode_attn_cascade() and decode_attn_fp8kv().
+ */
+int decode_attn_fp8kv_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                              const float *k_scale, const float *v_scale, const da_tensor *block_table,
+                              const da_tensor *seq_lens, int32_t shared_prefix_tokens, float scale, da_tensor *out,
+                              da_tensor *lse, void *prefix_scratch, size_t prefix_scratch_bytes, void *stream);
+size_t decode_attn_fp8kv_cascade_scratch_bytes(int32_t shared_prefix_tokens, int32_t Hkv, int32_t P);
+
+/*
  * decode_attn_append -- the step that precedes decode_attn() in each layer of a decoding loop:
  * writes the new token's key and value vectors into the paged cache (the per-token growth of the
  * sessions' contexts; paper Sec. 3.2, the dialog that every FSM iteration extends).

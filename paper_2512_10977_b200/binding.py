@@ -66,6 +66,10 @@ def lib() -> ctypes.CDLL:
             L.decode_attn_append_fp8kv.argtypes = [T, T, T, T, vp, vp, T, T, vp]
             L.decode_attn_cascade.restype = ctypes.c_int
             L.decode_attn_cascade.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
+            L.decode_attn_fp8kv_cascade.restype = ctypes.c_int
+            L.decode_attn_fp8kv_cascade.argtypes = [T, T, T, vp, vp, T, T, i32, ctypes.c_float, T, T, vp, ctypes.c_size_t, vp]
+            L.decode_attn_fp8kv_cascade_scratch_bytes.restype = ctypes.c_size_t
+            L.decode_attn_fp8kv_cascade_scratch_bytes.argtypes = [i32, i32, i32]
             L.decode_attn_append.restype = ctypes.c_int
             L.decode_attn_append.argtypes = [T, T, T, T, T, T, vp]
             L.decode_attn_extend.restype = ctypes.c_int
@@ -267,6 +271,38 @@ def decode_attn_cascade(q, k_pages, v_pages, block_table, seq_lens, shared_prefi
         _check(lib().decode_attn_cascade(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]), _ref(tv[3]), _ref(tv[4]),
                                          int(shared_prefix_tokens), float(scale), _ref(tv[5]), _ref(tv[6]),
                                          _stream_ptr(stream)))
+    return out, lse
+
+
+_prefix_scratch = {}   # device index -> torch uint8 tensor for the widened prefix of the 8-bit cascade
+
+
+def decode_attn_fp8kv_cascade(q, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens, shared_prefix_tokens: int,
+                              scale: float, out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                              stream: Optional[torch.cuda.Stream] = None, out_dtype=torch.float32,
+                              prefix_scratch: Optional[torch.Tensor] = None):
+    """``decode_attn_cascade`` over the 8-bit cache (pools of E4M3 codes, per-KV-head factors).  The bf16 copy
+    of the shared prefix goes to ``prefix_scratch`` (a uint8 device tensor; one is kept per device when not
+    given).  Returns (out, lse)."""
+    if out is None:
+        out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+    with torch.cuda.device(k_pages.device):
+        _auto_workspace(q, k_pages, block_table)
+        need = int(lib().decode_attn_fp8kv_cascade_scratch_bytes(int(shared_prefix_tokens), k_pages.shape[1], k_pages.shape[2]))
+        if prefix_scratch is None:
+            prefix_scratch = _prefix_scratch.get(k_pages.device.index)
+            if prefix_scratch is None or prefix_scratch.numel() < need:
+                prefix_scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=k_pages.device)
+                _prefix_scratch[k_pages.device.index] = prefix_scratch
+        tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
+        _check(lib().decode_attn_fp8kv_cascade(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]),
+                                               k_scale.data_ptr() if k_scale is not None else None,
+                                               v_scale.data_ptr() if v_scale is not None else None,
+                                               _ref(tv[3]), _ref(tv[4]), int(shared_prefix_tokens), float(scale),
+                                               _ref(tv[5]), _ref(tv[6]), prefix_scratch.data_ptr(), prefix_scratch.numel(),
+                                               _stream_ptr(stream)))
     return out, lse
 
 

@@ -78,6 +78,11 @@ struct PrefixParams {
     int32_t splits;               // KV ranges per (row tile, head)
     int32_t row_tiles;            // cascade: ceil(B*G / 128); extend: ceil(Lq*G / 128)
     float scale_log2;
+    // The shared prefix of an 8-bit cache, widened to bf16 in scratch (widen_prefix_kernel): the pools are
+    // then that scratch copy, whose page i holds tokens [i P, (i+1) P) (no block table), and the per-KV-head
+    // factors enter here -- k_scale[g] with the score scale, v_scale[g] with the result.  NULL / 0 otherwise.
+    const float *k_scale, *v_scale;
+    int32_t identity_pages;
 };
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -327,7 +332,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 const int t = (t_begin + j) * PF_TOK + box * p.box_rows;
                 if (p.ext && t >= L)
                     return 0;   // past the sequence's last page: the block table has no entry
-                return __ldg(bt_row + t / p.P);
+                return p.identity_pages ? t / p.P : __ldg(bt_row + t / p.P);
             };
             auto load_tile = [&](int j, int page) {   // tile j into buffer j % 3
                 const int buf = j % PF_NB;
@@ -523,7 +528,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         // The scale enters inside the exponent (one fma per score).  A masked raw score must come out as
         // -inf after scaling whatever the scale's sign; a scale of exactly 0 would turn it into NaN
         // (inf * 0), so 0 is replaced by 1e-30, which changes no weight by more than 1e-24.
-        const float sc = p.scale_log2 == 0.f ? 1e-30f : p.scale_log2;
+        const float sc_in = p.scale_log2 * (p.k_scale ? __ldg(p.k_scale + g) : 1.f);
+        const float sc = sc_in == 0.f ? 1e-30f : sc_in;
+        const float v_mul = p.v_scale ? __ldg(p.v_scale + g) : 1.f;
         const float neg_inf_raw = sc > 0.f ? -INFINITY : INFINITY;
         // extend: this row's query attends tokens below `limit` (0 for padding rows: nothing)
         const int rr = rt * PF_ROWS + r;
@@ -715,9 +722,11 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             if (rr < R) {
                 const int outer = rr / p.G, hd = rr % p.G;   // sequence (cascade) or query token (extend)
                 const bool any = ntiles > 0 && l_row > 0.f;
-                const bool poisoned = *poison_s != 0;   // (every copy of this block was issued long before)
+                // (every copy of this block was issued long before; a NaN sum of weights: NaN keys, e.g. the
+                //  NaN-filled page of a widened 8-bit prefix whose page id was bad)
+                const bool poisoned = *poison_s != 0 || l_row != l_row;
                 const float nan = __int_as_float(0x7fc00000);
-                const float inv = any ? 1.f / l_row : 0.f;
+                const float inv = any ? v_mul / l_row : 0.f;
                 const float lse_val = poisoned ? nan : (any ? (m_run + fast_log2(l_row)) * LN2 : -INFINITY);
                 float vals[PF_COLS];
 #pragma unroll
@@ -767,6 +776,54 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     __syncthreads();
     if (warp == PF_DRV)
         tmem_dealloc(tmem, PF_TMEM_COLS);
+}
+
+// =====================================================================================  8-bit prefix -> bf16
+// The shared prefix of an 8-bit (E4M3) cache is widened ONCE per call into a bf16 copy that the tensor-core
+// kernel above reads: every E4M3 value is a bf16 value, so the copy is exact; the per-KV-head factors stay
+// out of it (PrefixParams::k_scale / v_scale).  One block per (prefix page, KV head); the copy is laid out
+// [page index][head][token][128] for K, then the same for V.  A page id outside the pool sets the status
+// record and fills that page with NaN, which makes every row of the result NaN (every row attends it).
+struct WidenParams {
+    const uint8_t *k_pages, *v_pages;     // strides in bytes: page, head, token
+    int64_t k_sp, k_sh, k_st, v_sp, v_sh, v_st;
+    const int32_t *block_table;           // row 0 names the prefix pages
+    __nv_bfloat16 *k_out, *v_out;         // [pages][Hkv][P][128] each
+    int32_t *status;
+    int32_t Hkv, P, num_pages;
+};
+
+__global__ void __launch_bounds__(256) widen_prefix_kernel(const WidenParams p)
+{
+    const int pi = blockIdx.x / p.Hkv, g = blockIdx.x % p.Hkv;
+    const int page = __ldg(p.block_table + pi);
+    const bool bad = (uint32_t)page >= (uint32_t)p.num_pages;
+    if (bad && threadIdx.x == 0 && g == 0)
+        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, 0, pi, page);
+    const int chunks = p.P * 8;   // 16 codes each
+    for (int e = threadIdx.x; e < 2 * chunks; e += blockDim.x) {
+        const int is_v = e >= chunks, c = (is_v ? e - chunks : e), tok = c >> 3, ch = c & 7;
+        __nv_bfloat16 *dst = (is_v ? p.v_out : p.k_out) + (((int64_t)pi * p.Hkv + g) * p.P + tok) * HEAD_DIM + ch * 16;
+        uint32_t w[8];
+        if (bad) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                w[i] = 0x7fc07fc0u;   // two bf16 NaN
+        } else {
+            const uint8_t *src = is_v ? p.v_pages + (int64_t)page * p.v_sp + (int64_t)g * p.v_sh + (int64_t)tok * p.v_st
+                                      : p.k_pages + (int64_t)page * p.k_sp + (int64_t)g * p.k_sh + (int64_t)tok * p.k_st;
+            const uint4 in = *reinterpret_cast<const uint4 *>(src + ch * 16);
+            const uint32_t codes[4] = {in.x, in.y, in.z, in.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 lo = unpack_f16(e4m3x2_lo_to_f16x2(codes[i])), hi = unpack_f16(e4m3x2_hi_to_f16x2(codes[i]));
+                w[2 * i] = pack_bf16(lo.x, lo.y);       // exact: four significant bits, exponents well inside bf16's
+                w[2 * i + 1] = pack_bf16(hi.x, hi.y);
+            }
+        }
+        reinterpret_cast<uint4 *>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        reinterpret_cast<uint4 *>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
 }
 
 // =====================================================================================  cascade merge

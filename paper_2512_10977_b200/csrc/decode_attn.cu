@@ -609,18 +609,31 @@ int decode_attn_fp8kv(const da_tensor *q, const da_tensor *k_pages, const da_ten
                true, k_scale, v_scale);
 }
 
-int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
-                        const da_tensor *block_table, const da_tensor *seq_lens, int32_t shared_prefix_tokens, float scale,
-                        da_tensor *out, da_tensor *lse, void *stream_)
+}  // extern "C"
+
+namespace {
+// decode_attn_cascade / decode_attn_fp8kv_cascade.  For the 8-bit cache the shared prefix is first widened,
+// exactly, into a bf16 copy in the caller's scratch, which the tensor-core kernel then reads as a pool whose
+// page i holds tokens [i P, (i+1) P); the per-KV-head factors enter in that kernel.
+int run_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
+                const da_tensor *seq_lens, int32_t shared_prefix_tokens, float scale, da_tensor *out, da_tensor *lse,
+                cudaStream_t stream, bool kv8, const float *k_scale, const float *v_scale, void *prefix_scratch,
+                size_t prefix_scratch_bytes)
 {
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (shared_prefix_tokens <= 0)
-        return run(q, k_pages, v_pages, block_table, seq_lens, 0, scale, out, lse, stream);
+        return run(q, k_pages, v_pages, block_table, seq_lens, 0, scale, out, lse, stream, kv8, k_scale, v_scale);
     Dims d;
-    int rc = validate(q, k_pages, v_pages, block_table, seq_lens, out, lse, &d);
+    int rc = validate(q, k_pages, v_pages, block_table, seq_lens, out, lse, &d, kv8 ? DA_FP8_E4M3 : DA_BF16);
     if (rc != DA_OK) return rc;
     if (shared_prefix_tokens % PF_TOK != 0 || (int64_t)shared_prefix_tokens > d.max_pages * d.P) return DA_ERR_SHAPE;
     if (d.B * d.Hq > 0x7fffffffll / HEAD_DIM) return DA_ERR_UNSUPPORTED;
+    const int64_t prefix_pages = (shared_prefix_tokens + d.P - 1) / d.P;
+    const size_t half_copy = (size_t)prefix_pages * d.Hkv * d.P * HEAD_DIM * 2;   // bytes of the widened K (or V)
+    if (kv8) {
+        if (!prefix_scratch) return DA_ERR_NULL;
+        if (reinterpret_cast<uintptr_t>(prefix_scratch) & 255u) return DA_ERR_STRIDE_ALIGN;
+        if (prefix_scratch_bytes < 2 * half_copy) return DA_ERR_WORKSPACE;
+    }
 
     std::lock_guard<std::mutex> lock(g_mu);
     int dev;
@@ -650,19 +663,50 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     cudaEvent_t ev_before = g_ev_before, ev_after = g_ev_after;
     g_ev_before = g_ev_after = nullptr;
     rc = launch_path(st, d, ws, lay, nblocks, n_tail, q, k_pages, v_pages, block_table, seq_lens, 0, scale, &so, &sl, stream,
-                     shared_prefix_tokens);
+                     shared_prefix_tokens, kv8, k_scale, v_scale);
     g_ev_before = ev_before;
     g_ev_after = ev_after;
     if (rc != DA_OK) return rc;
 
     // 2. attention of every query row over the shared prefix, on the tensor cores
     const int box_rows = d.P < PF_TOK ? (int)d.P : PF_TOK;
+    da_tensor kw = *k_pages, vw = *v_pages;   // the pools the prefix kernel reads
+    if (kv8) {
+        // 2a. the prefix's E4M3 codes -> bf16 (exact), page i of the copy = prefix tokens [i P, (i+1) P)
+        WidenParams wp;
+        wp.k_pages = static_cast<const uint8_t *>(k_pages->data);
+        wp.v_pages = static_cast<const uint8_t *>(v_pages->data);
+        wp.k_sp = k_pages->stride[0]; wp.k_sh = k_pages->stride[1]; wp.k_st = k_pages->stride[2];
+        wp.v_sp = v_pages->stride[0]; wp.v_sh = v_pages->stride[1]; wp.v_st = v_pages->stride[2];
+        wp.block_table = static_cast<const int32_t *>(block_table->data);
+        wp.k_out = static_cast<__nv_bfloat16 *>(prefix_scratch);
+        wp.v_out = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(prefix_scratch) + half_copy);
+        wp.status = reinterpret_cast<int32_t *>(ws + lay.status);
+        wp.Hkv = (int32_t)d.Hkv;
+        wp.P = (int32_t)d.P;
+        wp.num_pages = (int32_t)d.num_pages;
+        widen_prefix_kernel<<<(unsigned)(prefix_pages * d.Hkv), 256, 0, stream>>>(wp);
+        g_launches.fetch_add(1);
+        DA_CUDA(cudaGetLastError());
+        for (da_tensor *t : {&kw, &vw}) {
+            t->dtype = DA_BF16;
+            t->shape[0] = prefix_pages;
+            t->stride[2] = HEAD_DIM;
+            t->stride[1] = d.P * HEAD_DIM;
+            t->stride[0] = d.Hkv * d.P * HEAD_DIM;
+        }
+        kw.data = wp.k_out;
+        vw.data = wp.v_out;
+    }
     CUtensorMap tm_k, tm_v;
-    rc = get_tmap(k_pages, box_rows, 1, &tm_k);
+    rc = get_tmap(&kw, box_rows, 1, &tm_k);
     if (rc != DA_OK) return rc;
-    rc = get_tmap(v_pages, box_rows, 2, &tm_v);   // (K: one plane per box; V: both)
+    rc = get_tmap(&vw, box_rows, 2, &tm_v);   // (K: one plane per box; V: both)
     if (rc != DA_OK) return rc;
     PrefixParams pf;
+    pf.k_scale = kv8 ? k_scale : nullptr;
+    pf.v_scale = kv8 ? v_scale : nullptr;
+    pf.identity_pages = kv8 ? 1 : 0;
     pf.q = static_cast<const __nv_bfloat16 *>(q->data);
     pf.q_sb = q->stride[0];
     pf.q_sq = 0;
@@ -687,7 +731,7 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     pf.G = (int32_t)d.G;
     pf.P = (int32_t)d.P;
     pf.box_rows = box_rows;
-    pf.num_pages = (int32_t)d.num_pages;
+    pf.num_pages = kv8 ? (int32_t)prefix_pages : (int32_t)d.num_pages;
     pf.prefix_tiles = shared_prefix_tokens / PF_TOK;
     pf.row_tiles = (int32_t)((d.B * d.G + PF_ROWS - 1) / PF_ROWS);
     // one block per SM at a time (its shared memory fills an SM): as many KV ranges as fit one wave
@@ -730,6 +774,33 @@ int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_t
     g_launches.fetch_add(1);
     DA_CUDA(cudaGetLastError());
     return DA_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int decode_attn_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                        const da_tensor *block_table, const da_tensor *seq_lens, int32_t shared_prefix_tokens, float scale,
+                        da_tensor *out, da_tensor *lse, void *stream)
+{
+    return run_cascade(q, k_pages, v_pages, block_table, seq_lens, shared_prefix_tokens, scale, out, lse,
+                       static_cast<cudaStream_t>(stream), false, nullptr, nullptr, nullptr, 0);
+}
+
+int decode_attn_fp8kv_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const float *k_scale,
+                              const float *v_scale, const da_tensor *block_table, const da_tensor *seq_lens,
+                              int32_t shared_prefix_tokens, float scale, da_tensor *out, da_tensor *lse,
+                              void *prefix_scratch, size_t prefix_scratch_bytes, void *stream)
+{
+    return run_cascade(q, k_pages, v_pages, block_table, seq_lens, shared_prefix_tokens, scale, out, lse,
+                       static_cast<cudaStream_t>(stream), true, k_scale, v_scale, prefix_scratch, prefix_scratch_bytes);
+}
+
+size_t decode_attn_fp8kv_cascade_scratch_bytes(int32_t shared_prefix_tokens, int32_t Hkv, int32_t P)
+{
+    if (shared_prefix_tokens <= 0 || Hkv <= 0 || P <= 0) return 0;
+    const size_t pages = ((size_t)shared_prefix_tokens + P - 1) / P;
+    return 2 * pages * Hkv * P * HEAD_DIM * 2;
 }
 
 int decode_attn_append(const da_tensor *k_new, const da_tensor *v_new, da_tensor *k_pages, da_tensor *v_pages,
@@ -945,6 +1016,8 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
     if (rc != DA_OK) return rc;
 
     PrefixParams pf;
+    pf.k_scale = pf.v_scale = nullptr;
+    pf.identity_pages = 0;
     pf.q = static_cast<const __nv_bfloat16 *>(q->data);
     pf.q_sb = q->stride[0];
     pf.q_sq = q->stride[1];

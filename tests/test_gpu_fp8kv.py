@@ -443,3 +443,71 @@ def test_few_new_tokens_over_the_fp8_cache(da, Hq, Hkv, Lq, P):
         big = torch.zeros((len(lens), 49, Hq, 128), dtype=torch.bfloat16, device="cuda")
         da.decode_attn_fp8kv_extend(big, dev.k_pages, dev.v_pages, None, None, dev.block_table, dev.seq_lens, 1.0)
     assert e.value.status == 5
+
+
+# ------------------------------------------------------------------ shared prefix over the 8-bit cache
+
+@pytest.mark.parametrize("P", [16, 64, 128])
+@pytest.mark.parametrize("prefix,B", [(128, 1), (256, 5), (1024, 22), (2048, 43)])
+def test_fp8_cascade_matches_the_oracle(da, P, prefix, B):
+    """decode_attn_fp8kv_cascade: the prefix's codes widened exactly to bf16 and attended once for the batch on
+    the tensor cores (per-head factors folded into the score scale and the result), the rest through the 8-bit
+    streaming kernels; the result is plain decode attention over the dequantised cache."""
+    rng = np.random.default_rng(prefix + B + P)
+    lens = prefix + rng.integers(0, 700, size=B)
+    lens[0] = prefix                      # a sequence that is nothing but the prefix
+    case = fp8_case("casc8", lens, P, 11 * B + P, shared_prefix_tokens=prefix)
+    ref, ref_lse = oracle_of(case)
+    dev = workloads.to_device(case, "cuda")
+    out, lse = da.decode_attn_fp8kv_cascade(dev.q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, dev.block_table,
+                                            dev.seq_lens, prefix, dev.scale)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    assert_close(out.cpu().numpy(), ref, f"fp8 cascade P={P} prefix={prefix} B={B} out")
+    assert_close(lse.cpu().numpy(), ref_lse, f"fp8 cascade P={P} prefix={prefix} B={B} lse")
+    plain, plain_lse = da.decode_attn_fp8kv(dev.q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, dev.block_table,
+                                            dev.seq_lens, 0, dev.scale)
+    np.testing.assert_allclose(out.cpu().numpy(), plain.cpu().numpy(), atol=3e-5, rtol=1e-4)
+
+
+def test_fp8_cascade_scratch_errors_and_marking(da):
+    case = workloads.to_device(fp8_case("casc8e", [300, 400, 256], 16, 97, shared_prefix_tokens=256), "cuda")
+    args = (case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table, case.seq_lens, 256, case.scale)
+    need = da.lib().decode_attn_fp8kv_cascade_scratch_bytes(256, 8, 16)
+    assert need == 2 * 256 * 8 * 128 * 2
+    with pytest.raises(da.DecodeAttnError) as e:          # scratch too small
+        da.decode_attn_fp8kv_cascade(*args, prefix_scratch=torch.empty(need - 256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 6
+    with pytest.raises(da.DecodeAttnError) as e:          # not 256-byte aligned
+        da.decode_attn_fp8kv_cascade(*args, prefix_scratch=torch.empty(need + 512, dtype=torch.uint8, device="cuda")[16:])
+    assert e.value.status == 4
+    want, want_lse = da.decode_attn_fp8kv_cascade(*args)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    # a page id outside the pool inside the shared prefix: every row attends it, so every row is NaN
+    bt = case.block_table.clone()
+    bt[:, 5] = 10 ** 6
+    out, lse = da.decode_attn_fp8kv_cascade(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt,
+                                            case.seq_lens, 256, case.scale)
+    st = da.read_device_status()
+    assert st[0] == 1 and st[3] == 10 ** 6
+    assert torch.isnan(out).all() and torch.isnan(lse).all()
+    # a sequence shorter than the prefix is refused and comes out empty
+    sl = case.seq_lens.clone()
+    sl[1] = 100
+    out, lse = da.decode_attn_fp8kv_cascade(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table,
+                                            sl, 256, case.scale)
+    assert da.read_device_status()[0] == 2
+    assert (out[1] == 0).all() and torch.isneginf(lse[1]).all()
+    assert torch.allclose(out[[0, 2]], want[[0, 2]], atol=2e-5, rtol=1e-4)
+
+
+def test_c5a_full_size_fp8_cascade_every_eighth_sequence(da):
+    case = workloads.c5("cuda", 0, kv_dtype="fp8")
+    out, lse = da.decode_attn_fp8kv_cascade(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table,
+                                            case.seq_lens, 16384, case.scale)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    assert torch.isfinite(out).all() and torch.isfinite(lse).all()
+    ids = sorted(set(range(0, case.B, 8)) | {int(np.argmin(case.lens)), int(np.argmax(case.lens))})
+    sub = workloads.host_subcase(case, ids)
+    ref, ref_lse = oracle_of(sub)
+    assert_close(out[ids].cpu().numpy(), ref, "c5a fp8 cascade out")
+    assert_close(lse[ids].cpu().numpy(), ref_lse, "c5a fp8 cascade lse")
