@@ -152,6 +152,7 @@ struct PartParams {
     const int32_t *seq_lens;
     int64_t sl_stride;
     int32_t *pair_counters;           // [DIRECT_MAX_PAIRS], zero between calls
+    int32_t *fold_counters;           // [unit_cap][2]: two-piece pairs folded by the second block to finish; zero between calls
 };
 
 struct PlanParams {
@@ -178,6 +179,7 @@ struct PlanParams {
     int32_t n_static, n_tail_max, static_frac_q8;   // large units; most ticketed units; share of the
                                                     // line given to the large units, in 1/256
     int64_t max_pages;
+    int32_t fold_pairs;       // pairs cut in two by neighbouring thread blocks' own ranges are folded by the partition kernel
 };
 
 struct MergeParams {
@@ -434,29 +436,57 @@ __global__ void __launch_bounds__(PLAN_THREADS, 1) plan_kernel(PlanParams p)
     // the segments one after another, which the merge kernel's walk over the per-block counts reads back
     // as one contiguous list
     [[maybe_unused]] const int list_room = nblk == 1 ? p.merge_seg * PLAN_BLOCKS : p.merge_seg;
+    // where tile w of the line lies: sequence, KV head, tile of the pair, tiles of the pair
+    struct Where { int b, g, rel, nt; };
+    auto locate = [&](long long w) {
+        const int x = (w < 0x7fffffffll) ? (int)((unsigned)w / (unsigned)p.Hkv) : (int)(w / p.Hkv);
+        // largest b with prefix[b] <= x; equal prefixes (empty sequences) resolve to the last
+        int lo_i = 0, hi_i = p.B;   // invariant: prefix[lo_i] <= x < prefix[hi_i]
+        while (hi_i - lo_i > 1) {
+            const int mid = (lo_i + hi_i) >> 1;
+            if (prefix[mid] <= x)
+                lo_i = mid;
+            else
+                hi_i = mid;
+        }
+        Where r;
+        r.b = lo_i;
+        r.nt = prefix[r.b + 1] - prefix[r.b];
+        const int rem = (int)(w - (long long)prefix[r.b] * p.Hkv);   // < Hkv * nt
+        r.g = rem / r.nt;
+        r.rel = rem - r.g * r.nt;
+        return r;
+    };
+    // Does static unit v (0 < v < n_full) start inside a pair that began in unit v-1 and ends inside v?  Such a
+    // pair has exactly two pieces, in two thread blocks' own ranges: the partition kernel folds it itself (the
+    // block that finishes its piece second), so it is kept off the merge lists.  bit 0: yes; bit 2: the pair
+    // is the FIRST item of unit v-1 (that unit starts at the pair's first tile).
+    auto two_piece_start = [&](int v) {
+        if (!p.fold_pairs || v <= 0 || v >= n_full)
+            return 0;
+        const long long vs = unit_start(h, v), ve = unit_start(h, v + 1);
+        if (ve <= vs)
+            return 0;
+        const Where at = locate(vs);
+        const long long w0 = vs - at.rel, prev_start = unit_start(h, v - 1);
+        if (at.rel == 0 || prev_start > w0 || w0 + at.nt > ve)
+            return 0;
+        return 1 | (prev_start == w0 ? 4 : 0);
+    };
     for (int u = u_begin + tid; u < u_end; u += PLAN_THREADS) {
         int4 uw = make_int4(0, 0, 0, 0);
         if (u < n_units) {
             const long long ws = unit_start(h, u), we = unit_start(h, u + 1);
             if (we > ws) {
-                const int x = (ws < 0x7fffffffll) ? (int)((unsigned)ws / (unsigned)p.Hkv) : (int)(ws / p.Hkv);
-                // largest b with prefix[b] <= x; equal prefixes (empty sequences) resolve to the last
-                int lo_i = 0, hi_i = p.B;   // invariant: prefix[lo_i] <= x < prefix[hi_i]
-                while (hi_i - lo_i > 1) {
-                    const int mid = (lo_i + hi_i) >> 1;
-                    if (prefix[mid] <= x)
-                        lo_i = mid;
-                    else
-                        hi_i = mid;
-                }
-                const int b = lo_i;
-                const int nt = prefix[b + 1] - prefix[b];
-                const int rem = (int)(ws - (long long)prefix[b] * p.Hkv);   // < Hkv * nt
-                const int g = rem / nt, rel = rem - g * nt;
-                uw = make_int4(b, g, rel, (int)(we - ws));
+                const Where at = locate(ws);
+                const int b = at.b, nt = at.nt, g = at.g, rel = at.rel;
+                // unit flags, above the KV head: 1 = my first item is the second piece of a two-piece pair,
+                // 2 = my last item is the first piece of one, 4 = (with 1) my partner is its unit's first item
+                const int mine = two_piece_start(u), next = two_piece_start(u + 1);
+                uw = make_int4(b, g | ((mine | ((next & 1) << 1)) << 16), rel, (int)(we - ws));
                 // A unit that starts inside a pair marks that pair as split.  The pair is listed once,
                 // by the first such unit: the one whose predecessor holds the pair's first tile.
-                if (rel > 0) {
+                if (rel > 0 && !(mine & 1)) {
                     const int prev = (u == h.n_static) ? n_full - 1 : u - 1;
                     const long long w0 = ws - rel, prev_start = unit_start(h, prev);
                     if (prev_start <= w0) {
@@ -570,7 +600,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         int b = 0, g = 0, rel = 0, remaining = 0, cnt = 0, i = 0;
         int4 si = make_int4(0, 0, 0, 0);
         bool first_item = true;
-        int direct_flags = 0;
+        int direct_flags = 0, unit_flags = 0;
         const int box_tok = box * p.box_rows;   // this lane's first token within a tile
         const int32_t *bt_row = p.block_table;  // block-table row of the cursor's sequence (set in open_pair)
         auto take_ticket = [&]() {
@@ -586,7 +616,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     return false;
                 const int4 uw = p.unit_work[u];
                 if (uw.w > 0) {
-                    b = uw.x; g = uw.y; rel = uw.z; remaining = uw.w;
+                    b = uw.x; g = uw.y & 0xffff; rel = uw.z; remaining = uw.w;
+                    unit_flags = uw.y >> 16;
                     first_item = true;
                     return true;
                 }
@@ -613,7 +644,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     return false;
             }
         };
-        struct Tile { int page, row, t0, g, b, lo, L, flags, slot; bool need, valid; };
+        struct Tile { int page, row, t0, g, b, lo, L, flags, slot, fold; bool need, valid; };
         auto fetch = [&](Tile &t) {   // describe the cursor's tile and start its block-table read
             t.t0 = (si.z + rel + i) * TT;
             const int tok0 = t.t0 + box_tok;
@@ -627,6 +658,15 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             t.g = g; t.b = b; t.lo = si.x; t.L = si.y;
             t.flags = (i == cnt - 1 ? TILE_ITEM_END : 0) | (cnt == si.w ? TILE_WHOLE : 0) | direct_flags;
             t.slot = direct ? (int)blockIdx.x : 2 * u + (first_item ? 0 : 1);
+            // A two-piece pair that this block and a neighbour share (the plan's unit flags): the item's last
+            // tile tells the consumers which piece this is (1 first, 2 second) and the partner's slot.
+            t.fold = 0;
+            if (i == cnt - 1 && unit_flags) {
+                if ((unit_flags & 1) && first_item && rel > 0)
+                    t.fold = 2 | ((2 * (u - 1) + ((unit_flags & 4) ? 0 : 1)) << 2);
+                else if ((unit_flags & 2) && remaining == cnt && cnt < si.w - rel)
+                    t.fold = 1 | ((2 * (u + 1)) << 2);
+            }
         };
         auto advance = [&]() {   // step to the next tile; false when the block has no more work
             if (++i == cnt) {
@@ -716,7 +756,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             const bool withheld = DA_WITHHOLD(0, blockIdx.x, it);
             if (lane == 0 && !withheld) {
                 meta[2 * stage] = make_int4(cur.b, cur.g, cur.t0, cur.flags);
-                meta[2 * stage + 1] = make_int4(cur.lo, cur.L, cur.slot, poisoned != 0u);
+                meta[2 * stage + 1] = make_int4(cur.lo, cur.L, cur.slot, (poisoned != 0u ? 1 : 0) | (cur.fold << 1));
                 mbar_arrive_expect_tx(bar_full + 8 * stage, (uint32_t)__popc(mask) * box_bytes);
             }
             __syncwarp();
@@ -785,6 +825,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const int col0 = cs * HS;                           // first (virtual) head of this warp's column tiles
     const uint32_t bar_epi = bar_epi0 + 16 * cs;
     uint32_t it = 0, items = 0;
+    uint32_t ph_a = 0, ph_b = 0;   // completed phases of this column set's two epilogue barriers
     // per-lane offsets used by the ldmatrix address patterns
     const int k_row = 16 * tw + (lane & 7) + ((lane >> 3) & 1) * 8;     // K: matrices 1,3 are rows +8
     const int k_chunk = lane >> 4;                                      //    matrices 2,3 are chunk +1
@@ -959,6 +1000,7 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         const int b = m0.x, g = m0.y, lo = m1.x, L = m1.y, slot = m1.z;
         const bool whole = (m0.w & TILE_WHOLE) != 0;
         const int pieces = m0.w >> TILE_SPLITS_SHIFT;   // direct mode: blocks that share this pair (else 0)
+        int fold = 0;             // a two-piece pair shared with a neighbouring block: piece (1, 2) | partner slot << 2
         bool poisoned = false;   // a tile of this item lost rows to a bad page id: the result is NaN
         float m_run[NT8][2], l_run[NT8][2], o[NT8][8][4];
 #pragma unroll
@@ -976,7 +1018,9 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             const int a = m0.z + WT * tw;       // first token of this warp's rows
             const int v_lo = max(a, lo), v_hi = min(a + WT, L);
             const bool item_end = (m0.w & TILE_ITEM_END) != 0;
-            poisoned |= m1.w != 0;
+            poisoned |= (m1.w & 1) != 0;
+            if (item_end)
+                fold = m1.w >> 1;
             if constexpr (KV8) {
               if (v_lo < v_hi) {
                 const uint32_t k_base = smem_base + stage * STAGE_BYTES;
@@ -1340,10 +1384,11 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         __syncwarp();
         if (lane == 0)
             mbar_arrive(bar_epi);
-        if (!mbar_wait_bounded(bar_epi, items & 1u, abort_flag)) {
+        if (!mbar_wait_bounded(bar_epi, ph_a & 1u, abort_flag)) {
             give_up(-4);
             return;
         }
+        ++ph_a;
         {
             // Warp w of a column set folds the set's heads w, w + 4, ...: lane -> output dims 4 lane .. 4 lane + 3.  A short loop
             // on purpose: this code runs once per item, so its instructions are fetched cold each time,
@@ -1399,46 +1444,65 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 }
             }
         }
-        if (pieces > 1)
-            __threadfence();   // direct mode: this thread's partial stores are visible device-wide before the count below
+        // A pair whose pieces are folded here rather than by the merge kernel: in direct mode every split pair
+        // (`pieces` blocks share it), otherwise a pair cut in two by this block's range and a neighbour's
+        // (`fold`).  The block that counts last on the pair's counter folds the pieces -- the merge kernel's
+        // rule: M = max lse_k; w_k = exp(lse_k - M); out = sum w_k O_k / sum w_k; lse = M + ln sum w_k -- and
+        // leaves the counter at zero for the next call.
+        const bool counted = pieces > 1 || fold != 0;
+        if (counted)
+            __threadfence();   // this thread's partial stores are visible device-wide before the count below
         __syncwarp();
         if (lane == 0)
             mbar_arrive(bar_epi + 8);
-        if (!mbar_wait_bounded(bar_epi + 8, items & 1u, abort_flag)) {
+        if (!mbar_wait_bounded(bar_epi + 8, ph_b & 1u, abort_flag)) {
             give_up(-5);
             return;
         }
-        if (pieces > 1) {
-            // Direct mode, a pair cut into pieces: the block that counts last folds them (the merge kernel's
-            // rule: M = max lse_k; w_k = exp(lse_k - M); out = sum w_k O_k / sum w_k; lse = M + ln sum w_k) and
-            // leaves the counter at zero for the next call.  A block has one item in this mode, so the first
-            // epilogue barrier is free for one more rendezvous (its second phase).
-            volatile int *fold_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAGS + 4);
-            const int pair = (int)blockIdx.x / p.direct_splits;
-            if (tid == 0) {
-                const int last = DA_IN_RANGE(p.status, pair, DIRECT_MAX_PAIRS, 16) && atomicAdd(p.pair_counters + pair, 1) == pieces - 1;
+        ++ph_b;
+        if (counted) {
+            volatile int *fold_flag = reinterpret_cast<volatile int *>(smem + C::OFF_FLAGS + 4 + 4 * cs);
+            int n_pieces, slot_a, slot_step;   // the pieces' slots: slot_a + k * slot_step
+            int32_t *counter;
+            if (fold) {
+                const int partner = fold >> 2, first = (fold & 3) == 1;
+                n_pieces = 2;
+                slot_a = slot;
+                slot_step = partner - slot;
+                // one counter per boundary between two units (the earlier unit's index) and column set
+                counter = p.fold_counters + (size_t)(first ? partner / 2 - 1 : partner / 2) * CSETS + cs;
+            } else {
+                const int pair = (int)blockIdx.x / p.direct_splits;
+                n_pieces = pieces;
+                slot_a = pair * p.direct_splits;
+                slot_step = 1;
+                counter = p.pair_counters + (DA_IN_RANGE(p.status, pair, DIRECT_MAX_PAIRS, 16) ? pair : 0);
+            }
+            if (tw == 0 && lane == 0) {
+                const int last = atomicAdd(counter, 1) == n_pieces - 1;
                 if (last)
-                    p.pair_counters[pair] = 0;
+                    *counter = 0;
                 *fold_flag = last;
             }
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_epi);
-            if (!mbar_wait_bounded(bar_epi, (items & 1u) ^ 1u, abort_flag)) {
+            if (!mbar_wait_bounded(bar_epi, ph_a & 1u, abort_flag)) {
                 give_up(-6);
                 return;
             }
+            ++ph_a;
             if (*fold_flag) {
                 __threadfence();   // the other blocks' partials were published before their counts
-                const int slot0 = pair * p.direct_splits;
-                for (int head = tw; head < p.Gv; head += NCW) {
+                for (int head = col0 + tw; head < min(p.Gv, col0 + HS); head += NCW) {
                     float lk[8], M = -INFINITY;
                     float4 ok_[8];
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        const bool on = k < pieces;
-                        lk[k] = on ? __ldcg(p.part_lse + (int64_t)(slot0 + k) * HEADS + head) : -INFINITY;
-                        ok_[k] = on ? __ldcg(reinterpret_cast<const float4 *>(p.part_o + ((int64_t)(slot0 + k) * HEADS + head) * HEAD_DIM) + lane)
+                        const bool on = k < n_pieces;
+                        const int64_t sl = slot_a + (int64_t)k * slot_step;
+                        lk[k] = on ? __ldcg(p.part_lse + sl * HEADS + head) : -INFINITY;
+                        ok_[k] = on ? __ldcg(reinterpret_cast<const float4 *>(p.part_o + (sl * HEADS + head) * HEAD_DIM) + lane)
                                     : make_float4(0.f, 0.f, 0.f, 0.f);
                         M = fmaxf(M, lk[k]);
                     }
@@ -1448,15 +1512,19 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     for (int k = 0; k < 8; ++k) {
                         // (a piece that saw no token has lse = -inf and weighs nothing; a NaN piece -- rows lost
                         //  to a bad page id -- makes the result NaN)
-                        const float w = (k < pieces && lk[k] != -INFINITY) ? __expf(lk[k] - M) : 0.f;
+                        const float w = (k < n_pieces && lk[k] != -INFINITY) ? __expf(lk[k] - M) : 0.f;
                         den += w;
                         acc.x += w * ok_[k].x;
                         acc.y += w * ok_[k].y;
                         acc.z += w * ok_[k].z;
                         acc.w += w * ok_[k].w;
                     }
-                    const float inv = 1.f / den;
-                    store_result(b, g, head, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv), M + __logf(den));
+                    if (den == 0.f) {   // a column whose query attends none of the pair's tokens
+                        store_result(b, g, head, make_float4(0.f, 0.f, 0.f, 0.f), -INFINITY);
+                    } else {
+                        const float inv = 1.f / den;
+                        store_result(b, g, head, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv), M + __logf(den));
+                    }
                 }
             }
         }

@@ -32,6 +32,9 @@ int64_t g_opt_grid_blocks = 0;   // 0 = two blocks per SM
 int64_t g_opt_tail_units = 4;    // ticketed units per thread block (0: one static range per block only)
 int64_t g_opt_static_frac = 224; // share of the work given to the static ranges, in 1/256
 int64_t g_opt_kv_evict_first = 2; // L2 policy of the K and V loads: 0 normal, 1 evict first, 2 chosen by the plan kernel
+int64_t g_opt_fold_pairs = 2;     // pairs cut in two by neighbouring blocks' own ranges are folded by the partition kernel:
+                                  // 0 never, 1 always, 2 when the results go to host memory (decode_attn_host_io)
+thread_local bool t_results_to_host = false;   // set by the host-buffer entry points around their call of run()
 int64_t g_opt_direct_path = 1;    // small calls (every pair fits one wave of blocks) skip the plan and merge kernels
 int64_t g_opt_extend_stream_rows = 16;   // decode_attn_extend: Lq * (Hq / Hkv) up to this many rows go through the
                                          // streaming (partition) kernel, more through the tcgen05 kernel; 0: never
@@ -123,10 +126,11 @@ int tail_units_for(int nblocks)
     return t > 0 ? (int)t : 0;
 }
 
-constexpr size_t kWsHeadBytes = 4096;   // status record and the direct path's pair counters: zero between calls
+// status record, the direct path's pair counters and the two-piece pairs' counters: zero between calls
+constexpr size_t kWsHeadBytes = 256 + 2048 + (size_t)kMaxUnits * 2 * 4;
 
 struct WsLayout {
-    size_t status, counters, hdr, merge_counts, seq_info, prefix, unit_work, merge_small, merge_big, part_lse, part_o;
+    size_t status, counters, fold_counters, hdr, merge_counts, seq_info, prefix, unit_work, merge_small, merge_big, part_lse, part_o;
     int merge_seg;
     size_t stg_q, stg_bt, stg_sl, stg_out, stg_lse;
     size_t pre_o, pre_lse, suf_o, suf_lse, total;   // cascade scratch
@@ -144,8 +148,9 @@ WsLayout ws_layout(int64_t B, int64_t Hq, int64_t D, int64_t max_pages, int unit
         return at;
     };
     w.status = take(16);
-    w.counters = take((size_t)DIRECT_MAX_PAIRS * 4);   // (256 + 2048 bytes: inside the head that set_workspace clears)
-    static_assert(256 + DIRECT_MAX_PAIRS * 4 <= kWsHeadBytes, "the cleared head holds the status record and the counters");
+    w.counters = take((size_t)DIRECT_MAX_PAIRS * 4);
+    w.fold_counters = take((size_t)kMaxUnits * 2 * 4);   // (a fixed size, so that the head does not move with the options)
+    static_assert(DIRECT_MAX_PAIRS * 4 == 2048, "the cleared head holds the status record and the two counter arrays");
     w.hdr = take(sizeof(PlanHeader));
     w.merge_counts = take(sizeof(MergeCounts));
     w.merge_seg = (units + PLAN_BLOCKS - 1) / PLAN_BLOCKS;   // a plan block lists at most one pair per unit it cuts
@@ -378,6 +383,7 @@ int launch_plan(const da_tensor *sl, int32_t window, int32_t first_token, const 
     pp.n_tail_max = n_tail;
     pp.static_frac_q8 = (int32_t)g_opt_static_frac;
     pp.max_pages = d.max_pages;
+    pp.fold_pairs = g_opt_fold_pairs == 1 || (g_opt_fold_pairs == 2 && t_results_to_host);
     // Programmatic stream serialization: the blocks may be placed while the kernel before this one in
     // the stream finishes; the kernel waits on the device before it reads or writes anything.
     cudaLaunchAttribute pdl;
@@ -486,6 +492,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     pa.seq_lens = static_cast<const int32_t *>(sl->data);
     pa.sl_stride = sl->stride[0];
     pa.pair_counters = reinterpret_cast<int32_t *>(ws + lay.counters);
+    pa.fold_counters = reinterpret_cast<int32_t *>(ws + lay.fold_counters);
     const bool timed = g_ev_before && g_ev_after;
     if (timed) DA_CUDA(cudaEventRecord(g_ev_before, stream));
     // Both dependent kernels are launched with programmatic stream serialization: their blocks may
@@ -1183,7 +1190,9 @@ int run_host_io(const da_tensor *q_host, const da_tensor *k_pages, const da_tens
         ld = *lse_host;
         ld.data = direct ? lse_dev : ws + lay.stg_lse;
     }
+    t_results_to_host = direct;   // results written across PCIe: spread them over the kernel's run (option "fold_pairs")
     rc = run(&qd, k_pages, v_pages, &btd, &sld, window, scale, &od, lse_host ? &ld : nullptr, stream, kv8, k_scale, v_scale);
+    t_results_to_host = false;
     if (rc != DA_OK) return rc;
     if (!direct) {
         DA_CUDA(cudaMemcpyAsync(out_host->data, ws + lay.stg_out, (size_t)d.B * d.Hq * HEAD_DIM * out_item, cudaMemcpyDeviceToHost, stream));
@@ -1357,6 +1366,8 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
                             stream));
     DA_CUDA(cudaStreamSynchronize(stream));
     *num_units = h.n_static + h.n_tail;
+    for (int u = 0; u < nblocks + n_tail; ++u)
+        host_unit_work[4 * u + 1] &= 0xffff;   // (the kernels keep per-unit flags above the KV head)
     return DA_OK;
 }
 
@@ -1387,6 +1398,11 @@ int decode_attn_set_option(const char *name, int64_t value)
     if (std::strcmp(name, "direct_path") == 0) {
         if (value < 0 || value > 1) return DA_ERR_UNSUPPORTED;
         g_opt_direct_path = value;
+        return DA_OK;
+    }
+    if (std::strcmp(name, "fold_pairs") == 0) {
+        if (value < 0 || value > 2) return DA_ERR_UNSUPPORTED;
+        g_opt_fold_pairs = value;
         return DA_OK;
     }
     if (std::strcmp(name, "extend_stream_rows") == 0) {
@@ -1425,6 +1441,7 @@ int64_t decode_attn_get_option(const char *name)
     if (std::strcmp(name, "kv_evict_first") == 0) return g_opt_kv_evict_first;
     if (std::strcmp(name, "extend_stream_rows") == 0) return g_opt_extend_stream_rows;
     if (std::strcmp(name, "direct_path") == 0) return g_opt_direct_path;
+    if (std::strcmp(name, "fold_pairs") == 0) return g_opt_fold_pairs;
 #ifdef DA_DIAG
     if (std::strcmp(name, "diag_wait_limit_us") == 0) return g_host_wait_limit_us;
     if (std::strcmp(name, "diag_withhold_partition_tile") == 0) return g_host_withhold[0];

@@ -416,6 +416,39 @@ def test_plan_covers_every_attended_token_exactly_once(da, window):
         da.set_option("tail_units", 4)
 
 
+# ------------------------------------------------------------------ two-piece pairs folded by the partition kernel
+
+@pytest.mark.parametrize("grid", [2, 3, 7, 64, 148, 296, 1000])
+def test_pairs_cut_in_two_are_folded_by_the_partition_kernel(da, grid):
+    """Option fold_pairs = 1 (the default folds only in the host-buffer calls): a pair that the own ranges of
+    two neighbouring thread blocks cut in two is folded by the block that finishes second, not by the merge
+    kernel.  Same answer as the oracle, for every split schedule, output type and twice in a row (the
+    counters are left at zero)."""
+    case = workloads.build_case("fold", [2500, 3, 900, 0, 64, 4097, 130, 9000, 700], 16, 17, "cpu")
+    try:
+        da.set_option("fold_pairs", 1)
+        da.set_option("tail_units", 1)
+        for _ in range(2):
+            check(da, case, f"fold grid={grid}", grid)
+        check(da, case, f"fold grid={grid} bf16", grid, torch.bfloat16)
+        da.set_option("tail_units", 0)
+        check(da, case, f"fold grid={grid}, no ticketed units", grid)
+    finally:
+        da.set_option("fold_pairs", 2)
+        da.set_option("tail_units", 4)
+        da.set_option("grid_blocks", 0)
+
+
+def test_c2_full_size_with_folded_pairs(da):
+    try:
+        da.set_option("fold_pairs", 1)
+        da.set_option("grid_blocks", 0)
+        case = workloads.c2("cuda")
+        _full_size(da, case, list(range(0, case.B, 4)), "c2 folded pairs")
+    finally:
+        da.set_option("fold_pairs", 2)
+
+
 # ------------------------------------------------------------------ small calls: one kernel instead of three
 
 @pytest.mark.parametrize("lens,P,window", [([512], 16, 0), ([1, 2, 63, 64, 65, 300], 16, 0), ([700, 0, 33, 129], 64, 0),
