@@ -451,7 +451,9 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
         e1.record(stream)
         barrier()
         e2e_ms = e0.elapsed_time(e1) / K
-    assert torch.equal(out_h, out.cpu()), "host-io result differs from the device-resident call"
+    # (not bit for bit: the host-buffer call folds two-piece pairs inside the partition kernel, the
+    #  device-resident one in the merge kernel -- the same sums in another order)
+    assert torch.allclose(out_h, out.cpu(), atol=2e-5, rtol=1e-4), "host-io result differs from the device-resident call"
 
     gbs, seqs, ms = aggregate_replicas(nbytes, case.B, ms_per_step, device)
     e2e_gbs, _, e2e_ms_max = aggregate_replicas(nbytes, case.B, e2e_ms, device)

@@ -10,6 +10,15 @@ import workloads
 
 pytestmark = pytest.mark.gpu
 
+
+def same(host, dev):
+    """A host-buffer call against the device-resident call on the same inputs: the same sums, but possibly
+    folded in another order (two-piece pairs are folded by the partition kernel in the host-buffer calls)."""
+    a, b = host.float(), dev.float().cpu()
+    both_ninf = torch.isneginf(a) & torch.isneginf(b)
+    return bool(torch.allclose(torch.where(both_ninf, torch.zeros_like(a), a), torch.where(both_ninf, torch.zeros_like(b), b),
+                               atol=2e-5 if host.dtype == torch.float32 else 8e-3, rtol=1e-4))
+
 ATOL, RTOL = 1e-3, 1e-3
 
 
@@ -406,12 +415,12 @@ def test_host_io_matches_device_call(da):
         da.decode_attn_fp8kv_host_io(q_h, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, bt_h, sl_h, 9, dev.scale,
                                      out_h, lse_h)
         torch.cuda.synchronize()
-        assert torch.equal(out_h, want.cpu()) and torch.equal(lse_h, want_lse.cpu())
+        assert same(out_h, want) and same(lse_h, want_lse)
     out_p = torch.full(case.q.shape, 5.0, dtype=torch.float32)     # pageable: the staged path
     da.decode_attn_fp8kv_host_io(case.q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, case.block_table,
                                  case.seq_lens, 9, dev.scale, out_p, None)
     torch.cuda.synchronize()
-    assert torch.equal(out_p, want.cpu())
+    assert same(out_p, want)
 
 
 # ------------------------------------------------------------------ a few new tokens over the 8-bit cache

@@ -12,6 +12,15 @@ import workloads
 
 pytestmark = pytest.mark.gpu
 
+
+def same(host, dev):
+    """A host-buffer call against the device-resident call on the same inputs: the same sums, but possibly
+    folded in another order (two-piece pairs are folded by the partition kernel in the host-buffer calls)."""
+    a, b = host.float(), dev.float().cpu()
+    both_ninf = torch.isneginf(a) & torch.isneginf(b)
+    return bool(torch.allclose(torch.where(both_ninf, torch.zeros_like(a), a), torch.where(both_ninf, torch.zeros_like(b), b),
+                               atol=2e-5 if host.dtype == torch.float32 else 8e-3, rtol=1e-4))
+
 ATOL, RTOL = 1e-3, 1e-3
 
 
@@ -232,7 +241,7 @@ def test_host_io_matches_device_call(da):
         out_h.fill_(5)
         da.decode_attn_host_io(q_h, dev.k_pages, dev.v_pages, bt_h, sl_h, 9, dev.scale, out_h, lse_h)
         torch.cuda.synchronize()
-        assert torch.equal(out_h, want.cpu()) and torch.equal(lse_h, want_lse.cpu())
+        assert same(out_h, want) and same(lse_h, want_lse)
 
 
 def test_host_io_with_pageable_buffers_takes_the_staged_path(da):
@@ -243,13 +252,13 @@ def test_host_io_with_pageable_buffers_takes_the_staged_path(da):
     lse_h = torch.full(case.q.shape[:2], 5.0, dtype=torch.float32)
     da.decode_attn_host_io(case.q, dev.k_pages, dev.v_pages, case.block_table, case.seq_lens, 0, dev.scale, out_h, lse_h)
     torch.cuda.synchronize()
-    assert torch.equal(out_h, want.cpu()) and torch.equal(lse_h, want_lse.cpu())
+    assert same(out_h, want) and same(lse_h, want_lse)
     # pinned out, pageable lse: still staged (both must be mapped for direct writes)
     out_p = torch.full(case.q.shape, 5.0, dtype=torch.float32).pin_memory()
     lse_h.fill_(5)
     da.decode_attn_host_io(case.q, dev.k_pages, dev.v_pages, case.block_table, case.seq_lens, 0, dev.scale, out_p, lse_h)
     torch.cuda.synchronize()
-    assert torch.equal(out_p, want.cpu()) and torch.equal(lse_h, want_lse.cpu())
+    assert same(out_p, want) and same(lse_h, want_lse)
     # bf16 results written directly into pinned memory
     out_b = torch.zeros(case.q.shape, dtype=torch.bfloat16).pin_memory()
     lse_p = torch.zeros(case.q.shape[:2], dtype=torch.float32).pin_memory()
@@ -258,7 +267,7 @@ def test_host_io_with_pageable_buffers_takes_the_staged_path(da):
     torch.cuda.synchronize()
     want_b, _ = da.decode_attn(dev.q, dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, 0, dev.scale,
                                out_dtype=torch.bfloat16)
-    assert torch.equal(out_b, want_b.cpu()) and torch.equal(lse_p, want_lse.cpu())
+    assert same(out_b, want_b) and same(lse_p, want_lse)
     assert da.read_device_status() == (0, 0, 0, 0)
 
 
