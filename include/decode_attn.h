@@ -378,6 +378,20 @@ int decode_attn_plan(const da_tensor *seq_lens, int32_t window, int32_t Hkv, int
  *                  2 (default) in the host-buffer calls only: on the device the two ways take the same time,
  *                  but results that cross PCIe then leave while the batch is still streaming instead of
  *                  all at the end (c2 from host buffers: 0.376 -> 0.358 ms).
+ *   "cascade_overlap"  decode_attn_cascade / decode_attn_fp8kv_cascade: whether the tensor-core pass over
+ *                  the shared prefix runs BESIDE the HBM-bound pass over the sequences' own tokens -- the prefix
+ *                  kernel on about a third of the SMs ("cascade_prefix_sms", 0 = a third), the other kernels on
+ *                  the rest, joined by the prefix kernel's SMs when it ends -- or before it on all SMs.  Side
+ *                  by side, the second pass is launched on a stream of the library's own (made, with two
+ *                  events, at the first such call on a device: the one thing the library creates besides its
+ *                  kernels), forked from `stream` at the start of the call and joined to it before the final
+ *                  merge, so the call is still ordered on `stream` like any other and can be captured into a
+ *                  CUDA graph.  0 never; 1 (default) when (row tiles x KV heads) fits half of the SMs and the
+ *                  host's estimate says the second pass lasts at least as long as the first on its share (the
+ *                  host cannot see the lengths: it assumes a sequence's own part is half of what its
+ *                  block-table row can hold beyond the prefix); 2 whenever the shapes allow.  A caller whose
+ *                  sequences are much shorter than their block-table rows should say 0.  While "grid_blocks"
+ *                  is not 0, or profile events are set, the passes run one after the other.
  *   "direct_path"  1 (default): a call small enough that every (sequence, KV head) pair, cut into at most
  *                  eight pieces of at most eight tiles, fits one wave of thread blocks (judged from B, the
  *                  block table's width and the window, since the lengths are on the device) runs as ONE

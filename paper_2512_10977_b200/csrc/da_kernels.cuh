@@ -596,7 +596,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         const uint64_t kv_policy = (!direct && p.hdr->kv_evict_first) ? l2_policy_evict_first() : l2_policy_evict_normal();
 
         // cursor over this block's tiles: unit u, pair (b, g), tile i of cnt
-        int u = (int)blockIdx.x < n_units ? (int)blockIdx.x : -1;
+        // (a grid may hold more blocks than the plan has static ranges: the extra ones live on tickets alone)
+        int u = (int)blockIdx.x < n_static ? (int)blockIdx.x : -1;
         int b = 0, g = 0, rel = 0, remaining = 0, cnt = 0, i = 0;
         int4 si = make_int4(0, 0, 0, 0);
         bool first_item = true;
@@ -610,6 +611,8 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             t = __shfl_sync(0xffffffffu, t, 0) + n_static;
             return t < n_units ? t : -1;
         };
+        if (!direct && (int)blockIdx.x >= n_static)
+            u = take_ticket();
         auto open_unit = [&]() {   // make u a unit that has tiles, taking tickets past empty ones
             while (u >= 0) {
                 if (!DA_IN_RANGE(p.status, u, p.unit_cap, 4))

@@ -76,6 +76,7 @@ struct PrefixParams {
     int64_t max_pages;
     int32_t prefix_tiles;         // cascade: shared prefix length / PF_TOK
     int32_t splits;               // KV ranges per (row tile, head)
+    int32_t split0;               // cascade: the first KV range of this launch (a call may launch the ranges in two groups)
     int32_t row_tiles;            // cascade: ceil(B*G / 128); extend: ceil(Lq*G / 128)
     float scale_log2;
     // The shared prefix of an 8-bit cache, widened to bf16 in scratch (widen_prefix_kernel): the pools are
@@ -216,7 +217,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     // block -> (row tile, kv head, [sequence,] split)
     const int rt = blockIdx.x % p.row_tiles;
     const int g = (blockIdx.x / p.row_tiles) % p.Hkv;
-    int split = blockIdx.x / (p.row_tiles * p.Hkv);
+    int split = blockIdx.x / (p.row_tiles * p.Hkv) + p.split0;
     int bseq = 0, L = 0, kv_tiles = p.prefix_tiles;
     int R = p.B * p.G;               // rows in this block's row space
     if (p.ext) {
@@ -602,20 +603,30 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     if (t_mine + i >= limit)
                         sv[i] = neg_inf_raw;
             }
-            float mx = sv[0];
+            // (three at a time; fifteen instructions, five deep, for 32 scores)
+            float mx;
             if (sc > 0.f) {
+                float t[11];
 #pragma unroll
-                for (int i = 1; i < PF_COLS; ++i)
-                    mx = fmaxf(mx, sv[i]);
+                for (int i = 0; i < 10; ++i)
+                    t[i] = fmax3(sv[3 * i], sv[3 * i + 1], sv[3 * i + 2]);
+                t[10] = fmaxf(sv[30], sv[31]);
+                const float u0 = fmax3(t[0], t[1], t[2]), u1 = fmax3(t[3], t[4], t[5]), u2 = fmax3(t[6], t[7], t[8]);
+                mx = fmax3(fmax3(u0, u1, u2), t[9], t[10]);
             } else {
+                float t[11];
 #pragma unroll
-                for (int i = 1; i < PF_COLS; ++i)
-                    mx = fminf(mx, sv[i]);
+                for (int i = 0; i < 10; ++i)
+                    t[i] = fmin3(sv[3 * i], sv[3 * i + 1], sv[3 * i + 2]);
+                t[10] = fminf(sv[30], sv[31]);
+                const float u0 = fmin3(t[0], t[1], t[2]), u1 = fmin3(t[3], t[4], t[5]), u2 = fmin3(t[6], t[7], t[8]);
+                mx = fmin3(fmin3(u0, u1, u2), t[9], t[10]);
             }
             mx = (mx == neg_inf_raw) ? -INFINITY : mx * sc;
-            // the row's threads must use one maximum: swap through shared memory
+            // the row's threads must use one maximum: swap through shared memory ([row][part]: a thread
+            // reads its row's four values with one 8-byte load)
             __nv_bfloat16 *xb = xchg + (j & 1) * (PF_TPR * 128);
-            xb[part * 128 + r] = __float2bfloat16_ru(mx);
+            xb[r * PF_TPR + part] = __float2bfloat16_ru(mx);
             __syncwarp();
             if (lane == 0)
                 mbar_arrive(bar_x);
@@ -623,25 +634,41 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 ok = false;
                 break;
             }
-            mx = __bfloat162float(xb[r]);
-#pragma unroll
-            for (int q = 1; q < PF_TPR; ++q)
-                mx = fmaxf(mx, __bfloat162float(xb[q * 128 + r]));
+            static_assert(PF_TPR == 4, "four bf16 maxima per row are read as one 8-byte word");
+            {
+                const uint2 four = *reinterpret_cast<const uint2 *>(xb + r * PF_TPR);
+                const uint32_t m2 = bf16x2_max(four.x, four.y);
+                mx = fmaxf(bf16_lo_to_float(m2), bf16_hi_to_float(m2));
+            }
             DA_PH(ph, 1, ph_t);
             const bool moved = (m_run == -INFINITY) || (mx > m_run + PF_RESCALE_LOG2);
             const float m_new = moved ? mx : m_run;
             const float alpha = !moved ? 1.f : (m_run == -INFINITY ? 0.f : fast_exp2(m_run - m_new));
             // weights, their sum, and P as bf16 high + low parts (kept in registers for now)
-            float lsum = 0.f;
+            // (two scores per instruction where the arithmetic allows: scale and shift, the sum, the low part)
             uint32_t phi[PF_COLS / 2], plo[PF_COLS / 2];
             const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // a row with nothing to attend yet
+            const uint64_t sc2 = f32x2(sc, sc), nm2 = f32x2(-m_use, -m_use);
+            uint64_t lsum_a = f32x2(0.f, 0.f), lsum_b = lsum_a;
 #pragma unroll
             for (int e = 0; e < PF_COLS / 2; ++e) {
-                const float p0 = fast_exp2(fmaf(sv[2 * e], sc, -m_use));
-                const float p1 = fast_exp2(fmaf(sv[2 * e + 1], sc, -m_use));
-                lsum += p0 + p1;
+                float x0, x1, l0, l1;
+                f32x2_split(f32x2_fma(f32x2(sv[2 * e], sv[2 * e + 1]), sc2, nm2), x0, x1);
+                const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                const uint64_t pp = f32x2(p0, p1);
+                if (e & 1)
+                    lsum_b = f32x2_add(lsum_b, pp);
+                else
+                    lsum_a = f32x2_add(lsum_a, pp);
                 phi[e] = pack_bf16(p0, p1);
-                plo[e] = pack_bf16(p0 - bf16_lo_to_float(phi[e]), p1 - bf16_hi_to_float(phi[e]));
+                f32x2_split(f32x2_sub(pp, f32x2(bf16_lo_to_float(phi[e]), bf16_hi_to_float(phi[e]))), l0, l1);
+                plo[e] = pack_bf16(l0, l1);
+            }
+            float lsum;
+            {
+                float s0, s1;
+                f32x2_split(f32x2_add(lsum_a, lsum_b), s0, s1);
+                lsum = s0 + s1;
             }
             // a row of O may be rescaled only once the previous tile's PV product is complete
             // (tcgen05.ld / .st are warp-wide: all lanes go)

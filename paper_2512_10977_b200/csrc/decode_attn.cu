@@ -17,7 +17,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 111;
+constexpr int kVersion = 112;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -32,6 +32,9 @@ int64_t g_opt_grid_blocks = 0;   // 0 = two blocks per SM
 int64_t g_opt_tail_units = 4;    // ticketed units per thread block (0: one static range per block only)
 int64_t g_opt_static_frac = 224; // share of the work given to the static ranges, in 1/256
 int64_t g_opt_kv_evict_first = 2; // L2 policy of the K and V loads: 0 normal, 1 evict first, 2 chosen by the plan kernel
+int64_t g_opt_cascade_overlap = 1;  // the cascade's prefix pass beside its pass over the sequences' own tokens: 0 never,
+                                    // 1 where the host's estimate favours it, 2 wherever the shapes allow
+int64_t g_opt_cascade_prefix_sms = 0;   // SMs given to the prefix kernel then (0: a third of them)
 int64_t g_opt_fold_pairs = 2;     // pairs cut in two by neighbouring blocks' own ranges are folded by the partition kernel:
                                   // 0 never, 1 always, 2 when the results go to host memory (decode_attn_host_io)
 thread_local bool t_results_to_host = false;   // set by the host-buffer entry points around their call of run()
@@ -48,6 +51,11 @@ struct DeviceState {
     size_t ws_bytes = 0;
     int sm_count = 0;
     bool attrs_set = false;
+    // decode_attn_cascade with its two passes side by side: the second pass runs on a stream of the library's
+    // own, forked from and joined to the caller's stream by these events (made at the first such call)
+    cudaStream_t side_hi = nullptr, side_lo = nullptr;   // prefix kernel (highest priority); plan / partition / merge
+    cudaEvent_t ev_fork = nullptr, ev_join_hi = nullptr, ev_join_lo = nullptr;
+    bool side_failed = false;
 };
 DeviceState g_dev[kMaxDevices];
 
@@ -338,6 +346,37 @@ int set_all_kernel_attrs(DeviceState *st)
     return DA_OK;
 }
 
+// The library's own stream and events for the cascade's side-by-side mode; false if they cannot be made
+// (then the passes run one after the other).
+bool ensure_side_stream(DeviceState *st)
+{
+    if (st->side_hi) return true;
+    if (st->side_failed) return false;
+    cudaStream_t hi = nullptr, lo = nullptr;
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    int least = 0, greatest = 0;
+    bool ok = cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess &&
+              cudaStreamCreateWithPriority(&hi, cudaStreamNonBlocking, greatest) == cudaSuccess &&
+              cudaStreamCreateWithPriority(&lo, cudaStreamNonBlocking, least) == cudaSuccess;
+    for (int i = 0; ok && i < 3; ++i)
+        ok = cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) == cudaSuccess;
+    if (ok) {
+        st->side_hi = hi;
+        st->side_lo = lo;
+        st->ev_fork = ev[0];
+        st->ev_join_hi = ev[1];
+        st->ev_join_lo = ev[2];
+        return true;
+    }
+    cudaGetLastError();   // not an error of the call being made
+    for (cudaEvent_t e : ev)
+        if (e) cudaEventDestroy(e);
+    if (hi) cudaStreamDestroy(hi);
+    if (lo) cudaStreamDestroy(lo);
+    st->side_failed = true;
+    return false;
+}
+
 // One instance of the partition kernel: NT8 column tiles of 8 heads per warp, CSETS column sets.
 template <int NT8, int CSETS>
 int launch_partition(cudaLaunchConfig_t &cfg, bool kv8, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PartParams &pa)
@@ -407,8 +446,12 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
                 const da_tensor *k, const da_tensor *v, const da_tensor *bt, const da_tensor *sl, int32_t window,
                 float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, int32_t first_token = 0,
                 bool kv8 = false, const float *k_scale = nullptr, const float *v_scale = nullptr, int Lq = 1,
-                int64_t q_sq = 0, int64_t o_sq = 0, int64_t l_sq = 0)
+                int64_t q_sq = 0, int64_t o_sq = 0, int64_t l_sq = 0, int late_blocks = 0)
 {
+    // late_blocks: of the nblocks thread blocks, the last late_blocks get no range of their own and live on
+    // tickets (they are expected to become resident late: the cascade's prefix kernel holds their SMs); the
+    // partition kernel is then launched the ordinary way, so that it starts after the plan kernel has ended
+    // and not while the prefix kernel's blocks may still be on their way to their SMs.
     int rc = set_all_kernel_attrs(st);
     if (rc != DA_OK) return rc;
     // Up to 16 (virtual) heads per KV group: one column set, two blocks per SM.  17 .. 48 (several new tokens
@@ -434,7 +477,8 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     // more launches, the plan's round trips) exceed the work of such a call.  The host cannot see the lengths:
     // it bounds a pair's tiles by the block-table row (and the window).
     int direct_splits = 0;
-    if (g_opt_direct_path && g_opt_grid_blocks <= 0 && Lq == 1 && first_token == 0 && d.B * d.Hkv <= DIRECT_MAX_PAIRS) {
+    if (g_opt_direct_path && g_opt_grid_blocks <= 0 && Lq == 1 && first_token == 0 && late_blocks == 0 &&
+        d.B * d.Hkv <= DIRECT_MAX_PAIRS) {
         int64_t tiles_max = (d.max_pages * d.P + tile_t - 1) / tile_t;
         if (window > 0) tiles_max = std::min<int64_t>(tiles_max, (int64_t)window / tile_t + 2);
         const int64_t pairs = d.B * d.Hkv, wave = 2 * (int64_t)st->sm_count;
@@ -447,7 +491,8 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
         nblocks = (int)(d.B * d.Hkv) * direct_splits;   // <= two per SM <= the slots the workspace was sized for
         n_tail = 0;
     } else {
-        rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks, n_tail, stream, tile_t, Lq > 1 ? Lq : 0, bt);
+        rc = launch_plan(sl, window, first_token, d, ws, lay, nblocks - late_blocks, n_tail, stream, tile_t, Lq > 1 ? Lq : 0,
+                         bt);
         if (rc != DA_OK) return rc;
     }
 
@@ -505,7 +550,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     cfg.gridDim = dim3((unsigned)nblocks);
     cfg.stream = stream;
     cfg.attrs = &pdl;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = late_blocks ? 0 : 1;
     if (csets == 1 && nt8 == 1)
         rc = launch_partition<1, 1>(cfg, kv8, tm_k, tm_v, pa);
     else if (csets == 1)
@@ -547,6 +592,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     mp.l_sq = l_sq;
     mp.unit_cap = pa.unit_cap;
     mp.status = pa.status;
+    cfg.numAttrs = 1;
     cfg.gridDim = dim3((unsigned)(4 * st->sm_count));
     cfg.blockDim = dim3((unsigned)MERGE_THREADS);
     cfg.dynamicSmemBytes = 0;
@@ -654,32 +700,11 @@ int run_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
     if (d.B == 0) return DA_OK;
     uint8_t *ws = static_cast<uint8_t *>(st->ws);
 
-    // 1. attention over the tokens past the prefix, per sequence, into fp32 scratch
-    da_tensor so, sl;
-    so.data = ws + lay.suf_o;
-    so.dtype = DA_F32;
-    so.ndim = 3;
-    so.shape[0] = d.B; so.shape[1] = d.Hq; so.shape[2] = HEAD_DIM; so.shape[3] = 0;
-    so.stride[0] = d.Hq * HEAD_DIM; so.stride[1] = HEAD_DIM; so.stride[2] = 1; so.stride[3] = 0;
-    sl.data = ws + lay.suf_lse;
-    sl.dtype = DA_F32;
-    sl.ndim = 2;
-    sl.shape[0] = d.B; sl.shape[1] = d.Hq; sl.shape[2] = sl.shape[3] = 0;
-    sl.stride[0] = d.Hq; sl.stride[1] = 1; sl.stride[2] = sl.stride[3] = 0;
-    // (profile events, if set, bracket the prefix kernel in this entry point, not the partition kernel)
-    cudaEvent_t ev_before = g_ev_before, ev_after = g_ev_after;
-    g_ev_before = g_ev_after = nullptr;
-    rc = launch_path(st, d, ws, lay, nblocks, n_tail, q, k_pages, v_pages, block_table, seq_lens, 0, scale, &so, &sl, stream,
-                     shared_prefix_tokens, kv8, k_scale, v_scale);
-    g_ev_before = ev_before;
-    g_ev_after = ev_after;
-    if (rc != DA_OK) return rc;
-
-    // 2. attention of every query row over the shared prefix, on the tensor cores
+    // 1. attention of every query row over the shared prefix, on the tensor cores
     const int box_rows = d.P < PF_TOK ? (int)d.P : PF_TOK;
     da_tensor kw = *k_pages, vw = *v_pages;   // the pools the prefix kernel reads
     if (kv8) {
-        // 2a. the prefix's E4M3 codes -> bf16 (exact), page i of the copy = prefix tokens [i P, (i+1) P)
+        // 1a. the prefix's E4M3 codes -> bf16 (exact), page i of the copy = prefix tokens [i P, (i+1) P)
         WidenParams wp;
         wp.k_pages = static_cast<const uint8_t *>(k_pages->data);
         wp.v_pages = static_cast<const uint8_t *>(v_pages->data);
@@ -705,6 +730,8 @@ int run_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
         kw.data = wp.k_out;
         vw.data = wp.v_out;
     }
+    rc = set_all_kernel_attrs(st);
+    if (rc != DA_OK) return rc;
     CUtensorMap tm_k, tm_v;
     rc = get_tmap(&kw, box_rows, 1, &tm_k);
     if (rc != DA_OK) return rc;
@@ -741,21 +768,103 @@ int run_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
     pf.num_pages = kv8 ? (int32_t)prefix_pages : (int32_t)d.num_pages;
     pf.prefix_tiles = shared_prefix_tokens / PF_TOK;
     pf.row_tiles = (int32_t)((d.B * d.G + PF_ROWS - 1) / PF_ROWS);
+    // (profile events, if set, bracket the prefix kernel in this entry point, not the partition kernel)
+    cudaEvent_t ev_before = g_ev_before, ev_after = g_ev_after;
+    const bool timed = ev_before && ev_after;
     // one block per SM at a time (its shared memory fills an SM): as many KV ranges as fit one wave
-    int splits = st->sm_count / (pf.row_tiles * pf.Hkv);
+    const int64_t pairs = (int64_t)pf.row_tiles * pf.Hkv;
+    int splits = (int)(st->sm_count / pairs);
     if (splits > kMaxPrefixSplits) splits = kMaxPrefixSplits;
     if (splits > pf.prefix_tiles) splits = pf.prefix_tiles;
     if (splits < 1) splits = 1;
     pf.splits = splits;
+    pf.split0 = 0;
     pf.scale_log2 = scale * LOG2E;
-    const long long grid = (long long)pf.row_tiles * pf.Hkv * splits;
-    if (grid > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
-    const bool timed = ev_before && ev_after;
+    if (pairs * splits > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+    // Side by side or one after the other.  The prefix pass is bound by the tensor cores and the pass over the
+    // sequences' own tokens by HBM, which a good half of the SMs saturate.  So, where the second is expected to
+    // last at least as long as the first would on a third of the SMs, the two run side by side on two streams of
+    // the library's own, forked from the caller's stream and joined to it before the final merge:
+    //  * the prefix kernel at the highest priority, its KV ranges in two launches -- the first range alone
+    //    (a block fills an SM's shared memory, so (row tiles x KV heads) SMs are taken and the others stay
+    //    free), then the remaining ranges, whose blocks follow on the SMs the first launch leaves;
+    //  * plan / partition / merge at the lowest priority.  The partition blocks find the other SMs; those that
+    //    find no room are given no range of their own and join, on tickets, once no prefix block is waiting
+    //    for an SM.  When the sequences' own parts turn out short, the waiting prefix blocks spread over the
+    //    SMs that the partition blocks leave (priority decides who gets a free SM).
+    // The partition kernel is launched to start only after the plan kernel has ended, microseconds after the
+    // first prefix launch could start; should its blocks be placed first all the same, they take every SM and
+    // the prefix kernel runs after them: slower, still correct.  The host cannot see the lengths: it takes
+    // half of what the block-table rows can hold beyond the prefix as the typical sequence's own part.
+    int first_splits = 0;   // KV ranges of the first prefix launch (0: one launch, passes one after the other)
+    if (g_opt_cascade_overlap && !timed && g_opt_grid_blocks <= 0 && splits >= 2) {
+        int64_t sa = g_opt_cascade_prefix_sms > 0 ? g_opt_cascade_prefix_sms / pairs : (splits + 1) / 3;
+        sa = std::max<int64_t>(1, std::min<int64_t>(sa, splits - 1));
+        const int64_t x = pairs * sa;
+        const double flops = 4.0 * PF_ROWS * (double)pairs * shared_prefix_tokens * HEAD_DIM;
+        const double t_prefix = flops / ((double)x * 4.4e12);                      // seconds, on x SMs
+        const double own = 0.5 * (double)(d.max_pages * d.P - shared_prefix_tokens);
+        const double t_own = (double)d.B * d.Hkv * own * (kv8 ? 256.0 : 512.0) / 7.0e12;
+        if (x <= st->sm_count / 2 && (g_opt_cascade_overlap == 2 || t_own >= t_prefix) && ensure_side_stream(st))
+            first_splits = (int)sa;
+    }
+    const int prefix_sms = first_splits ? (int)(pairs * first_splits) : 0;
+    cudaStream_t pre_stream = stream, own_stream = stream;
+    if (first_splits) {
+        DA_CUDA(cudaEventRecord(st->ev_fork, stream));
+        DA_CUDA(cudaStreamWaitEvent(st->side_hi, st->ev_fork, 0));
+        DA_CUDA(cudaStreamWaitEvent(st->side_lo, st->ev_fork, 0));
+        pre_stream = st->side_hi;
+        own_stream = st->side_lo;
+    }
     if (timed) DA_CUDA(cudaEventRecord(ev_before, stream));
-    prefix_kernel<<<(unsigned)grid, PF_THREADS, PF_SMEM_BYTES, stream>>>(tm_k, tm_v, pf);
-    g_launches.fetch_add(1);
-    DA_CUDA(cudaGetLastError());
+    {
+        const int n1 = first_splits ? first_splits : splits;
+        prefix_kernel<<<(unsigned)(pairs * n1), PF_THREADS, PF_SMEM_BYTES, pre_stream>>>(tm_k, tm_v, pf);
+        g_launches.fetch_add(1);
+        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess && n1 < splits) {
+            pf.split0 = n1;
+            prefix_kernel<<<(unsigned)(pairs * (splits - n1)), PF_THREADS, PF_SMEM_BYTES, pre_stream>>>(tm_k, tm_v, pf);
+            g_launches.fetch_add(1);
+            e = cudaGetLastError();
+        }
+        if (first_splits) {   // (also after a failed launch: the caller's stream must not be left forked)
+            cudaError_t e1 = cudaEventRecord(st->ev_join_hi, st->side_hi);
+            if (e1 == cudaSuccess) e1 = cudaStreamWaitEvent(stream, st->ev_join_hi, 0);
+            if (e == cudaSuccess) e = e1;
+        }
+        if (e != cudaSuccess) {
+            if (first_splits && cudaEventRecord(st->ev_join_lo, st->side_lo) == cudaSuccess)
+                cudaStreamWaitEvent(stream, st->ev_join_lo, 0);
+            return cuda_fail(e);
+        }
+    }
     if (timed) DA_CUDA(cudaEventRecord(ev_after, stream));
+
+    // 2. attention over the tokens past the prefix, per sequence, into fp32 scratch
+    da_tensor so, sl;
+    so.data = ws + lay.suf_o;
+    so.dtype = DA_F32;
+    so.ndim = 3;
+    so.shape[0] = d.B; so.shape[1] = d.Hq; so.shape[2] = HEAD_DIM; so.shape[3] = 0;
+    so.stride[0] = d.Hq * HEAD_DIM; so.stride[1] = HEAD_DIM; so.stride[2] = 1; so.stride[3] = 0;
+    sl.data = ws + lay.suf_lse;
+    sl.dtype = DA_F32;
+    sl.ndim = 2;
+    sl.shape[0] = d.B; sl.shape[1] = d.Hq; sl.shape[2] = sl.shape[3] = 0;
+    sl.stride[0] = d.Hq; sl.stride[1] = 1; sl.stride[2] = sl.stride[3] = 0;
+    g_ev_before = g_ev_after = nullptr;
+    rc = launch_path(st, d, ws, lay, nblocks, n_tail, q, k_pages, v_pages, block_table, seq_lens, 0, scale, &so, &sl, own_stream,
+                     shared_prefix_tokens, kv8, k_scale, v_scale, 1, 0, 0, 0, prefix_sms ? 2 * prefix_sms : 0);
+    g_ev_before = ev_before;
+    g_ev_after = ev_after;
+    if (first_splits) {   // (also after a failed launch: the caller's stream must not be left forked)
+        cudaError_t e1 = cudaEventRecord(st->ev_join_lo, st->side_lo);
+        if (e1 == cudaSuccess) e1 = cudaStreamWaitEvent(stream, st->ev_join_lo, 0);
+        if (rc == DA_OK) DA_CUDA(e1);
+    }
+    if (rc != DA_OK) return rc;
 
     // 3. fold prefix partials and suffix result
     CascadeMergeParams cm;
@@ -1064,6 +1173,7 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
     if ((long long)splits * Lq > kMaxPrefixSplits) splits = (int)(kMaxPrefixSplits / Lq);
     if (splits < 1) splits = 1;
     pf.splits = splits;
+    pf.split0 = 0;
     pf.scale_log2 = scale * LOG2E;
     const long long grid = base * splits;
     if (grid > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
@@ -1405,6 +1515,16 @@ int decode_attn_set_option(const char *name, int64_t value)
         g_opt_fold_pairs = value;
         return DA_OK;
     }
+    if (std::strcmp(name, "cascade_overlap") == 0) {
+        if (value < 0 || value > 2) return DA_ERR_UNSUPPORTED;
+        g_opt_cascade_overlap = value;
+        return DA_OK;
+    }
+    if (std::strcmp(name, "cascade_prefix_sms") == 0) {
+        if (value < 0 || value > 1024) return DA_ERR_UNSUPPORTED;
+        g_opt_cascade_prefix_sms = value;
+        return DA_OK;
+    }
     if (std::strcmp(name, "extend_stream_rows") == 0) {
         if (value < 0 || value > kMaxStreamRows) return DA_ERR_UNSUPPORTED;
         g_opt_extend_stream_rows = value;
@@ -1442,6 +1562,8 @@ int64_t decode_attn_get_option(const char *name)
     if (std::strcmp(name, "extend_stream_rows") == 0) return g_opt_extend_stream_rows;
     if (std::strcmp(name, "direct_path") == 0) return g_opt_direct_path;
     if (std::strcmp(name, "fold_pairs") == 0) return g_opt_fold_pairs;
+    if (std::strcmp(name, "cascade_overlap") == 0) return g_opt_cascade_overlap;
+    if (std::strcmp(name, "cascade_prefix_sms") == 0) return g_opt_cascade_prefix_sms;
 #ifdef DA_DIAG
     if (std::strcmp(name, "diag_wait_limit_us") == 0) return g_host_wait_limit_us;
     if (std::strcmp(name, "diag_withhold_partition_tile") == 0) return g_host_withhold[0];

@@ -20,6 +20,15 @@ def da():
     return pkg
 
 
+@pytest.fixture(params=[0, 2], ids=["one-after-the-other", "side-by-side"], autouse=True)
+def overlap(request, da):
+    """Every test of this file runs with the two passes one after the other and (wherever the shapes allow it)
+    side by side on the library's own streams."""
+    da.set_option("cascade_overlap", request.param)
+    yield request.param
+    da.set_option("cascade_overlap", 1)
+
+
 def run_both(da, case, prefix, out_dtype=torch.float32):
     ref, ref_lse = oracle.decode_attn_oracle(case.q, case.k_pages, case.v_pages, case.block_table,
                                              case.seq_lens, 0, case.scale)
@@ -129,3 +138,42 @@ def test_c5a_full_size_cascade_every_fourth_sequence(da):
     ref, ref_lse = oracle.decode_attn_oracle(sub.q, sub.k_pages, sub.v_pages, sub.block_table, sub.seq_lens, 0, sub.scale)
     assert_close(out[ids].cpu().numpy(), ref, "c5a cascade out")
     assert_close(lse[ids].cpu().numpy(), ref_lse, "c5a cascade lse")
+
+
+def test_cascade_side_by_side_replayed_from_a_cuda_graph(da, overlap):
+    """The fork onto the library's own streams and the join are part of what is captured: a replay runs the two
+    passes again (side by side if that is the mode) and reads seq_lens and q as they are then."""
+    prefix = 1024
+    lens = prefix + np.array([0, 5, 300, 2000, 64, 1500, 17, 900])
+    case = workloads.build_case("cascgraph", lens + 2, 16, 29, "cpu", shared_prefix_tokens=prefix, poison=False)
+    case.seq_lens[:] = torch.from_numpy(lens.astype(np.int32))
+    dev = workloads.to_device(case, "cuda")
+    out = torch.empty(dev.q.shape, dtype=torch.float32, device="cuda")
+    lse = torch.empty(dev.q.shape[:2], dtype=torch.float32, device="cuda")
+
+    def call(stream=None):
+        da.decode_attn_cascade(dev.q, dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, prefix, dev.scale,
+                               out=out, lse=lse, stream=stream)
+
+    call()   # one-time set-up (kernel attributes, the library's streams) outside the capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            call(side)
+    for step in range(3):
+        case.seq_lens += 1 if step else 0
+        dev.seq_lens.copy_(case.seq_lens)
+        qn = torch.randn(case.q.shape, generator=torch.Generator().manual_seed(step)).to(torch.bfloat16)
+        case.q.copy_(qn)
+        dev.q.copy_(qn)
+        out.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        ref, ref_lse = oracle.decode_attn_oracle(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
+                                                 0, case.scale)
+        assert_close(out.cpu().numpy(), ref, f"cascade replay {step} out")
+        assert_close(lse.cpu().numpy(), ref_lse, f"cascade replay {step} lse")
+    assert da.read_device_status() == (0, 0, 0, 0)

@@ -456,9 +456,16 @@ def test_few_new_tokens_over_the_fp8_cache(da, Hq, Hkv, Lq, P):
 
 # ------------------------------------------------------------------ shared prefix over the 8-bit cache
 
+@pytest.fixture(params=[0, 2], ids=["one-after-the-other", "side-by-side"])
+def overlap(request, da):
+    da.set_option("cascade_overlap", request.param)
+    yield request.param
+    da.set_option("cascade_overlap", 1)
+
+
 @pytest.mark.parametrize("P", [16, 64, 128])
 @pytest.mark.parametrize("prefix,B", [(128, 1), (256, 5), (1024, 22), (2048, 43)])
-def test_fp8_cascade_matches_the_oracle(da, P, prefix, B):
+def test_fp8_cascade_matches_the_oracle(da, overlap, P, prefix, B):
     """decode_attn_fp8kv_cascade: the prefix's codes widened exactly to bf16 and attended once for the batch on
     the tensor cores (per-head factors folded into the score scale and the result), the rest through the 8-bit
     streaming kernels; the result is plain decode attention over the dequantised cache."""
@@ -509,7 +516,7 @@ def test_fp8_cascade_scratch_errors_and_marking(da):
     assert torch.allclose(out[[0, 2]], want[[0, 2]], atol=2e-5, rtol=1e-4)
 
 
-def test_c5a_full_size_fp8_cascade_every_eighth_sequence(da):
+def test_c5a_full_size_fp8_cascade_every_eighth_sequence(da, overlap):
     case = workloads.c5("cuda", 0, kv_dtype="fp8")
     out, lse = da.decode_attn_fp8kv_cascade(case.q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table,
                                             case.seq_lens, 16384, case.scale)
