@@ -440,18 +440,18 @@ int decode_attn_set_profile_events(void *before, void *after);
  *              for the plan, 2 first tile ready, 3 last tile consumed, 4 exit, 5 tiles consumed,
  *              6 (sequence, KV head) items finished); rows 1024..1031 = the merge kernel's first eight
  *              blocks (0 resident, 1 released, 2 exit); row 1032 column 2 = the last merge block's
- *              exit; rows 1036..1043 = the plan kernel's blocks (0 entry, 1 exit, 2 past the wait for the
+ *              exit; rows 1036..1051 = the plan kernel's blocks (0 entry, 1 exit, 2 past the wait for the
  *              kernel before it in the stream, 3 lengths scanned, 4 cut made, 5 units written);
- *              rows 1044..1049 = thread block 0 of the prefix kernel (decode_attn_cascade, decode_attn_extend),
- *              CYCLES one warp of each role spent in its phases, summed over the block's tiles: 1044 a softmax
+ *              rows 1052..1057 = thread block 0 of the prefix kernel (decode_attn_cascade, decode_attn_extend),
+ *              CYCLES one warp of each role spent in its phases, summed over the block's tiles: 1052 a softmax
  *              warp (0 waiting for scores, 1 loading them and agreeing on row maxima, 2 weights, 3 storing P,
- *              4 after the last tile, 5 tiles, 6 cycles entry to end, 7 the same span in ns), 1045 the score
- *              MMA warp (0 waiting for the PV products, 1 for K, 2 issuing), 1046 / 1047 the PV MMA warps
- *              (0 waiting for P, 1 for V, 2 issuing), 1048 / 1049 the K / V loader warps (0 waiting for a
+ *              4 after the last tile, 5 tiles, 6 cycles entry to end, 7 the same span in ns), 1053 the score
+ *              MMA warp (0 waiting for the PV products, 1 for K, 2 issuing), 1054 / 1055 the PV MMA warps
+ *              (0 waiting for P, 1 for V, 2 issuing), 1056 / 1057 the K / V loader warps (0 waiting for a
  *              free buffer, 1 issuing copies)
  *   capacity   values `host_out` can hold; DA_ERR_SHAPE if fewer than rows x cols
  */
-#define DECODE_ATTN_TIMELINE_ROWS 1056
+#define DECODE_ATTN_TIMELINE_ROWS 1064
 #define DECODE_ATTN_TIMELINE_COLS 8
 int decode_attn_timeline(unsigned long long *host_out, int64_t capacity, int32_t clear);
 

@@ -148,7 +148,7 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     return s.cuda_stream
 
 
-TIMELINE_ROWS, TIMELINE_COLS = 1056, 8
+TIMELINE_ROWS, TIMELINE_COLS = 1064, 8
 
 
 def timeline(clear: bool = True):

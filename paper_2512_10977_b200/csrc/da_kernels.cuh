@@ -48,7 +48,7 @@ constexpr float LN2 = 0.6931471805599453f;
 // in ns; score MMA warp: 0 waiting for the PV products, 1 for K, 2 issuing; the two PV MMA warps: 0 waiting for
 // P, 1 for V, 2 issuing; the K and V loader warps: 0 waiting for a free buffer, 1 issuing the copies.
 // In the normal build DA_TL() is empty and nothing is kept.
-constexpr int TL_ROWS = 1056, TL_COLS = 8, TL_MERGE = 1024, TL_PLAN = 1036, TL_PREFIX = 1044;
+constexpr int TL_ROWS = 1064, TL_COLS = 8, TL_MERGE = 1024, TL_PLAN = 1036, TL_PREFIX = 1052;
 #ifdef DA_TIMELINE
 __device__ unsigned long long g_timeline[TL_ROWS][TL_COLS];
 #define DA_TL(row, col) (g_timeline[(row)][(col)] = globaltimer_ns())
@@ -1566,6 +1566,10 @@ partition_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 constexpr int MERGE_LANES = HEAD_DIM / 4;
 constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_THREADS = MERGE_WARPS * MERGE_LANES;
+#ifndef DA_MERGE_BLOCKS_PER_SM
+#define DA_MERGE_BLOCKS_PER_SM 3
+#endif
+constexpr int MERGE_BLOCKS_PER_SM = DA_MERGE_BLOCKS_PER_SM;   // resident blocks an SM holds (three: 78 registers a thread, no spills to speak of)
 
 struct MergeAcc {
     float M, den;
@@ -1587,7 +1591,7 @@ __device__ __forceinline__ void merge_fold(MergeAcc &a, const MergeAcc &b)
     a.M = m_new;
 }
 
-__global__ void __launch_bounds__(MERGE_THREADS, 4) merge_kernel(const MergeParams p)
+__global__ void __launch_bounds__(MERGE_THREADS, MERGE_BLOCKS_PER_SM) merge_kernel(const MergeParams p)
 {
     __shared__ MergeAcc s_part[MERGE_WARPS][MERGE_LANES];
     const int warp = threadIdx.x / MERGE_LANES, ln = threadIdx.x % MERGE_LANES, d = ln * 4;

@@ -32,6 +32,13 @@ constexpr int PF_DRV = 4 * PF_TPR;           // warps 0..15: softmax; warp 16: i
 constexpr int PF_PV = PF_DRV + 1;            // allocation); warps 17, 18: issue the P_hi V and the P_lo V MMAs;
 constexpr int PF_LOADER = PF_DRV + 3;        // warp 19: issues the TMA loads of K, warp 20 those of V
 constexpr int PF_THREADS = (PF_LOADER + 5) * 32;   // + one idle warp: whole warpgroups, for the register hand-over   // (one tensor copy costs its issuing warp ~90 cycles)
+// Registers.  The block is launched with PF_REGS_LAUNCH a thread (the kernel's compiled count, checked on the
+// host before the first launch); the sixteen softmax warps then take PF_REGS_SOFTMAX each and the other eight
+// (two whole warpgroups) keep PF_REGS_OTHER: the sum must not exceed what the block was launched with, or the
+// increase would wait for registers that never come.
+constexpr int PF_REGS_LAUNCH = 80, PF_REGS_SOFTMAX = 96, PF_REGS_OTHER = 40;
+static_assert(PF_DRV * PF_REGS_SOFTMAX + (PF_THREADS / 32 - PF_DRV) * PF_REGS_OTHER <= (PF_THREADS / 32) * PF_REGS_LAUNCH,
+              "the register shares of the warps must fit what the block is launched with");
 constexpr int PF_OFF_Q = 0;
 constexpr float PF_RESCALE_LOG2 = 8.f;       // a row's reference maximum moves only when the maximum grew by more
 constexpr uint32_t PF_WAIT_SLEEP_NS = 32;     // softmax warps yield while they wait: the driver warp shares their schedulers
@@ -293,14 +300,10 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     const uint32_t tmem = tmem_base_s;
     const uint32_t tmem_s = tmem, tmem_o = tmem + 256, tmem_o2 = tmem + 384;   // S(j) lives at tmem_s + 128 * (j & 1)
 
-    // Registers: the block is launched with 80 a thread; the MMA-issuing, loader and idle warps (two whole
-    // warpgroups) give theirs back down to 40 and the sixteen softmax warps take 96 -- 16 x 32 x 96 + 8 x 32 x 40
-    // = 59,392 of the 24 x 32 x 80 = 61,440 the block holds, so the increase cannot wait for registers that
-    // never come.
     if (warp >= PF_LOADER + 4) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");   // the idle warp
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PF_REGS_OTHER));   // the idle warp
     } else if (warp >= PF_LOADER) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PF_REGS_OTHER));
         // ------------------------------------------------------------------ loader warps: TMA
         // Warp PF_LOADER loads the K tiles, warp PF_LOADER + 1 the V tiles (issuing a tile's 16 tensor
         // copies takes a warp ~1500 cycles: one warp for both was the slowest stage of the block).
@@ -403,7 +406,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         }
     } else if (warp == PF_DRV) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PF_REGS_OTHER));
         // ------------------------------------------------------------------ score MMA warp
         // All lanes wait together; lane 0 issues.  S(0), S(1), then S(j+2) into the S buffer of tile j as
         // soon as both PV products of tile j are complete (they read P(j) from that buffer) -- so the scores
@@ -460,7 +463,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         }
     } else if (warp == PF_PV || warp == PF_PV + 1) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(PF_REGS_OTHER));
         // ------------------------------------------------------------------ PV MMA warps
         // Warp PF_PV accumulates P_hi V in tmem_o, warp PF_PV + 1 P_lo V in tmem_o2: for every tile, as soon
         // as P is written and V has landed.  A = P from tensor memory (16 tokens = 8 columns per step);
@@ -506,7 +509,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
         }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 96;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(PF_REGS_SOFTMAX));
         // ------------------------------------------------------------------ softmax warps
         // PF_TPR threads per row: warps w, w + 4, w + 8, ... read the same TMEM lanes (32 * (w % 4) ...),
         // each its own PF_COLS columns -- of S (tokens) and of O_tile (head_dim).

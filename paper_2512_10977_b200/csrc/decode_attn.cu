@@ -17,7 +17,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 112;
+constexpr int kVersion = 113;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -342,6 +342,12 @@ int set_all_kernel_attrs(DeviceState *st)
     rc = set_kernel_attrs<3, 2>();
     if (rc != DA_OK) return rc;
     DA_CUDA(cudaFuncSetAttribute(prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PF_SMEM_BYTES));
+    // The prefix kernel's warps redistribute the block's registers among themselves (setmaxnreg): the shares
+    // are written for a block launched with PF_REGS_LAUNCH registers a thread, and a block launched with
+    // fewer would wait forever for the increase.  Refuse rather than launch.
+    cudaFuncAttributes fa;
+    DA_CUDA(cudaFuncGetAttributes(&fa, prefix_kernel));
+    if (fa.numRegs < PF_REGS_LAUNCH) return DA_ERR_UNSUPPORTED;
     st->attrs_set = true;
     return DA_OK;
 }
@@ -593,7 +599,7 @@ int launch_path(DeviceState *st, const Dims &d, uint8_t *ws, const WsLayout &lay
     mp.unit_cap = pa.unit_cap;
     mp.status = pa.status;
     cfg.numAttrs = 1;
-    cfg.gridDim = dim3((unsigned)(4 * st->sm_count));
+    cfg.gridDim = dim3((unsigned)(MERGE_BLOCKS_PER_SM * st->sm_count));
     cfg.blockDim = dim3((unsigned)MERGE_THREADS);
     cfg.dynamicSmemBytes = 0;
     DA_CUDA(cudaLaunchKernelEx(&cfg, merge_kernel, mp));

@@ -101,12 +101,13 @@ def prefix_report(args, binding, case, out, lse) -> None:
     else:
         call = lambda: binding.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
                                                    16384, case.scale, out=out, lse=lse)
+    binding.set_option("cascade_overlap", 0)   # the prefix kernel alone on all SMs
     for _ in range(max(args.calls, 1)):
         call()
     torch.cuda.synchronize()
     binding.timeline(clear=True)
     call()
-    tl = binding.timeline()[1044:1050]
+    tl = binding.timeline()[1052:1058]
     tiles = max(int(tl[0, 5]), 1)
     ghz = tl[0, 6] / max(tl[0, 7], 1)
     per = lambda x: f"{x / tiles:7.0f}"
