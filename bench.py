@@ -284,6 +284,7 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
         if workload != "c5a":
             raise SystemExit("--cascade applies to the shared-prefix workload c5a (full attention)")
         prefix = 16384
+        da.set_option("cascade_overlap", args.cascade_overlap)
 
     Lq = int(args.extend)
     if Lq:
@@ -518,6 +519,10 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
                            (("cascade over the 8-bit cache (shared prefix widened to bf16, then tcgen05)" if kv8 else
                              "cascade (shared prefix on tcgen05)") if prefix else
                             ("decode_attn_fp8kv" if kv8 else "decode_attn"))},
+    }
+    if prefix:
+        line["config"]["cascade_overlap"] = args.cascade_overlap
+    line.update({
         "frac_of_8TBs": gbs / world / NOMINAL_HBM_GBS, "seq_per_s": seqs,
         "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
         "roofline": roofline,
@@ -526,7 +531,7 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
                 "note": "q, block_table, seq_lens from pinned host memory and out, lse back to it every step; "
                         "the KV cache is resident state"},
         "gpu_launches": launches, "clocks": clocks,
-    }
+    })
     if with_cpu:
         sample = oracle_sample(case, args.ref_every)
         line["cpu_baseline"] = {k: v for k, v in sample.items() if k in ("value", "unit", "cores", "kind", "sample")}
@@ -555,6 +560,9 @@ def main():
                     help="cache element type: bf16 (decode_attn, the headline) or fp8 (decode_attn_fp8kv)")
     ap.add_argument("--cascade", action="store_true",
                     help="c5a only: attend the shared 16384-token prefix once for the batch (decode_attn_cascade)")
+    ap.add_argument("--cascade-overlap", type=int, default=1, choices=[0, 1, 2],
+                    help="--cascade: the library's option of that name (0: the two passes one after the other, "
+                         "1: side by side where the library's estimate favours it, 2: wherever the shapes allow)")
     args = ap.parse_args()
     return run_reference(args) if args.impl == "reference" else run_ours(args)
 
