@@ -32,7 +32,10 @@
  * memory: scratch comes from the caller through decode_attn_set_workspace()
  * (one entry point, decode_attn_static_scratch(), uses a fixed array inside the
  * library image instead).  Work is
- * enqueued on the given CUDA stream and the call returns at once.  Arguments a
+ * enqueued on the given CUDA stream and the call returns at once (the cascade
+ * calls may run part of their work on two streams of the library's own, created
+ * with three events at the first such call on a device and ordered inside the
+ * given stream by a fork and a join: option "cascade_overlap").  Arguments a
  * host can check (NULL, dtype, shape, stride, alignment, workspace size) are
  * rejected before anything is launched.  Errors that depend on device data are
  * found on the device (never a trap, never an unbounded wait); a status record
