@@ -522,6 +522,12 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
     }
     if prefix:
         line["config"]["cascade_overlap"] = args.cascade_overlap
+    if workload in ("c5a", "c5b") and not Lq:
+        # sequences share prefix pages: `value` counts every sequence's reads (logical bytes); these count
+        # each physical K/V row once
+        uniq = case.unique_kv_bytes()
+        line["config"]["unique_kv_bytes"] = uniq
+        line["unique_kv_gbs"] = uniq * world / (ms * 1e-3) / 1e9
     line.update({
         "frac_of_8TBs": gbs / world / NOMINAL_HBM_GBS, "seq_per_s": seqs,
         "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),

@@ -72,3 +72,19 @@ def test_reference_arm_prints_the_contract_line():
     assert line["impl"] == "reference" and line["value"] > 0 and line["unit"] == "GB/s"
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def test_byte_accounting_of_the_workloads():
+    """algorithmic_bytes counts every sequence's attended K/V rows (exact token counts, not pages);
+    unique_kv_bytes counts a physical row once however many sequences share its page."""
+    sys.path.insert(0, ROOT)
+    import workloads
+    row = 2 * 8 * 128 * 2                                   # K + V, 8 KV heads, 128 values, bf16
+    shared = workloads.build_case("acct", [40, 50, 33], 16, 7, "cpu", shared_prefix_tokens=32)
+    assert shared.unique_kv_bytes() == (32 + 8 + 18 + 1) * row
+    per_seq = 48 * 128 * 2 + 48 * 128 * 4 + 48 * 4 + 4       # q, out, lse, seq_len
+    pages = 3 + 4 + 3                                        # block-table entries touched
+    assert shared.algorithmic_bytes(4) == (40 + 50 + 33) * row + 3 * per_seq + pages * 4
+    windowed = workloads.build_case("acct", [40, 50, 33], 16, 7, "cpu", window=20)
+    assert windowed.unique_kv_bytes() == 60 * row            # nothing shared: 20 rows each
+    assert list(windowed.attended_tokens()) == [20, 20, 20]

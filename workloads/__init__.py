@@ -72,6 +72,29 @@ class Case:
         return int(per_seq.sum()) + scales
 
 
+    def unique_kv_bytes(self) -> int:
+        """Bytes of the K+V rows attended by at least one sequence, each physical row counted once
+        (sequences that share pages -- a common prefix -- read the same rows): what has to come from
+        HBM at least once per call, where ``algorithmic_bytes`` counts every sequence's reads."""
+        Hkv, Dh = self.k_pages.shape[1], self.k_pages.shape[3]
+        P = self.P
+        n = self.attended_tokens()
+        L = np.maximum(self.lens.astype(np.int64), 0)
+        bt = self.block_table.cpu().numpy().astype(np.int64)
+        rows_in_page = np.zeros(int(self.k_pages.shape[0]), dtype=np.int64)   # most rows any sequence attends
+        for b in range(len(L)):
+            if n[b] <= 0:
+                continue
+            lo = int(L[b] - n[b])
+            first, last = lo // P, (int(L[b]) - 1) // P
+            pages = bt[b, first:last + 1]
+            cnt = np.full(len(pages), P, dtype=np.int64)
+            cnt[0] -= lo - first * P
+            cnt[-1] -= (last + 1) * P - int(L[b])
+            np.maximum.at(rows_in_page, pages, cnt)
+        return int(rows_in_page.sum()) * 2 * Hkv * Dh * self.k_pages.element_size()
+
+
 def _randn_bf16(shape, gen: torch.Generator, device) -> torch.Tensor:
     return torch.randn(shape, generator=gen, device=device, dtype=torch.float32).to(torch.bfloat16)
 
