@@ -301,7 +301,7 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
 
     def step():
         if Lq and kv8:
-            da.decode_attn_fp8kv_extend(q_ext, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
+            da.decode_attn_fp8kv_extend_wide(q_ext, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
                                         case.block_table, case.seq_lens, case.scale, out=out, lse=lse, stream=stream)
         elif Lq:
             da.decode_attn_extend(q_ext, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
@@ -409,7 +409,7 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
         if Lq:
             q_d.copy_(q_h, non_blocking=True); bt_d.copy_(bt_h, non_blocking=True); sl_d.copy_(sl_h, non_blocking=True)
             if kv8:
-                da.decode_attn_fp8kv_extend(q_d, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt_d, sl_d,
+                da.decode_attn_fp8kv_extend_wide(q_d, case.k_pages, case.v_pages, case.k_scale, case.v_scale, bt_d, sl_d,
                                             case.scale, out=out, lse=lse, stream=stream)
             else:
                 da.decode_attn_extend(q_d, case.k_pages, case.v_pages, bt_d, sl_d, case.scale, out=out, lse=lse,
@@ -472,7 +472,7 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
                 "kernel_ms": kms, "traffic": traffic, "traffic_capture_library_version": traffic_ver,
                 "library_version": da.version()}
     G_ = case.q.shape[1] // case.k_pages.shape[1]
-    ext_stream = bool(Lq) and (kv8 or Lq * G_ <= da.get_option("extend_stream_rows"))
+    ext_stream = bool(Lq) and ((kv8 and Lq * G_ <= 48) or Lq * G_ <= da.get_option("extend_stream_rows"))
     if ext_stream:
         # a few new tokens ride through the streaming kernels as a wider group: still bound by HBM
         roofline["kernel"] = f"partition_kernel ({Lq} query tokens x {G_} heads per KV head)"
@@ -515,7 +515,8 @@ def measure(args, da, workload, device, rank, world, local, with_cpu):
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "grid_blocks": da.get_option("grid_blocks"),
                    "path": (f"decode_attn{'_fp8kv' if kv8 else ''}_extend, {Lq} new tokens per sequence (causal, " +
-                            ("streaming kernels)" if ext_stream else "tcgen05)")) if Lq else
+                            ("streaming kernels)" if ext_stream else
+                             ("pages widened to bf16, then tcgen05)" if kv8 else "tcgen05)"))) if Lq else
                            (("cascade over the 8-bit cache (shared prefix widened to bf16, then tcgen05)" if kv8 else
                              "cascade (shared prefix on tcgen05)") if prefix else
                             ("decode_attn_fp8kv" if kv8 else "decode_attn"))},

@@ -255,7 +255,8 @@ int decode_attn_extend(const da_tensor *q, const da_tensor *k_pages, const da_te
 /*
  * decode_attn_fp8kv_extend -- decode_attn_extend() over the 8-bit cache of decode_attn_fp8kv(), for a
  * few new tokens per sequence (speculated tokens): Lq * Hq / Hkv must not exceed 48 (else
- * DA_ERR_UNSUPPORTED: longer query blocks need the tensor-core kernel, which reads a bf16 cache).
+ * DA_ERR_UNSUPPORTED: longer query blocks need the tensor-core kernel, which reads a bf16 cache; see
+ * decode_attn_fp8kv_extend_wide() below).
  * Runs on the streaming kernels with per-column causal limits.  Arguments as decode_attn_extend()
  * and decode_attn_fp8kv().
  */
@@ -263,6 +264,29 @@ int decode_attn_fp8kv_extend(const da_tensor *q, const da_tensor *k_pages, const
                              const float *k_scale, const float *v_scale, const da_tensor *block_table,
                              const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse,
                              void *stream);
+
+/*
+ * decode_attn_fp8kv_extend_wide -- decode_attn_fp8kv_extend() for query blocks of any length (a
+ * multi-thousand-token feedback prompt ingested into a context whose cache is kept in 8 bits; Sec. 3.2,
+ * "Feedback").  Up to 48 query rows per KV head it is decode_attn_fp8kv_extend().  Beyond that the pages
+ * every sequence attends are first widened, exactly (every E4M3 value is a bf16 value), into a bf16 copy in
+ * `scratch` -- page i of sequence b becomes page b * max_pages + i of the copy -- and the tensor-core kernel
+ * of decode_attn_extend() runs over that copy; the per-KV-head factors enter in that kernel (k_scale with
+ * the score scale, v_scale with the result), so the result is extend attention over the dequantised cache.
+ *   scratch        DEVICE, 256-byte aligned, caller-owned, at least
+ *                  decode_attn_fp8kv_extend_wide_scratch_bytes(B, max_pages, Hkv, P) bytes
+ *                  (= 2 * B * max_pages * Hkv * P * 256: the bf16 size of what the block table can name;
+ *                  pages past a sequence's end are not written or read).  DA_ERR_NULL / DA_ERR_STRIDE_ALIGN
+ *                  / DA_ERR_WORKSPACE otherwise, before any launch.  May be reused by the next call on the
+ *                  same stream.
+ * A page id outside the pool fills that page of the copy with NaN (DA_DEV_BAD_PAGE); the rows that attend
+ * it come out NaN.  Other arguments and conventions as decode_attn_fp8kv_extend().
+ */
+int decode_attn_fp8kv_extend_wide(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages,
+                                  const float *k_scale, const float *v_scale, const da_tensor *block_table,
+                                  const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse,
+                                  void *scratch, size_t scratch_bytes, void *stream);
+size_t decode_attn_fp8kv_extend_wide_scratch_bytes(int32_t B, int64_t max_pages, int32_t Hkv, int32_t P);
 
 /*
  * decode_attn_host_io -- the same call for a caller whose per-step tensors are in HOST memory.

@@ -76,6 +76,10 @@ def lib() -> ctypes.CDLL:
             L.decode_attn_extend.argtypes = [T, T, T, T, T, ctypes.c_float, T, T, vp]
             L.decode_attn_fp8kv_extend.restype = ctypes.c_int
             L.decode_attn_fp8kv_extend.argtypes = [T, T, T, vp, vp, T, T, ctypes.c_float, T, T, vp]
+            L.decode_attn_fp8kv_extend_wide.restype = ctypes.c_int
+            L.decode_attn_fp8kv_extend_wide.argtypes = [T, T, T, vp, vp, T, T, ctypes.c_float, T, T, vp, ctypes.c_size_t, vp]
+            L.decode_attn_fp8kv_extend_wide_scratch_bytes.restype = ctypes.c_size_t
+            L.decode_attn_fp8kv_extend_wide_scratch_bytes.argtypes = [i32, i64, i32, i32]
             L.decode_attn_host_io.restype = ctypes.c_int
             L.decode_attn_host_io.argtypes = [T, T, T, T, T, i32, ctypes.c_float, T, T, vp]
             L.decode_attn_fp8kv_host_io.restype = ctypes.c_int
@@ -366,6 +370,39 @@ def decode_attn_fp8kv_extend(q, k_pages, v_pages, k_scale, v_scale, block_table,
                                               v_scale.data_ptr() if v_scale is not None else None,
                                               _ref(tv[3]), _ref(tv[4]), float(scale), _ref(tv[5]), _ref(tv[6]),
                                               _stream_ptr(stream)))
+    return out, lse
+
+
+_wide_scratch = {}   # device index -> torch uint8 tensor for the widened cache of decode_attn_fp8kv_extend_wide
+
+
+def decode_attn_fp8kv_extend_wide(q, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens, scale: float,
+                                  out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                                  stream: Optional[torch.cuda.Stream] = None, out_dtype=torch.float32,
+                                  scratch: Optional[torch.Tensor] = None):
+    """``decode_attn_extend`` over the 8-bit cache for query blocks of any length: beyond 48 query rows per KV
+    head the attended pages are widened to bf16 in ``scratch`` (a uint8 device tensor; one is kept per device
+    when not given) and the tensor-core kernel runs over that copy.  Returns (out, lse)."""
+    if out is None:
+        out = torch.empty(q.shape, dtype=out_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    with torch.cuda.device(k_pages.device):
+        ensure_workspace(q.shape[0], q.shape[2], k_pages.shape[1], q.shape[3], k_pages.shape[2],
+                         block_table.shape[1], k_pages.device)
+        need = int(lib().decode_attn_fp8kv_extend_wide_scratch_bytes(q.shape[0], block_table.shape[1], k_pages.shape[1],
+                                                                     k_pages.shape[2]))
+        if scratch is None:
+            scratch = _wide_scratch.get(k_pages.device.index)
+            if scratch is None or scratch.numel() < need:
+                scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=k_pages.device)
+                _wide_scratch[k_pages.device.index] = scratch
+        tv = [_view(t) for t in (q, k_pages, v_pages, block_table, seq_lens, out, lse)]
+        _check(lib().decode_attn_fp8kv_extend_wide(_ref(tv[0]), _ref(tv[1]), _ref(tv[2]),
+                                                   k_scale.data_ptr() if k_scale is not None else None,
+                                                   v_scale.data_ptr() if v_scale is not None else None,
+                                                   _ref(tv[3]), _ref(tv[4]), float(scale), _ref(tv[5]), _ref(tv[6]),
+                                                   scratch.data_ptr(), scratch.numel(), _stream_ptr(stream)))
     return out, lse
 
 

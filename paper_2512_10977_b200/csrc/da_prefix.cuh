@@ -90,7 +90,7 @@ struct PrefixParams {
     // then that scratch copy, whose page i holds tokens [i P, (i+1) P) (no block table), and the per-KV-head
     // factors enter here -- k_scale[g] with the score scale, v_scale[g] with the result.  NULL / 0 otherwise.
     const float *k_scale, *v_scale;
-    int32_t identity_pages;
+    int32_t identity_pages;       // > 0: page t / P of sequence b is page b * identity_pages + t / P of the pools
 };
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -336,7 +336,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                 const int t = (t_begin + j) * PF_TOK + box * p.box_rows;
                 if (p.ext && t >= L)
                     return 0;   // past the sequence's last page: the block table has no entry
-                return p.identity_pages ? t / p.P : __ldg(bt_row + t / p.P);
+                return p.identity_pages ? bseq * p.identity_pages + t / p.P : __ldg(bt_row + t / p.P);
             };
             auto load_tile = [&](int j, int page) {   // tile j into buffer j % 3
                 const int buf = j % PF_NB;
@@ -817,23 +817,35 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
 struct WidenParams {
     const uint8_t *k_pages, *v_pages;     // strides in bytes: page, head, token
     int64_t k_sp, k_sh, k_st, v_sp, v_sh, v_st;
-    const int32_t *block_table;           // row 0 names the prefix pages
-    __nv_bfloat16 *k_out, *v_out;         // [pages][Hkv][P][128] each
+    const int32_t *block_table;           // cascade: row 0 names the prefix pages; extend: every row its sequence's
+    int64_t bt_sb;
+    const int32_t *seq_lens;              // extend: pages wholly past a sequence's end are left out; NULL: all pages
+    int64_t sl_stride;
+    __nv_bfloat16 *k_out, *v_out;         // [sequences][pages_per_seq][Hkv][P][128] each (cascade: one "sequence")
     int32_t *status;
     int32_t Hkv, P, num_pages;
+    int32_t pages_per_seq;                // cascade: pages of the prefix; extend: width of the block table
 };
 
 __global__ void __launch_bounds__(256) widen_prefix_kernel(const WidenParams p)
 {
-    const int pi = blockIdx.x / p.Hkv, g = blockIdx.x % p.Hkv;
-    const int page = __ldg(p.block_table + pi);
+    const int g = blockIdx.x % p.Hkv;
+    const int pi = (blockIdx.x / p.Hkv) % p.pages_per_seq, b = blockIdx.x / (p.Hkv * p.pages_per_seq);
+    if (p.seq_lens) {
+        const int L = __ldg(p.seq_lens + (int64_t)b * p.sl_stride);
+        // (a length the attention kernel refuses counts as empty there too)
+        if (L <= 0 || (int64_t)L > (int64_t)p.pages_per_seq * p.P || (int64_t)pi * p.P >= L)
+            return;
+    }
+    const int page = __ldg(p.block_table + (int64_t)b * p.bt_sb + pi);
     const bool bad = (uint32_t)page >= (uint32_t)p.num_pages;
     if (bad && threadIdx.x == 0 && g == 0)
-        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, 0, pi, page);
+        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, b, pi, page);
+    const int64_t slot = (int64_t)b * p.pages_per_seq + pi;   // page of the copy
     const int chunks = p.P * 8;   // 16 codes each
     for (int e = threadIdx.x; e < 2 * chunks; e += blockDim.x) {
         const int is_v = e >= chunks, c = (is_v ? e - chunks : e), tok = c >> 3, ch = c & 7;
-        __nv_bfloat16 *dst = (is_v ? p.v_out : p.k_out) + (((int64_t)pi * p.Hkv + g) * p.P + tok) * HEAD_DIM + ch * 16;
+        __nv_bfloat16 *dst = (is_v ? p.v_out : p.k_out) + ((slot * p.Hkv + g) * p.P + tok) * HEAD_DIM + ch * 16;
         uint32_t w[8];
         if (bad) {
 #pragma unroll

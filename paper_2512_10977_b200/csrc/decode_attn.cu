@@ -17,7 +17,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 113;
+constexpr int kVersion = 114;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -717,6 +717,10 @@ int run_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
         wp.k_sp = k_pages->stride[0]; wp.k_sh = k_pages->stride[1]; wp.k_st = k_pages->stride[2];
         wp.v_sp = v_pages->stride[0]; wp.v_sh = v_pages->stride[1]; wp.v_st = v_pages->stride[2];
         wp.block_table = static_cast<const int32_t *>(block_table->data);
+        wp.bt_sb = 0;
+        wp.seq_lens = nullptr;
+        wp.sl_stride = 0;
+        wp.pages_per_seq = (int32_t)prefix_pages;
         wp.k_out = static_cast<__nv_bfloat16 *>(prefix_scratch);
         wp.v_out = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(prefix_scratch) + half_copy);
         wp.status = reinterpret_cast<int32_t *>(ws + lay.status);
@@ -746,7 +750,7 @@ int run_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
     PrefixParams pf;
     pf.k_scale = kv8 ? k_scale : nullptr;
     pf.v_scale = kv8 ? v_scale : nullptr;
-    pf.identity_pages = kv8 ? 1 : 0;
+    pf.identity_pages = kv8 ? (int32_t)prefix_pages : 0;
     pf.q = static_cast<const __nv_bfloat16 *>(q->data);
     pf.q_sb = q->stride[0];
     pf.q_sq = 0;
@@ -1068,7 +1072,8 @@ namespace {
 // decode_attn_extend / decode_attn_fp8kv_extend
 int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
                const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, bool kv8,
-               const float *k_scale, const float *v_scale)
+               const float *k_scale, const float *v_scale, void *wide_scratch = nullptr, size_t wide_scratch_bytes = 0,
+               bool has_scratch_arg = false)
 {
     if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return DA_ERR_NULL;
     if (!q->data || !block_table->data || !seq_lens->data || !out->data || (lse && !lse->data)) return DA_ERR_NULL;
@@ -1128,18 +1133,60 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
                            lse ? &l3 : nullptr, stream, 0, kv8, k_scale, v_scale, (int)Lq, q->stride[1], out->stride[1],
                            lse ? lse->stride[1] : 0);
     }
-    if (kv8)
-        return DA_ERR_UNSUPPORTED;   // the tensor-core kernel reads a bf16 cache only
+    // The tensor-core kernel reads a bf16 cache.  Over the 8-bit cache, the pages every sequence attends are
+    // first widened, exactly, into a bf16 copy in the caller's scratch -- page i of sequence b becomes page
+    // b * max_pages + i of the copy, so the kernel needs no block table -- and the per-KV-head factors enter in
+    // the kernel (k_scale with the score scale, v_scale with the result), as in the cascade.
+    if (kv8 && !has_scratch_arg)
+        return DA_ERR_UNSUPPORTED;
     const int box_rows = P < PF_TOK ? (int)P : PF_TOK;
+    da_tensor kw = *k_pages, vw = *v_pages;   // the pools the kernel reads
+    if (kv8) {
+        const int64_t copy_pages = B * max_pages;
+        if (copy_pages > 0x7fffffffll || copy_pages * Hkv > 0x7fffffffll) return DA_ERR_UNSUPPORTED;
+        const size_t half_copy = (size_t)copy_pages * Hkv * P * HEAD_DIM * 2;   // bytes of the widened K (or V)
+        if (!wide_scratch) return DA_ERR_NULL;
+        if (reinterpret_cast<uintptr_t>(wide_scratch) & 255u) return DA_ERR_STRIDE_ALIGN;
+        if (wide_scratch_bytes < 2 * half_copy) return DA_ERR_WORKSPACE;
+        WidenParams wp;
+        wp.k_pages = static_cast<const uint8_t *>(k_pages->data);
+        wp.v_pages = static_cast<const uint8_t *>(v_pages->data);
+        wp.k_sp = k_pages->stride[0]; wp.k_sh = k_pages->stride[1]; wp.k_st = k_pages->stride[2];
+        wp.v_sp = v_pages->stride[0]; wp.v_sh = v_pages->stride[1]; wp.v_st = v_pages->stride[2];
+        wp.block_table = static_cast<const int32_t *>(block_table->data);
+        wp.bt_sb = block_table->stride[0];
+        wp.seq_lens = static_cast<const int32_t *>(seq_lens->data);
+        wp.sl_stride = seq_lens->stride[0];
+        wp.pages_per_seq = (int32_t)max_pages;
+        wp.k_out = static_cast<__nv_bfloat16 *>(wide_scratch);
+        wp.v_out = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(wide_scratch) + half_copy);
+        wp.status = reinterpret_cast<int32_t *>(ws + lay.status);
+        wp.Hkv = (int32_t)Hkv;
+        wp.P = (int32_t)P;
+        wp.num_pages = (int32_t)k_pages->shape[0];
+        widen_prefix_kernel<<<(unsigned)(copy_pages * Hkv), 256, 0, stream>>>(wp);
+        g_launches.fetch_add(1);
+        DA_CUDA(cudaGetLastError());
+        for (da_tensor *t : {&kw, &vw}) {
+            t->dtype = DA_BF16;
+            t->shape[0] = copy_pages;
+            t->stride[2] = HEAD_DIM;
+            t->stride[1] = P * HEAD_DIM;
+            t->stride[0] = Hkv * P * HEAD_DIM;
+        }
+        kw.data = wp.k_out;
+        vw.data = wp.v_out;
+    }
     CUtensorMap tm_k, tm_v;
-    rc = get_tmap(k_pages, box_rows, 1, &tm_k);
+    rc = get_tmap(&kw, box_rows, 1, &tm_k);
     if (rc != DA_OK) return rc;
-    rc = get_tmap(v_pages, box_rows, 2, &tm_v);   // (K: one plane per box; V: both)
+    rc = get_tmap(&vw, box_rows, 2, &tm_v);   // (K: one plane per box; V: both)
     if (rc != DA_OK) return rc;
 
     PrefixParams pf;
-    pf.k_scale = pf.v_scale = nullptr;
-    pf.identity_pages = 0;
+    pf.k_scale = kv8 ? k_scale : nullptr;
+    pf.v_scale = kv8 ? v_scale : nullptr;
+    pf.identity_pages = kv8 ? (int32_t)max_pages : 0;
     pf.q = static_cast<const __nv_bfloat16 *>(q->data);
     pf.q_sb = q->stride[0];
     pf.q_sq = q->stride[1];
@@ -1164,7 +1211,7 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
     pf.G = (int32_t)G;
     pf.P = (int32_t)P;
     pf.box_rows = box_rows;
-    pf.num_pages = (int32_t)k_pages->shape[0];
+    pf.num_pages = (int32_t)kw.shape[0];
     pf.out_bf16 = out->dtype == DA_BF16;
     pf.ext = 1;
     pf.Lq = (int32_t)Lq;
@@ -1232,6 +1279,20 @@ int decode_attn_fp8kv_extend(const da_tensor *q, const da_tensor *k_pages, const
 {
     return run_extend(q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, static_cast<cudaStream_t>(stream), true,
                       k_scale, v_scale);
+}
+
+int decode_attn_fp8kv_extend_wide(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const float *k_scale,
+                                  const float *v_scale, const da_tensor *block_table, const da_tensor *seq_lens, float scale,
+                                  da_tensor *out, da_tensor *lse, void *scratch, size_t scratch_bytes, void *stream)
+{
+    return run_extend(q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, static_cast<cudaStream_t>(stream), true,
+                      k_scale, v_scale, scratch, scratch_bytes, true);
+}
+
+size_t decode_attn_fp8kv_extend_wide_scratch_bytes(int32_t B, int64_t max_pages, int32_t Hkv, int32_t P)
+{
+    if (B <= 0 || max_pages <= 0 || Hkv <= 0 || P <= 0) return 0;
+    return (size_t)B * (size_t)max_pages * (size_t)Hkv * (size_t)P * HEAD_DIM * 2 * 2;
 }
 
 }  // extern "C"

@@ -454,6 +454,65 @@ def test_few_new_tokens_over_the_fp8_cache(da, Hq, Hkv, Lq, P):
     assert e.value.status == 5
 
 
+# ------------------------------------------------------------------ long query blocks over the 8-bit cache
+
+@pytest.mark.parametrize("Hq,Hkv,Lq", [(48, 8, 9), (48, 8, 64), (8, 8, 130), (32, 8, 100), (16, 1, 300)])
+@pytest.mark.parametrize("P", [16, 64, 128])
+def test_long_query_blocks_over_the_fp8_cache(da, Hq, Hkv, Lq, P):
+    """decode_attn_fp8kv_extend_wide: the attended pages widened exactly to bf16 in scratch, then the
+    tensor-core kernel with the per-head factors folded into the score scale and the result; the oracle is
+    causal extend attention over the dequantised cache."""
+    lens = [Lq, Lq + 1, 127 + Lq, 128 + Lq, 129 + Lq, 1000 + Lq, 0, 2500]
+    lens = [L if L == 0 else max(L, Lq) for L in lens]
+    case = fp8_case("wide8", lens, P, 5 * Lq + P + Hq, Hq=Hq, Hkv=Hkv, poison=True)
+    q = torch.randn((len(lens), Lq, Hq, 128), generator=torch.Generator().manual_seed(Lq + P)).to(torch.bfloat16)
+    ref, ref_lse = oracle.extend_attn_fp8kv_oracle(q, case.k_pages, case.v_pages, case.k_scale, case.v_scale,
+                                                   case.block_table, case.seq_lens, case.scale)
+    dev = workloads.to_device(case, "cuda")
+    out, lse = da.decode_attn_fp8kv_extend_wide(q.cuda(), dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale,
+                                                dev.block_table, dev.seq_lens, dev.scale)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    assert_close(out.cpu().numpy(), ref, f"fp8 wide extend Lq={Lq} P={P} out")
+    assert_close(lse.cpu().numpy(), ref_lse, f"fp8 wide extend Lq={Lq} P={P} lse")
+
+
+def test_long_query_blocks_fp8_scratch_errors_and_marking(da):
+    Lq = 40
+    lens = [500, 41, 900, 0]
+    case = fp8_case("wide8err", lens, 16, 77, poison=True)
+    dev = workloads.to_device(case, "cuda")
+    q = torch.randn((len(lens), Lq, 48, 128), generator=torch.Generator().manual_seed(3)).to(torch.bfloat16).cuda()
+    args = (q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, dev.block_table, dev.seq_lens, dev.scale)
+    need = da.lib().decode_attn_fp8kv_extend_wide_scratch_bytes(len(lens), dev.block_table.shape[1], 8, 16)
+    assert need == 2 * len(lens) * dev.block_table.shape[1] * 8 * 16 * 256
+    with pytest.raises(da.DecodeAttnError) as e:
+        da.decode_attn_fp8kv_extend_wide(*args, scratch=torch.empty(need - 256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 6
+    with pytest.raises(da.DecodeAttnError) as e:
+        da.decode_attn_fp8kv_extend_wide(*args, scratch=torch.empty(need + 512, dtype=torch.uint8, device="cuda")[16:])
+    assert e.value.status == 4
+    want, want_lse = da.decode_attn_fp8kv_extend_wide(*args)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    # a page id outside the pool, in the middle of sequence 2: its rows are NaN, the others as before
+    bt = dev.block_table.clone()
+    bt[2, 10] = dev.k_pages.shape[0] + 5
+    out, lse = da.decode_attn_fp8kv_extend_wide(q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, bt, dev.seq_lens,
+                                                dev.scale)
+    st = da.read_device_status()
+    assert st[0] == 1 and st[1] == 2
+    assert torch.isnan(out[2]).all() and torch.isnan(lse[2]).all()
+    keep = [0, 1, 3]
+    assert torch.equal(out[keep], want[keep]) and torch.equal(lse[keep], want_lse[keep])
+    # a sequence shorter than its new tokens: refused, empty
+    sl = dev.seq_lens.clone()
+    sl[1] = Lq - 1
+    out, lse = da.decode_attn_fp8kv_extend_wide(q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, dev.block_table, sl,
+                                                dev.scale)
+    assert da.read_device_status()[0] == 2
+    assert (out[1] == 0).all() and torch.isneginf(lse[1]).all()
+    assert torch.equal(out[[0, 2, 3]], want[[0, 2, 3]])
+
+
 # ------------------------------------------------------------------ shared prefix over the 8-bit cache
 
 @pytest.fixture(params=[0, 2], ids=["one-after-the-other", "side-by-side"])
@@ -527,3 +586,23 @@ def test_c5a_full_size_fp8_cascade_every_eighth_sequence(da, overlap):
     ref, ref_lse = oracle_of(sub)
     assert_close(out[ids].cpu().numpy(), ref, "c5a fp8 cascade out")
     assert_close(lse[ids].cpu().numpy(), ref_lse, "c5a fp8 cascade lse")
+
+
+def test_c2_full_size_long_query_block_over_the_fp8_cache_sampled(da):
+    """c2's 8-bit cache with 512 new tokens per sequence, as `bench.py --kv fp8 --extend 512` times it; sampled
+    sequences and query tokens against the single-token oracle on a cache cut at each query's position."""
+    Lq = 512
+    case = workloads.c2("cuda", kv_dtype="fp8")
+    q = torch.randn((case.B, Lq, 48, 128), device="cuda", generator=torch.Generator(device="cuda").manual_seed(7)).to(torch.bfloat16)
+    out, lse = da.decode_attn_fp8kv_extend_wide(q, case.k_pages, case.v_pages, case.k_scale, case.v_scale, case.block_table,
+                                                case.seq_lens, case.scale)
+    assert da.read_device_status() == (0, 0, 0, 0)
+    assert torch.isfinite(out).all() and torch.isfinite(lse).all()
+    ids = sorted({int(np.argmin(case.lens)), int(np.argmax(case.lens)), 17})
+    sub = workloads.host_subcase(case, ids)
+    for qi in (0, Lq // 2, Lq - 1):
+        cut = torch.from_numpy((sub.lens - Lq + qi + 1).astype(np.int32))
+        ref, ref_lse = oracle.decode_attn_fp8kv_oracle(q[ids, qi].cpu().contiguous(), sub.k_pages, sub.v_pages, sub.k_scale,
+                                                       sub.v_scale, sub.block_table, cut, 0, sub.scale)
+        assert_close(out[ids, qi].cpu().numpy(), ref, f"c2 fp8 extend qi={qi} out")
+        assert_close(lse[ids, qi].cpu().numpy(), ref_lse, f"c2 fp8 extend qi={qi} lse")
