@@ -220,13 +220,17 @@ def run_reference(args):
     best["value"] = best["value"] * best["seconds"] / sec
     best["seq_per_s"] = best["seq_per_s"] * best["seconds"] / sec
     ms = sec * 1e3
+    nbytes_ref = case.algorithmic_bytes(4)
     line = {
         "impl": "reference", "metric": METRIC, "value": best["value"], "unit": "GB/s", "n_gpus": args.gpus,
         "steps": len(res), "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        # the same keys and values as the other arm's line for this workload (what was sampled is in cpu_baseline)
         "config": {"workload": WORKLOAD_TEXT[args.workload] + kv_text(args), "sequences": case.B,
-                   "attended_tokens": int(case.attended_tokens().sum()), "algorithmic_bytes": case.algorithmic_bytes(4),
-                   "sample": best["sample"]},
+                   "attended_tokens": int(case.attended_tokens().sum()), "algorithmic_bytes": nbytes_ref,
+                   "l2": "inputs exceed L2 (no flush)" if nbytes_ref > 4 * 126e6 else "inputs fit L2; not flushed",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU", "grid_blocks": 0,
+                   "path": "decode_attn_fp8kv" if args.kv == "fp8" else "decode_attn"},
         "seq_per_s": best["seq_per_s"], "frac_of_8TBs": best["value"] / NOMINAL_HBM_GBS,
         "cpu_baseline": {k: best[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": best["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
