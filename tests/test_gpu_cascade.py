@@ -138,6 +138,21 @@ def test_c5a_full_size_cascade_every_fourth_sequence(da):
     ref, ref_lse = oracle.decode_attn_oracle(sub.q, sub.k_pages, sub.v_pages, sub.block_table, sub.seq_lens, 0, sub.scale)
     assert_close(out[ids].cpu().numpy(), ref, "c5a cascade out")
     assert_close(lse[ids].cpu().numpy(), ref_lse, "c5a cascade lse")
+    # the library's own choice (option 1) on this workload: own parts of up to 8192 tokens beside a 16384-token
+    # prefix -> side by side, which shows as two launches of the prefix kernel (six launches instead of five)
+    da.set_option("cascade_overlap", 1)
+    before = da.launch_count()
+    out1, lse1 = da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, case.block_table, case.seq_lens,
+                                        16384, case.scale)
+    assert da.launch_count() - before == 6
+    assert torch.allclose(out1, out, atol=2e-5, rtol=1e-4) and torch.allclose(lse1, lse, atol=2e-5, rtol=1e-4)
+    # ... and with block-table rows that can hold no more than the prefix and a page, one after the other
+    narrow = case.block_table[:, :1025].contiguous()
+    short = torch.clamp(case.seq_lens, max=16384 + 16)
+    before = da.launch_count()
+    da.decode_attn_cascade(case.q, case.k_pages, case.v_pages, narrow, short, 16384, case.scale)
+    assert da.launch_count() - before == 5
+    assert da.read_device_status() == (0, 0, 0, 0)
 
 
 def test_cascade_side_by_side_replayed_from_a_cuda_graph(da, overlap):
