@@ -273,12 +273,14 @@ int decode_attn_fp8kv_extend(const da_tensor *q, const da_tensor *k_pages, const
  * `scratch` -- page i of sequence b becomes page b * max_pages + i of the copy -- and the tensor-core kernel
  * of decode_attn_extend() runs over that copy; the per-KV-head factors enter in that kernel (k_scale with
  * the score scale, v_scale with the result), so the result is extend attention over the dequantised cache.
- *   scratch        DEVICE, 256-byte aligned, caller-owned, at least
+ *   scratch        DEVICE, 256-byte aligned, caller-owned.
  *                  decode_attn_fp8kv_extend_wide_scratch_bytes(B, max_pages, Hkv, P) bytes
  *                  (= 2 * B * max_pages * Hkv * P * 256: the bf16 size of what the block table can name;
- *                  pages past a sequence's end are not written or read).  DA_ERR_NULL / DA_ERR_STRIDE_ALIGN
- *                  / DA_ERR_WORKSPACE otherwise, before any launch.  May be reused by the next call on the
- *                  same stream.
+ *                  pages past a sequence's end are not written or read) serve all B sequences at once; with
+ *                  less, down to one sequence's share (that figure for B = 1), the sequences are served in
+ *                  groups of as many as fit, one group after the other on the stream.  Less than one
+ *                  sequence's share: DA_ERR_WORKSPACE; NULL: DA_ERR_NULL; misaligned: DA_ERR_STRIDE_ALIGN;
+ *                  all before any launch.  May be reused by the next call on the same stream.
  * A page id outside the pool fills that page of the copy with NaN (DA_DEV_BAD_PAGE); the rows that attend
  * it come out NaN.  Other arguments and conventions as decode_attn_fp8kv_extend().
  */

@@ -91,6 +91,7 @@ struct PrefixParams {
     // factors enter here -- k_scale[g] with the score scale, v_scale[g] with the result.  NULL / 0 otherwise.
     const float *k_scale, *v_scale;
     int32_t identity_pages;       // > 0: page t / P of sequence b is page b * identity_pages + t / P of the pools
+    int32_t seq0;                 // sequence number of row 0 in the caller's batch (a call may be made in groups): status records
 };
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -234,7 +235,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         L = p.seq_lens[(int64_t)bseq * p.sl_stride];
         if (L < 0 || (L > 0 && L < p.Lq) || (int64_t)L > p.max_pages * (int64_t)p.P) {
             if (tid == 0)
-                report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, bseq, 2, L);
+                report_status(p.status, 2 /* DA_DEV_BAD_SEQLEN */, bseq + p.seq0, 2, L);
             L = 0;
         }
         // causal: the block's last row attends tokens below L - Lq + qi_max + 1
@@ -351,7 +352,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
                     // tensor map fills zeros there and still counts the bytes), and the block is marked:
                     // its rows are written as NaN, not as a finite result over zeroed keys.
                     if (!is_v && pl == 0)
-                        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, bseq, t / p.P, page);
+                        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, bseq + p.seq0, t / p.P, page);
                     *poison_s = 1;
                     page = p.num_pages;
                 }
@@ -825,6 +826,7 @@ struct WidenParams {
     int32_t *status;
     int32_t Hkv, P, num_pages;
     int32_t pages_per_seq;                // cascade: pages of the prefix; extend: width of the block table
+    int32_t seq0;                         // sequence number of row 0 in the caller's batch (status records)
 };
 
 __global__ void __launch_bounds__(256) widen_prefix_kernel(const WidenParams p)
@@ -840,7 +842,7 @@ __global__ void __launch_bounds__(256) widen_prefix_kernel(const WidenParams p)
     const int page = __ldg(p.block_table + (int64_t)b * p.bt_sb + pi);
     const bool bad = (uint32_t)page >= (uint32_t)p.num_pages;
     if (bad && threadIdx.x == 0 && g == 0)
-        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, b, pi, page);
+        report_status(p.status, 1 /* DA_DEV_BAD_PAGE */, b + p.seq0, pi, page);
     const int64_t slot = (int64_t)b * p.pages_per_seq + pi;   // page of the copy
     const int chunks = p.P * 8;   // 16 codes each
     for (int e = threadIdx.x; e < 2 * chunks; e += blockDim.x) {

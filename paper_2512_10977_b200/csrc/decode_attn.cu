@@ -17,7 +17,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 114;
+constexpr int kVersion = 115;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
@@ -721,6 +721,7 @@ int run_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
         wp.seq_lens = nullptr;
         wp.sl_stride = 0;
         wp.pages_per_seq = (int32_t)prefix_pages;
+        wp.seq0 = 0;
         wp.k_out = static_cast<__nv_bfloat16 *>(prefix_scratch);
         wp.v_out = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(prefix_scratch) + half_copy);
         wp.status = reinterpret_cast<int32_t *>(ws + lay.status);
@@ -751,6 +752,7 @@ int run_cascade(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v
     pf.k_scale = kv8 ? k_scale : nullptr;
     pf.v_scale = kv8 ? v_scale : nullptr;
     pf.identity_pages = kv8 ? (int32_t)prefix_pages : 0;
+    pf.seq0 = 0;
     pf.q = static_cast<const __nv_bfloat16 *>(q->data);
     pf.q_sb = q->stride[0];
     pf.q_sq = 0;
@@ -1073,7 +1075,7 @@ namespace {
 int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_pages, const da_tensor *block_table,
                const da_tensor *seq_lens, float scale, da_tensor *out, da_tensor *lse, cudaStream_t stream, bool kv8,
                const float *k_scale, const float *v_scale, void *wide_scratch = nullptr, size_t wide_scratch_bytes = 0,
-               bool has_scratch_arg = false)
+               bool has_scratch_arg = false, int32_t seq0 = 0)
 {
     if (!q || !k_pages || !v_pages || !block_table || !seq_lens || !out) return DA_ERR_NULL;
     if (!q->data || !block_table->data || !seq_lens->data || !out->data || (lse && !lse->data)) return DA_ERR_NULL;
@@ -1158,6 +1160,7 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
         wp.seq_lens = static_cast<const int32_t *>(seq_lens->data);
         wp.sl_stride = seq_lens->stride[0];
         wp.pages_per_seq = (int32_t)max_pages;
+        wp.seq0 = seq0;
         wp.k_out = static_cast<__nv_bfloat16 *>(wide_scratch);
         wp.v_out = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(wide_scratch) + half_copy);
         wp.status = reinterpret_cast<int32_t *>(ws + lay.status);
@@ -1187,6 +1190,7 @@ int run_extend(const da_tensor *q, const da_tensor *k_pages, const da_tensor *v_
     pf.k_scale = kv8 ? k_scale : nullptr;
     pf.v_scale = kv8 ? v_scale : nullptr;
     pf.identity_pages = kv8 ? (int32_t)max_pages : 0;
+    pf.seq0 = seq0;
     pf.q = static_cast<const __nv_bfloat16 *>(q->data);
     pf.q_sb = q->stride[0];
     pf.q_sq = q->stride[1];
@@ -1285,6 +1289,40 @@ int decode_attn_fp8kv_extend_wide(const da_tensor *q, const da_tensor *k_pages, 
                                   const float *v_scale, const da_tensor *block_table, const da_tensor *seq_lens, float scale,
                                   da_tensor *out, da_tensor *lse, void *scratch, size_t scratch_bytes, void *stream)
 {
+    // A scratch buffer that holds the widened pages of some, not all, of the sequences: the call is made in
+    // groups of as many sequences as fit, one after the other on the stream (the next group's copy follows the
+    // kernel that read the last one's).  Everything else about the arguments is checked by the calls themselves.
+    if (q && q->ndim == 4 && k_pages && k_pages->ndim == 4 && block_table && block_table->ndim == 2 && seq_lens &&
+        seq_lens->ndim == 1 && out && out->ndim == 4 && (!lse || lse->ndim == 3) && scratch && q->data && out->data &&
+        block_table->data && seq_lens->data && (!lse || lse->data)) {
+        const int64_t B = q->shape[0], Lq = q->shape[1], Hq = q->shape[2];
+        const int64_t Hkv = k_pages->shape[1], P = k_pages->shape[2], max_pages = block_table->shape[1];
+        if (B > 1 && Lq > 0 && Hkv > 0 && Hq > 0 && Hq % Hkv == 0 && P > 0 && P <= 128 && max_pages > 0 &&
+            max_pages <= 0x7fffffffll && Lq * (Hq / Hkv) > kMaxStreamRows && out->shape[0] == B &&
+            block_table->shape[0] == B && seq_lens->shape[0] == B && (!lse || lse->shape[0] == B)) {
+            const size_t per_seq = (size_t)max_pages * (size_t)Hkv * (size_t)P * HEAD_DIM * 2 * 2;
+            if (scratch_bytes >= per_seq && scratch_bytes / per_seq < (size_t)B) {
+                const int64_t group = (int64_t)(scratch_bytes / per_seq);
+                auto rows = [](const da_tensor *t, int64_t b0, int64_t n, int64_t item) {
+                    da_tensor v = *t;
+                    v.data = static_cast<uint8_t *>(t->data) + b0 * t->stride[0] * item;
+                    v.shape[0] = n;
+                    return v;
+                };
+                for (int64_t b0 = 0; b0 < B; b0 += group) {
+                    const int64_t n = std::min<int64_t>(group, B - b0);
+                    da_tensor qg = rows(q, b0, n, 2), btg = rows(block_table, b0, n, 4), slg = rows(seq_lens, b0, n, 4);
+                    da_tensor og = rows(out, b0, n, out->dtype == DA_BF16 ? 2 : 4), lg;
+                    if (lse) lg = rows(lse, b0, n, 4);
+                    const int rc = run_extend(&qg, k_pages, v_pages, &btg, &slg, scale, &og, lse ? &lg : nullptr,
+                                              static_cast<cudaStream_t>(stream), true, k_scale, v_scale, scratch,
+                                              scratch_bytes, true, (int32_t)b0);
+                    if (rc != DA_OK) return rc;
+                }
+                return DA_OK;
+            }
+        }
+    }
     return run_extend(q, k_pages, v_pages, block_table, seq_lens, scale, out, lse, static_cast<cudaStream_t>(stream), true,
                       k_scale, v_scale, scratch, scratch_bytes, true);
 }

@@ -486,13 +486,27 @@ def test_long_query_blocks_fp8_scratch_errors_and_marking(da):
     need = da.lib().decode_attn_fp8kv_extend_wide_scratch_bytes(len(lens), dev.block_table.shape[1], 8, 16)
     assert need == 2 * len(lens) * dev.block_table.shape[1] * 8 * 16 * 256
     with pytest.raises(da.DecodeAttnError) as e:
-        da.decode_attn_fp8kv_extend_wide(*args, scratch=torch.empty(need - 256, dtype=torch.uint8, device="cuda"))
-    assert e.value.status == 6
-    with pytest.raises(da.DecodeAttnError) as e:
         da.decode_attn_fp8kv_extend_wide(*args, scratch=torch.empty(need + 512, dtype=torch.uint8, device="cuda")[16:])
     assert e.value.status == 4
     want, want_lse = da.decode_attn_fp8kv_extend_wide(*args)
     assert da.read_device_status() == (0, 0, 0, 0)
+    # scratch for two of the four sequences, and for one: served in groups, same result
+    one = need // len(lens)
+    for room in (2 * one, one + 256):
+        got, got_lse = da.decode_attn_fp8kv_extend_wide(*args, scratch=torch.empty(room, dtype=torch.uint8, device="cuda"))
+        assert da.read_device_status() == (0, 0, 0, 0)
+        assert torch.equal(got, want) and torch.equal(got_lse, want_lse)
+    with pytest.raises(da.DecodeAttnError) as e:
+        da.decode_attn_fp8kv_extend_wide(*args, scratch=torch.empty(one - 256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 6
+    # (the status record names the sequence by its place in the whole batch, whichever group it was served in)
+    bt = dev.block_table.clone()
+    bt[2, 10] = dev.k_pages.shape[0] + 5
+    out, lse = da.decode_attn_fp8kv_extend_wide(q, dev.k_pages, dev.v_pages, dev.k_scale, dev.v_scale, bt, dev.seq_lens,
+                                                dev.scale, scratch=torch.empty(one, dtype=torch.uint8, device="cuda"))
+    st = da.read_device_status()
+    assert st[0] == 1 and st[1] == 2
+    assert torch.isnan(out[2]).all() and torch.equal(out[[0, 1, 3]], want[[0, 1, 3]])
     # a page id outside the pool, in the middle of sequence 2: its rows are NaN, the others as before
     bt = dev.block_table.clone()
     bt[2, 10] = dev.k_pages.shape[0] + 5
