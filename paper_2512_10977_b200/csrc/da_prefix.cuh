@@ -45,7 +45,7 @@ constexpr uint32_t PF_WAIT_SLEEP_NS = 32;     // softmax warps yield while they 
 constexpr int PF_NB = 3;                     // K and V buffers (tiles in flight)
 constexpr int PF_OFF_K = PF_TILE;
 constexpr int PF_OFF_V = (1 + PF_NB) * PF_TILE;
-constexpr int PF_OFF_BARS = (1 + 2 * PF_NB) * PF_TILE;   // kfull[3], vfull[3], kfree[3], o[3], s[2], p, x[4]
+constexpr int PF_OFF_BARS = (1 + 2 * PF_NB) * PF_TILE;   // kfull[3], vfull[3], kfree[3], o[3], s[2], p[2], x[4]
 constexpr int PF_OFF_MISC = PF_OFF_BARS + 160;  // TMEM base address, abort flag, "a page id was bad" flag
 constexpr int PF_OFF_XCHG = PF_OFF_MISC + 16;   // row maxima / sums swapped between a row's two threads
 constexpr int PF_SMEM_BYTES = PF_OFF_XCHG + PF_TPR * 128 * 4;   // 2 buffers of bf16 maxima, or one of fp32 sums
@@ -219,7 +219,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
     // per K/V buffer (tile t uses buffer t % 3): K loaded, V loaded, K no longer needed (scores complete),
     // PV product complete; per S buffer (t & 1): scores complete; P written; row-maximum exchange
     const uint32_t bar_kfull = sb + PF_OFF_BARS, bar_vfull = bar_kfull + 24, bar_kfree = bar_kfull + 48, bar_o = bar_kfull + 72,
-                   bar_s = bar_kfull + 96, bar_p = bar_kfull + 112, bar_x0 = bar_kfull + 120;   // x: one per 32 rows
+                   bar_s = bar_kfull + 96, bar_p = bar_kfull + 112, bar_x0 = bar_kfull + 128;   // s, p: one per S buffer; x: one per 32 rows
     volatile int *abort_flag = &abort_s;
 
     // block -> (row tile, kv head, [sequence,] split)
@@ -266,7 +266,11 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
         }
         mbar_init(bar_s, 1);
         mbar_init(bar_s + 8, 1);
+        // (one hand-over barrier per S buffer: a warp cannot arrive for tile j + 2 before the hand-over of tile j is
+        //  complete -- those scores are only written after it -- so no arrival can be counted for the wrong tile,
+        //  however far one warp runs ahead of another)
         mbar_init(bar_p, PF_DRV);
+        mbar_init(bar_p + 8, PF_DRV);
         for (int i = 0; i < 4; ++i)
             mbar_init(bar_x0 + 8 * i, PF_TPR);   // the row-maximum exchange of one quarter of the rows: its PF_TPR warps
         mbar_fence_init();
@@ -480,7 +484,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             const uint32_t acc = low ? tmem_o2 : tmem_o;
             DA_PH_DECL(ph, ph_t);
             for (int j = 0; ok && j < ntiles; ++j) {
-                ok = mbar_wait_bounded(bar_p, (uint32_t)(j & 1), abort_flag);
+                ok = mbar_wait_bounded(bar_p + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag);
                 DA_PH(ph, 0, ph_t);
                 ok = ok && mbar_wait_bounded(bar_vfull + 8 * (j % PF_NB), (uint32_t)((j / PF_NB) & 1), abort_flag);
                 DA_PH(ph, 1, ph_t);
@@ -575,9 +579,9 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             }
             __syncwarp();
             if (lane == 0)
-                mbar_arrive(bar_p);
+                mbar_arrive(bar_p + 8 * (j & 1));
             // (no second arrival before every warp has made its first: wait for this tile's hand-over)
-            if (!mbar_wait_bounded(bar_p, (uint32_t)(j & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
+            if (!mbar_wait_bounded(bar_p + 8 * (j & 1), (uint32_t)((j >> 1) & 1), abort_flag, DA_WAIT_LIMIT_NS, PF_WAIT_SLEEP_NS)) {
                 ok = false;
                 break;
             }
@@ -709,7 +713,7 @@ prefix_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ 
             tc_fence_before();          // this thread's TMEM reads and writes precede the MMAs that follow
             __syncwarp();
             if (lane == 0)
-                mbar_arrive(bar_p);     // one arrival per warp: 512 arrivals on one barrier cost hundreds of cycles
+                mbar_arrive(bar_p + 8 * (j & 1));     // one arrival per warp: 512 arrivals on one barrier cost hundreds of cycles
             DA_PH(ph, 3, ph_t);
         }
         uint32_t o_raw[PF_COLS];

@@ -17,7 +17,7 @@ namespace {
 
 using namespace da;
 
-constexpr int kVersion = 115;
+constexpr int kVersion = 116;
 constexpr int kMaxDevices = 64;
 constexpr int kMaxGridBlocks = 4096;
 constexpr int kMaxUnits = 8192;
