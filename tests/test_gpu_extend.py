@@ -174,3 +174,23 @@ def test_c2_full_size_extend_sampled(da, Lq):
                                                  cut, 0, sub.scale)
         assert_close(out[ids, qi].cpu().numpy(), ref, f"c2 extend Lq={Lq} qi={qi} out")
         assert_close(lse[ids, qi].cpu().numpy(), ref_lse, f"c2 extend Lq={Lq} qi={qi} lse")
+
+
+@pytest.mark.parametrize("Lq,Hq", [(4, 48), (22, 48), (130, 8), (40, 16)])
+def test_repeated_tensor_core_calls_give_identical_results(da, Lq, Hq):
+    """The tensor-core kernel adds in a fixed order, so identical calls must agree bit for bit; a hand-over
+    race between its warps would show up here as an occasional difference (partly filled row tiles included)."""
+    lens = [Lq + 700, Lq, 2600, 1300 + Lq]
+    case = workloads.build_case("rep", lens, 16, 90 + Lq, "cpu", Hq=Hq, Hkv=8)
+    q = torch.randn((len(lens), Lq, Hq, 128), generator=torch.Generator().manual_seed(Lq)).to(torch.bfloat16).cuda()
+    dev = workloads.to_device(case, "cuda")
+    da.set_option("extend_stream_rows", 0)      # always the tensor-core kernel
+    try:
+        first, first_lse = da.decode_attn_extend(q, dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, dev.scale)
+        first, first_lse = first.clone(), first_lse.clone()
+        for _ in range(40):
+            out, lse = da.decode_attn_extend(q, dev.k_pages, dev.v_pages, dev.block_table, dev.seq_lens, dev.scale)
+            assert torch.equal(out, first) and torch.equal(lse, first_lse)
+    finally:
+        da.set_option("extend_stream_rows", 16)
+    assert da.read_device_status() == (0, 0, 0, 0)
